@@ -1,0 +1,179 @@
+/*
+ * caote.h — C ABI of the CAOTE eviction-scoring attention step for NVIDIA B200 (sm_100a).
+ *
+ * CAOTE ("Cache selection via Attention Output error-based Token Eviction") scores every cached
+ * token j of a (sequence, KV head) unit by the change in attention output that evicting it would
+ * cause, c_j = w_j / (1 - w_j) * || X - v_j ||_2, keeps the highest-scoring tokens up to a budget
+ * and drops the rest from the K/V cache.
+ *
+ * Conventions shared by every entry point
+ * ---------------------------------------
+ * Notation (Sec. 2 "Background" and Sec. 3 of the paper): B sequences, Hq query heads, Hkv KV heads,
+ * G = Hq / Hkv query heads per KV head (query head hq belongs to KV head hq / G), d = head_dim,
+ * cap = slots per unit, n = len[b] valid slots of sequence b (the m = n_new newest tokens included),
+ * budget b. A "unit" is one (sequence, KV head) pair; unit index u = b * Hkv + hkv.
+ *
+ * Layout. All arrays are dense, row-major, innermost dimension last:
+ *   q            [B, Hq,  m,   d]   I/O dtype (bf16 or fp32)
+ *   K, V         [B, Hkv, cap, d]   I/O dtype; slot j of unit u holds one cached token
+ *   o            [B, Hq,  m,   d]   I/O dtype
+ *   base, scores [B, Hkv, cap]      fp32
+ *   pos          [B, Hkv, cap]      int32, original position of the token held by each slot
+ *   len, budget, n_evict, n_seen [B] int32
+ *   evict_idx    [B, Hkv, max_evict] int32
+ * Every pointer named below is a DEVICE pointer unless it says "host". K, V, q, o must be 16-byte
+ * aligned; the others 4-byte aligned; workspace 256-byte aligned.
+ *
+ * Ownership. The caller owns every buffer and the stream. The library allocates no device memory,
+ * keeps no per-call state, never synchronises (except caote_read_status) and only enqueues work on
+ * the stream it is given. Calls on the same stream compose in order.
+ *
+ * Errors. Every entry point returns CAOTE_OK (0) or a negative caote_status_t. Arguments that the
+ * host can see (null pointers, shapes, workspace size, dtype, head_dim) are validated before any
+ * launch and yield CAOTE_ERR_INVALID_ARG / CAOTE_ERR_UNSUPPORTED; nothing is enqueued in that case.
+ * Conditions only the device can see (len[b] > cap, len[b] < n_new, more evictions than max_evict,
+ * an append that would overflow cap) make the kernel skip that sequence and record a code in the
+ * workspace status word, read back with caote_read_status. No entry point throws, aborts or traps.
+ */
+#ifndef CAOTE_H_
+#define CAOTE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* A CUDA stream handle (cudaStream_t), passed as an opaque pointer so that this header needs no CUDA
+ * include. NULL is the legacy default stream. */
+typedef void* caote_stream_t;
+
+typedef enum {
+  CAOTE_OK = 0,
+  CAOTE_ERR_INVALID_ARG = -1, /* null pointer, bad shape, workspace too small                     */
+  CAOTE_ERR_UNSUPPORTED = -2, /* dtype / head_dim / mode not built, or the device is not sm_100   */
+  CAOTE_ERR_CUDA = -3,        /* a CUDA runtime or driver call failed (see caote_last_cuda_error) */
+  CAOTE_ERR_TIMEOUT = -4,     /* a bounded device-side wait gave up (status word only)            */
+  CAOTE_ERR_BAD_LENGTH = -5,  /* device saw len[b] > cap or 0 < len[b] < n_new (status word only) */
+  CAOTE_ERR_OVERFLOW = -6     /* device saw n_evict > max_evict or len + n_new > cap (status word) */
+} caote_status_t;
+
+typedef enum { CAOTE_BF16 = 0, CAOTE_F32 = 1 } caote_dtype_t;
+
+/* How the base retention score h_j is obtained from the attention matrix A (rows = this call's
+ * queries, columns = cached tokens), Sec. 2 (f_score) and Sec. 3.2:
+ *   LAST_QUERY  h_j = sum_g A^g[m-1, j]                 (TOVA: the last query row of every group head)
+ *   CHUNK_SUM   h_j = sum_g sum_i A^g[i, j]             (H2O over this call's block of m queries only)
+ *   ACCUM       base_j += sum_g sum_i A^g[i, j]; h = base   (H2O carried across calls; base is in/out)
+ *   EXTERNAL    h_j = base_j                            (any non-negative score the caller computed)
+ */
+typedef enum {
+  CAOTE_BASE_LAST_QUERY = 0,
+  CAOTE_BASE_CHUNK_SUM = 1,
+  CAOTE_BASE_ACCUM = 2,
+  CAOTE_BASE_EXTERNAL = 3
+} caote_base_mode_t;
+
+/* How the cache is repacked after eviction.
+ *   FILL    surviving tokens of the last k slots move into the holes left below the new length;
+ *           at most k rows move per unit; slot order is not position order afterwards (use pos).
+ *   STABLE  surviving tokens keep their relative order (everything behind the first hole shifts).
+ */
+typedef enum { CAOTE_COMPACT_FILL = 0, CAOTE_COMPACT_STABLE = 1 } caote_compact_mode_t;
+
+typedef struct {
+  int32_t batch;      /* B >= 1                                                                    */
+  int32_t n_q_heads;  /* Hq, a multiple of n_kv_heads; G = Hq / Hkv <= 16                          */
+  int32_t n_kv_heads; /* Hkv >= 1                                                                  */
+  int32_t head_dim;   /* d in {64, 128}                                                            */
+  int32_t capacity;   /* cap: slots per unit in K, V, base, scores, pos                            */
+  int32_t n_new;      /* m >= 1: the last m valid slots of every sequence are the keys of this
+                         call's own m queries; query i sees slots j <= n - m + i (causal inside
+                         the block, Sec. 2 "Block-wise prompt prefill")                            */
+  int32_t dtype;      /* caote_dtype_t of q, K, V, o                                               */
+  float scale;        /* logits are scale * <q, k>; the paper writes Softmax(QK^T) without a scale,
+                         callers normally pass 1/sqrt(head_dim)                                    */
+  int32_t base_mode;  /* caote_base_mode_t                                                         */
+  int32_t flags;      /* reserved, must be 0                                                       */
+} caote_params_t;
+
+/* Bytes of scratch that caote_score / caote_select_evict / caote_compact / caote_append need for these
+ * parameters (the maximum over the four; one buffer serves all). Returns 0 if params is invalid.
+ * The first 256 bytes hold the status word; zero them once (cudaMemsetAsync) before first use. */
+size_t caote_workspace_bytes(const caote_params_t* params);
+
+/* Append the m = n_new newest tokens of every sequence to its cache (Sec. 2: the block
+ * [K_{:t}, K_{t+1:t+m}] the new queries attend to). For sequence b with n = len[b]:
+ * K/V[b, h, n + i, :] = k_new/v_new[b, h, i, :], base[...] = 0, pos[...] = n_seen[b] + i for
+ * i in [0, m); then len[b] = n + m and n_seen[b] += m.
+ *   k_new, v_new  [B, Hkv, m, d] I/O dtype, in.     base, pos, n_seen: nullable (skipped when NULL).
+ * A sequence with n + m > cap is skipped and CAOTE_ERR_OVERFLOW is recorded. */
+int caote_append(const caote_params_t* params, void* K, void* V, float* base, int32_t* pos,
+                 int32_t* len, int32_t* n_seen, const void* k_new, const void* v_new,
+                 void* workspace, size_t workspace_bytes, caote_stream_t stream);
+
+/* Attention + CAOTE scores for every unit.
+ *   1. alpha^g_i = softmax_j(scale * <q^g_i, k_j>) over visible slots j <= n - m + i, and the
+ *      pre-eviction attention output o^g_i = sum_j alpha^g_{i,j} v_j   (Sec. 2, generation and
+ *      block-wise prefill equations; Sec. 3.1, X_attn = V A^T).
+ *   2. base score h per base_mode (Sec. 2 f_score; Sec. 3.2 "CAOTE for H2O"), summed over the G
+ *      query heads that share the KV head.
+ *   3. w_j = h_j / sum_i h_i (Sec. 3.2, normalisation equation) and X = sum_j w_j v_j.
+ *   4. scores[u, j] = w_j / (1 - w_j) * || X - v_j ||_2  (Sec. 3.1 CAOTE score; Sec. 3.2 general
+ *      form; Theorem 3.2 shows it equals the output error of evicting j and renormalising).
+ *      1 - w_j == 0 gives +inf; sum_i h_i == 0 gives 0. Scores are >= +0 and never NaN for finite
+ *      inputs.
+ *   q in; K, V in; len in (n = len[b]; 0 skips the sequence; n_new <= n <= cap required);
+ *   base: in/out for ACCUM, in for EXTERNAL, ignored (may be NULL) otherwise;
+ *   o out (all m rows of all Hq heads); scores out for slots j < n, slots >= n are left untouched. */
+int caote_score(const caote_params_t* params, const void* q, const void* K, const void* V,
+                const int32_t* len, float* base, void* o, float* scores, void* workspace,
+                size_t workspace_bytes, caote_stream_t stream);
+
+/* Choose the tokens to evict: for sequence b, k = max(0, len[b] - budget[b]) (Sec. 2: the top-b tokens
+ * by score are retained; Sec. 4.1 "Prompt consumption": evict once the cache exceeds the budget), and
+ * every unit of b evicts its k smallest entries under the total order (score bits, pos) ascending —
+ * among equal scores the older token goes first. pos == NULL uses the slot index as pos.
+ *   evict_idx[u, 0..k) out: the evicted SLOT indices in ascending order; n_evict[b] = k out.
+ * budget[b] >= 1 required (a smaller value is treated as 1). k > max_evict records
+ * CAOTE_ERR_OVERFLOW, sets n_evict[b] = 0 and evicts nothing for that sequence. */
+int caote_select_evict(const caote_params_t* params, const float* scores, const int32_t* len,
+                       const int32_t* budget, const int32_t* pos, int32_t* evict_idx,
+                       int32_t max_evict, int32_t* n_evict, void* workspace,
+                       size_t workspace_bytes, caote_stream_t stream);
+
+/* Remove the evicted slots from K, V, base, pos in place and set len[b] -= n_evict[b], so that the
+ * cache is back within budget before the next block arrives (Sec. 2, budgeted block-wise flow).
+ * mode is a caote_compact_mode_t. base, pos nullable. evict_idx rows must be ascending and unique
+ * (what caote_select_evict writes). */
+int caote_compact(const caote_params_t* params, void* K, void* V, float* base, int32_t* pos,
+                  int32_t* len, const int32_t* evict_idx, int32_t max_evict, const int32_t* n_evict,
+                  int32_t mode, void* workspace, size_t workspace_bytes, caote_stream_t stream);
+
+/* One whole eviction step on the stream: caote_append (skipped when k_new is NULL), caote_score,
+ * caote_select_evict, caote_compact, with the same arguments and the same results as the four
+ * separate calls. */
+int caote_step(const caote_params_t* params, const void* q, const void* k_new, const void* v_new,
+               void* K, void* V, float* base, int32_t* pos, int32_t* len, int32_t* n_seen,
+               const int32_t* budget, void* o, float* scores, int32_t* evict_idx, int32_t max_evict,
+               int32_t* n_evict, int32_t compact_mode, void* workspace, size_t workspace_bytes,
+               caote_stream_t stream);
+
+/* Synchronise the stream, copy the status word to *status_out (host pointer) and reset it to CAOTE_OK.
+ * The word holds the first device-side error since the last reset. */
+int caote_read_status(void* workspace, caote_stream_t stream, int32_t* status_out);
+
+/* Static, NUL-terminated description of a status code. */
+const char* caote_status_string(int status);
+
+/* Text of the last CUDA error seen by the calling thread inside this library ("" if none). */
+const char* caote_last_cuda_error(void);
+
+/* Number of kernels this library has launched from this process since it was loaded. */
+int64_t caote_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CAOTE_H_ */
