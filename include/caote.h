@@ -16,7 +16,7 @@
  * Layout. All arrays are dense, row-major, innermost dimension last:
  *   q            [B, Hq,  m,   d]   I/O dtype (bf16 or fp32)
  *   K, V         [B, Hkv, cap, d]   I/O dtype; slot j of unit u holds one cached token
- *   o            [B, Hq,  m,   d]   I/O dtype
+ *   o            [B, Hq,  m,   d]   fp32 (the fp32 accumulator is handed out unrounded)
  *   base, scores [B, Hkv, cap]      fp32
  *   pos          [B, Hkv, cap]      int32, original position of the token held by each slot
  *   len, budget, n_evict, n_seen [B] int32
@@ -40,6 +40,12 @@
 
 #include <stddef.h>
 #include <stdint.h>
+
+#if defined(__GNUC__)
+#define CAOTE_API __attribute__((visibility("default")))
+#else
+#define CAOTE_API
+#endif
 
 #ifdef __cplusplus
 extern "C" {
@@ -91,7 +97,7 @@ typedef struct {
   int32_t n_new;      /* m >= 1: the last m valid slots of every sequence are the keys of this
                          call's own m queries; query i sees slots j <= n - m + i (causal inside
                          the block, Sec. 2 "Block-wise prompt prefill")                            */
-  int32_t dtype;      /* caote_dtype_t of q, K, V, o                                               */
+  int32_t dtype;      /* caote_dtype_t of q, K, V                                                  */
   float scale;        /* logits are scale * <q, k>; the paper writes Softmax(QK^T) without a scale,
                          callers normally pass 1/sqrt(head_dim)                                    */
   int32_t base_mode;  /* caote_base_mode_t                                                         */
@@ -101,7 +107,7 @@ typedef struct {
 /* Bytes of scratch that caote_score / caote_select_evict / caote_compact / caote_append need for these
  * parameters (the maximum over the four; one buffer serves all). Returns 0 if params is invalid.
  * The first 256 bytes hold the status word; zero them once (cudaMemsetAsync) before first use. */
-size_t caote_workspace_bytes(const caote_params_t* params);
+CAOTE_API size_t caote_workspace_bytes(const caote_params_t* params);
 
 /* Append the m = n_new newest tokens of every sequence to its cache (Sec. 2: the block
  * [K_{:t}, K_{t+1:t+m}] the new queries attend to). For sequence b with n = len[b]:
@@ -109,7 +115,7 @@ size_t caote_workspace_bytes(const caote_params_t* params);
  * i in [0, m); then len[b] = n + m and n_seen[b] += m.
  *   k_new, v_new  [B, Hkv, m, d] I/O dtype, in.     base, pos, n_seen: nullable (skipped when NULL).
  * A sequence with n + m > cap is skipped and CAOTE_ERR_OVERFLOW is recorded. */
-int caote_append(const caote_params_t* params, void* K, void* V, float* base, int32_t* pos,
+CAOTE_API int caote_append(const caote_params_t* params, void* K, void* V, float* base, int32_t* pos,
                  int32_t* len, int32_t* n_seen, const void* k_new, const void* v_new,
                  void* workspace, size_t workspace_bytes, caote_stream_t stream);
 
@@ -127,8 +133,8 @@ int caote_append(const caote_params_t* params, void* K, void* V, float* base, in
  *   q in; K, V in; len in (n = len[b]; 0 skips the sequence; n_new <= n <= cap required);
  *   base: in/out for ACCUM, in for EXTERNAL, ignored (may be NULL) otherwise;
  *   o out (all m rows of all Hq heads); scores out for slots j < n, slots >= n are left untouched. */
-int caote_score(const caote_params_t* params, const void* q, const void* K, const void* V,
-                const int32_t* len, float* base, void* o, float* scores, void* workspace,
+CAOTE_API int caote_score(const caote_params_t* params, const void* q, const void* K, const void* V,
+                const int32_t* len, float* base, float* o, float* scores, void* workspace,
                 size_t workspace_bytes, caote_stream_t stream);
 
 /* Choose the tokens to evict: for sequence b, k = max(0, len[b] - budget[b]) (Sec. 2: the top-b tokens
@@ -138,7 +144,7 @@ int caote_score(const caote_params_t* params, const void* q, const void* K, cons
  *   evict_idx[u, 0..k) out: the evicted SLOT indices in ascending order; n_evict[b] = k out.
  * budget[b] >= 1 required (a smaller value is treated as 1). k > max_evict records
  * CAOTE_ERR_OVERFLOW, sets n_evict[b] = 0 and evicts nothing for that sequence. */
-int caote_select_evict(const caote_params_t* params, const float* scores, const int32_t* len,
+CAOTE_API int caote_select_evict(const caote_params_t* params, const float* scores, const int32_t* len,
                        const int32_t* budget, const int32_t* pos, int32_t* evict_idx,
                        int32_t max_evict, int32_t* n_evict, void* workspace,
                        size_t workspace_bytes, caote_stream_t stream);
@@ -147,31 +153,44 @@ int caote_select_evict(const caote_params_t* params, const float* scores, const 
  * cache is back within budget before the next block arrives (Sec. 2, budgeted block-wise flow).
  * mode is a caote_compact_mode_t. base, pos nullable. evict_idx rows must be ascending and unique
  * (what caote_select_evict writes). */
-int caote_compact(const caote_params_t* params, void* K, void* V, float* base, int32_t* pos,
+CAOTE_API int caote_compact(const caote_params_t* params, void* K, void* V, float* base, int32_t* pos,
                   int32_t* len, const int32_t* evict_idx, int32_t max_evict, const int32_t* n_evict,
                   int32_t mode, void* workspace, size_t workspace_bytes, caote_stream_t stream);
 
 /* One whole eviction step on the stream: caote_append (skipped when k_new is NULL), caote_score,
  * caote_select_evict, caote_compact, with the same arguments and the same results as the four
  * separate calls. */
-int caote_step(const caote_params_t* params, const void* q, const void* k_new, const void* v_new,
+CAOTE_API int caote_step(const caote_params_t* params, const void* q, const void* k_new, const void* v_new,
                void* K, void* V, float* base, int32_t* pos, int32_t* len, int32_t* n_seen,
-               const int32_t* budget, void* o, float* scores, int32_t* evict_idx, int32_t max_evict,
+               const int32_t* budget, float* o, float* scores, int32_t* evict_idx, int32_t max_evict,
                int32_t* n_evict, int32_t compact_mode, void* workspace, size_t workspace_bytes,
                caote_stream_t stream);
 
 /* Synchronise the stream, copy the status word to *status_out (host pointer) and reset it to CAOTE_OK.
  * The word holds the first device-side error since the last reset. */
-int caote_read_status(void* workspace, caote_stream_t stream, int32_t* status_out);
+CAOTE_API int caote_read_status(void* workspace, caote_stream_t stream, int32_t* status_out);
 
 /* Static, NUL-terminated description of a status code. */
-const char* caote_status_string(int status);
+CAOTE_API const char* caote_status_string(int status);
 
 /* Text of the last CUDA error seen by the calling thread inside this library ("" if none). */
-const char* caote_last_cuda_error(void);
+CAOTE_API const char* caote_last_cuda_error(void);
+
+/* Per-kernel timing, for benchmarks and profiling. While tracing is on (process-wide switch), every
+ * kernel launch of this library is bracketed by two CUDA events recorded on the launching stream.
+ * caote_trace_collect waits for the outstanding events, adds up launches and elapsed milliseconds per
+ * kernel name into out[0..*n_out) (host memory, at most max_entries names) and forgets them.
+ * Do not enable tracing while a stream is being captured into a CUDA graph. */
+typedef struct {
+  char name[48];
+  int64_t launches;
+  double total_ms;
+} caote_trace_entry_t;
+CAOTE_API int caote_trace_enable(int on);
+CAOTE_API int caote_trace_collect(caote_trace_entry_t* out, int32_t max_entries, int32_t* n_out);
 
 /* Number of kernels this library has launched from this process since it was loaded. */
-int64_t caote_launch_count(void);
+CAOTE_API int64_t caote_launch_count(void);
 
 #ifdef __cplusplus
 }

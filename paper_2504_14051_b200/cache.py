@@ -1,0 +1,65 @@
+"""A budgeted KV cache driven through the C ABI: the call a user of the library makes per step.
+
+Holds the caller-owned device buffers (K, V, base, pos, len, scores, ...) and forwards each step to
+``caote_step`` (append the new tokens, score, select, compact). No arithmetic happens here.
+"""
+from __future__ import annotations
+
+from typing import Optional
+
+import torch
+
+from . import binding as C
+
+
+class EvictionCache:
+    def __init__(self, batch, n_q_heads, n_kv_heads, head_dim, capacity, n_new, dtype, budget,
+                 base_mode="last_query", compact_mode="fill", scale: Optional[float] = None,
+                 max_evict: Optional[int] = None, device="cuda"):
+        self.device = torch.device(device)
+        scale = head_dim ** -0.5 if scale is None else scale
+        self.params = C.make_params(batch, n_q_heads, n_kv_heads, head_dim, capacity, n_new, dtype, scale,
+                                    base_mode)
+        self.dtype = dtype
+        self.compact_mode = C.COMPACT_MODES[compact_mode] if isinstance(compact_mode, str) else compact_mode
+        B, Hkv, Hq, d, cap, m = batch, n_kv_heads, n_q_heads, head_dim, capacity, n_new
+        dev = self.device
+        self.K = torch.zeros((B, Hkv, cap, d), dtype=dtype, device=dev)
+        self.V = torch.zeros((B, Hkv, cap, d), dtype=dtype, device=dev)
+        self.base = torch.zeros((B, Hkv, cap), dtype=torch.float32, device=dev)
+        self.pos = torch.zeros((B, Hkv, cap), dtype=torch.int32, device=dev)
+        self.scores = torch.zeros((B, Hkv, cap), dtype=torch.float32, device=dev)
+        self.lens = torch.zeros((B,), dtype=torch.int32, device=dev)
+        self.n_seen = torch.zeros((B,), dtype=torch.int32, device=dev)
+        if isinstance(budget, int):
+            budget = torch.full((B,), budget, dtype=torch.int32)
+        self.budget = budget.to(device=dev, dtype=torch.int32).contiguous()
+        self.max_evict = max_evict if max_evict is not None else max(n_new, 1)
+        self.evict_idx = torch.zeros((B, Hkv, self.max_evict), dtype=torch.int32, device=dev)
+        self.n_evict = torch.zeros((B,), dtype=torch.int32, device=dev)
+        self.o = torch.zeros((B, Hq, m, d), dtype=torch.float32, device=dev)
+        self.workspace = C.alloc_workspace(self.params, dev)
+
+    def load(self, K, V, lens, base=None, pos=None):
+        """Install an existing cache state (copied into the owned buffers)."""
+        self.K.copy_(K)
+        self.V.copy_(V)
+        self.lens.copy_(lens)
+        self.n_seen.copy_(lens)
+        if base is not None:
+            self.base.copy_(base)
+        if pos is not None:
+            self.pos.copy_(pos)
+        else:
+            cap = self.K.shape[2]
+            self.pos.copy_(torch.arange(cap, dtype=torch.int32, device=self.device).expand_as(self.pos))
+
+    def step(self, q, k_new, v_new, stream=None):
+        """One eviction step; returns the pre-eviction attention output o [B, Hq, m, d]."""
+        C.caote_step(self.params, q, k_new, v_new, self.K, self.V, self.base, self.pos, self.lens, self.n_seen,
+                     self.budget, self.o, self.scores, self.evict_idx, self.n_evict, self.compact_mode,
+                     self.workspace, stream)
+        return self.o
+
+    def status(self) -> int:
+        return C.caote_read_status(self.workspace)

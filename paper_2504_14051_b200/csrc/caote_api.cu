@@ -1,0 +1,358 @@
+// C ABI of the CAOTE library: argument validation, workspace carving and kernel dispatch.
+// Every entry point only enqueues work on the caller's stream.
+#include <atomic>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+#include <vector>
+
+#include "common.cuh"
+#include "generic_score.cuh"
+#include "select_compact.cuh"
+
+namespace caote {
+
+static std::atomic<long long> g_launches{0};
+static thread_local char g_cuda_error[256] = "";
+
+static int cuda_fail(cudaError_t e, const char* what) {
+  snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: %s", what, cudaGetErrorString(e));
+  return CAOTE_ERR_CUDA;
+}
+#define CAOTE_CUDA(call)                                  \
+  do {                                                    \
+    cudaError_t e__ = (call);                             \
+    if (e__ != cudaSuccess) return cuda_fail(e__, #call); \
+  } while (0)
+
+static int after_launch(const char* name) {
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e, name);
+  return CAOTE_OK;
+}
+
+// ---- optional per-kernel tracing: CUDA events recorded on the launching stream around each kernel ----
+struct TraceRec {
+  const char* name;
+  cudaEvent_t a, b;
+};
+static std::atomic<bool> g_trace_on{false};
+static std::mutex g_trace_mu;
+static std::vector<TraceRec> g_trace_pending;
+static std::vector<cudaEvent_t> g_trace_pool;
+
+static cudaEvent_t trace_event() {
+  std::lock_guard<std::mutex> lk(g_trace_mu);
+  if (!g_trace_pool.empty()) {
+    cudaEvent_t e = g_trace_pool.back();
+    g_trace_pool.pop_back();
+    return e;
+  }
+  cudaEvent_t e = nullptr;
+  if (cudaEventCreate(&e) != cudaSuccess) return nullptr;
+  return e;
+}
+
+struct TraceScope {
+  const char* name;
+  cudaStream_t st;
+  cudaEvent_t a = nullptr, b = nullptr;
+  TraceScope(const char* n, cudaStream_t s) : name(n), st(s) {
+    if (!g_trace_on.load(std::memory_order_relaxed)) return;
+    a = trace_event();
+    b = trace_event();
+    if (a && b) cudaEventRecord(a, st);
+  }
+  ~TraceScope() {
+    if (!a || !b) return;
+    cudaEventRecord(b, st);
+    std::lock_guard<std::mutex> lk(g_trace_mu);
+    g_trace_pending.push_back({name, a, b});
+  }
+};
+
+// Launch a kernel (the statement after the stream argument), count it, trace it when tracing is on,
+// and return from the calling function if the launch failed.
+#define CAOTE_LAUNCH(name, st, ...)        \
+  do {                                     \
+    int rc__;                              \
+    {                                      \
+      TraceScope ts__(name, st);           \
+      __VA_ARGS__;                         \
+      rc__ = after_launch(name);           \
+    }                                      \
+    if (rc__ != CAOTE_OK) return rc__;     \
+  } while (0)
+
+static bool params_ok(const caote_params_t* p) {
+  if (!p) return false;
+  if (p->batch < 1 || p->n_kv_heads < 1 || p->n_q_heads < 1 || p->capacity < 1 || p->n_new < 1) return false;
+  if (p->n_q_heads % p->n_kv_heads != 0) return false;
+  if (p->n_q_heads / p->n_kv_heads > 16) return false;
+  if (p->n_new > p->capacity) return false;
+  if (p->flags != 0) return false;
+  if (p->base_mode < CAOTE_BASE_LAST_QUERY || p->base_mode > CAOTE_BASE_EXTERNAL) return false;
+  if (!(p->scale == p->scale)) return false;
+  return true;
+}
+static bool params_supported(const caote_params_t* p) {
+  if (p->dtype != CAOTE_BF16 && p->dtype != CAOTE_F32) return false;
+  if (p->head_dim != 64 && p->head_dim != 128) return false;
+  return true;
+}
+
+static Dims make_dims(const caote_params_t* p) {
+  Dims d;
+  d.B = p->batch;
+  d.Hq = p->n_q_heads;
+  d.Hkv = p->n_kv_heads;
+  d.G = d.Hq / d.Hkv;
+  d.D = p->head_dim;
+  d.cap = p->capacity;
+  d.m = p->n_new;
+  d.R = d.G * d.m;
+  d.units = d.B * d.Hkv;
+  d.scale = p->scale;
+  d.base_mode = p->base_mode;
+  return d;
+}
+
+// The device must be a compute-capability 10.x part; checked once per device.
+static int check_device() {
+  static std::atomic<int> ok[64];
+  int dev = 0;
+  CAOTE_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return CAOTE_ERR_UNSUPPORTED;
+  int st = ok[dev].load(std::memory_order_acquire);
+  if (st == 0) {
+    int major = 0;
+    CAOTE_CUDA(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+    st = (major == 10) ? 1 : -1;
+    ok[dev].store(st, std::memory_order_release);
+  }
+  return st == 1 ? CAOTE_OK : CAOTE_ERR_UNSUPPORTED;
+}
+
+template <typename KernelT>
+static int allow_smem(KernelT kernel, size_t bytes) {
+  if (bytes > 48 * 1024)
+    CAOTE_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
+  return CAOTE_OK;
+}
+
+template <typename T, int D>
+static int launch_generic_score(const Dims& dm, const void* q, const void* K, const void* V, const int* len,
+                                float* base, float* o, float* scores, char* ws, cudaStream_t st) {
+  generic::Scratch sc;
+  generic::carve(dm, ws + kHeaderBytes, &sc);
+  int* status = reinterpret_cast<int*>(ws);
+  const int row_tiles = (dm.R + generic::kRT - 1) / generic::kRT;
+  {
+    const size_t smem = generic::partial_smem(D);
+    int rc = allow_smem(generic::attn_partial_kernel<T, D>, smem);
+    if (rc) return rc;
+    dim3 grid(row_tiles, sc.splits, dm.units);
+    CAOTE_LAUNCH("attn_partial_kernel", st, generic::attn_partial_kernel<T, D><<<grid, generic::kThreads, smem, st>>>(
+        dm, (const T*)q, (const T*)K, (const T*)V, len, base, sc, status));
+  }
+  {
+    dim3 grid(sc.chunks, dm.units);
+    CAOTE_LAUNCH("attn_combine_kernel", st, generic::attn_combine_kernel<T, D><<<grid, D, 0, st>>>(dm, len, sc, o));
+  }
+  {
+    const size_t smem = generic::score_smem(D);
+    int rc = allow_smem(generic::score_pass_kernel<T, D>, smem);
+    if (rc) return rc;
+    dim3 grid((dm.cap + generic::kKT - 1) / generic::kKT, dm.units);
+    CAOTE_LAUNCH("score_pass_kernel", st, generic::score_pass_kernel<T, D><<<grid, generic::kThreads, smem, st>>>(
+        dm, (const T*)q, (const T*)K, (const T*)V, len, base, sc, scores));
+  }
+  return CAOTE_OK;
+}
+
+static size_t workspace_bytes(const caote_params_t* p) {
+  const Dims dm = make_dims(p);
+  size_t need = generic::carve(dm, nullptr, nullptr);
+  return kHeaderBytes + need;
+}
+
+static inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+}  // namespace caote
+
+using namespace caote;
+
+extern "C" {
+
+size_t caote_workspace_bytes(const caote_params_t* params) {
+  if (!params_ok(params) || !params_supported(params)) return 0;
+  return workspace_bytes(params);
+}
+
+int caote_append(const caote_params_t* p, void* K, void* V, float* base, int32_t* pos, int32_t* len,
+                 int32_t* n_seen, const void* k_new, const void* v_new, void* workspace,
+                 size_t workspace_bytes_, caote_stream_t stream) {
+  if (!params_ok(p) || !K || !V || !len || !k_new || !v_new || !workspace) return CAOTE_ERR_INVALID_ARG;
+  if (!params_supported(p)) return CAOTE_ERR_UNSUPPORTED;
+  if (workspace_bytes_ < kHeaderBytes || !aligned(workspace, 256)) return CAOTE_ERR_INVALID_ARG;
+  if (!aligned(K, 16) || !aligned(V, 16) || !aligned(k_new, 16) || !aligned(v_new, 16)) return CAOTE_ERR_INVALID_ARG;
+  int rc = check_device();
+  if (rc) return rc;
+  const Dims dm = make_dims(p);
+  const int row_bytes = dm.D * (p->dtype == CAOTE_BF16 ? 2 : 4);
+  cudaStream_t st = (cudaStream_t)stream;
+  CAOTE_LAUNCH("append_kernel", st, sel::append_kernel<<<dm.units, 256, 0, st>>>(dm.Hkv, dm.cap, dm.m, row_bytes, (char*)K, (char*)V, base, pos,
+                                               len, n_seen, (const char*)k_new, (const char*)v_new,
+                                               (int*)workspace));
+  CAOTE_LAUNCH("bump_len_kernel", st, sel::bump_len_kernel<<<(dm.B + 127) / 128, 128, 0, st>>>(dm.B, dm.cap, dm.m, len, n_seen));
+  return CAOTE_OK;
+}
+
+int caote_score(const caote_params_t* p, const void* q, const void* K, const void* V, const int32_t* len,
+                float* base, float* o, float* scores, void* workspace, size_t workspace_bytes_,
+                caote_stream_t stream) {
+  if (!params_ok(p) || !q || !K || !V || !len || !o || !scores || !workspace) return CAOTE_ERR_INVALID_ARG;
+  if (!params_supported(p)) return CAOTE_ERR_UNSUPPORTED;
+  if ((p->base_mode == CAOTE_BASE_ACCUM || p->base_mode == CAOTE_BASE_EXTERNAL) && !base)
+    return CAOTE_ERR_INVALID_ARG;
+  if (workspace_bytes_ < workspace_bytes(p) || !aligned(workspace, 256)) return CAOTE_ERR_INVALID_ARG;
+  if (!aligned(q, 16) || !aligned(K, 16) || !aligned(V, 16) || !aligned(o, 16)) return CAOTE_ERR_INVALID_ARG;
+  int rc = check_device();
+  if (rc) return rc;
+  const Dims dm = make_dims(p);
+  cudaStream_t st = (cudaStream_t)stream;
+  char* ws = (char*)workspace;
+  if (p->dtype == CAOTE_BF16) {
+    if (dm.D == 128) return launch_generic_score<__nv_bfloat16, 128>(dm, q, K, V, len, base, o, scores, ws, st);
+    return launch_generic_score<__nv_bfloat16, 64>(dm, q, K, V, len, base, o, scores, ws, st);
+  }
+  if (dm.D == 128) return launch_generic_score<float, 128>(dm, q, K, V, len, base, o, scores, ws, st);
+  return launch_generic_score<float, 64>(dm, q, K, V, len, base, o, scores, ws, st);
+}
+
+int caote_select_evict(const caote_params_t* p, const float* scores, const int32_t* len, const int32_t* budget,
+                       const int32_t* pos, int32_t* evict_idx, int32_t max_evict, int32_t* n_evict,
+                       void* workspace, size_t workspace_bytes_, caote_stream_t stream) {
+  if (!params_ok(p) || !scores || !len || !budget || !evict_idx || !n_evict || !workspace || max_evict < 1)
+    return CAOTE_ERR_INVALID_ARG;
+  if (workspace_bytes_ < kHeaderBytes || !aligned(workspace, 256)) return CAOTE_ERR_INVALID_ARG;
+  int rc = check_device();
+  if (rc) return rc;
+  const Dims dm = make_dims(p);
+  cudaStream_t st = (cudaStream_t)stream;
+  CAOTE_LAUNCH("select_kernel", st, sel::select_kernel<<<dm.units, sel::kSelThreads, 0, st>>>(
+      dm.Hkv, dm.cap, scores, len, budget, pos, evict_idx, max_evict, n_evict, (int*)workspace));
+  return CAOTE_OK;
+}
+
+int caote_compact(const caote_params_t* p, void* K, void* V, float* base, int32_t* pos, int32_t* len,
+                  const int32_t* evict_idx, int32_t max_evict, const int32_t* n_evict, int32_t mode,
+                  void* workspace, size_t workspace_bytes_, caote_stream_t stream) {
+  if (!params_ok(p) || !K || !V || !len || !evict_idx || !n_evict || !workspace || max_evict < 1)
+    return CAOTE_ERR_INVALID_ARG;
+  if (!params_supported(p)) return CAOTE_ERR_UNSUPPORTED;
+  if (mode != CAOTE_COMPACT_FILL && mode != CAOTE_COMPACT_STABLE) return CAOTE_ERR_INVALID_ARG;
+  if (workspace_bytes_ < kHeaderBytes || !aligned(workspace, 256)) return CAOTE_ERR_INVALID_ARG;
+  if (!aligned(K, 16) || !aligned(V, 16)) return CAOTE_ERR_INVALID_ARG;
+  int rc = check_device();
+  if (rc) return rc;
+  const Dims dm = make_dims(p);
+  const int row_bytes = dm.D * (p->dtype == CAOTE_BF16 ? 2 : 4);
+  cudaStream_t st = (cudaStream_t)stream;
+  if (mode == CAOTE_COMPACT_FILL) {
+    CAOTE_LAUNCH("compact_fill_kernel", st, sel::compact_fill_kernel<<<dm.units, 256, 0, st>>>(dm.Hkv, dm.cap, row_bytes, (char*)K, (char*)V, base, pos,
+                                                       len, evict_idx, max_evict, n_evict));
+  } else {
+    dim3 grid(dm.units, 3);
+    CAOTE_LAUNCH("compact_stable_kernel", st, sel::compact_stable_kernel<<<grid, 256, (size_t)sel::kStableTile * row_bytes, st>>>(
+        dm.Hkv, dm.cap, row_bytes, (char*)K, (char*)V, base, pos, len, evict_idx, max_evict, n_evict));
+  }
+  CAOTE_LAUNCH("update_len_kernel", st, sel::update_len_kernel<<<(dm.B + 127) / 128, 128, 0, st>>>(dm.B, len, n_evict));
+  return CAOTE_OK;
+}
+
+int caote_step(const caote_params_t* p, const void* q, const void* k_new, const void* v_new, void* K, void* V,
+               float* base, int32_t* pos, int32_t* len, int32_t* n_seen, const int32_t* budget, float* o,
+               float* scores, int32_t* evict_idx, int32_t max_evict, int32_t* n_evict, int32_t compact_mode,
+               void* workspace, size_t workspace_bytes_, caote_stream_t stream) {
+  int rc;
+  if (k_new || v_new) {
+    rc = caote_append(p, K, V, base, pos, len, n_seen, k_new, v_new, workspace, workspace_bytes_, stream);
+    if (rc) return rc;
+  }
+  rc = caote_score(p, q, K, V, len, base, o, scores, workspace, workspace_bytes_, stream);
+  if (rc) return rc;
+  rc = caote_select_evict(p, scores, len, budget, pos, evict_idx, max_evict, n_evict, workspace,
+                          workspace_bytes_, stream);
+  if (rc) return rc;
+  return caote_compact(p, K, V, base, pos, len, evict_idx, max_evict, n_evict, compact_mode, workspace,
+                       workspace_bytes_, stream);
+}
+
+int caote_read_status(void* workspace, caote_stream_t stream, int32_t* status_out) {
+  if (!workspace || !status_out) return CAOTE_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  CAOTE_CUDA(cudaMemcpyAsync(status_out, workspace, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+  CAOTE_CUDA(cudaMemsetAsync(workspace, 0, sizeof(int32_t), st));
+  CAOTE_CUDA(cudaStreamSynchronize(st));
+  return CAOTE_OK;
+}
+
+const char* caote_status_string(int status) {
+  switch (status) {
+    case CAOTE_OK: return "ok";
+    case CAOTE_ERR_INVALID_ARG: return "invalid argument";
+    case CAOTE_ERR_UNSUPPORTED: return "unsupported dtype, head_dim, mode or device";
+    case CAOTE_ERR_CUDA: return "CUDA call failed";
+    case CAOTE_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+    case CAOTE_ERR_BAD_LENGTH: return "a cache length is outside [n_new, capacity]";
+    case CAOTE_ERR_OVERFLOW: return "more evictions than max_evict, or an append past capacity";
+    default: return "unknown status";
+  }
+}
+
+const char* caote_last_cuda_error(void) { return g_cuda_error; }
+
+int caote_trace_enable(int on) {
+  g_trace_on.store(on != 0, std::memory_order_relaxed);
+  return CAOTE_OK;
+}
+
+int caote_trace_collect(caote_trace_entry_t* out, int32_t max_entries, int32_t* n_out) {
+  if (!out || !n_out || max_entries < 1) return CAOTE_ERR_INVALID_ARG;
+  std::vector<TraceRec> recs;
+  {
+    std::lock_guard<std::mutex> lk(g_trace_mu);
+    recs.swap(g_trace_pending);
+  }
+  int n = 0;
+  int rc = CAOTE_OK;
+  for (const TraceRec& r : recs) {
+    float ms = 0.f;
+    cudaError_t e = cudaEventSynchronize(r.b);
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, r.a, r.b);
+    if (e != cudaSuccess) rc = cuda_fail(e, "caote_trace_collect");
+    int i = 0;
+    for (; i < n; ++i)
+      if (strncmp(out[i].name, r.name, sizeof(out[i].name) - 1) == 0) break;
+    if (i == n && n < max_entries) {
+      memset(&out[n], 0, sizeof(out[n]));
+      strncpy(out[n].name, r.name, sizeof(out[n].name) - 1);
+      ++n;
+    }
+    if (i < n && e == cudaSuccess) {
+      out[i].launches += 1;
+      out[i].total_ms += (double)ms;
+    }
+    std::lock_guard<std::mutex> lk(g_trace_mu);
+    g_trace_pool.push_back(r.a);
+    g_trace_pool.push_back(r.b);
+  }
+  *n_out = n;
+  return rc;
+}
+
+int64_t caote_launch_count(void) { return (int64_t)g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

@@ -1,0 +1,272 @@
+// Selection of the tokens to evict (block radix-select on the bit patterns of the non-negative fp32
+// scores, ties broken by original position), in-place compaction of the cache, and the append of new
+// tokens. These are bandwidth-trivial next to the scoring pass: n * 4 bytes per unit for selection,
+// at most k rows per unit for FILL compaction.
+#pragma once
+
+#include "common.cuh"
+
+namespace caote {
+namespace sel {
+
+constexpr int kSelThreads = 1024;
+
+// 64-bit sort key: score bits in the high word (scores are >= +0, so the unsigned order of the bit
+// patterns is the numeric order; +inf sorts last), original position in the low word.
+__device__ __forceinline__ unsigned long long make_key(float score, int pos) {
+  return ((unsigned long long)__float_as_uint(score) << 32) | (unsigned int)pos;
+}
+
+// One CTA per unit. k = max(0, n - budget). Finds the k-th smallest key by 8 passes of an 8-bit
+// radix histogram (most significant digit first), then writes the slots whose key is <= that key in
+// ascending slot order with a block-wide ordered compaction.
+__global__ void __launch_bounds__(kSelThreads)
+select_kernel(int Hkv, int cap, const float* __restrict__ scores, const int* __restrict__ len,
+              const int* __restrict__ budget, const int* __restrict__ pos, int* __restrict__ evict_idx,
+              int max_evict, int* __restrict__ n_evict, int* status) {
+  __shared__ unsigned int hist[256];
+  __shared__ unsigned long long s_prefix;
+  __shared__ int s_remaining;
+  __shared__ int s_warp_tot[kSelThreads / 32];
+  __shared__ int s_running;
+  __shared__ unsigned long long s_min[kSelThreads / 32];
+
+  const int unit = blockIdx.x, b = unit / Hkv, h = unit % Hkv;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int n = len[b];
+  int bud = budget[b];
+  if (bud < 1) bud = 1;
+  int k = n - bud;
+  if (k < 0) k = 0;
+  if (n > cap) k = 0;
+  if (k > max_evict) {
+    if (tid == 0) set_status(status, CAOTE_ERR_OVERFLOW);
+    k = 0;
+  }
+  if (h == 0 && tid == 0) n_evict[b] = k;
+  if (k == 0) return;
+  const float* sc = scores + (size_t)unit * cap;
+  const int* ps = pos ? pos + (size_t)unit * cap : nullptr;
+  int* out = evict_idx + (size_t)unit * max_evict;
+
+  if (k == 1) {  // argmin
+    unsigned long long best = ~0ull;
+    int best_slot = 0;
+    for (int j = tid; j < n; j += kSelThreads) {
+      const unsigned long long key = make_key(sc[j], ps ? ps[j] : j);
+      if (key < best) { best = key; best_slot = j; }
+    }
+    // reduce (key, slot): keys are unique when pos is, else the lower slot wins
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const unsigned long long ok = __shfl_xor_sync(0xffffffffu, best, o);
+      const int os = __shfl_xor_sync(0xffffffffu, best_slot, o);
+      if (ok < best || (ok == best && os < best_slot)) { best = ok; best_slot = os; }
+    }
+    if (lane == 0) { s_min[warp] = best; s_warp_tot[warp] = best_slot; }
+    __syncthreads();
+    if (warp == 0) {
+      best = s_min[lane];
+      best_slot = s_warp_tot[lane];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const unsigned long long ok = __shfl_xor_sync(0xffffffffu, best, o);
+        const int os = __shfl_xor_sync(0xffffffffu, best_slot, o);
+        if (ok < best || (ok == best && os < best_slot)) { best = ok; best_slot = os; }
+      }
+      if (lane == 0) out[0] = best_slot;
+    }
+    return;
+  }
+
+  if (tid == 0) { s_prefix = 0ull; s_remaining = k; }
+  for (int pass = 0; pass < 8; ++pass) {
+    const int shift = 56 - 8 * pass;
+    if (tid < 256) hist[tid] = 0u;
+    __syncthreads();
+    const unsigned long long prefix = s_prefix;
+    const unsigned long long mask = (pass == 0) ? 0ull : (~0ull << (shift + 8));
+    for (int j = tid; j < n; j += kSelThreads) {
+      const unsigned long long key = make_key(sc[j], ps ? ps[j] : j);
+      if ((key & mask) == prefix) atomicAdd(&hist[(unsigned int)(key >> shift) & 255u], 1u);
+    }
+    __syncthreads();
+    if (tid == 0) {
+      int rem = s_remaining;
+      int dgt = 0;
+      for (; dgt < 256; ++dgt) {
+        const int c = (int)hist[dgt];
+        if (rem <= c) break;
+        rem -= c;
+      }
+      if (dgt > 255) dgt = 255;
+      s_remaining = rem;
+      s_prefix = prefix | ((unsigned long long)dgt << shift);
+    }
+    __syncthreads();
+  }
+  const unsigned long long kth = s_prefix;  // the k-th smallest key
+  if (tid == 0) s_running = 0;
+  __syncthreads();
+  for (int j0 = 0; j0 < n; j0 += kSelThreads) {
+    const int j = j0 + tid;
+    const int flag = (j < n) && (make_key(sc[j], ps ? ps[j] : j) <= kth);
+    const unsigned int ballot = __ballot_sync(0xffffffffu, flag);
+    const int in_warp = __popc(ballot & ((1u << lane) - 1u));
+    if (lane == 0) s_warp_tot[warp] = __popc(ballot);
+    __syncthreads();
+    int before = s_running;
+    for (int w = 0; w < warp; ++w) before += s_warp_tot[w];
+    const int idx = before + in_warp;
+    if (flag && idx < k) out[idx] = j;
+    __syncthreads();
+    if (tid == 0) {
+      int tot = s_running;
+      for (int w = 0; w < kSelThreads / 32; ++w) tot += s_warp_tot[w];
+      s_running = tot;
+    }
+    __syncthreads();
+  }
+}
+
+// Copy one row of `bytes` bytes (a multiple of 16, 16-byte aligned on both sides) with one warp.
+__device__ __forceinline__ void warp_copy_row(char* dst, const char* src, int bytes, int lane) {
+  for (int o = lane * 16; o < bytes; o += 32 * 16)
+    *reinterpret_cast<uint4*>(dst + o) = *reinterpret_cast<const uint4*>(src + o);
+}
+
+// First index in sorted a[0..n) whose value is >= x.
+__device__ __forceinline__ int lower_bound(const int* a, int n, int x) {
+  int lo = 0, hi = n;
+  while (lo < hi) {
+    const int mid = (lo + hi) >> 1;
+    if (a[mid] < x) lo = mid + 1; else hi = mid;
+  }
+  return lo;
+}
+
+// FILL compaction, one CTA per unit. With n' = n - k, the evicted slots below n' are holes, and the
+// k slots [n', n) hold exactly as many survivors; the i-th surviving tail slot moves into the i-th
+// hole. Sources lie in [n', n) and destinations in [0, n'), so no move can clobber another's source.
+__global__ void __launch_bounds__(256)
+compact_fill_kernel(int Hkv, int cap, int row_bytes, char* __restrict__ K, char* __restrict__ V,
+                    float* __restrict__ base, int* __restrict__ pos, const int* __restrict__ len,
+                    const int* __restrict__ evict_idx, int max_evict, const int* __restrict__ n_evict) {
+  const int unit = blockIdx.x, b = unit / Hkv;
+  const int k = n_evict[b];
+  if (k <= 0) return;
+  const int n = len[b], n_new = n - k;
+  const int* E = evict_idx + (size_t)unit * max_evict;
+  const int nh = lower_bound(E, k, n_new);  // holes = E[0..nh)
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  for (int t = warp; t < k; t += nwarps) {
+    const int s = n_new + t;
+    const int lb = nh + lower_bound(E + nh, k - nh, s);
+    if (lb < k && E[lb] == s) continue;  // this tail slot is itself evicted
+    const int rank = t - (lb - nh);      // its rank among the surviving tail slots
+    const int dst = E[rank];
+    const size_t so = ((size_t)unit * cap + s), dof = ((size_t)unit * cap + dst);
+    warp_copy_row(K + dof * row_bytes, K + so * row_bytes, row_bytes, lane);
+    warp_copy_row(V + dof * row_bytes, V + so * row_bytes, row_bytes, lane);
+    if (lane == 0) {
+      if (base) base[dof] = base[so];
+      if (pos) pos[dof] = pos[so];
+    }
+  }
+}
+
+// STABLE compaction: survivors keep their order. grid = (units, 3): y = 0 moves K, 1 moves V,
+// 2 moves base and pos. Tiles of 64 slots are processed front to back; a tile is read completely
+// into shared memory before any of it is written, and every destination index is <= its source
+// index, so a write can only land on slots whose old contents were already read.
+constexpr int kStableTile = 64;
+__global__ void __launch_bounds__(256)
+compact_stable_kernel(int Hkv, int cap, int row_bytes, char* __restrict__ K, char* __restrict__ V,
+                      float* __restrict__ base, int* __restrict__ pos, const int* __restrict__ len,
+                      const int* __restrict__ evict_idx, int max_evict, const int* __restrict__ n_evict) {
+  extern __shared__ __align__(16) char tile[];  // kStableTile * max(row_bytes, 8)
+  const int unit = blockIdx.x, b = unit / Hkv, which = blockIdx.y;
+  const int k = n_evict[b];
+  if (k <= 0) return;
+  const int n = len[b];
+  const int* E = evict_idx + (size_t)unit * max_evict;
+  char* arr = (which == 0) ? K : V;
+  if (which == 2 && !base && !pos) return;
+  const int rb = (which == 2) ? 8 : row_bytes;
+  const int chunks_per_row = rb / ((which == 2) ? 8 : 16);
+  for (int s0 = E[0]; s0 < n; s0 += kStableTile) {
+    const int rows = min(kStableTile, n - s0);
+    for (int idx = threadIdx.x; idx < rows * chunks_per_row; idx += blockDim.x) {
+      const int r = idx / chunks_per_row, c = idx % chunks_per_row;
+      const size_t slot = (size_t)unit * cap + s0 + r;
+      if (which == 2) {
+        float bv = base ? base[slot] : 0.f;
+        int pv = pos ? pos[slot] : 0;
+        *reinterpret_cast<float*>(tile + r * 8) = bv;
+        *reinterpret_cast<int*>(tile + r * 8 + 4) = pv;
+      } else {
+        *reinterpret_cast<uint4*>(tile + (size_t)r * rb + c * 16) =
+            *reinterpret_cast<const uint4*>(arr + slot * rb + c * 16);
+      }
+    }
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < rows * chunks_per_row; idx += blockDim.x) {
+      const int r = idx / chunks_per_row, c = idx % chunks_per_row;
+      const int s = s0 + r;
+      const int lb = lower_bound(E, k, s);
+      if (lb < k && E[lb] == s) continue;  // evicted
+      const size_t dst = (size_t)unit * cap + (s - lb);
+      if (which == 2) {
+        if (base) base[dst] = *reinterpret_cast<float*>(tile + r * 8);
+        if (pos) pos[dst] = *reinterpret_cast<int*>(tile + r * 8 + 4);
+      } else {
+        *reinterpret_cast<uint4*>(arr + dst * rb + c * 16) =
+            *reinterpret_cast<const uint4*>(tile + (size_t)r * rb + c * 16);
+      }
+    }
+    __syncthreads();
+  }
+}
+
+// len[b] -= n_evict[b], after every unit of the sequence has been compacted.
+__global__ void update_len_kernel(int B, int* __restrict__ len, const int* __restrict__ n_evict) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b < B) len[b] -= n_evict[b];
+}
+
+// Append m new rows per unit: one CTA per unit, one warp per row.
+__global__ void __launch_bounds__(256)
+append_kernel(int Hkv, int cap, int m, int row_bytes, char* __restrict__ K, char* __restrict__ V,
+              float* __restrict__ base, int* __restrict__ pos, const int* __restrict__ len,
+              const int* __restrict__ n_seen, const char* __restrict__ k_new,
+              const char* __restrict__ v_new, int* status) {
+  const int unit = blockIdx.x, b = unit / Hkv;
+  const int n = len[b];
+  if (n < 0 || n + m > cap) {
+    if (threadIdx.x == 0) set_status(status, CAOTE_ERR_OVERFLOW);
+    return;
+  }
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  const int seen = n_seen ? n_seen[b] : n;
+  for (int i = warp; i < m; i += nwarps) {
+    const size_t dst = (size_t)unit * cap + n + i, src = (size_t)unit * m + i;
+    warp_copy_row(K + dst * row_bytes, k_new + src * row_bytes, row_bytes, lane);
+    warp_copy_row(V + dst * row_bytes, v_new + src * row_bytes, row_bytes, lane);
+    if (lane == 0) {
+      if (base) base[dst] = 0.f;
+      if (pos) pos[dst] = seen + i;
+    }
+  }
+}
+
+// len[b] += m and n_seen[b] += m for the sequences append_kernel did not skip.
+__global__ void bump_len_kernel(int B, int cap, int m, int* __restrict__ len, int* __restrict__ n_seen) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b < B && len[b] >= 0 && len[b] + m <= cap) {
+    len[b] += m;
+    if (n_seen) n_seen[b] += m;
+  }
+}
+
+}  // namespace sel
+}  // namespace caote
