@@ -7,6 +7,7 @@
 #include <vector>
 
 #include "common.cuh"
+#include "decode_score.cuh"
 #include "generic_score.cuh"
 #include "select_compact.cuh"
 
@@ -171,9 +172,102 @@ static int launch_generic_score(const Dims& dm, const void* q, const void* K, co
   return CAOTE_OK;
 }
 
+// ---- single-query fast path ---------------------------------------------------------------------
+typedef CUresult (*TensorMapEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                      const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                      CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static TensorMapEncodeFn tensor_map_encoder() {
+  static std::atomic<TensorMapEncodeFn> fn{nullptr};
+  TensorMapEncodeFn f = fn.load(std::memory_order_acquire);
+  if (!f) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qr) == cudaSuccess &&
+        qr == cudaDriverEntryPointSuccess)
+      f = reinterpret_cast<TensorMapEncodeFn>(ptr);
+    fn.store(f, std::memory_order_release);
+  }
+  return f;
+}
+
+// Resident CTAs of the persistent decode kernel on the current device (SMs x CTAs per SM); 0 on error.
+static int decode_grid_limit() {
+  static std::atomic<int> cached[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+  int g = cached[dev].load(std::memory_order_acquire);
+  if (g == 0) {
+    int sms = 0, per_sm = 0;
+    const size_t smem = decode::smem_bytes();
+    if (cudaFuncSetAttribute(decode::decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode::decode_kernel, decode::kThreads, smem) != cudaSuccess)
+      return 0;
+    g = sms * per_sm;
+    cached[dev].store(g > 0 ? g : -1, std::memory_order_release);
+  }
+  return g > 0 ? g : 0;
+}
+
+// Shapes the persistent decode kernel covers; everything else takes the generic path.
+static bool decode_shape_ok(const caote_params_t* p) {
+  const int G = p->n_q_heads / p->n_kv_heads;
+  const bool carried = p->base_mode == CAOTE_BASE_ACCUM || p->base_mode == CAOTE_BASE_EXTERNAL;
+  return p->dtype == CAOTE_BF16 && p->head_dim == 128 && p->n_new == 1 && G <= 8 && !(carried && G > 7) &&
+         (long long)p->batch * p->n_kv_heads * p->capacity < (1LL << 31);
+}
+
+static int launch_decode_score(const Dims& dm, const void* q, const void* K, const void* V, const int* len,
+                               float* base, float* o, float* scores, char* ws, cudaStream_t st, bool* used) {
+  *used = false;
+  const int grid_limit = decode_grid_limit();
+  TensorMapEncodeFn encode = tensor_map_encoder();
+  const int chunks_per_unit = (dm.cap + decode::kT - 1) / decode::kT;
+  // a unit's chunks must all fall within one round of the resident CTAs (see decode_score.cuh)
+  if (grid_limit <= 0 || !encode || chunks_per_unit > grid_limit) return CAOTE_OK;
+  decode::Plan pl;
+  decode::carve(dm, ws + kHeaderBytes, &pl);
+  int* status = reinterpret_cast<int*>(ws);
+  CUtensorMap tmK, tmV;
+  const cuuint64_t gdim[2] = {(cuuint64_t)dm.D, (cuuint64_t)dm.units * (cuuint64_t)dm.cap};
+  const cuuint64_t gstride[1] = {(cuuint64_t)dm.D * 2};
+  const cuuint32_t box[2] = {64, (cuuint32_t)decode::kT};
+  const cuuint32_t estride[2] = {1, 1};
+  for (int i = 0; i < 2; ++i) {
+    CUresult r = encode(i == 0 ? &tmK : &tmV, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(i == 0 ? K : V), gdim,
+                        gstride, box, estride, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+      snprintf(g_cuda_error, sizeof(g_cuda_error), "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+      return CAOTE_ERR_CUDA;
+    }
+  }
+  CAOTE_LAUNCH("decode_plan_kernel", st,
+               decode::plan_kernel<<<1, 1024, 0, st>>>(dm.units, dm.Hkv, dm.cap, len, pl, status));
+  const long long max_chunks = (long long)dm.units * chunks_per_unit;
+  const int grid = (int)(max_chunks < grid_limit ? max_chunks : grid_limit);
+  const __nv_bfloat16* qp = (const __nv_bfloat16*)q;
+  Dims dmv = dm;
+  void* args[] = {&tmK, &tmV, &dmv, &qp, &len, &base, &o, &scores, &pl, &status};
+  {
+    TraceScope ts("decode_kernel", st);
+    cudaError_t e = cudaLaunchCooperativeKernel((const void*)decode::decode_kernel, dim3(grid), dim3(decode::kThreads),
+                                                args, decode::smem_bytes(), st);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    if (e != cudaSuccess) return cuda_fail(e, "decode_kernel");
+  }
+  *used = true;
+  return CAOTE_OK;
+}
+
 static size_t workspace_bytes(const caote_params_t* p) {
   const Dims dm = make_dims(p);
   size_t need = generic::carve(dm, nullptr, nullptr);
+  if (decode_shape_ok(p)) {
+    const size_t need2 = decode::carve(dm, nullptr, nullptr);
+    if (need2 > need) need = need2;
+  }
   return kHeaderBytes + need;
 }
 
@@ -223,6 +317,11 @@ int caote_score(const caote_params_t* p, const void* q, const void* K, const voi
   const Dims dm = make_dims(p);
   cudaStream_t st = (cudaStream_t)stream;
   char* ws = (char*)workspace;
+  if (decode_shape_ok(p) && !(p->flags & 0)) {
+    bool used = false;
+    rc = launch_decode_score(dm, q, K, V, len, base, o, scores, ws, st, &used);
+    if (rc || used) return rc;
+  }
   if (p->dtype == CAOTE_BF16) {
     if (dm.D == 128) return launch_generic_score<__nv_bfloat16, 128>(dm, q, K, V, len, base, o, scores, ws, st);
     return launch_generic_score<__nv_bfloat16, 64>(dm, q, K, V, len, base, o, scores, ws, st);

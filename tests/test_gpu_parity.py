@@ -48,6 +48,12 @@ SHAPES = [
     (2, 8, 4, 64, 272, 128, [272, 130]),
     (1, 4, 1, 128, 520, 128, [515]),
     (1, 32, 2, 128, 96, 5, [5]),
+    # single-query shapes that span several chunks, several rounds of the persistent kernel, ragged tails
+    (4, 8, 8, 128, 2100, 1, [2049, 2100, 1, 127]),
+    (2, 28, 4, 128, 1000, 1, [999, 513]),
+    (40, 8, 8, 128, 704, 1, [704 - 13 * (i % 7) for i in range(40)]),
+    (1, 8, 1, 128, 16400, 1, [16385]),
+    (2, 6, 2, 128, 384, 1, [384, 256]),
 ]
 
 
