@@ -62,7 +62,8 @@ typedef enum {
   CAOTE_ERR_CUDA = -3,        /* a CUDA runtime or driver call failed (see caote_last_cuda_error) */
   CAOTE_ERR_TIMEOUT = -4,     /* a bounded device-side wait gave up (status word only)            */
   CAOTE_ERR_BAD_LENGTH = -5,  /* device saw len[b] > cap or 0 < len[b] < n_new (status word only) */
-  CAOTE_ERR_OVERFLOW = -6     /* device saw n_evict > max_evict or len + n_new > cap (status word) */
+  CAOTE_ERR_OVERFLOW = -6,    /* device saw n_evict > max_evict or len + n_new > cap (status word) */
+  CAOTE_ERR_TOO_LARGE = -7    /* caote_score_static: the shape needs more than CAOTE_STATIC_SCRATCH_BYTES */
 } caote_status_t;
 
 typedef enum { CAOTE_BF16 = 0, CAOTE_F32 = 1 } caote_dtype_t;
@@ -136,6 +137,35 @@ CAOTE_API int caote_append(const caote_params_t* params, void* K, void* V, float
 CAOTE_API int caote_score(const caote_params_t* params, const void* q, const void* K, const void* V,
                 const int32_t* len, float* base, float* o, float* scores, void* workspace,
                 size_t workspace_bytes, caote_stream_t stream);
+
+/* caote_score for callers that cannot allocate device memory. (The paper has no counterpart: this is
+ * a packaging variant of caote_score, same arithmetic, same kernels.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - inside a serving engine whose memory
+ * pool has already claimed the whole GPU, in a plug-in that is handed tensors but no allocator, or on
+ * a latency path where an allocation (which may synchronise the device) is not acceptable - and that
+ * therefore has nowhere to get the workspace caote_score asks for.
+ *
+ * Here the scratch is an array of CAOTE_STATIC_SCRATCH_BYTES bytes built into the library's device
+ * image; every GPU that loads the library holds it from load until the process exits. The caller
+ * passes only inputs and outputs, with the meaning, layout and alignment they have in caote_score.
+ *   status_out  device pointer to one int32, or NULL. Receives the status word of this call (CAOTE_OK
+ *               or the first device-side error); stream-ordered like the other outputs.
+ * Limits and rules:
+ *   - A shape with caote_workspace_bytes(params) > CAOTE_STATIC_SCRATCH_BYTES is rejected with
+ *     CAOTE_ERR_TOO_LARGE before anything is enqueued.
+ *   - The call itself allocates and frees nothing: no cudaMalloc / cudaFree, no allocating library
+ *     routine. It enqueues a 256-byte memset of the scratch header, the kernels of caote_score and a
+ *     4-byte device-to-device copy.
+ *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
+ *     that device current). Make that first call outside any stream capture.
+ *   - All calls on one device share the one array, and it keeps the previous call's contents (the call
+ *     clears what has to start at zero). Two calls that may overlap on the GPU - different streams
+ *     without an ordering between them - race on it and give undefined results; serialise them. */
+#define CAOTE_STATIC_SCRATCH_BYTES (16u << 20)
+CAOTE_API int caote_score_static(const caote_params_t* params, const void* q, const void* K, const void* V,
+                       const int32_t* len, float* base, float* o, float* scores, int32_t* status_out,
+                       caote_stream_t stream);
 
 /* Choose the tokens to evict: for sequence b, k = max(0, len[b] - budget[b]) (Sec. 2: the top-b tokens
  * by score are retained; Sec. 4.1 "Prompt consumption": evict once the cache exceeds the budget), and

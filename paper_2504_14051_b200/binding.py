@@ -19,6 +19,8 @@ BASE_MODES = {"last_query": 0, "chunk_sum": 1, "accum": 2, "external": 3}
 COMPACT_MODES = {"fill": 0, "stable": 1}
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT, ERR_BAD_LENGTH, ERR_OVERFLOW = 0, -1, -2, -3, -4, -5, -6
+ERR_TOO_LARGE = -7
+STATIC_SCRATCH_BYTES = 16 << 20
 
 
 class Params(ctypes.Structure):
@@ -76,6 +78,8 @@ def lib() -> ctypes.CDLL:
     L.caote_append.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     L.caote_score.restype = ctypes.c_int
     L.caote_score.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    L.caote_score_static.restype = ctypes.c_int
+    L.caote_score_static.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     L.caote_select_evict.restype = ctypes.c_int
     L.caote_select_evict.argtypes = [pp, vp, vp, vp, vp, vp, i32, vp, vp, sz, vp]
     L.caote_compact.restype = ctypes.c_int
@@ -142,6 +146,14 @@ def caote_append(p, K, V, base, pos, lens, n_seen, k_new, v_new, workspace, stre
 def caote_score(p, q, K, V, lens, base, o, scores, workspace, stream=None):
     _check("caote_score", lib().caote_score(ctypes.byref(p), _p(q), _p(K), _p(V), _p(lens), _p(base), _p(o),
                                             _p(scores), _p(workspace), workspace.numel(), _stream(stream)))
+
+
+def caote_score_static(p, q, K, V, lens, base, o, scores, status_out=None, stream=None):
+    """caote_score on the library's built-in scratch array: for callers that may not allocate device
+    memory (no workspace argument). ``status_out``: optional int32 device tensor of one element."""
+    _check("caote_score_static",
+           lib().caote_score_static(ctypes.byref(p), _p(q), _p(K), _p(V), _p(lens), _p(base), _p(o), _p(scores),
+                                    _p(status_out), _stream(stream)))
 
 
 def caote_select_evict(p, scores, lens, budget, pos, evict_idx, n_evict, workspace, stream=None):

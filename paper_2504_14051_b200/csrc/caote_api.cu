@@ -273,6 +273,30 @@ static size_t workspace_bytes(const caote_params_t* p) {
 
 static inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
+// ---- built-in scratch of caote_score_static ------------------------------------------------------
+// Lives in the library's device image: every GPU that loads the library holds these bytes until the
+// process exits. The name below is only a host-side handle; the device address is looked up once per
+// device with cudaGetSymbolAddress.
+constexpr size_t kStaticScratchBytes = CAOTE_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+static int static_scratch_address(char** out) {
+  static std::mutex mu;
+  static char* addr[64] = {};
+  int dev = 0;
+  CAOTE_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return CAOTE_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lk(mu);
+  if (!addr[dev]) {
+    void* p = nullptr;
+    CAOTE_CUDA(cudaGetSymbolAddress(&p, g_static_scratch));
+    if (!p) return CAOTE_ERR_CUDA;
+    addr[dev] = static_cast<char*>(p);
+  }
+  *out = addr[dev];
+  return CAOTE_OK;
+}
+
 }  // namespace caote
 
 using namespace caote;
@@ -328,6 +352,25 @@ int caote_score(const caote_params_t* p, const void* q, const void* K, const voi
   }
   if (dm.D == 128) return launch_generic_score<float, 128>(dm, q, K, V, len, base, o, scores, ws, st);
   return launch_generic_score<float, 64>(dm, q, K, V, len, base, o, scores, ws, st);
+}
+
+int caote_score_static(const caote_params_t* p, const void* q, const void* K, const void* V, const int32_t* len,
+                       float* base, float* o, float* scores, int32_t* status_out, caote_stream_t stream) {
+  if (!params_ok(p)) return CAOTE_ERR_INVALID_ARG;
+  if (!params_supported(p)) return CAOTE_ERR_UNSUPPORTED;
+  if (workspace_bytes(p) > kStaticScratchBytes) return CAOTE_ERR_TOO_LARGE;
+  int rc = check_device();
+  if (rc) return rc;
+  char* scratch = nullptr;
+  rc = static_scratch_address(&scratch);  // first call on this device: looks the address up
+  if (rc) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  // the array keeps whatever the previous call left: the status word has to start at zero
+  CAOTE_CUDA(cudaMemsetAsync(scratch, 0, kHeaderBytes, st));
+  rc = caote_score(p, q, K, V, len, base, o, scores, scratch, kStaticScratchBytes, stream);
+  if (rc) return rc;
+  if (status_out) CAOTE_CUDA(cudaMemcpyAsync(status_out, scratch, sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
+  return CAOTE_OK;
 }
 
 int caote_select_evict(const caote_params_t* p, const float* scores, const int32_t* len, const int32_t* budget,
@@ -407,6 +450,7 @@ const char* caote_status_string(int status) {
     case CAOTE_ERR_TIMEOUT: return "a bounded device-side wait gave up";
     case CAOTE_ERR_BAD_LENGTH: return "a cache length is outside [n_new, capacity]";
     case CAOTE_ERR_OVERFLOW: return "more evictions than max_evict, or an append past capacity";
+    case CAOTE_ERR_TOO_LARGE: return "the problem needs more scratch than the built-in array of caote_score_static holds";
     default: return "unknown status";
   }
 }

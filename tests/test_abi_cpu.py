@@ -41,7 +41,7 @@ def test_params_struct_matches_header():
 
 
 def test_status_strings_and_workspace_size():
-    for code in range(0, -7, -1):
+    for code in range(0, -8, -1):
         assert C.caote_status_string(code) != "unknown status"
     assert C.caote_status_string(-99) == "unknown status"
     p = C.make_params(2, 8, 2, 128, 1024, 1, torch.bfloat16, 0.1, "accum")
