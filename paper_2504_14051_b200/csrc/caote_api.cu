@@ -7,7 +7,7 @@
 #include <vector>
 
 #include "common.cuh"
-#include "decode_score.cuh"
+#include "decode_stream.cuh"
 #include "generic_score.cuh"
 #include "select_compact.cuh"
 
@@ -210,11 +210,15 @@ static int decode_grid_limit() {
   return g > 0 ? g : 0;
 }
 
+static inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
 // Shapes the persistent decode kernel covers; everything else takes the generic path.
 static bool decode_shape_ok(const caote_params_t* p) {
   const int G = p->n_q_heads / p->n_kv_heads;
   const bool carried = p->base_mode == CAOTE_BASE_ACCUM || p->base_mode == CAOTE_BASE_EXTERNAL;
-  return p->dtype == CAOTE_BF16 && p->head_dim == 128 && p->n_new == 1 && G <= 8 && !(carried && G > 7) &&
+  // a carried base score rides in row 7 of the P operand (G <= 7) and is staged by 16-byte bulk copies
+  return p->dtype == CAOTE_BF16 && p->head_dim == 128 && p->n_new == 1 && G <= 8 &&
+         !(carried && (G > 7 || p->capacity % 4 != 0)) &&
          (long long)p->batch * p->n_kv_heads * p->capacity < (1LL << 31);
 }
 
@@ -223,11 +227,10 @@ static int launch_decode_score(const Dims& dm, const void* q, const void* K, con
   *used = false;
   const int grid_limit = decode_grid_limit();
   TensorMapEncodeFn encode = tensor_map_encoder();
-  const int chunks_per_unit = (dm.cap + decode::kT - 1) / decode::kT;
-  // a unit's chunks must all fall within one round of the resident CTAs (see decode_score.cuh)
-  if (grid_limit <= 0 || !encode || chunks_per_unit > grid_limit) return CAOTE_OK;
+  const bool carried = dm.base_mode == CAOTE_BASE_ACCUM || dm.base_mode == CAOTE_BASE_EXTERNAL;
+  if (grid_limit <= 0 || !encode || (carried && !aligned(base, 16))) return CAOTE_OK;
   decode::Plan pl;
-  decode::carve(dm, ws + kHeaderBytes, &pl);
+  decode::carve(dm, ws + kHeaderBytes, &pl, grid_limit);
   int* status = reinterpret_cast<int*>(ws);
   CUtensorMap tmK, tmV;
   const cuuint64_t gdim[2] = {(cuuint64_t)dm.D, (cuuint64_t)dm.units * (cuuint64_t)dm.cap};
@@ -245,18 +248,12 @@ static int launch_decode_score(const Dims& dm, const void* q, const void* K, con
   }
   CAOTE_LAUNCH("decode_plan_kernel", st,
                decode::plan_kernel<<<1, 1024, 0, st>>>(dm.units, dm.Hkv, dm.cap, len, pl, status));
-  const long long max_chunks = (long long)dm.units * chunks_per_unit;
-  const int grid = (int)(max_chunks < grid_limit ? max_chunks : grid_limit);
-  const __nv_bfloat16* qp = (const __nv_bfloat16*)q;
-  Dims dmv = dm;
-  void* args[] = {&tmK, &tmV, &dmv, &qp, &len, &base, &o, &scores, &pl, &status};
-  {
-    TraceScope ts("decode_kernel", st);
-    cudaError_t e = cudaLaunchCooperativeKernel((const void*)decode::decode_kernel, dim3(grid), dim3(decode::kThreads),
-                                                args, decode::smem_bytes(), st);
-    g_launches.fetch_add(1, std::memory_order_relaxed);
-    if (e != cudaSuccess) return cuda_fail(e, "decode_kernel");
-  }
+  const int tiles_per_unit = (dm.cap + decode::kT - 1) / decode::kT;
+  const long long max_items = (long long)dm.units * ((tiles_per_unit + pl.tpi - 1) / pl.tpi);
+  const int grid = (int)(max_items < grid_limit ? max_items : grid_limit);
+  CAOTE_LAUNCH("decode_kernel", st,
+               decode::decode_kernel<<<grid, decode::kThreads, decode::smem_bytes(), st>>>(
+                   tmK, tmV, dm, (const __nv_bfloat16*)q, len, base, o, scores, pl, status));
   *used = true;
   return CAOTE_OK;
 }
@@ -265,13 +262,11 @@ static size_t workspace_bytes(const caote_params_t* p) {
   const Dims dm = make_dims(p);
   size_t need = generic::carve(dm, nullptr, nullptr);
   if (decode_shape_ok(p)) {
-    const size_t need2 = decode::carve(dm, nullptr, nullptr);
+    const size_t need2 = decode::carve(dm, nullptr, nullptr, 0);
     if (need2 > need) need = need2;
   }
   return kHeaderBytes + need;
 }
-
-static inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
 // ---- built-in scratch of caote_score_static ------------------------------------------------------
 // Lives in the library's device image: every GPU that loads the library holds these bytes until the
