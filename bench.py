@@ -371,8 +371,12 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--pool", type=int, default=64, help="distinct per-step input sets kept on the device")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=None,
+                    help="override the workload's batch (smaller cases for profiler captures; not a bench line)")
     args = ap.parse_args()
     w = wl.WORKLOADS[args.workload]
+    if args.batch is not None:
+        w = wl.scaled(w, batch=args.batch)
     if w.n_new > 1:
         # chunked prefill is timed in its steady state: the cache already holds `budget` tokens, so every
         # timed step scores budget + m tokens per unit and evicts m (the regime of all but the first chunks)

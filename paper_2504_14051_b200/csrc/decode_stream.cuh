@@ -43,9 +43,8 @@ constexpr int kConsumers = kConsumerWarps * 32;
 constexpr int kThreads = kConsumers + 32;  // + one producer warp
 constexpr int kHalfBytes = kT * 128;       // one 64-channel box: kT rows of 128 bytes
 constexpr int kTileBytes = 2 * kHalfBytes;
-constexpr int kSideBytes = 8 * kT * 4;     // per slot: 8 rows of kT floats (logits / base / P fragments)
-constexpr int kSlotBytes = kTileBytes + kSideBytes;
-constexpr int kMaxTilesPerItem = 4;
+constexpr int kRowsBytes = 8 * kT * 4;     // per slot: 8 rows of kT floats (logits / base / q / P fragments)
+constexpr int kMaxTilesPerItem = 16;
 constexpr long long kWaitCycles = 2000000000LL;  // ~1 s: far beyond any legitimate wait
 
 enum SlotType { kSlotKA = 0, kSlotVA = 1, kSlotVB = 2, kSlotStop = 3 };
@@ -62,10 +61,12 @@ struct FinalRec {     // per unit
   float m[8];
   float inv_l[8];
   float H;            // normaliser of the base score: counted rows + sum of carried base scores
-  float pad[7];
+  float XX;           // ||X||^2
+  float pad[2];
   float X[kD];
 };
-constexpr int kFinalFloats = sizeof(FinalRec) / sizeof(float);
+constexpr int kFinalBytes = sizeof(FinalRec);          // 592, a multiple of 16
+constexpr int kSideBytes = kRowsBytes + kFinalBytes;   // the rows, then the unit's FinalRec (score-pass slots)
 
 struct Desc {         // what a slot holds
   int type, unit, tile, n_valid, flags, item, item0, nitems;
@@ -86,7 +87,7 @@ struct Plan {
 
 inline int tiles_per_item(const Dims& dm, int grid) {
   const long long max_tiles = (long long)dm.units * ((dm.cap + kT - 1) / kT);
-  long long t = max_tiles / (4LL * (grid > 0 ? grid : 1));
+  long long t = max_tiles / (2LL * (grid > 0 ? grid : 1));
   if (t < 1) t = 1;
   if (t > kMaxTilesPerItem) t = kMaxTilesPerItem;
   return (int)t;
@@ -120,7 +121,7 @@ inline size_t carve(const Dims& dm, char* base, Plan* out, int grid) {
 }
 
 inline size_t smem_bytes() {
-  return 1024 /* alignment slack */ + (size_t)kSlots * kSlotBytes + sizeof(Desc) * kSlots + sizeof(FinalRec) +
+  return 1024 /* alignment slack */ + (size_t)kSlots * (kTileBytes + kSideBytes) + sizeof(Desc) * kSlots +
          sizeof(float) * (2 * kConsumerWarps * 8 + kConsumerWarps * 8 + kConsumerWarps + 8 + kD) + 8 * 2 * kSlots + 64;
 }
 
@@ -258,13 +259,31 @@ __device__ __forceinline__ bool consumer_any(bool pred) {
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
-// bf16 hi/lo split of a non-negative float: x ~= hi + lo with ~16 significant bits.
+// Two floats -> packed bf16x2 (x0 in the low half), round to nearest even.
+__device__ __forceinline__ uint32_t pack_bf16(float x0, float x1) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(x1), "f"(x0));
+  return r;
+}
+// bf16 hi/lo split of two floats: x ~= hi + lo with ~16 significant bits.
 __device__ __forceinline__ void split_pair(float x0, float x1, uint32_t& hi, uint32_t& lo) {
-  const __nv_bfloat16 h0 = __float2bfloat16_rn(x0), h1 = __float2bfloat16_rn(x1);
-  const __nv_bfloat16 l0 = __float2bfloat16_rn(x0 - __bfloat162float(h0));
-  const __nv_bfloat16 l1 = __float2bfloat16_rn(x1 - __bfloat162float(h1));
-  hi = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-  lo = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+  hi = pack_bf16(x0, x1);
+  lo = pack_bf16(x0 - __uint_as_float(hi << 16), x1 - __uint_as_float(hi & 0xffff0000u));
+}
+// 2^x, hardware approximation (2 ulp); 2^-inf = 0.
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+// One lane polls the barrier, the others sleep at the warp barrier; every lane then observes the
+// completed phase itself (which is what makes the copied data visible to it). Warp-uniform result.
+__device__ __forceinline__ bool warp_mbar_wait(uint64_t* bar, uint32_t parity, const volatile int* stop, int lane) {
+  int ok = 1;
+  if (lane == 0) ok = mbar_wait(bar, parity, stop) ? 1 : 0;
+  ok = __shfl_sync(0xffffffffu, ok, 0);
+  if (ok) ok = mbar_try_wait(bar, parity) ? 1 : 0;
+  return __all_sync(0xffffffffu, ok) != 0;
 }
 
 // Byte offset of 16-byte chunk `chunk16` (0..15 along the 128 channels) of row `row` inside a staged
@@ -293,10 +312,10 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
               float* __restrict__ o, float* __restrict__ scores, Plan pl, int* status) {
   extern __shared__ char smem_raw[];
   char* sm = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  char* slots = sm;                                                              // [kSlots][kSlotBytes]
-  Desc* desc = reinterpret_cast<Desc*>(slots + kSlots * kSlotBytes);             // [kSlots]
-  FinalRec* frec = reinterpret_cast<FinalRec*>(desc + kSlots);
-  float* wmax = reinterpret_cast<float*>(frec + 1);                              // [2][kConsumerWarps][8]
+  char* tiles = sm;                                                              // [kSlots][kTileBytes]
+  char* sides = tiles + kSlots * kTileBytes;                                     // [kSlots][kSideBytes]
+  Desc* desc = reinterpret_cast<Desc*>(sides + kSlots * kSideBytes);             // [kSlots]
+  float* wmax = reinterpret_cast<float*>(desc + kSlots);                         // [2][kConsumerWarps][8]
   float* wl = wmax + 2 * kConsumerWarps * 8;                                     // [kConsumerWarps][8]
   float* whb = wl + kConsumerWarps * 8;                                          // [kConsumerWarps]
   float* wm = whb + kConsumerWarps;                                              // [8]
@@ -386,37 +405,44 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
           int s;
           if (!is_b) {
             if (!(ok = acquire_slot(s))) break;
-            char* sl = slots + s * kSlotBytes;
+            char* tl = tiles + s * kTileBytes;
+            char* sd = sides + s * kSideBytes;
             d.type = kSlotKA;
             desc[s] = d;
-            mbar_expect_tx(&full[s], kTileBytes + base_bytes);
-            tma_load_2d(sl, &tmK, 0, row, &full[s], pol_stream);
-            tma_load_2d(sl + kHalfBytes, &tmK, 64, row, &full[s], pol_stream);
-            if (use_base) bulk_load(sl + kTileBytes + 7 * kT * 4, base_src, base_bytes, &full[s]);
+            // the unit's G query rows ride along with the item's first K tile (rows 0..3 of the side area)
+            const uint32_t q_bytes = (d.flags & kFlagFirst) ? (uint32_t)G * kD * 2u : 0u;
+            mbar_expect_tx(&full[s], kTileBytes + base_bytes + q_bytes);
+            tma_load_2d(tl, &tmK, 0, row, &full[s], pol_stream);
+            tma_load_2d(tl + kHalfBytes, &tmK, 64, row, &full[s], pol_stream);
+            if (use_base) bulk_load(sd + 7 * kT * 4, base_src, base_bytes, &full[s]);
+            if (q_bytes)
+              bulk_load(sd, q + ((size_t)(u / dm.Hkv) * dm.Hq + (size_t)(u % dm.Hkv) * G) * kD, q_bytes, &full[s]);
             ctl[2] = ++issued;
             if (!(ok = acquire_slot(s))) break;
-            sl = slots + s * kSlotBytes;
+            tl = tiles + s * kTileBytes;
             d.type = kSlotVA;
             desc[s] = d;
             mbar_expect_tx(&full[s], kTileBytes);
-            tma_load_2d(sl, &tmV, 0, row, &full[s], pol_keep);
-            tma_load_2d(sl + kHalfBytes, &tmV, 64, row, &full[s], pol_keep);
+            tma_load_2d(tl, &tmV, 0, row, &full[s], pol_keep);
+            tma_load_2d(tl + kHalfBytes, &tmV, 64, row, &full[s], pol_keep);
             ctl[2] = ++issued;
           } else {
             if (!(ok = acquire_slot(s))) break;
-            char* sl = slots + s * kSlotBytes;
+            char* tl = tiles + s * kTileBytes;
+            char* sd = sides + s * kSideBytes;
             d.type = kSlotVB;
             desc[s] = d;
             const uint32_t s_bytes = softmax_counted ? (uint32_t)G * kT * 4u : 0u;
-            mbar_expect_tx(&full[s], kTileBytes + s_bytes + base_bytes);
-            tma_load_2d(sl, &tmV, 0, row, &full[s], pol_stream);
-            tma_load_2d(sl + kHalfBytes, &tmV, 64, row, &full[s], pol_stream);
+            mbar_expect_tx(&full[s], kTileBytes + s_bytes + base_bytes + kFinalBytes);
+            tma_load_2d(tl, &tmV, 0, row, &full[s], pol_stream);
+            tma_load_2d(tl + kHalfBytes, &tmV, 64, row, &full[s], pol_stream);
             if (softmax_counted) {
               const float* ssrc = pl.S + ((size_t)u * G) * pl.capS + (size_t)t * kT;
               for (int g = 0; g < G; ++g)
-                bulk_load(sl + kTileBytes + g * kT * 4, ssrc + (size_t)g * pl.capS, kT * 4, &full[s]);
+                bulk_load(sd + g * kT * 4, ssrc + (size_t)g * pl.capS, kT * 4, &full[s]);
             }
-            if (use_base) bulk_load(sl + kTileBytes + 7 * kT * 4, base_src, base_bytes, &full[s]);
+            if (use_base) bulk_load(sd + 7 * kT * 4, base_src, base_bytes, &full[s]);
+            bulk_load(sd + kRowsBytes, pl.fin + u, kFinalBytes, &full[s]);
             ctl[2] = ++issued;
           }
         }
@@ -450,9 +476,9 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 
     for (;; ++consumed) {
       const int s = consumed % kSlots;
-      char* sl = slots + s * kSlotBytes;
-      float* side = reinterpret_cast<float*>(sl + kTileBytes);  // [8][kT]
-      const bool got = mbar_wait(&full[s], (consumed / kSlots) & 1, &ctl[0]);
+      char* sl = tiles + s * kTileBytes;
+      float* side = reinterpret_cast<float*>(sides + s * kSideBytes);  // [8][kT], then a FinalRec
+      const bool got = warp_mbar_wait(&full[s], (consumed / kSlots) & 1, &ctl[0], lane);
       if (consumer_any(!got)) {  // uniform: either every consumer thread leaves here or none does
         if (tid == 0 && !ctl[0]) {
           set_status(status, CAOTE_ERR_TIMEOUT);
@@ -468,7 +494,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         // ===================== logits and softmax numerators of one tile =====================
         if (d.flags & kFlagFirst) {
           // Q fragments: row = lane / 4 (rows 8..15 duplicate rows 0..7), zero for heads >= G
-          const __nv_bfloat16* qrow = q + ((size_t)b * dm.Hq + h * G + (head < G ? head : 0)) * kD + 2 * quad;
+          const __nv_bfloat16* qrow = reinterpret_cast<const __nv_bfloat16*>(side) + (head < G ? head : 0) * kD + 2 * quad;
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks) {
             qa[ks][0] = (head < G) ? *reinterpret_cast<const uint32_t*>(qrow + 16 * ks) : 0u;
@@ -526,11 +552,11 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
 #pragma unroll
         for (int w = 0; w < kConsumerWarps; ++w) m_new = fmaxf(m_new, wmx[w * 8 + head]);
         tile_par ^= 1;
-        corr = (m_run == -INFINITY) ? 0.f : exp2f(m_run - m_new);
+        corr = fast_exp2(m_run - m_new);  // m_new is finite (a tile holds a valid token); 2^-inf = 0
         m_run = m_new;
         float p[4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) p[i] = (sv[i] == -INFINITY) ? 0.f : exp2f(sv[i] - m_new);
+        for (int i = 0; i < 4; ++i) p[i] = fast_exp2(sv[i] - m_new);
         l_priv = fmaf(l_priv, corr, (p[0] + p[1]) + (p[2] + p[3]));
         if (head >= G) { p[0] = p[1] = p[2] = p[3] = 0.f; }
         if (use_base && head == 7) {
@@ -541,7 +567,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         split_pair(p[0], p[1], frag.x, frag.y);
         split_pair(p[2], p[3], frag.z, frag.w);
         // the P fragments wait in the side area of the next slot, which will hold this tile's V
-        uint4* Pbuf = reinterpret_cast<uint4*>(slots + ((consumed + 1) % kSlots) * kSlotBytes + kTileBytes);
+        uint4* Pbuf = reinterpret_cast<uint4*>(sides + ((consumed + 1) % kSlots) * kSideBytes);
         Pbuf[warp * 32 + lane] = frag;
       } else if (d.type == kSlotVA) {
         // ===================== partial output of one tile =====================
@@ -659,8 +685,14 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
             }
             if ((tid & 31) == 0) { fr->m[hd] = mfin; fr->inv_l[hd] = inv_l; }
             if (tid == 0) fr->H = Htot;
-            if (tid < kD) fr->X[tid] = (Htot > 0.f) ? xrow[tid] / Htot : 0.f;
+            if (tid < kD) {
+              const float xv = (Htot > 0.f) ? xrow[tid] / Htot : 0.f;
+              fr->X[tid] = xv;
+              float xx = warp_sum(xv * xv);
+              if (lane == 0) wl[warp] = xx;  // warps 0..3
+            }
             consumer_sync();
+            if (tid == 0) fr->XX = (wl[0] + wl[1]) + (wl[2] + wl[3]);
             if (tid == 0) {
               __threadfence();
               st_release(&pl.ready[d.unit], 1);
@@ -669,51 +701,101 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         }
       } else {
         // ===================== score pass of one tile =====================
-        if (d.flags & kFlagFirst) {
-          if (tid < kFinalFloats)
-            reinterpret_cast<float*>(frec)[tid] = __ldcg(reinterpret_cast<const float*>(pl.fin + d.unit) + tid);
-          consumer_sync();
-        }
-        const int row = tid >> 1, half = tid & 1;
-        float acc = 0.f;
+        // ||X - v_j||^2 = ||v_j||^2 - 2 <v_j, X> + ||X||^2 for this warp's 16 tokens on the tensor
+        // cores: the V rows are the A operand; used again as the B operand they give the Gram
+        // blocks whose diagonals are ||v_j||^2; X, split into bf16 hi + lo columns, gives <v_j, X>.
+        // Tokens for which that difference cancels (v_j close to X) or that hold most of the weight
+        // are redone below by plain subtraction, so v_j = X still scores exactly 0.
+        const FinalRec* fr = reinterpret_cast<const FinalRec*>(side + 8 * kT);
+        uint32_t xb[8][2];
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          const int cc = c ^ (half << 2);
-          const uint4 raw = *reinterpret_cast<const uint4*>(sl + tile_off(row, half * 8 + cc));
-          const uint32_t wv[4] = {raw.x, raw.y, raw.z, raw.w};
-          const float4 xa = *reinterpret_cast<const float4*>(frec->X + half * 64 + cc * 8);
-          const float4 xb = *reinterpret_cast<const float4*>(frec->X + half * 64 + cc * 8 + 4);
-          const float x[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&wv[e]));
-            const float d0 = x[2 * e] - f.x, d1 = x[2 * e + 1] - f.y;
-            acc = fmaf(d0, d0, acc);
-            acc = fmaf(d1, d1, acc);
+        for (int ks = 0; ks < 8; ++ks) {
+          xb[ks][0] = 0u;
+          xb[ks][1] = 0u;
+          if (head < 2) {
+            const float2 x0 = *reinterpret_cast<const float2*>(fr->X + 16 * ks + 2 * quad);
+            const float2 x1 = *reinterpret_cast<const float2*>(fr->X + 16 * ks + 8 + 2 * quad);
+            uint32_t h0, l0, h1, l1;
+            split_pair(x0.x, x0.y, h0, l0);
+            split_pair(x1.x, x1.y, h1, l1);
+            xb[ks][0] = head == 0 ? h0 : l0;
+            xb[ks][1] = head == 0 ? h1 : l1;
           }
         }
-        acc += __shfl_xor_sync(0xffffffffu, acc, 1);
-        if (half == 0 && row < d.n_valid) {
-          float hj = 0.f;
-          if (softmax_counted) {
+        float ca[4] = {0.f, 0.f, 0.f, 0.f}, cb[4] = {0.f, 0.f, 0.f, 0.f}, cx[4] = {0.f, 0.f, 0.f, 0.f};
+        {
+          const uint32_t vaddr = smem_u32(sl);
+          const int mi = lane >> 3, r = lane & 7;
+          const int tok = 16 * warp + 8 * (mi & 1) + r;
 #pragma unroll
-            for (int g = 0; g < 8; ++g)
-              if (g < G) hj += exp2f(side[g * kT + row] - frec->m[g]) * frec->inv_l[g];
+          for (int ks = 0; ks < 8; ++ks) {
+            uint32_t a0, a1, a2, a3;
+            ldmatrix_x4(vaddr + tile_off(tok, 2 * ks + (mi >> 1)), a0, a1, a2, a3);
+            mma_bf16(ca, a0, a1, a2, a3, a0, a2);  // rows x tokens 0..7 of the warp
+            mma_bf16(cb, a0, a1, a2, a3, a1, a3);  // rows x tokens 8..15
+            mma_bf16(cx, a0, a1, a2, a3, xb[ks][0], xb[ks][1]);
           }
-          const size_t slot = (size_t)d.unit * dm.cap + (size_t)d.tile * kT + row;
+        }
+        // lane (head, quad): token `head` of the warp if quad == 0, token head + 8 if quad == 1
+        const int src = (lane & ~3) | (head >> 1);
+        const float vva = __shfl_sync(0xffffffffu, (head & 1) ? ca[1] : ca[0], src);
+        const float vvb = __shfl_sync(0xffffffffu, (head & 1) ? cb[3] : cb[2], src);
+        const float vxa = __shfl_sync(0xffffffffu, cx[0] + cx[1], lane & ~3);
+        const float vxb = __shfl_sync(0xffffffffu, cx[2] + cx[3], lane & ~3);
+        // base score: heads quad and quad + 4 of both tokens, then a sum over the quad
+        const int ra = 16 * warp + head, rb = ra + 8;
+        float ha = 0.f, hbv = 0.f;
+        if (softmax_counted) {
+#pragma unroll
+          for (int gg = 0; gg < 2; ++gg) {
+            const int g = quad + 4 * gg;
+            if (g < G) {
+              const float mg = fr->m[g], il = fr->inv_l[g];
+              ha = fmaf(fast_exp2(side[g * kT + ra] - mg), il, ha);
+              hbv = fmaf(fast_exp2(side[g * kT + rb] - mg), il, hbv);
+            }
+          }
+          ha += __shfl_xor_sync(0xffffffffu, ha, 1);
+          ha += __shfl_xor_sync(0xffffffffu, ha, 2);
+          hbv += __shfl_xor_sync(0xffffffffu, hbv, 1);
+          hbv += __shfl_xor_sync(0xffffffffu, hbv, 2);
+        }
+        const int row = quad == 0 ? ra : rb;
+        const bool mine = quad < 2 && row < d.n_valid;
+        float hj = quad == 0 ? ha : hbv;
+        const float vv = quad == 0 ? vva : vvb, vx = quad == 0 ? vxa : vxb;
+        const size_t slot = (size_t)d.unit * dm.cap + (size_t)d.tile * kT + row;
+        if (mine) {
           if (mode == CAOTE_BASE_ACCUM) {
             hj += side[7 * kT + row];
             base[slot] = hj;
           } else if (mode == CAOTE_BASE_EXTERNAL) {
             hj = side[7 * kT + row];
           }
-          const float Htot = frec->H;
+        }
+        const float Htot = fr->H, XX = fr->XX;
+        float n2 = fmaxf(vv - 2.f * vx + XX, 0.f);
+        const bool redo = mine && (n2 < 2e-3f * (vv + XX) || 2.f * hj > Htot);
+        unsigned todo = __ballot_sync(0xffffffffu, redo);
+        while (todo) {
+          const int l = __ffs((int)todo) - 1;
+          todo &= todo - 1;
+          const int rr = 16 * warp + (l >> 2) + 8 * (l & 3);  // the row lane l is responsible for
+          const uint2 raw = *reinterpret_cast<const uint2*>(sl + tile_off(rr, lane >> 1) + (lane & 1) * 8);
+          const float4 xv = *reinterpret_cast<const float4*>(fr->X + 4 * lane);
+          const float2 f0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
+          const float2 f1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
+          const float d0 = xv.x - f0.x, d1 = xv.y - f0.y, d2 = xv.z - f1.x, d3 = xv.w - f1.y;
+          const float exact = warp_sum(fmaf(d0, d0, d1 * d1) + fmaf(d2, d2, d3 * d3));
+          if (lane == l) n2 = exact;
+        }
+        if (mine) {
           float ratio = 0.f;
           if (Htot > 0.f) {
             const float rest = Htot - hj;
             ratio = (rest > 0.f) ? hj / rest : INFINITY;
           }
-          scores[slot] = (ratio == 0.f) ? 0.f : ((ratio == INFINITY) ? INFINITY : ratio * sqrtf(acc));
+          scores[slot] = (ratio == 0.f) ? 0.f : ((ratio == INFINITY) ? INFINITY : ratio * sqrtf(n2));
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&empty[s]);
