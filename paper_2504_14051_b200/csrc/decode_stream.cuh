@@ -37,14 +37,14 @@ namespace decode {
 
 constexpr int kT = 128;                 // tokens per tile
 constexpr int kD = 128;
-constexpr int kSlots = 3;
+constexpr int kSlots = 4;
 constexpr int kConsumerWarps = 8;
 constexpr int kConsumers = kConsumerWarps * 32;
 constexpr int kThreads = kConsumers + 32;  // + one producer warp
 constexpr int kHalfBytes = kT * 128;       // one 64-channel box: kT rows of 128 bytes
 constexpr int kTileBytes = 2 * kHalfBytes;
 constexpr int kRowsBytes = 8 * kT * 4;     // per slot: 8 rows of kT floats (logits / base / q / P fragments)
-constexpr int kMaxTilesPerItem = 16;
+constexpr int kMaxTilesPerItem = 8;
 constexpr long long kWaitCycles = 2000000000LL;  // ~1 s: far beyond any legitimate wait
 
 enum SlotType { kSlotKA = 0, kSlotVA = 1, kSlotVB = 2, kSlotStop = 3 };
@@ -120,9 +120,14 @@ inline size_t carve(const Dims& dm, char* base, Plan* out, int grid) {
   return off;
 }
 
+// Staging area in which the eight consumer warps put their partial results at the end of an item
+// (two copies, used by alternate items): per warp 8 heads x kD floats, then max, sum and base sum.
+constexpr int kStageFloats = kConsumerWarps * 8 * kD + 2 * kConsumerWarps * 8 + kConsumerWarps;
+constexpr int kStageBytes = (kStageFloats * 4 + 255) / 256 * 256;
+
 inline size_t smem_bytes() {
-  return 1024 /* alignment slack */ + (size_t)kSlots * (kTileBytes + kSideBytes) + sizeof(Desc) * kSlots +
-         sizeof(float) * (2 * kConsumerWarps * 8 + kConsumerWarps * 8 + kConsumerWarps + 8 + kD) + 8 * 2 * kSlots + 64;
+  return 1024 /* alignment slack */ + (size_t)kSlots * (kTileBytes + kSideBytes) + 2 * (size_t)kStageBytes +
+         sizeof(Desc) * kSlots + 8 * (2 * kSlots + 2) + 64;
 }
 
 // ---- plan: items per unit, their prefix sum, and cleared counters / flags (one CTA) -------------
@@ -306,7 +311,7 @@ __device__ __forceinline__ void work_entry(int w, int N, int L, bool& is_b, int&
   item = w - N;
 }
 
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, 1)
 decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, Dims dm,
               const __nv_bfloat16* __restrict__ q, const int* __restrict__ len, float* __restrict__ base,
               float* __restrict__ o, float* __restrict__ scores, Plan pl, int* status) {
@@ -314,16 +319,13 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
   char* sm = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   char* tiles = sm;                                                              // [kSlots][kTileBytes]
   char* sides = tiles + kSlots * kTileBytes;                                     // [kSlots][kSideBytes]
-  Desc* desc = reinterpret_cast<Desc*>(sides + kSlots * kSideBytes);             // [kSlots]
-  float* wmax = reinterpret_cast<float*>(desc + kSlots);                         // [2][kConsumerWarps][8]
-  float* wl = wmax + 2 * kConsumerWarps * 8;                                     // [kConsumerWarps][8]
-  float* whb = wl + kConsumerWarps * 8;                                          // [kConsumerWarps]
-  float* wm = whb + kConsumerWarps;                                              // [8]
-  float* xrow = wm + 8;                                                          // [kD]
-  uint64_t* full = reinterpret_cast<uint64_t*>(xrow + kD);                       // [kSlots]
+  char* stages = sides + kSlots * kSideBytes;                                    // [2][kStageBytes]
+  Desc* desc = reinterpret_cast<Desc*>(stages + 2 * kStageBytes);                // [kSlots]
+  uint64_t* full = reinterpret_cast<uint64_t*>(desc + kSlots);                   // [kSlots]
   uint64_t* empty = full + kSlots;                                               // [kSlots]
-  volatile int* ctl = reinterpret_cast<volatile int*>(empty + kSlots);           // [0] stop, [1] last arriver,
-                                                                                 // [2] slots issued
+  uint64_t* stage_free = empty + kSlots;                                         // [2]
+  volatile int* ctl = reinterpret_cast<volatile int*>(stage_free + 2);           // [0] stop, [2] slots issued,
+  int* stage_cnt = const_cast<int*>(ctl) + 4;                                    // [2] warps that have staged
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int G = dm.G, mode = dm.base_mode;
@@ -337,15 +339,19 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
       mbar_init(&full[i], 1);
       mbar_init(&empty[i], kConsumerWarps);
     }
+    mbar_init(&stage_free[0], 1);
+    mbar_init(&stage_free[1], 1);
     ctl[0] = 0;
     ctl[1] = 0;
     ctl[2] = 0;
+    stage_cnt[0] = 0;
+    stage_cnt[1] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (tid < kSlots * (int)(sizeof(Desc) / sizeof(int))) reinterpret_cast<int*>(desc)[tid] = 0;
   __syncthreads();
 
-  int consumed = 0;  // slots the consumers have finished (uniform over the consumer threads)
+  int consumed = 0;  // slots this warp has finished
 
   if (warp == kConsumerWarps) {
     // ================================ producer warp ================================
@@ -467,339 +473,389 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
     }
   } else {
     // ================================ consumer warps ================================
+    // Each warp is on its own: it owns tokens [16 warp, 16 warp + 16) of every tile, keeps its own
+    // softmax reference and its own full-width output accumulator, and never waits for a sibling.
     const int head = lane >> 2, quad = lane & 3;
-    const int t0 = 16 * warp + 2 * quad;  // this thread's tokens: t0, t0 + 1, t0 + 8, t0 + 9
-    uint32_t qa[8][2];
-    float m_run = -INFINITY, l_priv = 0.f, hb_priv = 0.f, corr = 0.f;
-    float o0[4] = {0.f, 0.f, 0.f, 0.f}, o1[4] = {0.f, 0.f, 0.f, 0.f};
-    int tile_par = 0;
+    const int t0 = 16 * warp + 2 * quad;  // this thread's tokens in a tile: t0, t0 + 1, t0 + 8, t0 + 9
+    const int mi = lane >> 3, mr = lane & 7;
+    bool alive = true;
+    int items_done = 0;  // A items this warp has finished (selects the staging copy)
+    int s = 0;
+    Desc d;
+    auto next_slot = [&]() -> bool {
+      s = consumed % kSlots;
+      if (!warp_mbar_wait(&full[s], (consumed / kSlots) & 1, &ctl[0], lane)) return false;
+      d = desc[s];
+      return true;
+    };
+    auto release = [&]() {
+      __syncwarp();
+      fence_async_smem();
+      if (lane == 0) mbar_arrive(&empty[s]);
+      ++consumed;
+    };
 
-    for (;; ++consumed) {
-      const int s = consumed % kSlots;
-      char* sl = tiles + s * kTileBytes;
-      float* side = reinterpret_cast<float*>(sides + s * kSideBytes);  // [8][kT], then a FinalRec
-      const bool got = warp_mbar_wait(&full[s], (consumed / kSlots) & 1, &ctl[0], lane);
-      if (consumer_any(!got)) {  // uniform: either every consumer thread leaves here or none does
-        if (tid == 0 && !ctl[0]) {
-          set_status(status, CAOTE_ERR_TIMEOUT);
-          ctl[0] = 1;
-        }
-        break;
-      }
-      const Desc d = desc[s];
+    while (alive) {
+      if (!next_slot()) { alive = false; break; }
       if (d.type == kSlotStop) { ++consumed; break; }
-      const int b = d.unit / dm.Hkv, h = d.unit % dm.Hkv;
 
       if (d.type == kSlotKA) {
-        // ===================== logits and softmax numerators of one tile =====================
-        if (d.flags & kFlagFirst) {
+        // =============================== one A item ===============================
+        const bool base_row = use_base && head == 7;
+        uint32_t qa[8][2];
+        float oacc[16][4];
+        float m_ref = base_row ? 0.f : -INFINITY, l_priv = 0.f, hb_priv = 0.f;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) { oacc[j][0] = 0.f; oacc[j][1] = 0.f; oacc[j][2] = 0.f; oacc[j][3] = 0.f; }
+        {
           // Q fragments: row = lane / 4 (rows 8..15 duplicate rows 0..7), zero for heads >= G
-          const __nv_bfloat16* qrow = reinterpret_cast<const __nv_bfloat16*>(side) + (head < G ? head : 0) * kD + 2 * quad;
+          const __nv_bfloat16* qrow = reinterpret_cast<const __nv_bfloat16*>(sides + s * kSideBytes) +
+                                      (head < G ? head : 0) * kD + 2 * quad;
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks) {
             qa[ks][0] = (head < G) ? *reinterpret_cast<const uint32_t*>(qrow + 16 * ks) : 0u;
             qa[ks][1] = (head < G) ? *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 8) : 0u;
           }
-          m_run = -INFINITY;
-          l_priv = 0.f;
-          hb_priv = 0.f;
-#pragma unroll
-          for (int i = 0; i < 4; ++i) { o0[i] = 0.f; o1[i] = 0.f; }
         }
-        const uint32_t kaddr = smem_u32(sl);
-        float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
-        {
-          const int mi = lane >> 3, r = lane & 7;
-          const int tok = 16 * warp + 8 * (mi >> 1) + r;
-#pragma unroll
-          for (int ks = 0; ks < 8; ++ks) {
-            uint32_t b0, b1, b2, b3;
-            ldmatrix_x4(kaddr + tile_off(tok, 2 * ks + (mi & 1)), b0, b1, b2, b3);
-            mma_bf16(s0, qa[ks][0], qa[ks][0], qa[ks][1], qa[ks][1], b0, b1);
-            mma_bf16(s1, qa[ks][0], qa[ks][0], qa[ks][1], qa[ks][1], b2, b3);
-          }
-        }
-        const bool v0 = t0 < d.n_valid, v1 = t0 + 1 < d.n_valid, v2 = t0 + 8 < d.n_valid, v3 = t0 + 9 < d.n_valid;
-        float bv[4] = {0.f, 0.f, 0.f, 0.f};
-        if (use_base && head == 7) {
-          const float* Bb = side + 7 * kT;
-          bv[0] = v0 ? Bb[t0] : 0.f;
-          bv[1] = v1 ? Bb[t0 + 1] : 0.f;
-          bv[2] = v2 ? Bb[t0 + 8] : 0.f;
-          bv[3] = v3 ? Bb[t0 + 9] : 0.f;
-          hb_priv += (bv[0] + bv[1]) + (bv[2] + bv[3]);
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&empty[s]);  // this warp is done with the K tile and its base row
-
-        float sv[4];
-        sv[0] = v0 ? s0[0] * scale2 : -INFINITY;
-        sv[1] = v1 ? s0[1] * scale2 : -INFINITY;
-        sv[2] = v2 ? s1[0] * scale2 : -INFINITY;
-        sv[3] = v3 ? s1[1] * scale2 : -INFINITY;
-        if (softmax_counted && head < G) {
-          float* Sg = pl.S + ((size_t)d.unit * G + head) * pl.capS + (size_t)d.tile * kT + t0;
-          __stcg(reinterpret_cast<float2*>(Sg), make_float2(sv[0], sv[1]));
-          __stcg(reinterpret_cast<float2*>(Sg + 8), make_float2(sv[2], sv[3]));
-        }
-        float mx = fmaxf(fmaxf(sv[0], sv[1]), fmaxf(sv[2], sv[3]));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-        float* wmx = wmax + tile_par * kConsumerWarps * 8;
-        if (quad == 0) wmx[warp * 8 + head] = mx;
-        consumer_sync();
-        float m_new = m_run;
-#pragma unroll
-        for (int w = 0; w < kConsumerWarps; ++w) m_new = fmaxf(m_new, wmx[w * 8 + head]);
-        tile_par ^= 1;
-        corr = fast_exp2(m_run - m_new);  // m_new is finite (a tile holds a valid token); 2^-inf = 0
-        m_run = m_new;
-        float p[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) p[i] = fast_exp2(sv[i] - m_new);
-        l_priv = fmaf(l_priv, corr, (p[0] + p[1]) + (p[2] + p[3]));
-        if (head >= G) { p[0] = p[1] = p[2] = p[3] = 0.f; }
-        if (use_base && head == 7) {
-          p[0] = bv[0]; p[1] = bv[1]; p[2] = bv[2]; p[3] = bv[3];
-          corr = 1.f;
-        }
-        uint4 frag;  // a0 = hi(n-tile 0), a1 = lo(n-tile 0), a2 = hi(n-tile 1), a3 = lo(n-tile 1)
-        split_pair(p[0], p[1], frag.x, frag.y);
-        split_pair(p[2], p[3], frag.z, frag.w);
-        // the P fragments wait in the side area of the next slot, which will hold this tile's V
-        uint4* Pbuf = reinterpret_cast<uint4*>(sides + ((consumed + 1) % kSlots) * kSideBytes);
-        Pbuf[warp * 32 + lane] = frag;
-      } else if (d.type == kSlotVA) {
-        // ===================== partial output of one tile =====================
-        const uint4* Pbuf = reinterpret_cast<const uint4*>(side);
-        if (d.n_valid < kT) {
-          // rows behind the unit's length hold whatever the cache has there: clear them so that a
-          // zero weight times a stray NaN cannot reach the accumulators
-          const int rows = kT - d.n_valid;
-          for (int i = tid; i < rows * 16; i += kConsumers) {
-            const int row = d.n_valid + (i >> 4), c = i & 15;
-            *reinterpret_cast<uint4*>(sl + tile_off(row, c)) = make_uint4(0u, 0u, 0u, 0u);
-          }
-          consumer_sync();
-        }
-#pragma unroll
-        for (int i = 0; i < 4; ++i) { o0[i] *= corr; o1[i] *= corr; }
-        const uint32_t vaddr = smem_u32(sl);
-        {
-          const int mi = lane >> 3, r = lane & 7;
-#pragma unroll
-          for (int kk = 0; kk < kT / 16; ++kk) {
-            const uint4 a = Pbuf[kk * 32 + lane];
-            uint32_t b0, b1, b2, b3;
-            ldmatrix_x4_trans(vaddr + tile_off(16 * kk + 8 * (mi & 1) + r, 2 * warp + (mi >> 1)), b0, b1, b2, b3);
-            mma_bf16(o0, a.x, a.y, a.z, a.w, b0, b1);
-            mma_bf16(o1, a.x, a.y, a.z, a.w, b2, b3);
-          }
-        }
-        __syncwarp();
-        fence_async_smem();
-        if (lane == 0) mbar_arrive(&empty[s]);
-
-        if (d.flags & kFlagLast) {
-          // ---------- the item's record ----------
-          PartialRec* pr = pl.part + d.item;
+        for (;;) {
+          // ---------------- K tile: logits, softmax numerators ----------------
+          if (d.type != kSlotKA) { alive = false; break; }
+          uint4 frag;  // P as an A fragment: a0 = hi(tokens 0..7), a1 = lo(0..7), a2 = hi(8..15), a3 = lo(8..15)
           {
-            const int c0 = 16 * warp + 2 * quad;
-            *reinterpret_cast<float2*>(&pr->o[head][c0]) = make_float2(o0[0] + o0[2], o0[1] + o0[3]);
-            *reinterpret_cast<float2*>(&pr->o[head][c0 + 8]) = make_float2(o1[0] + o1[2], o1[1] + o1[3]);
-          }
-          float ls = l_priv;
-          ls += __shfl_xor_sync(0xffffffffu, ls, 1);
-          ls += __shfl_xor_sync(0xffffffffu, ls, 2);
-          float hs = hb_priv;
-          hs += __shfl_xor_sync(0xffffffffu, hs, 1);
-          hs += __shfl_xor_sync(0xffffffffu, hs, 2);
-          if (quad == 0) {
-            wl[warp * 8 + head] = ls;
-            if (head == 7) whb[warp] = hs;
-            if (warp == 0) wm[head] = m_run;
-          }
-          consumer_sync();
-          if (warp == 0) {
-            if (lane < 8) {
-              float ll = 0.f;
-              for (int w = 0; w < kConsumerWarps; ++w) ll += wl[w * 8 + lane];
-              pr->m[lane] = wm[lane];
-              pr->l[lane] = ll;
+            const uint32_t kaddr = smem_u32(tiles + s * kTileBytes);
+            const float* side = reinterpret_cast<const float*>(sides + s * kSideBytes);
+            uint32_t kb[8][4];
+            const int tok = 16 * warp + 8 * (mi >> 1) + mr;
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks)
+              ldmatrix_x4(kaddr + tile_off(tok, 2 * ks + (mi & 1)), kb[ks][0], kb[ks][1], kb[ks][2], kb[ks][3]);
+            float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+              mma_bf16(s0, qa[ks][0], qa[ks][0], qa[ks][1], qa[ks][1], kb[ks][0], kb[ks][1]);
+              mma_bf16(s1, qa[ks][0], qa[ks][0], qa[ks][1], qa[ks][1], kb[ks][2], kb[ks][3]);
             }
-            if (lane == 8) {
-              float hb = 0.f;
-              for (int w = 0; w < kConsumerWarps; ++w) hb += whb[w];
-              pr->hb = use_base ? hb : 0.f;
+            const bool v0 = t0 < d.n_valid, v1 = t0 + 1 < d.n_valid, v2 = t0 + 8 < d.n_valid, v3 = t0 + 9 < d.n_valid;
+            float bv[4] = {0.f, 0.f, 0.f, 0.f};
+            if (base_row) {
+              const float* Bb = side + 7 * kT;
+              bv[0] = v0 ? Bb[t0] : 0.f;
+              bv[1] = v1 ? Bb[t0 + 1] : 0.f;
+              bv[2] = v2 ? Bb[t0 + 8] : 0.f;
+              bv[3] = v3 ? Bb[t0 + 9] : 0.f;
+              hb_priv += (bv[0] + bv[1]) + (bv[2] + bv[3]);
             }
+            const int tile = d.tile, unit = d.unit;
+            release();  // done with the K tile and its side rows
+
+            float sv[4];
+            sv[0] = v0 ? s0[0] * scale2 : -INFINITY;
+            sv[1] = v1 ? s0[1] * scale2 : -INFINITY;
+            sv[2] = v2 ? s1[0] * scale2 : -INFINITY;
+            sv[3] = v3 ? s1[1] * scale2 : -INFINITY;
+            if (softmax_counted && head < G) {
+              float* Sg = pl.S + ((size_t)unit * G + head) * pl.capS + (size_t)tile * kT + t0;
+              __stcg(reinterpret_cast<float2*>(Sg), make_float2(sv[0], sv[1]));
+              __stcg(reinterpret_cast<float2*>(Sg + 8), make_float2(sv[2], sv[3]));
+            }
+            float mx = fmaxf(fmaxf(sv[0], sv[1]), fmaxf(sv[2], sv[3]));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+            // The reference moves only when a logit exceeds it by more than 8 (p stays <= 256), so
+            // the 64 accumulator registers are rescaled a handful of times per item, not every tile.
+            const bool need = !base_row && mx > m_ref + 8.f;  // also true for the first finite maximum
+            if (__any_sync(0xffffffffu, need)) {
+              const float corr = need ? fast_exp2(m_ref - mx) : 1.f;
+              if (need) m_ref = mx;
+              l_priv *= corr;
+#pragma unroll
+              for (int j = 0; j < 16; ++j) { oacc[j][0] *= corr; oacc[j][1] *= corr; oacc[j][2] *= corr; oacc[j][3] *= corr; }
+            }
+            float p[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) p[i] = (sv[i] == -INFINITY) ? 0.f : fast_exp2(sv[i] - m_ref);
+            l_priv += (p[0] + p[1]) + (p[2] + p[3]);
+            if (head >= G) { p[0] = p[1] = p[2] = p[3] = 0.f; }
+            if (base_row) { p[0] = bv[0]; p[1] = bv[1]; p[2] = bv[2]; p[3] = bv[3]; }
+            split_pair(p[0], p[1], frag.x, frag.y);
+            split_pair(p[2], p[3], frag.z, frag.w);
           }
-          consumer_sync();
-          if (tid == 0) {
-            __threadfence();
-            const int old = atomicAdd(&pl.counter[d.unit], 1);
-            ctl[1] = (old == d.nitems - 1);
-          }
-          consumer_sync();
-          if (ctl[1]) {
-            // ---------- last arriver: merge the unit's records ----------
-            __threadfence();
-            const PartialRec* p0 = pl.part + d.item0;
-            const int hd = tid >> 5, c4 = (tid & 31) * 4;
-            const bool base_row = use_base && hd == 7;
-            float mfin = -INFINITY;
-            for (int c = 0; c < d.nitems; ++c) mfin = fmaxf(mfin, __ldcg(&p0[c].m[hd]));
-            float lfin = 0.f, hbsum = 0.f;
-            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 4
-            for (int c = 0; c < d.nitems; ++c) {
-              const float f = base_row ? 1.f : exp2f(__ldcg(&p0[c].m[hd]) - mfin);
-              lfin = fmaf(__ldcg(&p0[c].l[hd]), f, lfin);
-              const float4 v = __ldcg(reinterpret_cast<const float4*>(&p0[c].o[hd][c4]));
-              acc.x = fmaf(v.x, f, acc.x);
-              acc.y = fmaf(v.y, f, acc.y);
-              acc.z = fmaf(v.z, f, acc.z);
-              acc.w = fmaf(v.w, f, acc.w);
-              hbsum += __ldcg(&p0[c].hb);
-            }
-            const float inv_l = (hd < G) ? 1.f / lfin : 0.f;
-            FinalRec* fr = pl.fin + d.unit;
-            float4 contrib = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (hd < G) {
-              const float4 on = make_float4(acc.x * inv_l, acc.y * inv_l, acc.z * inv_l, acc.w * inv_l);
-              *reinterpret_cast<float4*>(o + ((size_t)b * dm.Hq + h * G + hd) * kD + c4) = on;
-              if (softmax_counted) contrib = on;
-            } else if (base_row) {
-              contrib = acc;
-            }
-            const float Htot = (softmax_counted ? (float)G : 0.f) + (use_base ? hbsum : 0.f);
-            // X = (sum of the 8 rows of contrib) / Htot; row hd lives in warp hd, so the warps add
-            // their rows one after the other (fixed order: bit-reproducible)
-            for (int r = 0; r < 8; ++r) {
-              if (hd == r) {
-                float4* xp = reinterpret_cast<float4*>(&xrow[c4]);
-                float4 t = (r == 0) ? make_float4(0.f, 0.f, 0.f, 0.f) : *xp;
-                t.x += contrib.x; t.y += contrib.y; t.z += contrib.z; t.w += contrib.w;
-                *xp = t;
+          // ---------------- V tile: partial output of this warp's 16 tokens ----------------
+          if (!next_slot() || d.type != kSlotVA) { alive = false; break; }
+          {
+            char* sl = tiles + s * kTileBytes;
+            if (d.n_valid < 16 * warp + 16) {
+              // rows behind the unit's length hold whatever the cache has there: clear this warp's
+              // so that a zero weight times a stray NaN cannot reach the accumulators
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                const int row = 16 * warp + 2 * i + (lane >> 4), c = lane & 15;
+                if (row >= d.n_valid) *reinterpret_cast<uint4*>(sl + tile_off(row, c)) = make_uint4(0u, 0u, 0u, 0u);
               }
-              consumer_sync();
+              __syncwarp();
             }
-            if ((tid & 31) == 0) { fr->m[hd] = mfin; fr->inv_l[hd] = inv_l; }
-            if (tid == 0) fr->H = Htot;
-            if (tid < kD) {
-              const float xv = (Htot > 0.f) ? xrow[tid] / Htot : 0.f;
-              fr->X[tid] = xv;
-              float xx = warp_sum(xv * xv);
-              if (lane == 0) wl[warp] = xx;  // warps 0..3
-            }
-            consumer_sync();
-            if (tid == 0) fr->XX = (wl[0] + wl[1]) + (wl[2] + wl[3]);
-            if (tid == 0) {
-              __threadfence();
-              st_release(&pl.ready[d.unit], 1);
+            const uint32_t vaddr = smem_u32(sl);
+            const int vrow = 16 * warp + 8 * (mi & 1) + mr;
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+              uint32_t vb[4][4];
+#pragma unroll
+              for (int jj = 0; jj < 4; ++jj)
+                ldmatrix_x4_trans(vaddr + tile_off(vrow, 2 * (4 * half + jj) + (mi >> 1)), vb[jj][0], vb[jj][1], vb[jj][2], vb[jj][3]);
+#pragma unroll
+              for (int jj = 0; jj < 4; ++jj) {
+                mma_bf16(oacc[2 * (4 * half + jj)], frag.x, frag.y, frag.z, frag.w, vb[jj][0], vb[jj][1]);
+                mma_bf16(oacc[2 * (4 * half + jj) + 1], frag.x, frag.y, frag.z, frag.w, vb[jj][2], vb[jj][3]);
+              }
             }
           }
+          if (!(d.flags & kFlagLast)) {
+            release();
+            if (!next_slot()) { alive = false; break; }
+            continue;
+          }
+          // ---------------- end of the item: stage this warp's partial result ----------------
+          {
+            const int buf = items_done & 1;
+            float* stage = reinterpret_cast<float*>(stages + buf * kStageBytes);
+            float* sm_m = stage + kConsumerWarps * 8 * kD;   // [warp][head]
+            float* sm_l = sm_m + kConsumerWarps * 8;         // [warp][head]
+            float* sm_hb = sm_l + kConsumerWarps * 8;        // [warp]
+            // the copy was last used two items ago; its merger signals when it is done with it
+            if (items_done >= 2 && !warp_mbar_wait(&stage_free[buf], ((items_done >> 1) - 1) & 1, &ctl[0], lane)) {
+              alive = false;
+              break;
+            }
+            float* mine = stage + (warp * 8 + head) * kD;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const int c = (4 * j + quad) ^ (4 * (head & 3));  // float2 slot, swizzled against bank conflicts
+              *reinterpret_cast<float2*>(mine + 2 * c) = make_float2(oacc[j][0] + oacc[j][2], oacc[j][1] + oacc[j][3]);
+            }
+            float ls = l_priv;
+            ls += __shfl_xor_sync(0xffffffffu, ls, 1);
+            ls += __shfl_xor_sync(0xffffffffu, ls, 2);
+            float hs = hb_priv;
+            hs += __shfl_xor_sync(0xffffffffu, hs, 1);
+            hs += __shfl_xor_sync(0xffffffffu, hs, 2);
+            if (quad == 0) {
+              sm_m[warp * 8 + head] = m_ref;
+              sm_l[warp * 8 + head] = ls;
+              if (head == 7) sm_hb[warp] = hs;
+            }
+            __syncwarp();
+            int arrived = 0;
+            if (lane == 0) {
+              __threadfence_block();
+              arrived = atomicAdd_block(&stage_cnt[buf], 1);
+              __threadfence_block();
+            }
+            arrived = __shfl_sync(0xffffffffu, arrived, 0);
+            if (arrived == kConsumerWarps - 1) {
+              // ---------- last warp of the CTA: merge the eight partial results into the item's record ----------
+              PartialRec* pr = pl.part + d.item;
+              float hb_tot = 0.f;
+#pragma unroll
+              for (int w = 0; w < kConsumerWarps; ++w) hb_tot += sm_hb[w];
+#pragma unroll 2
+              for (int hh = 0; hh < 8; ++hh) {
+                const bool brow = use_base && hh == 7;
+                float M = -INFINITY;
+#pragma unroll
+                for (int w = 0; w < kConsumerWarps; ++w) M = fmaxf(M, sm_m[w * 8 + hh]);
+                float L = 0.f;
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int w = 0; w < kConsumerWarps; ++w) {
+                  const float f = brow ? 1.f : fast_exp2(sm_m[w * 8 + hh] - M);
+                  L = fmaf(sm_l[w * 8 + hh], f, L);
+                  const float4 v = *reinterpret_cast<const float4*>(stage + (w * 8 + hh) * kD + 2 * ((2 * lane) ^ (4 * (hh & 3))));
+                  acc.x = fmaf(v.x, f, acc.x);
+                  acc.y = fmaf(v.y, f, acc.y);
+                  acc.z = fmaf(v.z, f, acc.z);
+                  acc.w = fmaf(v.w, f, acc.w);
+                }
+                *reinterpret_cast<float4*>(&pr->o[hh][4 * lane]) = acc;
+                if (lane == 0) { pr->m[hh] = M; pr->l[hh] = L; }
+              }
+              if (lane == 0) pr->hb = use_base ? hb_tot : 0.f;
+              __syncwarp();
+              int last_of_unit = 0;
+              if (lane == 0) {
+                stage_cnt[buf] = 0;
+                mbar_arrive(&stage_free[buf]);
+                __threadfence();
+                last_of_unit = (atomicAdd(&pl.counter[d.unit], 1) == d.nitems - 1) ? 1 : 0;
+                __threadfence();
+              }
+              last_of_unit = __shfl_sync(0xffffffffu, last_of_unit, 0);
+              if (last_of_unit) {
+                // ---------- last item of the unit: merge its records (this warp alone; lane = 4 channels) ----------
+                const PartialRec* p0 = pl.part + d.item0;
+                const int b = d.unit / dm.Hkv, h = d.unit % dm.Hkv;
+                float hbsum = 0.f;
+                for (int c = 0; c < d.nitems; ++c) hbsum += __ldcg(&p0[c].hb);
+                const float Htot = (softmax_counted ? (float)G : 0.f) + (use_base ? hbsum : 0.f);
+                FinalRec* fr = pl.fin + d.unit;
+                float4 xs = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int hh = 0; hh < 8; ++hh) {
+                  const bool brow = use_base && hh == 7;
+                  if (hh >= G && !brow) {
+                    if (lane == 0) { fr->m[hh] = 0.f; fr->inv_l[hh] = 0.f; }
+                    continue;
+                  }
+                  float mfin = -INFINITY;
+                  for (int c = 0; c < d.nitems; ++c) mfin = fmaxf(mfin, __ldcg(&p0[c].m[hh]));
+                  float lfin = 0.f;
+                  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+                  for (int c = 0; c < d.nitems; ++c) {
+                    const float f = brow ? 1.f : fast_exp2(__ldcg(&p0[c].m[hh]) - mfin);
+                    lfin = fmaf(__ldcg(&p0[c].l[hh]), f, lfin);
+                    const float4 v = __ldcg(reinterpret_cast<const float4*>(&p0[c].o[hh][4 * lane]));
+                    acc.x = fmaf(v.x, f, acc.x);
+                    acc.y = fmaf(v.y, f, acc.y);
+                    acc.z = fmaf(v.z, f, acc.z);
+                    acc.w = fmaf(v.w, f, acc.w);
+                  }
+                  if (brow) {
+                    xs.x += acc.x; xs.y += acc.y; xs.z += acc.z; xs.w += acc.w;
+                    if (lane == 0) { fr->m[hh] = 0.f; fr->inv_l[hh] = 0.f; }
+                  } else {
+                    const float inv_l = 1.f / lfin;
+                    const float4 on = make_float4(acc.x * inv_l, acc.y * inv_l, acc.z * inv_l, acc.w * inv_l);
+                    *reinterpret_cast<float4*>(o + ((size_t)b * dm.Hq + h * G + hh) * kD + 4 * lane) = on;
+                    if (softmax_counted) { xs.x += on.x; xs.y += on.y; xs.z += on.z; xs.w += on.w; }
+                    if (lane == 0) { fr->m[hh] = mfin; fr->inv_l[hh] = inv_l; }
+                  }
+                }
+                const float inv_h = (Htot > 0.f) ? 1.f / Htot : 0.f;
+                const float4 X = make_float4(xs.x * inv_h, xs.y * inv_h, xs.z * inv_h, xs.w * inv_h);
+                *reinterpret_cast<float4*>(&fr->X[4 * lane]) = X;
+                const float xx = warp_sum(fmaf(X.x, X.x, X.y * X.y) + fmaf(X.z, X.z, X.w * X.w));
+                if (lane == 0) { fr->H = Htot; fr->XX = xx; }
+                __syncwarp();
+                if (lane == 0) {
+                  __threadfence();
+                  st_release(&pl.ready[d.unit], 1);
+                }
+              }
+            }
+            ++items_done;
+          }
+          release();
+          break;
+        }
+      } else if (d.type == kSlotVB) {
+        // =============================== one B item ===============================
+        for (;;) {
+          if (d.type != kSlotVB) { alive = false; break; }
+          // ||X - v_j||^2 = ||v_j||^2 - 2 <v_j, X> + ||X||^2 for this warp's 16 tokens on the tensor
+          // cores: the V rows are the A operand; used again as the B operand they give the Gram
+          // blocks whose diagonals are ||v_j||^2; X, split into bf16 hi + lo columns, gives <v_j, X>.
+          // Tokens for which that difference cancels (v_j close to X) or that hold most of the weight
+          // are redone below by plain subtraction, so v_j = X still scores exactly 0.
+          const char* sl = tiles + s * kTileBytes;
+          const float* side = reinterpret_cast<const float*>(sides + s * kSideBytes);
+          const FinalRec* fr = reinterpret_cast<const FinalRec*>(side + 8 * kT);
+          float ca[4] = {0.f, 0.f, 0.f, 0.f}, cb[4] = {0.f, 0.f, 0.f, 0.f}, cx[4] = {0.f, 0.f, 0.f, 0.f};
+          {
+            const uint32_t vaddr = smem_u32(sl);
+            const int tok = 16 * warp + 8 * (mi & 1) + mr;
+            uint32_t va[8][4];
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks)
+              ldmatrix_x4(vaddr + tile_off(tok, 2 * ks + (mi >> 1)), va[ks][0], va[ks][1], va[ks][2], va[ks][3]);
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+              uint32_t x0 = 0u, x1 = 0u;
+              if (head < 2) {
+                const float2 f0 = *reinterpret_cast<const float2*>(fr->X + 16 * ks + 2 * quad);
+                const float2 f1 = *reinterpret_cast<const float2*>(fr->X + 16 * ks + 8 + 2 * quad);
+                uint32_t h0, l0, h1, l1;
+                split_pair(f0.x, f0.y, h0, l0);
+                split_pair(f1.x, f1.y, h1, l1);
+                x0 = head == 0 ? h0 : l0;
+                x1 = head == 0 ? h1 : l1;
+              }
+              mma_bf16(ca, va[ks][0], va[ks][1], va[ks][2], va[ks][3], va[ks][0], va[ks][2]);  // x tokens 0..7
+              mma_bf16(cb, va[ks][0], va[ks][1], va[ks][2], va[ks][3], va[ks][1], va[ks][3]);  // x tokens 8..15
+              mma_bf16(cx, va[ks][0], va[ks][1], va[ks][2], va[ks][3], x0, x1);
+            }
+          }
+          // lane (head, quad): token `head` of the warp if quad == 0, token head + 8 if quad == 1
+          const int src = (lane & ~3) | (head >> 1);
+          const float vva = __shfl_sync(0xffffffffu, (head & 1) ? ca[1] : ca[0], src);
+          const float vvb = __shfl_sync(0xffffffffu, (head & 1) ? cb[3] : cb[2], src);
+          const float vxa = __shfl_sync(0xffffffffu, cx[0] + cx[1], lane & ~3);
+          const float vxb = __shfl_sync(0xffffffffu, cx[2] + cx[3], lane & ~3);
+          // base score: heads quad and quad + 4 of both tokens, then a sum over the quad
+          const int ra = 16 * warp + head, rb = ra + 8;
+          float ha = 0.f, hbv = 0.f;
+          if (softmax_counted) {
+#pragma unroll
+            for (int gg = 0; gg < 2; ++gg) {
+              const int g = quad + 4 * gg;
+              if (g < G) {
+                const float mg = fr->m[g], il = fr->inv_l[g];
+                ha = fmaf(fast_exp2(side[g * kT + ra] - mg), il, ha);
+                hbv = fmaf(fast_exp2(side[g * kT + rb] - mg), il, hbv);
+              }
+            }
+            ha += __shfl_xor_sync(0xffffffffu, ha, 1);
+            ha += __shfl_xor_sync(0xffffffffu, ha, 2);
+            hbv += __shfl_xor_sync(0xffffffffu, hbv, 1);
+            hbv += __shfl_xor_sync(0xffffffffu, hbv, 2);
+          }
+          const int row = quad == 0 ? ra : rb;
+          const bool mine = quad < 2 && row < d.n_valid;
+          float hj = quad == 0 ? ha : hbv;
+          const float vv = quad == 0 ? vva : vvb, vx = quad == 0 ? vxa : vxb;
+          const size_t slot = (size_t)d.unit * dm.cap + (size_t)d.tile * kT + row;
+          if (mine) {
+            if (mode == CAOTE_BASE_ACCUM) {
+              hj += side[7 * kT + row];
+              base[slot] = hj;
+            } else if (mode == CAOTE_BASE_EXTERNAL) {
+              hj = side[7 * kT + row];
+            }
+          }
+          const float Htot = fr->H, XX = fr->XX;
+          float n2 = fmaxf(vv - 2.f * vx + XX, 0.f);
+          const bool redo = mine && (n2 < 2e-3f * (vv + XX) || 2.f * hj > Htot);
+          unsigned todo = __ballot_sync(0xffffffffu, redo);
+          while (todo) {
+            const int l = __ffs((int)todo) - 1;
+            todo &= todo - 1;
+            const int rr = 16 * warp + (l >> 2) + 8 * (l & 3);  // the row lane l is responsible for
+            const uint2 raw = *reinterpret_cast<const uint2*>(sl + tile_off(rr, lane >> 1) + (lane & 1) * 8);
+            const float4 xv = *reinterpret_cast<const float4*>(fr->X + 4 * lane);
+            const float2 f0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
+            const float2 f1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
+            const float d0 = xv.x - f0.x, d1 = xv.y - f0.y, d2 = xv.z - f1.x, d3 = xv.w - f1.y;
+            const float exact = warp_sum(fmaf(d0, d0, d1 * d1) + fmaf(d2, d2, d3 * d3));
+            if (lane == l) n2 = exact;
+          }
+          if (mine) {
+            float ratio = 0.f;
+            if (Htot > 0.f) {
+              const float rest = Htot - hj;
+              ratio = (rest > 0.f) ? hj / rest : INFINITY;
+            }
+            scores[slot] = (ratio == 0.f) ? 0.f : ((ratio == INFINITY) ? INFINITY : ratio * sqrtf(n2));
+          }
+          const bool last = (d.flags & kFlagLast) != 0;
+          release();
+          if (last) break;
+          if (!next_slot()) { alive = false; break; }
         }
       } else {
-        // ===================== score pass of one tile =====================
-        // ||X - v_j||^2 = ||v_j||^2 - 2 <v_j, X> + ||X||^2 for this warp's 16 tokens on the tensor
-        // cores: the V rows are the A operand; used again as the B operand they give the Gram
-        // blocks whose diagonals are ||v_j||^2; X, split into bf16 hi + lo columns, gives <v_j, X>.
-        // Tokens for which that difference cancels (v_j close to X) or that hold most of the weight
-        // are redone below by plain subtraction, so v_j = X still scores exactly 0.
-        const FinalRec* fr = reinterpret_cast<const FinalRec*>(side + 8 * kT);
-        uint32_t xb[8][2];
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-          xb[ks][0] = 0u;
-          xb[ks][1] = 0u;
-          if (head < 2) {
-            const float2 x0 = *reinterpret_cast<const float2*>(fr->X + 16 * ks + 2 * quad);
-            const float2 x1 = *reinterpret_cast<const float2*>(fr->X + 16 * ks + 8 + 2 * quad);
-            uint32_t h0, l0, h1, l1;
-            split_pair(x0.x, x0.y, h0, l0);
-            split_pair(x1.x, x1.y, h1, l1);
-            xb[ks][0] = head == 0 ? h0 : l0;
-            xb[ks][1] = head == 0 ? h1 : l1;
-          }
-        }
-        float ca[4] = {0.f, 0.f, 0.f, 0.f}, cb[4] = {0.f, 0.f, 0.f, 0.f}, cx[4] = {0.f, 0.f, 0.f, 0.f};
-        {
-          const uint32_t vaddr = smem_u32(sl);
-          const int mi = lane >> 3, r = lane & 7;
-          const int tok = 16 * warp + 8 * (mi & 1) + r;
-#pragma unroll
-          for (int ks = 0; ks < 8; ++ks) {
-            uint32_t a0, a1, a2, a3;
-            ldmatrix_x4(vaddr + tile_off(tok, 2 * ks + (mi >> 1)), a0, a1, a2, a3);
-            mma_bf16(ca, a0, a1, a2, a3, a0, a2);  // rows x tokens 0..7 of the warp
-            mma_bf16(cb, a0, a1, a2, a3, a1, a3);  // rows x tokens 8..15
-            mma_bf16(cx, a0, a1, a2, a3, xb[ks][0], xb[ks][1]);
-          }
-        }
-        // lane (head, quad): token `head` of the warp if quad == 0, token head + 8 if quad == 1
-        const int src = (lane & ~3) | (head >> 1);
-        const float vva = __shfl_sync(0xffffffffu, (head & 1) ? ca[1] : ca[0], src);
-        const float vvb = __shfl_sync(0xffffffffu, (head & 1) ? cb[3] : cb[2], src);
-        const float vxa = __shfl_sync(0xffffffffu, cx[0] + cx[1], lane & ~3);
-        const float vxb = __shfl_sync(0xffffffffu, cx[2] + cx[3], lane & ~3);
-        // base score: heads quad and quad + 4 of both tokens, then a sum over the quad
-        const int ra = 16 * warp + head, rb = ra + 8;
-        float ha = 0.f, hbv = 0.f;
-        if (softmax_counted) {
-#pragma unroll
-          for (int gg = 0; gg < 2; ++gg) {
-            const int g = quad + 4 * gg;
-            if (g < G) {
-              const float mg = fr->m[g], il = fr->inv_l[g];
-              ha = fmaf(fast_exp2(side[g * kT + ra] - mg), il, ha);
-              hbv = fmaf(fast_exp2(side[g * kT + rb] - mg), il, hbv);
-            }
-          }
-          ha += __shfl_xor_sync(0xffffffffu, ha, 1);
-          ha += __shfl_xor_sync(0xffffffffu, ha, 2);
-          hbv += __shfl_xor_sync(0xffffffffu, hbv, 1);
-          hbv += __shfl_xor_sync(0xffffffffu, hbv, 2);
-        }
-        const int row = quad == 0 ? ra : rb;
-        const bool mine = quad < 2 && row < d.n_valid;
-        float hj = quad == 0 ? ha : hbv;
-        const float vv = quad == 0 ? vva : vvb, vx = quad == 0 ? vxa : vxb;
-        const size_t slot = (size_t)d.unit * dm.cap + (size_t)d.tile * kT + row;
-        if (mine) {
-          if (mode == CAOTE_BASE_ACCUM) {
-            hj += side[7 * kT + row];
-            base[slot] = hj;
-          } else if (mode == CAOTE_BASE_EXTERNAL) {
-            hj = side[7 * kT + row];
-          }
-        }
-        const float Htot = fr->H, XX = fr->XX;
-        float n2 = fmaxf(vv - 2.f * vx + XX, 0.f);
-        const bool redo = mine && (n2 < 2e-3f * (vv + XX) || 2.f * hj > Htot);
-        unsigned todo = __ballot_sync(0xffffffffu, redo);
-        while (todo) {
-          const int l = __ffs((int)todo) - 1;
-          todo &= todo - 1;
-          const int rr = 16 * warp + (l >> 2) + 8 * (l & 3);  // the row lane l is responsible for
-          const uint2 raw = *reinterpret_cast<const uint2*>(sl + tile_off(rr, lane >> 1) + (lane & 1) * 8);
-          const float4 xv = *reinterpret_cast<const float4*>(fr->X + 4 * lane);
-          const float2 f0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
-          const float2 f1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
-          const float d0 = xv.x - f0.x, d1 = xv.y - f0.y, d2 = xv.z - f1.x, d3 = xv.w - f1.y;
-          const float exact = warp_sum(fmaf(d0, d0, d1 * d1) + fmaf(d2, d2, d3 * d3));
-          if (lane == l) n2 = exact;
-        }
-        if (mine) {
-          float ratio = 0.f;
-          if (Htot > 0.f) {
-            const float rest = Htot - hj;
-            ratio = (rest > 0.f) ? hj / rest : INFINITY;
-          }
-          scores[slot] = (ratio == 0.f) ? 0.f : ((ratio == INFINITY) ? INFINITY : ratio * sqrtf(n2));
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&empty[s]);
+        alive = false;
       }
+    }
+    if (!alive && lane == 0 && !ctl[0]) {
+      set_status(status, CAOTE_ERR_TIMEOUT);
+      ctl[0] = 1;
     }
   }
 
