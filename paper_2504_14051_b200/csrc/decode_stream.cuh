@@ -1,28 +1,32 @@
 // Single-query (decode) scoring path for bf16, head_dim 128, group size <= 8: one persistent kernel
 // that reads K and V from HBM once and takes the second pass over V out of L2.
 //
-// Work list. A unit's cached tokens are cut into tiles of kT tokens and items of `tpi` consecutive
-// tiles. Every item appears twice in one global, statically ordered work list:
+// Work. A unit's cached tokens are cut into tiles of kT tokens and items of `tpi` consecutive tiles.
+// Every item is processed twice:
 //   A(i)  attention pass: logits of the G group heads (tensor cores, mma.sync bf16), online softmax
 //         over the item's tiles, partial output sum_j p_j v_j; the logits go to a scratch array, the
-//         (max, sum, partial output) record to another; the CTA that completes a unit's last A item
-//         merges the records into the final softmax statistics, the attention output o and the
-//         reference vector X, and raises the unit's ready flag;
-//   B(i)  score pass: re-reads the item's V tiles (still in L2: B(i) trails A(i) by `lag` items, a few
-//         tens of MB) and its logits, and writes c_j = w_j / (1 - w_j) * ||X - v_j|| once.
-// The list is A(0..lag-1), then B(0), A(lag), B(1), A(lag+1), ..., then the remaining B items. CTAs
-// take entries with one atomic counter, so a CTA that is busy merging simply takes fewer entries.
+//         item's (max, sum, partial output) record to another;
+//   B(i)  score pass: re-reads the item's V tiles (from L2: B work of a unit becomes available as
+//         soon as the unit's records are merged and is taken before any further A work) and its
+//         logits, and writes c_j = w_j / (1 - w_j) * ||X - v_j|| once.
+// A items are handed out in order by one atomic counter. When the last record of a unit is written,
+// the CTA that wrote it merges the unit's records into the final softmax statistics, the attention
+// output o and the reference vector X, and appends the unit's B items to a global queue. Nothing
+// ever waits for another CTA except at the very end (A work exhausted, last merges in flight).
 //
-// Inside a CTA one producer warp walks the work list and fills a ring of shared-memory slots by TMA
-// (a K tile, a V tile, or a V tile plus the tile's logits and carried base scores); eight consumer
-// warps process the slots in order. Full/empty mbarriers hand the slots back and forth.
-//
-// Waits. B(i) needs its unit's ready flag. `lag` is at least the number of items of the longest
-// unit, so every A item of that unit was taken from the list before B(i) was, by a CTA that is
-// running and that only has earlier list entries in front of it; by induction over the list order
-// every flag is raised. No co-residency of the whole grid is needed. Every wait is still bounded by a
-// clock limit; when one runs out the CTA records CAOTE_ERR_TIMEOUT, stops taking work, lets its own
-// copies land and returns.
+// Inside a CTA (one per SM):
+//   producer warp   claims work (B first, then A) and fills a ring of shared-memory slots by TMA:
+//                   a K tile (+ q, + carried base scores), a V tile, or a V tile with the tile's
+//                   logits, base scores and the unit's final record;
+//   8 consumer warps process the slots in order, each on its own 16 tokens of every tile, with its
+//                   own softmax reference and full-width output accumulator (P never leaves the
+//                   registers); at the end of an item they merge their partial results through a
+//                   staging area in shared memory, one head per warp;
+//   merge warp      counts finished records per unit, merges a completed unit, publishes its B items.
+// Full/empty mbarriers hand slots back and forth; every wait in the kernel is bounded by a clock
+// limit, after which the CTA records CAOTE_ERR_TIMEOUT, stops taking work, lets its own copies land
+// and returns. No hardware barrier is used after start-up, so a warp that gives up cannot strand
+// its siblings.
 //
 // For the base modes that carry a score (ACCUM, EXTERNAL; G <= 7) row 7 of the P operand carries
 // base_j, which yields sum_j base_j v_j from the same tensor-core product.
@@ -40,18 +44,21 @@ constexpr int kD = 128;
 constexpr int kSlots = 4;
 constexpr int kConsumerWarps = 8;
 constexpr int kConsumers = kConsumerWarps * 32;
-constexpr int kThreads = kConsumers + 32;  // + one producer warp
+constexpr int kProducerWarp = kConsumerWarps;
+constexpr int kMergeWarp = kConsumerWarps + 1;
+constexpr int kThreads = kConsumers + 64;  // + producer warp + merge warp
 constexpr int kHalfBytes = kT * 128;       // one 64-channel box: kT rows of 128 bytes
 constexpr int kTileBytes = 2 * kHalfBytes;
-constexpr int kRowsBytes = 8 * kT * 4;     // per slot: 8 rows of kT floats (logits / base / q / P fragments)
+constexpr int kRowsBytes = 8 * kT * 4;     // per slot: 8 rows of kT floats (logits / base / q)
 constexpr int kMaxTilesPerItem = 8;
+constexpr int kJobs = 8;                   // mailbox entries between the consumers and the merge warp
 constexpr long long kWaitCycles = 2000000000LL;  // ~1 s: far beyond any legitimate wait
 
 enum SlotType { kSlotKA = 0, kSlotVA = 1, kSlotVB = 2, kSlotStop = 3 };
 enum { kFlagFirst = 1, kFlagLast = 2 };
 
 struct PartialRec {   // per item
-  float m[8];         // running max of the log2-domain logits per head
+  float m[8];         // reference of the log2-domain logits per head
   float l[8];         // sum of 2^(s - m)
   float hb;           // sum of the carried base scores of the item
   float pad[7];
@@ -73,29 +80,27 @@ struct Desc {         // what a slot holds
 };
 
 struct Plan {
-  int* item_prefix;   // [units + 1] exclusive prefix of items per unit
-  int* counter;       // [units] A items of the unit whose records are written
-  int* ready;         // [units] 1 once FinalRec is written
-  int* work;          // [1] next entry of the work list
-  PartialRec* part;   // [max items]
-  FinalRec* fin;      // [units]
-  float* S;           // [units][G][capS] log2-domain logits
-  int tpi;            // tiles per item
-  int capS;           // cap rounded up to a multiple of kT
-  int lag;            // items by which the score pass trails the attention pass
+  int* item_prefix;        // [units + 1] exclusive prefix of items per unit
+  int* counter;            // [units] records of the unit that are written
+  int* ctr;                // [0] next A item, [1] B entries claimed, [2] B entries reserved
+  unsigned long long* bq;  // [max items] B queue: (unit << 32) | (item + 1), 0 = not yet written
+  PartialRec* part;        // [max items]
+  FinalRec* fin;           // [units]
+  float* S;                // [units][G][capS] log2-domain logits
+  int tpi;                 // tiles per item
+  int capS;                // cap rounded up to a multiple of kT
+  int max_items;
 };
 
 inline int tiles_per_item(const Dims& dm, int grid) {
   const long long max_tiles = (long long)dm.units * ((dm.cap + kT - 1) / kT);
-  long long t = max_tiles / (2LL * (grid > 0 ? grid : 1));
+  long long t = max_tiles / (4LL * (grid > 0 ? grid : 1));
   if (t < 1) t = 1;
   if (t > kMaxTilesPerItem) t = kMaxTilesPerItem;
   return (int)t;
 }
 
-// `grid` only shapes the item size and the lag; the carve must be called with the same value by
-// caote_workspace_bytes and by the launch (both use the resident-CTA count, or 0 without a device:
-// the sizes below are upper bounds for every grid because tpi >= 1).
+// `grid` only shapes the item size; the sizes below hold for every grid (they assume tpi = 1).
 inline size_t carve(const Dims& dm, char* base, Plan* out, int grid) {
   size_t off = 0;
   auto take = [&](size_t bytes) {
@@ -107,12 +112,12 @@ inline size_t carve(const Dims& dm, char* base, Plan* out, int grid) {
   const int tiles_per_unit = (dm.cap + kT - 1) / kT;
   pl.tpi = tiles_per_item(dm, grid);
   pl.capS = tiles_per_unit * kT;
-  pl.lag = (tiles_per_unit + pl.tpi - 1) / pl.tpi + (grid > 0 ? grid : 1);
-  const size_t max_items = (size_t)dm.units * tiles_per_unit;  // sized for tpi = 1
+  const size_t max_items = (size_t)dm.units * tiles_per_unit;
+  pl.max_items = (int)max_items;
   pl.item_prefix = (int*)take(sizeof(int) * ((size_t)dm.units + 1));
   pl.counter = (int*)take(sizeof(int) * (size_t)dm.units);
-  pl.ready = (int*)take(sizeof(int) * (size_t)dm.units);
-  pl.work = (int*)take(sizeof(int) * 4);
+  pl.ctr = (int*)take(sizeof(int) * 4);
+  pl.bq = (unsigned long long*)take(sizeof(unsigned long long) * max_items);
   pl.fin = (FinalRec*)take(sizeof(FinalRec) * (size_t)dm.units);
   pl.S = (float*)take(sizeof(float) * (size_t)dm.units * dm.G * pl.capS);
   pl.part = (PartialRec*)take(sizeof(PartialRec) * max_items);
@@ -121,22 +126,29 @@ inline size_t carve(const Dims& dm, char* base, Plan* out, int grid) {
 }
 
 // Staging area in which the eight consumer warps put their partial results at the end of an item
-// (two copies, used by alternate items): per warp 8 heads x kD floats, then max, sum and base sum.
+// (two copies, used by alternate items): per warp 8 heads x kD floats, then reference, sum, base sum.
 constexpr int kStageFloats = kConsumerWarps * 8 * kD + 2 * kConsumerWarps * 8 + kConsumerWarps;
 constexpr int kStageBytes = (kStageFloats * 4 + 255) / 256 * 256;
 
+struct Job {  // a finished record, handed to the merge warp
+  int seq, unit, item0, nitems;
+};
+
 inline size_t smem_bytes() {
   return 1024 /* alignment slack */ + (size_t)kSlots * (kTileBytes + kSideBytes) + 2 * (size_t)kStageBytes +
-         sizeof(Desc) * kSlots + 8 * (2 * kSlots + 2) + 64;
+         sizeof(Desc) * kSlots + sizeof(Job) * kJobs + 8 * (2 * kSlots + 4) + 64;
 }
 
-// ---- plan: items per unit, their prefix sum, and cleared counters / flags (one CTA) -------------
+// ---- plan: items per unit, their prefix sum, and cleared counters and queue ----------------------
+// grid = any number of CTAs of 1024 threads; CTA 0 computes the prefix, all clear the queue.
 __global__ void __launch_bounds__(1024)
 plan_kernel(int units, int Hkv, int cap, const int* __restrict__ len, Plan pl, int* status) {
   __shared__ int warp_tot[32];
   __shared__ int carry;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (tid == 0) { carry = 0; pl.item_prefix[0] = 0; pl.work[0] = 0; }
+  for (int i = blockIdx.x * 1024 + tid; i < pl.max_items; i += gridDim.x * 1024) pl.bq[i] = 0ull;
+  if (blockIdx.x != 0) return;
+  if (tid == 0) { carry = 0; pl.item_prefix[0] = 0; pl.ctr[0] = 0; pl.ctr[1] = 0; pl.ctr[2] = 0; }
   __syncthreads();
   for (int u0 = 0; u0 < units; u0 += 1024) {
     const int u = u0 + tid;
@@ -146,7 +158,6 @@ plan_kernel(int units, int Hkv, int cap, const int* __restrict__ len, Plan pl, i
       if (n < 0 || n > cap) set_status(status, CAOTE_ERR_BAD_LENGTH);
       else ni = ((n + kT - 1) / kT + pl.tpi - 1) / pl.tpi;
       pl.counter[u] = 0;
-      pl.ready[u] = 0;
     }
     int incl = ni;
 #pragma unroll
@@ -297,18 +308,21 @@ __device__ __forceinline__ uint32_t tile_off(int row, int chunk16) {
   return (uint32_t)((chunk16 >> 3) * kHalfBytes + row * 128 + (((chunk16 & 7) ^ (row & 7)) << 4));
 }
 
-// Entry w of the work list -> (is_B, item). N items, lag L (see the file comment).
-__device__ __forceinline__ void work_entry(int w, int N, int L, bool& is_b, int& item) {
-  if (L > N) L = N;
-  if (w < L) { is_b = false; item = w; return; }
-  if (w < 2 * N - L) {
-    const int r = w - L;
-    is_b = (r & 1) == 0;
-    item = is_b ? (r >> 1) : (L + (r >> 1));
-    return;
-  }
-  is_b = true;
-  item = w - N;
+__device__ __forceinline__ int lds_acquire(const volatile int* p) {
+  int v;
+  asm volatile("ld.acquire.cta.shared::cta.s32 %0, [%1];" : "=r"(v) : "r"(smem_u32(const_cast<const int*>(p))) : "memory");
+  return v;
+}
+__device__ __forceinline__ void sts_release(volatile int* p, int v) {
+  asm volatile("st.release.cta.shared::cta.s32 [%0], %1;" ::"r"(smem_u32(const_cast<int*>(p))), "r"(v) : "memory");
+}
+__device__ __forceinline__ unsigned long long ld_acquire64(const unsigned long long* p) {
+  unsigned long long v;
+  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release64(unsigned long long* p, unsigned long long v) {
+  asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -321,11 +335,14 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
   char* sides = tiles + kSlots * kTileBytes;                                     // [kSlots][kSideBytes]
   char* stages = sides + kSlots * kSideBytes;                                    // [2][kStageBytes]
   Desc* desc = reinterpret_cast<Desc*>(stages + 2 * kStageBytes);                // [kSlots]
-  uint64_t* full = reinterpret_cast<uint64_t*>(desc + kSlots);                   // [kSlots]
+  Job* jobs = reinterpret_cast<Job*>(desc + kSlots);                             // [kJobs]
+  uint64_t* full = reinterpret_cast<uint64_t*>(jobs + kJobs);                    // [kSlots]
   uint64_t* empty = full + kSlots;                                               // [kSlots]
-  uint64_t* stage_free = empty + kSlots;                                         // [2]
-  volatile int* ctl = reinterpret_cast<volatile int*>(stage_free + 2);           // [0] stop, [2] slots issued,
-  int* stage_cnt = const_cast<int*>(ctl) + 4;                                    // [2] warps that have staged
+  uint64_t* stage_full = empty + kSlots;                                         // [2]
+  uint64_t* stage_free = stage_full + 2;                                         // [2]
+  // [0] stop, [2] slots issued, [3] jobs taken by the merge warp, [4] consumer warps that have left,
+  // [5] jobs posted in total, [6..7] warps that finished merging their head (per staging copy)
+  volatile int* ctl = reinterpret_cast<volatile int*>(stage_free + 2);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int G = dm.G, mode = dm.base_mode;
@@ -339,21 +356,20 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
       mbar_init(&full[i], 1);
       mbar_init(&empty[i], kConsumerWarps);
     }
-    mbar_init(&stage_free[0], 1);
-    mbar_init(&stage_free[1], 1);
-    ctl[0] = 0;
-    ctl[1] = 0;
-    ctl[2] = 0;
-    stage_cnt[0] = 0;
-    stage_cnt[1] = 0;
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&stage_full[i], kConsumerWarps);
+      mbar_init(&stage_free[i], kConsumerWarps);
+    }
+    for (int i = 0; i < 8; ++i) ctl[i] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (tid < kSlots * (int)(sizeof(Desc) / sizeof(int))) reinterpret_cast<int*>(desc)[tid] = 0;
+  if (tid < kJobs * (int)(sizeof(Job) / sizeof(int))) reinterpret_cast<int*>(jobs)[tid] = 0;
   __syncthreads();
 
   int consumed = 0;  // slots this warp has finished
 
-  if (warp == kConsumerWarps) {
+  if (warp == kProducerWarp) {
     // ================================ producer warp ================================
     const uint64_t pol_stream = policy_evict_first(), pol_keep = policy_evict_last();
     int issued = 0;
@@ -363,39 +379,61 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
       return mbar_wait(&empty[s], ((issued / kSlots) & 1) ^ 1, &ctl[0]);
     };
     while (ok) {
-      int w = 0;
-      if (lane == 0) w = atomicAdd(pl.work, 1);
-      w = __shfl_sync(0xffffffffu, w, 0);
-      if (w >= 2 * N) break;
-      bool is_b;
-      int item;
-      work_entry(w, N, pl.lag, is_b, item);
-      // unit of the item: 32-ary search over the item prefix, one probe per lane
-      int lo = 0, hi = dm.units;
-      while (hi - lo > 1) {
-        const int step = (hi - lo + 31) / 32;
-        const int probe = lo + lane * step;
-        const int val = (probe < hi) ? __ldg(pl.item_prefix + probe) : 0x7fffffff;
-        const unsigned mask = __ballot_sync(0xffffffffu, val <= item);
-        const int k = 31 - __clz((int)mask);
-        lo = lo + k * step;
-        hi = min(hi, lo + step);
+      // ---- claim work: a published B item if there is one, else the next A item
+      int kind = 0, item = 0, u = 0;  // kind: 0 = all work handed out, 1 = A, 2 = B, -1 = gave up
+      if (lane == 0) {
+        const long long t0c = clock64();
+        for (;;) {
+          const int bh = *reinterpret_cast<volatile int*>(&pl.ctr[1]);
+          const int bt = ld_acquire(&pl.ctr[2]);
+          if (bh < bt) {
+            if (atomicCAS(&pl.ctr[1], bh, bh + 1) != bh) continue;
+            unsigned long long e = ld_acquire64(&pl.bq[bh]);
+            while (e == 0ull) {  // reserved, about to be written
+              if (ctl[0] || clock64() - t0c > kWaitCycles) break;
+              __nanosleep(32);
+              e = ld_acquire64(&pl.bq[bh]);
+            }
+            if (e == 0ull) { kind = -1; break; }
+            u = (int)(e >> 32);
+            item = (int)(e & 0xffffffffull) - 1;
+            kind = 2;
+            break;
+          }
+          if (*reinterpret_cast<volatile int*>(&pl.ctr[0]) < N) {
+            const int a = atomicAdd(&pl.ctr[0], 1);
+            if (a < N) { item = a; kind = 1; break; }
+          }
+          if (bh >= N) { kind = 0; break; }
+          if (ctl[0] || clock64() - t0c > kWaitCycles) { kind = -1; break; }
+          __nanosleep(128);
+        }
       }
-      const int u = lo;
+      kind = __shfl_sync(0xffffffffu, kind, 0);
+      item = __shfl_sync(0xffffffffu, item, 0);
+      u = __shfl_sync(0xffffffffu, u, 0);
+      if (kind <= 0) { ok = (kind == 0); break; }
+      const bool is_b = kind == 2;
+      if (!is_b) {
+        // unit of the item: 32-ary search over the item prefix, one probe per lane
+        int lo = 0, hi = dm.units;
+        while (hi - lo > 1) {
+          const int step = (hi - lo + 31) / 32;
+          const int probe = lo + lane * step;
+          const int val = (probe < hi) ? __ldg(pl.item_prefix + probe) : 0x7fffffff;
+          const unsigned mask = __ballot_sync(0xffffffffu, val <= item);
+          const int k = 31 - __clz((int)mask);
+          lo = lo + k * step;
+          hi = min(hi, lo + step);
+        }
+        u = lo;
+      }
       if (lane == 0) {
         const int item0 = pl.item_prefix[u], nitems = pl.item_prefix[u + 1] - item0;
         const int n = len[u / dm.Hkv];
         const int ntiles = (n + kT - 1) / kT;
         const int t_begin = (item - item0) * pl.tpi, t_end = min(t_begin + pl.tpi, ntiles);
-        if (is_b) {
-          // the item's logits and the unit's final record must be complete before they are copied
-          const long long t0c = clock64();
-          while (ld_acquire(&pl.ready[u]) == 0) {
-            if (ctl[0] || clock64() - t0c > kWaitCycles) { ok = false; break; }
-            __nanosleep(64);
-          }
-          fence_async_all();
-        }
+        if (is_b) fence_async_all();  // the logits and the final record were written by ordinary stores
         for (int t = t_begin; ok && t < t_end; ++t) {
           Desc d;
           d.unit = u;
@@ -471,10 +509,124 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         ctl[0] = 1;
       }
     }
+  } else if (warp == kMergeWarp) {
+    // ================================ merge warp ================================
+    int idx = 0;
+    long long t_idle = clock64();
+    for (;;) {
+      int state = 0;  // 1 = a job is waiting, 2 = all done, 3 = give up
+      if (lane == 0) {
+        if (lds_acquire(&jobs[idx % kJobs].seq) == idx + 1) state = 1;
+        else if (lds_acquire(&ctl[4]) == kConsumerWarps && ctl[5] == idx) state = 2;
+        else if (ctl[0]) state = 2;
+        else if (clock64() - t_idle > kWaitCycles) state = 3;
+      }
+      state = __shfl_sync(0xffffffffu, state, 0);
+      if (state == 2) break;
+      if (state == 3) {
+        if (lane == 0) { set_status(status, CAOTE_ERR_TIMEOUT); ctl[0] = 1; }
+        break;
+      }
+      if (state == 0) { __nanosleep(100); continue; }
+      const int unit = jobs[idx % kJobs].unit, item0 = jobs[idx % kJobs].item0, nitems = jobs[idx % kJobs].nitems;
+      __syncwarp();
+      ++idx;
+      if (lane == 0) sts_release(&ctl[3], idx);  // the mailbox entry may be reused
+      t_idle = clock64();
+      int last_of_unit = 0;
+      if (lane == 0) {
+        __threadfence();
+        last_of_unit = (atomicAdd(&pl.counter[unit], 1) == nitems - 1) ? 1 : 0;
+        __threadfence();
+      }
+      last_of_unit = __shfl_sync(0xffffffffu, last_of_unit, 0);
+      if (!last_of_unit) continue;
+
+      // ---------- the unit's last record is in: merge its records (lane = 4 channels) ----------
+      const PartialRec* p0 = pl.part + item0;
+      const int b = unit / dm.Hkv, h = unit % dm.Hkv;
+      float M[8], L[8], hbsum = 0.f;
+#pragma unroll
+      for (int hh = 0; hh < 8; ++hh) { M[hh] = -INFINITY; L[hh] = 0.f; }
+      for (int c0 = 0; c0 < nitems; c0 += 32) {
+        const int c = c0 + lane;
+        if (c < nitems) {
+#pragma unroll
+          for (int hh = 0; hh < 8; ++hh) M[hh] = fmaxf(M[hh], __ldcg(&p0[c].m[hh]));
+        }
+      }
+#pragma unroll
+      for (int hh = 0; hh < 8; ++hh) M[hh] = warp_max(M[hh]);
+      for (int c0 = 0; c0 < nitems; c0 += 32) {
+        const int c = c0 + lane;
+        if (c < nitems) {
+#pragma unroll
+          for (int hh = 0; hh < 8; ++hh)
+            L[hh] = fmaf(__ldcg(&p0[c].l[hh]), fast_exp2(__ldcg(&p0[c].m[hh]) - M[hh]), L[hh]);
+          hbsum += __ldcg(&p0[c].hb);
+        }
+      }
+#pragma unroll
+      for (int hh = 0; hh < 8; ++hh) L[hh] = warp_sum(L[hh]);
+      hbsum = warp_sum(hbsum);
+      float4 acc[8];
+#pragma unroll
+      for (int hh = 0; hh < 8; ++hh) acc[hh] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 2
+      for (int c = 0; c < nitems; ++c) {
+        float f[8];
+        float4 v[8];
+#pragma unroll
+        for (int hh = 0; hh < 8; ++hh) {
+          f[hh] = __ldcg(&p0[c].m[hh]);
+          v[hh] = __ldcg(reinterpret_cast<const float4*>(&p0[c].o[hh][4 * lane]));
+        }
+#pragma unroll
+        for (int hh = 0; hh < 8; ++hh) {
+          const float ff = (use_base && hh == 7) ? 1.f : fast_exp2(f[hh] - M[hh]);
+          acc[hh].x = fmaf(v[hh].x, ff, acc[hh].x);
+          acc[hh].y = fmaf(v[hh].y, ff, acc[hh].y);
+          acc[hh].z = fmaf(v[hh].z, ff, acc[hh].z);
+          acc[hh].w = fmaf(v[hh].w, ff, acc[hh].w);
+        }
+      }
+      const float Htot = (softmax_counted ? (float)G : 0.f) + (use_base ? hbsum : 0.f);
+      FinalRec* fr = pl.fin + unit;
+      float4 xs = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int hh = 0; hh < 8; ++hh) {
+        const bool brow = use_base && hh == 7;
+        float mo = 0.f, il = 0.f;
+        if (brow) {
+          xs.x += acc[hh].x; xs.y += acc[hh].y; xs.z += acc[hh].z; xs.w += acc[hh].w;
+        } else if (hh < G) {
+          mo = M[hh];
+          il = 1.f / L[hh];
+          const float4 on = make_float4(acc[hh].x * il, acc[hh].y * il, acc[hh].z * il, acc[hh].w * il);
+          *reinterpret_cast<float4*>(o + ((size_t)b * dm.Hq + h * G + hh) * kD + 4 * lane) = on;
+          if (softmax_counted) { xs.x += on.x; xs.y += on.y; xs.z += on.z; xs.w += on.w; }
+        }
+        if (lane == 0) { fr->m[hh] = mo; fr->inv_l[hh] = il; }
+      }
+      const float inv_h = (Htot > 0.f) ? 1.f / Htot : 0.f;
+      const float4 X = make_float4(xs.x * inv_h, xs.y * inv_h, xs.z * inv_h, xs.w * inv_h);
+      *reinterpret_cast<float4*>(&fr->X[4 * lane]) = X;
+      const float xx = warp_sum(fmaf(X.x, X.x, X.y * X.y) + fmaf(X.z, X.z, X.w * X.w));
+      if (lane == 0) { fr->H = Htot; fr->XX = xx; }
+      // ---------- publish the unit's B items ----------
+      __syncwarp();
+      int first = 0;
+      if (lane == 0) first = atomicAdd(&pl.ctr[2], nitems);
+      first = __shfl_sync(0xffffffffu, first, 0);
+      __threadfence();
+      for (int k = lane; k < nitems; k += 32)
+        st_release64(&pl.bq[first + k], ((unsigned long long)(unsigned)unit << 32) | (unsigned)(item0 + k + 1));
+    }
   } else {
     // ================================ consumer warps ================================
     // Each warp is on its own: it owns tokens [16 warp, 16 warp + 16) of every tile, keeps its own
-    // softmax reference and its own full-width output accumulator, and never waits for a sibling.
+    // softmax reference and its own full-width output accumulator, and never waits for a sibling
+    // except where the item's eight partial results are merged.
     const int head = lane >> 2, quad = lane & 3;
     const int t0 = 16 * warp + 2 * quad;  // this thread's tokens in a tile: t0, t0 + 1, t0 + 8, t0 + 9
     const int mi = lane >> 3, mr = lane & 7;
@@ -609,23 +761,22 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
               }
             }
           }
-          if (!(d.flags & kFlagLast)) {
-            release();
+          const bool last_tile = (d.flags & kFlagLast) != 0;
+          const int unit = d.unit, item = d.item, item0 = d.item0, nitems = d.nitems;
+          release();
+          if (!last_tile) {
             if (!next_slot()) { alive = false; break; }
             continue;
           }
-          // ---------------- end of the item: stage this warp's partial result ----------------
+          // ---------------- end of the item: merge the eight warps' partial results ----------------
           {
-            const int buf = items_done & 1;
+            const int buf = items_done & 1, use = items_done >> 1;
             float* stage = reinterpret_cast<float*>(stages + buf * kStageBytes);
             float* sm_m = stage + kConsumerWarps * 8 * kD;   // [warp][head]
             float* sm_l = sm_m + kConsumerWarps * 8;         // [warp][head]
             float* sm_hb = sm_l + kConsumerWarps * 8;        // [warp]
-            // the copy was last used two items ago; its merger signals when it is done with it
-            if (items_done >= 2 && !warp_mbar_wait(&stage_free[buf], ((items_done >> 1) - 1) & 1, &ctl[0], lane)) {
-              alive = false;
-              break;
-            }
+            // the copy was last used two items ago; every warp signals when it is done reading it
+            if (use >= 1 && !warp_mbar_wait(&stage_free[buf], (use - 1) & 1, &ctl[0], lane)) { alive = false; break; }
             float* mine = stage + (warp * 8 + head) * kD;
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
@@ -644,106 +795,65 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
               if (head == 7) sm_hb[warp] = hs;
             }
             __syncwarp();
-            int arrived = 0;
+            if (lane == 0) mbar_arrive(&stage_full[buf]);
+            if (!warp_mbar_wait(&stage_full[buf], use & 1, &ctl[0], lane)) { alive = false; break; }
+            // this warp merges head `warp`; lane = 4 channels
+            {
+              PartialRec* pr = pl.part + item;
+              const int hh = warp;
+              const bool brow = use_base && hh == 7;
+              float mw[kConsumerWarps], M = -INFINITY;
+#pragma unroll
+              for (int w = 0; w < kConsumerWarps; ++w) { mw[w] = sm_m[w * 8 + hh]; M = fmaxf(M, mw[w]); }
+              float L = 0.f;
+              float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+              for (int w = 0; w < kConsumerWarps; ++w) {
+                const float f = brow ? 1.f : fast_exp2(mw[w] - M);
+                L = fmaf(sm_l[w * 8 + hh], f, L);
+                const float4 v = *reinterpret_cast<const float4*>(stage + (w * 8 + hh) * kD + 2 * ((2 * lane) ^ (4 * (hh & 3))));
+                acc.x = fmaf(v.x, f, acc.x);
+                acc.y = fmaf(v.y, f, acc.y);
+                acc.z = fmaf(v.z, f, acc.z);
+                acc.w = fmaf(v.w, f, acc.w);
+              }
+              *reinterpret_cast<float4*>(&pr->o[hh][4 * lane]) = acc;
+              if (lane == 0) { pr->m[hh] = M; pr->l[hh] = L; }
+              if (hh == 7 && lane == 0) {
+                float hb_tot = 0.f;
+#pragma unroll
+                for (int w = 0; w < kConsumerWarps; ++w) hb_tot += sm_hb[w];
+                pr->hb = use_base ? hb_tot : 0.f;
+              }
+            }
+            __syncwarp();
+            int last_warp = 0;
             if (lane == 0) {
+              mbar_arrive(&stage_free[buf]);
               __threadfence_block();
-              arrived = atomicAdd_block(&stage_cnt[buf], 1);
+              last_warp = (atomicAdd_block(const_cast<int*>(&ctl[6 + buf]), 1) == kConsumerWarps - 1) ? 1 : 0;
               __threadfence_block();
-            }
-            arrived = __shfl_sync(0xffffffffu, arrived, 0);
-            if (arrived == kConsumerWarps - 1) {
-              // ---------- last warp of the CTA: merge the eight partial results into the item's record ----------
-              PartialRec* pr = pl.part + d.item;
-              float hb_tot = 0.f;
-#pragma unroll
-              for (int w = 0; w < kConsumerWarps; ++w) hb_tot += sm_hb[w];
-#pragma unroll 2
-              for (int hh = 0; hh < 8; ++hh) {
-                const bool brow = use_base && hh == 7;
-                float M = -INFINITY;
-#pragma unroll
-                for (int w = 0; w < kConsumerWarps; ++w) M = fmaxf(M, sm_m[w * 8 + hh]);
-                float L = 0.f;
-                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-                for (int w = 0; w < kConsumerWarps; ++w) {
-                  const float f = brow ? 1.f : fast_exp2(sm_m[w * 8 + hh] - M);
-                  L = fmaf(sm_l[w * 8 + hh], f, L);
-                  const float4 v = *reinterpret_cast<const float4*>(stage + (w * 8 + hh) * kD + 2 * ((2 * lane) ^ (4 * (hh & 3))));
-                  acc.x = fmaf(v.x, f, acc.x);
-                  acc.y = fmaf(v.y, f, acc.y);
-                  acc.z = fmaf(v.z, f, acc.z);
-                  acc.w = fmaf(v.w, f, acc.w);
+              if (last_warp) {
+                // the record is complete: hand it to the merge warp
+                ctl[6 + buf] = 0;
+                const long long t0c = clock64();
+                while (items_done - lds_acquire(&ctl[3]) >= kJobs) {
+                  if (ctl[0] || clock64() - t0c > kWaitCycles) { last_warp = -1; break; }
+                  __nanosleep(64);
                 }
-                *reinterpret_cast<float4*>(&pr->o[hh][4 * lane]) = acc;
-                if (lane == 0) { pr->m[hh] = M; pr->l[hh] = L; }
-              }
-              if (lane == 0) pr->hb = use_base ? hb_tot : 0.f;
-              __syncwarp();
-              int last_of_unit = 0;
-              if (lane == 0) {
-                stage_cnt[buf] = 0;
-                mbar_arrive(&stage_free[buf]);
-                __threadfence();
-                last_of_unit = (atomicAdd(&pl.counter[d.unit], 1) == d.nitems - 1) ? 1 : 0;
-                __threadfence();
-              }
-              last_of_unit = __shfl_sync(0xffffffffu, last_of_unit, 0);
-              if (last_of_unit) {
-                // ---------- last item of the unit: merge its records (this warp alone; lane = 4 channels) ----------
-                const PartialRec* p0 = pl.part + d.item0;
-                const int b = d.unit / dm.Hkv, h = d.unit % dm.Hkv;
-                float hbsum = 0.f;
-                for (int c = 0; c < d.nitems; ++c) hbsum += __ldcg(&p0[c].hb);
-                const float Htot = (softmax_counted ? (float)G : 0.f) + (use_base ? hbsum : 0.f);
-                FinalRec* fr = pl.fin + d.unit;
-                float4 xs = make_float4(0.f, 0.f, 0.f, 0.f);
-                for (int hh = 0; hh < 8; ++hh) {
-                  const bool brow = use_base && hh == 7;
-                  if (hh >= G && !brow) {
-                    if (lane == 0) { fr->m[hh] = 0.f; fr->inv_l[hh] = 0.f; }
-                    continue;
-                  }
-                  float mfin = -INFINITY;
-                  for (int c = 0; c < d.nitems; ++c) mfin = fmaxf(mfin, __ldcg(&p0[c].m[hh]));
-                  float lfin = 0.f;
-                  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 4
-                  for (int c = 0; c < d.nitems; ++c) {
-                    const float f = brow ? 1.f : fast_exp2(__ldcg(&p0[c].m[hh]) - mfin);
-                    lfin = fmaf(__ldcg(&p0[c].l[hh]), f, lfin);
-                    const float4 v = __ldcg(reinterpret_cast<const float4*>(&p0[c].o[hh][4 * lane]));
-                    acc.x = fmaf(v.x, f, acc.x);
-                    acc.y = fmaf(v.y, f, acc.y);
-                    acc.z = fmaf(v.z, f, acc.z);
-                    acc.w = fmaf(v.w, f, acc.w);
-                  }
-                  if (brow) {
-                    xs.x += acc.x; xs.y += acc.y; xs.z += acc.z; xs.w += acc.w;
-                    if (lane == 0) { fr->m[hh] = 0.f; fr->inv_l[hh] = 0.f; }
-                  } else {
-                    const float inv_l = 1.f / lfin;
-                    const float4 on = make_float4(acc.x * inv_l, acc.y * inv_l, acc.z * inv_l, acc.w * inv_l);
-                    *reinterpret_cast<float4*>(o + ((size_t)b * dm.Hq + h * G + hh) * kD + 4 * lane) = on;
-                    if (softmax_counted) { xs.x += on.x; xs.y += on.y; xs.z += on.z; xs.w += on.w; }
-                    if (lane == 0) { fr->m[hh] = mfin; fr->inv_l[hh] = inv_l; }
-                  }
-                }
-                const float inv_h = (Htot > 0.f) ? 1.f / Htot : 0.f;
-                const float4 X = make_float4(xs.x * inv_h, xs.y * inv_h, xs.z * inv_h, xs.w * inv_h);
-                *reinterpret_cast<float4*>(&fr->X[4 * lane]) = X;
-                const float xx = warp_sum(fmaf(X.x, X.x, X.y * X.y) + fmaf(X.z, X.z, X.w * X.w));
-                if (lane == 0) { fr->H = Htot; fr->XX = xx; }
-                __syncwarp();
-                if (lane == 0) {
-                  __threadfence();
-                  st_release(&pl.ready[d.unit], 1);
+                if (last_warp > 0) {
+                  Job* jb = &jobs[items_done % kJobs];
+                  jb->unit = unit;
+                  jb->item0 = item0;
+                  jb->nitems = nitems;
+                  sts_release(&jb->seq, items_done + 1);
                 }
               }
             }
+            last_warp = __shfl_sync(0xffffffffu, last_warp, 0);
+            if (last_warp < 0) { alive = false; break; }
             ++items_done;
           }
-          release();
           break;
         }
       } else if (d.type == kSlotVB) {
@@ -762,25 +872,26 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
           {
             const uint32_t vaddr = smem_u32(sl);
             const int tok = 16 * warp + 8 * (mi & 1) + mr;
-            uint32_t va[8][4];
+            uint32_t va[8][4], xb[8][2];
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks)
               ldmatrix_x4(vaddr + tile_off(tok, 2 * ks + (mi >> 1)), va[ks][0], va[ks][1], va[ks][2], va[ks][3]);
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
-              uint32_t x0 = 0u, x1 = 0u;
-              if (head < 2) {
-                const float2 f0 = *reinterpret_cast<const float2*>(fr->X + 16 * ks + 2 * quad);
-                const float2 f1 = *reinterpret_cast<const float2*>(fr->X + 16 * ks + 8 + 2 * quad);
-                uint32_t h0, l0, h1, l1;
-                split_pair(f0.x, f0.y, h0, l0);
-                split_pair(f1.x, f1.y, h1, l1);
-                x0 = head == 0 ? h0 : l0;
-                x1 = head == 0 ? h1 : l1;
-              }
+              // B operand for <v, X>: column 0 = bf16 hi part of X, column 1 = lo part, the rest zero
+              const float2 f0 = *reinterpret_cast<const float2*>(fr->X + 16 * ks + 2 * quad);
+              const float2 f1 = *reinterpret_cast<const float2*>(fr->X + 16 * ks + 8 + 2 * quad);
+              uint32_t h0, l0, h1, l1;
+              split_pair(f0.x, f0.y, h0, l0);
+              split_pair(f1.x, f1.y, h1, l1);
+              xb[ks][0] = head == 0 ? h0 : (head == 1 ? l0 : 0u);
+              xb[ks][1] = head == 0 ? h1 : (head == 1 ? l1 : 0u);
+            }
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
               mma_bf16(ca, va[ks][0], va[ks][1], va[ks][2], va[ks][3], va[ks][0], va[ks][2]);  // x tokens 0..7
               mma_bf16(cb, va[ks][0], va[ks][1], va[ks][2], va[ks][3], va[ks][1], va[ks][3]);  // x tokens 8..15
-              mma_bf16(cx, va[ks][0], va[ks][1], va[ks][2], va[ks][3], x0, x1);
+              mma_bf16(cx, va[ks][0], va[ks][1], va[ks][2], va[ks][3], xb[ks][0], xb[ks][1]);
             }
           }
           // lane (head, quad): token `head` of the warp if quad == 0, token head + 8 if quad == 1
@@ -853,9 +964,14 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         alive = false;
       }
     }
-    if (!alive && lane == 0 && !ctl[0]) {
-      set_status(status, CAOTE_ERR_TIMEOUT);
-      ctl[0] = 1;
+    if (lane == 0) {
+      if (!alive && !ctl[0]) {
+        set_status(status, CAOTE_ERR_TIMEOUT);
+        ctl[0] = 1;
+      }
+      if (warp == 0) ctl[5] = items_done;
+      __threadfence_block();
+      atomicAdd_block(const_cast<int*>(&ctl[4]), 1);
     }
   }
 
