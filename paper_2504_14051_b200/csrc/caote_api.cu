@@ -247,7 +247,7 @@ static int launch_decode_score(const Dims& dm, const void* q, const void* K, con
     }
   }
   CAOTE_LAUNCH("decode_plan_kernel", st,
-               decode::plan_kernel<<<(pl.max_items + 16383) / 16384 > 0 ? (pl.max_items + 16383) / 16384 : 1, 1024, 0, st>>>(dm.units, dm.Hkv, dm.cap, len, pl, status));
+               decode::plan_kernel<<<1, 1024, 0, st>>>(dm.units, dm.Hkv, dm.cap, len, pl, status));
   const int tiles_per_unit = (dm.cap + decode::kT - 1) / decode::kT;
   const long long max_items = (long long)dm.units * ((tiles_per_unit + pl.tpi - 1) / pl.tpi);
   const int grid = (int)(max_items < grid_limit ? max_items : grid_limit);

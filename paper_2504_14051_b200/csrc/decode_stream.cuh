@@ -1,32 +1,28 @@
 // Single-query (decode) scoring path for bf16, head_dim 128, group size <= 8: one persistent kernel
 // that reads K and V from HBM once and takes the second pass over V out of L2.
 //
-// Work. A unit's cached tokens are cut into tiles of kT tokens and items of `tpi` consecutive tiles.
-// Every item is processed twice:
+// Work list. A unit's cached tokens are cut into tiles of kT tokens and items of `tpi` consecutive
+// tiles. Every item appears twice in one global, statically ordered work list:
 //   A(i)  attention pass: logits of the G group heads (tensor cores, mma.sync bf16), online softmax
 //         over the item's tiles, partial output sum_j p_j v_j; the logits go to a scratch array, the
-//         item's (max, sum, partial output) record to another;
-//   B(i)  score pass: re-reads the item's V tiles (from L2: B work of a unit becomes available as
-//         soon as the unit's records are merged and is taken before any further A work) and its
-//         logits, and writes c_j = w_j / (1 - w_j) * ||X - v_j|| once.
-// A items are handed out in order by one atomic counter. When the last record of a unit is written,
-// the CTA that wrote it merges the unit's records into the final softmax statistics, the attention
-// output o and the reference vector X, and appends the unit's B items to a global queue. Nothing
-// ever waits for another CTA except at the very end (A work exhausted, last merges in flight).
+//         (max, sum, partial output) record to another; the CTA that completes a unit's last A item
+//         merges the records into the final softmax statistics, the attention output o and the
+//         reference vector X, and raises the unit's ready flag;
+//   B(i)  score pass: re-reads the item's V tiles (still in L2: B(i) trails A(i) by `lag` items, a few
+//         tens of MB) and its logits, and writes c_j = w_j / (1 - w_j) * ||X - v_j|| once.
+// The list is A(0..lag-1), then B(0), A(lag), B(1), A(lag+1), ..., then the remaining B items. CTAs
+// take entries with one atomic counter, so a CTA that is busy merging simply takes fewer entries.
 //
-// Inside a CTA (one per SM):
-//   producer warp   claims work (B first, then A) and fills a ring of shared-memory slots by TMA:
-//                   a K tile (+ q, + carried base scores), a V tile, or a V tile with the tile's
-//                   logits, base scores and the unit's final record;
-//   8 consumer warps process the slots in order, each on its own 16 tokens of every tile, with its
-//                   own softmax reference and full-width output accumulator (P never leaves the
-//                   registers); at the end of an item they merge their partial results through a
-//                   staging area in shared memory, one head per warp;
-//   merge warp      counts finished records per unit, merges a completed unit, publishes its B items.
-// Full/empty mbarriers hand slots back and forth; every wait in the kernel is bounded by a clock
-// limit, after which the CTA records CAOTE_ERR_TIMEOUT, stops taking work, lets its own copies land
-// and returns. No hardware barrier is used after start-up, so a warp that gives up cannot strand
-// its siblings.
+// Inside a CTA one producer warp walks the work list and fills a ring of shared-memory slots by TMA
+// (a K tile, a V tile, or a V tile plus the tile's logits and carried base scores); eight consumer
+// warps process the slots in order. Full/empty mbarriers hand the slots back and forth.
+//
+// Waits. B(i) needs its unit's ready flag. `lag` is at least the number of items of the longest
+// unit, so every A item of that unit was taken from the list before B(i) was, by a CTA that is
+// running and that only has earlier list entries in front of it; by induction over the list order
+// every flag is raised. No co-residency of the whole grid is needed. Every wait is still bounded by a
+// clock limit; when one runs out the CTA records CAOTE_ERR_TIMEOUT, stops taking work, lets its own
+// copies land and returns.
 //
 // For the base modes that carry a score (ACCUM, EXTERNAL; G <= 7) row 7 of the P operand carries
 // base_j, which yields sum_j base_j v_j from the same tensor-core product.
@@ -41,24 +37,21 @@ namespace decode {
 
 constexpr int kT = 128;                 // tokens per tile
 constexpr int kD = 128;
-constexpr int kSlots = 4;
+constexpr int kSlots = 3;
 constexpr int kConsumerWarps = 8;
 constexpr int kConsumers = kConsumerWarps * 32;
-constexpr int kProducerWarp = kConsumerWarps;
-constexpr int kMergeWarp = kConsumerWarps + 1;
-constexpr int kThreads = kConsumers + 64;  // + producer warp + merge warp
+constexpr int kThreads = kConsumers + 32;  // + one producer warp
 constexpr int kHalfBytes = kT * 128;       // one 64-channel box: kT rows of 128 bytes
 constexpr int kTileBytes = 2 * kHalfBytes;
-constexpr int kRowsBytes = 8 * kT * 4;     // per slot: 8 rows of kT floats (logits / base / q)
-constexpr int kMaxTilesPerItem = 8;
-constexpr int kJobs = 8;                   // mailbox entries between the consumers and the merge warp
+constexpr int kRowsBytes = 8 * kT * 4;     // per slot: 8 rows of kT floats (logits / base / q / P fragments)
+constexpr int kMaxTilesPerItem = 16;
 constexpr long long kWaitCycles = 2000000000LL;  // ~1 s: far beyond any legitimate wait
 
 enum SlotType { kSlotKA = 0, kSlotVA = 1, kSlotVB = 2, kSlotStop = 3 };
 enum { kFlagFirst = 1, kFlagLast = 2 };
 
 struct PartialRec {   // per item
-  float m[8];         // reference of the log2-domain logits per head
+  float m[8];         // running max of the log2-domain logits per head
   float l[8];         // sum of 2^(s - m)
   float hb;           // sum of the carried base scores of the item
   float pad[7];
@@ -80,27 +73,29 @@ struct Desc {         // what a slot holds
 };
 
 struct Plan {
-  int* item_prefix;        // [units + 1] exclusive prefix of items per unit
-  int* counter;            // [units] records of the unit that are written
-  int* ctr;                // [0] next A item, [1] B entries claimed, [2] B entries reserved
-  unsigned long long* bq;  // [max items] B queue: (unit << 32) | (item + 1), 0 = not yet written
-  PartialRec* part;        // [max items]
-  FinalRec* fin;           // [units]
-  float* S;                // [units][G][capS] log2-domain logits
-  int tpi;                 // tiles per item
-  int capS;                // cap rounded up to a multiple of kT
-  int max_items;
+  int* item_prefix;   // [units + 1] exclusive prefix of items per unit
+  int* counter;       // [units] A items of the unit whose records are written
+  int* ready;         // [units] 1 once FinalRec is written
+  int* work;          // [1] next entry of the work list
+  PartialRec* part;   // [max items]
+  FinalRec* fin;      // [units]
+  float* S;           // [units][G][capS] log2-domain logits
+  int tpi;            // tiles per item
+  int capS;           // cap rounded up to a multiple of kT
+  int lag;            // items by which the score pass trails the attention pass
 };
 
 inline int tiles_per_item(const Dims& dm, int grid) {
   const long long max_tiles = (long long)dm.units * ((dm.cap + kT - 1) / kT);
-  long long t = max_tiles / (4LL * (grid > 0 ? grid : 1));
+  long long t = max_tiles / (2LL * (grid > 0 ? grid : 1));
   if (t < 1) t = 1;
   if (t > kMaxTilesPerItem) t = kMaxTilesPerItem;
   return (int)t;
 }
 
-// `grid` only shapes the item size; the sizes below hold for every grid (they assume tpi = 1).
+// `grid` only shapes the item size and the lag; the carve must be called with the same value by
+// caote_workspace_bytes and by the launch (both use the resident-CTA count, or 0 without a device:
+// the sizes below are upper bounds for every grid because tpi >= 1).
 inline size_t carve(const Dims& dm, char* base, Plan* out, int grid) {
   size_t off = 0;
   auto take = [&](size_t bytes) {
@@ -112,12 +107,12 @@ inline size_t carve(const Dims& dm, char* base, Plan* out, int grid) {
   const int tiles_per_unit = (dm.cap + kT - 1) / kT;
   pl.tpi = tiles_per_item(dm, grid);
   pl.capS = tiles_per_unit * kT;
-  const size_t max_items = (size_t)dm.units * tiles_per_unit;
-  pl.max_items = (int)max_items;
+  pl.lag = (tiles_per_unit + pl.tpi - 1) / pl.tpi + (grid > 0 ? grid : 1);
+  const size_t max_items = (size_t)dm.units * tiles_per_unit;  // sized for tpi = 1
   pl.item_prefix = (int*)take(sizeof(int) * ((size_t)dm.units + 1));
   pl.counter = (int*)take(sizeof(int) * (size_t)dm.units);
-  pl.ctr = (int*)take(sizeof(int) * 4);
-  pl.bq = (unsigned long long*)take(sizeof(unsigned long long) * max_items);
+  pl.ready = (int*)take(sizeof(int) * (size_t)dm.units);
+  pl.work = (int*)take(sizeof(int) * 4);
   pl.fin = (FinalRec*)take(sizeof(FinalRec) * (size_t)dm.units);
   pl.S = (float*)take(sizeof(float) * (size_t)dm.units * dm.G * pl.capS);
   pl.part = (PartialRec*)take(sizeof(PartialRec) * max_items);
@@ -125,30 +120,18 @@ inline size_t carve(const Dims& dm, char* base, Plan* out, int grid) {
   return off;
 }
 
-// Staging area in which the eight consumer warps put their partial results at the end of an item
-// (two copies, used by alternate items): per warp 8 heads x kD floats, then reference, sum, base sum.
-constexpr int kStageFloats = kConsumerWarps * 8 * kD + 2 * kConsumerWarps * 8 + kConsumerWarps;
-constexpr int kStageBytes = (kStageFloats * 4 + 255) / 256 * 256;
-
-struct Job {  // a finished record, handed to the merge warp
-  int seq, unit, item0, nitems;
-};
-
 inline size_t smem_bytes() {
-  return 1024 /* alignment slack */ + (size_t)kSlots * (kTileBytes + kSideBytes) + 2 * (size_t)kStageBytes +
-         sizeof(Desc) * kSlots + sizeof(Job) * kJobs + 8 * (2 * kSlots + 4) + 64;
+  return 1024 /* alignment slack */ + (size_t)kSlots * (kTileBytes + kSideBytes) + sizeof(Desc) * kSlots +
+         sizeof(float) * (2 * kConsumerWarps * 8 + kConsumerWarps * 8 + kConsumerWarps + 8 + kD) + 8 * 2 * kSlots + 64;
 }
 
-// ---- plan: items per unit, their prefix sum, and cleared counters and queue ----------------------
-// grid = any number of CTAs of 1024 threads; CTA 0 computes the prefix, all clear the queue.
+// ---- plan: items per unit, their prefix sum, and cleared counters / flags (one CTA) -------------
 __global__ void __launch_bounds__(1024)
 plan_kernel(int units, int Hkv, int cap, const int* __restrict__ len, Plan pl, int* status) {
   __shared__ int warp_tot[32];
   __shared__ int carry;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  for (int i = blockIdx.x * 1024 + tid; i < pl.max_items; i += gridDim.x * 1024) pl.bq[i] = 0ull;
-  if (blockIdx.x != 0) return;
-  if (tid == 0) { carry = 0; pl.item_prefix[0] = 0; pl.ctr[0] = 0; pl.ctr[1] = 0; pl.ctr[2] = 0; }
+  if (tid == 0) { carry = 0; pl.item_prefix[0] = 0; pl.work[0] = 0; }
   __syncthreads();
   for (int u0 = 0; u0 < units; u0 += 1024) {
     const int u = u0 + tid;
@@ -158,6 +141,7 @@ plan_kernel(int units, int Hkv, int cap, const int* __restrict__ len, Plan pl, i
       if (n < 0 || n > cap) set_status(status, CAOTE_ERR_BAD_LENGTH);
       else ni = ((n + kT - 1) / kT + pl.tpi - 1) / pl.tpi;
       pl.counter[u] = 0;
+      pl.ready[u] = 0;
     }
     int incl = ni;
 #pragma unroll
@@ -308,24 +292,21 @@ __device__ __forceinline__ uint32_t tile_off(int row, int chunk16) {
   return (uint32_t)((chunk16 >> 3) * kHalfBytes + row * 128 + (((chunk16 & 7) ^ (row & 7)) << 4));
 }
 
-__device__ __forceinline__ int lds_acquire(const volatile int* p) {
-  int v;
-  asm volatile("ld.acquire.cta.shared::cta.s32 %0, [%1];" : "=r"(v) : "r"(smem_u32(const_cast<const int*>(p))) : "memory");
-  return v;
-}
-__device__ __forceinline__ void sts_release(volatile int* p, int v) {
-  asm volatile("st.release.cta.shared::cta.s32 [%0], %1;" ::"r"(smem_u32(const_cast<int*>(p))), "r"(v) : "memory");
-}
-__device__ __forceinline__ unsigned long long ld_acquire64(const unsigned long long* p) {
-  unsigned long long v;
-  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
-  return v;
-}
-__device__ __forceinline__ void st_release64(unsigned long long* p, unsigned long long v) {
-  asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+// Entry w of the work list -> (is_B, item). N items, lag L (see the file comment).
+__device__ __forceinline__ void work_entry(int w, int N, int L, bool& is_b, int& item) {
+  if (L > N) L = N;
+  if (w < L) { is_b = false; item = w; return; }
+  if (w < 2 * N - L) {
+    const int r = w - L;
+    is_b = (r & 1) == 0;
+    item = is_b ? (r >> 1) : (L + (r >> 1));
+    return;
+  }
+  is_b = true;
+  item = w - N;
 }
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, 2)
 decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, Dims dm,
               const __nv_bfloat16* __restrict__ q, const int* __restrict__ len, float* __restrict__ base,
               float* __restrict__ o, float* __restrict__ scores, Plan pl, int* status) {
@@ -333,16 +314,16 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
   char* sm = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   char* tiles = sm;                                                              // [kSlots][kTileBytes]
   char* sides = tiles + kSlots * kTileBytes;                                     // [kSlots][kSideBytes]
-  char* stages = sides + kSlots * kSideBytes;                                    // [2][kStageBytes]
-  Desc* desc = reinterpret_cast<Desc*>(stages + 2 * kStageBytes);                // [kSlots]
-  Job* jobs = reinterpret_cast<Job*>(desc + kSlots);                             // [kJobs]
-  uint64_t* full = reinterpret_cast<uint64_t*>(jobs + kJobs);                    // [kSlots]
+  Desc* desc = reinterpret_cast<Desc*>(sides + kSlots * kSideBytes);             // [kSlots]
+  float* wmax = reinterpret_cast<float*>(desc + kSlots);                         // [2][kConsumerWarps][8]
+  float* wl = wmax + 2 * kConsumerWarps * 8;                                     // [kConsumerWarps][8]
+  float* whb = wl + kConsumerWarps * 8;                                          // [kConsumerWarps]
+  float* wm = whb + kConsumerWarps;                                              // [8]
+  float* xrow = wm + 8;                                                          // [kD]
+  uint64_t* full = reinterpret_cast<uint64_t*>(xrow + kD);                       // [kSlots]
   uint64_t* empty = full + kSlots;                                               // [kSlots]
-  uint64_t* stage_full = empty + kSlots;                                         // [2]
-  uint64_t* stage_free = stage_full + 2;                                         // [2]
-  // [0] stop, [2] slots issued, [3] jobs taken by the merge warp, [4] consumer warps that have left,
-  // [5] jobs posted in total, [6..7] warps that finished merging their head (per staging copy)
-  volatile int* ctl = reinterpret_cast<volatile int*>(stage_free + 2);
+  volatile int* ctl = reinterpret_cast<volatile int*>(empty + kSlots);           // [0] stop, [1] last arriver,
+                                                                                 // [2] slots issued
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int G = dm.G, mode = dm.base_mode;
@@ -356,20 +337,17 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
       mbar_init(&full[i], 1);
       mbar_init(&empty[i], kConsumerWarps);
     }
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(&stage_full[i], kConsumerWarps);
-      mbar_init(&stage_free[i], kConsumerWarps);
-    }
-    for (int i = 0; i < 8; ++i) ctl[i] = 0;
+    ctl[0] = 0;
+    ctl[1] = 0;
+    ctl[2] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (tid < kSlots * (int)(sizeof(Desc) / sizeof(int))) reinterpret_cast<int*>(desc)[tid] = 0;
-  if (tid < kJobs * (int)(sizeof(Job) / sizeof(int))) reinterpret_cast<int*>(jobs)[tid] = 0;
   __syncthreads();
 
-  int consumed = 0;  // slots this warp has finished
+  int consumed = 0;  // slots the consumers have finished (uniform over the consumer threads)
 
-  if (warp == kProducerWarp) {
+  if (warp == kConsumerWarps) {
     // ================================ producer warp ================================
     const uint64_t pol_stream = policy_evict_first(), pol_keep = policy_evict_last();
     int issued = 0;
@@ -379,61 +357,39 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
       return mbar_wait(&empty[s], ((issued / kSlots) & 1) ^ 1, &ctl[0]);
     };
     while (ok) {
-      // ---- claim work: a published B item if there is one, else the next A item
-      int kind = 0, item = 0, u = 0;  // kind: 0 = all work handed out, 1 = A, 2 = B, -1 = gave up
-      if (lane == 0) {
-        const long long t0c = clock64();
-        for (;;) {
-          const int bh = *reinterpret_cast<volatile int*>(&pl.ctr[1]);
-          const int bt = ld_acquire(&pl.ctr[2]);
-          if (bh < bt) {
-            if (atomicCAS(&pl.ctr[1], bh, bh + 1) != bh) continue;
-            unsigned long long e = ld_acquire64(&pl.bq[bh]);
-            while (e == 0ull) {  // reserved, about to be written
-              if (ctl[0] || clock64() - t0c > kWaitCycles) break;
-              __nanosleep(32);
-              e = ld_acquire64(&pl.bq[bh]);
-            }
-            if (e == 0ull) { kind = -1; break; }
-            u = (int)(e >> 32);
-            item = (int)(e & 0xffffffffull) - 1;
-            kind = 2;
-            break;
-          }
-          if (*reinterpret_cast<volatile int*>(&pl.ctr[0]) < N) {
-            const int a = atomicAdd(&pl.ctr[0], 1);
-            if (a < N) { item = a; kind = 1; break; }
-          }
-          if (bh >= N) { kind = 0; break; }
-          if (ctl[0] || clock64() - t0c > kWaitCycles) { kind = -1; break; }
-          __nanosleep(128);
-        }
+      int w = 0;
+      if (lane == 0) w = atomicAdd(pl.work, 1);
+      w = __shfl_sync(0xffffffffu, w, 0);
+      if (w >= 2 * N) break;
+      bool is_b;
+      int item;
+      work_entry(w, N, pl.lag, is_b, item);
+      // unit of the item: 32-ary search over the item prefix, one probe per lane
+      int lo = 0, hi = dm.units;
+      while (hi - lo > 1) {
+        const int step = (hi - lo + 31) / 32;
+        const int probe = lo + lane * step;
+        const int val = (probe < hi) ? __ldg(pl.item_prefix + probe) : 0x7fffffff;
+        const unsigned mask = __ballot_sync(0xffffffffu, val <= item);
+        const int k = 31 - __clz((int)mask);
+        lo = lo + k * step;
+        hi = min(hi, lo + step);
       }
-      kind = __shfl_sync(0xffffffffu, kind, 0);
-      item = __shfl_sync(0xffffffffu, item, 0);
-      u = __shfl_sync(0xffffffffu, u, 0);
-      if (kind <= 0) { ok = (kind == 0); break; }
-      const bool is_b = kind == 2;
-      if (!is_b) {
-        // unit of the item: 32-ary search over the item prefix, one probe per lane
-        int lo = 0, hi = dm.units;
-        while (hi - lo > 1) {
-          const int step = (hi - lo + 31) / 32;
-          const int probe = lo + lane * step;
-          const int val = (probe < hi) ? __ldg(pl.item_prefix + probe) : 0x7fffffff;
-          const unsigned mask = __ballot_sync(0xffffffffu, val <= item);
-          const int k = 31 - __clz((int)mask);
-          lo = lo + k * step;
-          hi = min(hi, lo + step);
-        }
-        u = lo;
-      }
+      const int u = lo;
       if (lane == 0) {
         const int item0 = pl.item_prefix[u], nitems = pl.item_prefix[u + 1] - item0;
         const int n = len[u / dm.Hkv];
         const int ntiles = (n + kT - 1) / kT;
         const int t_begin = (item - item0) * pl.tpi, t_end = min(t_begin + pl.tpi, ntiles);
-        if (is_b) fence_async_all();  // the logits and the final record were written by ordinary stores
+        if (is_b) {
+          // the item's logits and the unit's final record must be complete before they are copied
+          const long long t0c = clock64();
+          while (ld_acquire(&pl.ready[u]) == 0) {
+            if (ctl[0] || clock64() - t0c > kWaitCycles) { ok = false; break; }
+            __nanosleep(64);
+          }
+          fence_async_all();
+        }
         for (int t = t_begin; ok && t < t_end; ++t) {
           Desc d;
           d.unit = u;
@@ -509,469 +465,341 @@ decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ C
         ctl[0] = 1;
       }
     }
-  } else if (warp == kMergeWarp) {
-    // ================================ merge warp ================================
-    int idx = 0;
-    long long t_idle = clock64();
-    for (;;) {
-      int state = 0;  // 1 = a job is waiting, 2 = all done, 3 = give up
-      if (lane == 0) {
-        if (lds_acquire(&jobs[idx % kJobs].seq) == idx + 1) state = 1;
-        else if (lds_acquire(&ctl[4]) == kConsumerWarps && ctl[5] == idx) state = 2;
-        else if (ctl[0]) state = 2;
-        else if (clock64() - t_idle > kWaitCycles) state = 3;
-      }
-      state = __shfl_sync(0xffffffffu, state, 0);
-      if (state == 2) break;
-      if (state == 3) {
-        if (lane == 0) { set_status(status, CAOTE_ERR_TIMEOUT); ctl[0] = 1; }
-        break;
-      }
-      if (state == 0) { __nanosleep(100); continue; }
-      const int unit = jobs[idx % kJobs].unit, item0 = jobs[idx % kJobs].item0, nitems = jobs[idx % kJobs].nitems;
-      __syncwarp();
-      ++idx;
-      if (lane == 0) sts_release(&ctl[3], idx);  // the mailbox entry may be reused
-      t_idle = clock64();
-      int last_of_unit = 0;
-      if (lane == 0) {
-        __threadfence();
-        last_of_unit = (atomicAdd(&pl.counter[unit], 1) == nitems - 1) ? 1 : 0;
-        __threadfence();
-      }
-      last_of_unit = __shfl_sync(0xffffffffu, last_of_unit, 0);
-      if (!last_of_unit) continue;
-
-      // ---------- the unit's last record is in: merge its records (lane = 4 channels) ----------
-      const PartialRec* p0 = pl.part + item0;
-      const int b = unit / dm.Hkv, h = unit % dm.Hkv;
-      float M[8], L[8], hbsum = 0.f;
-#pragma unroll
-      for (int hh = 0; hh < 8; ++hh) { M[hh] = -INFINITY; L[hh] = 0.f; }
-      for (int c0 = 0; c0 < nitems; c0 += 32) {
-        const int c = c0 + lane;
-        if (c < nitems) {
-#pragma unroll
-          for (int hh = 0; hh < 8; ++hh) M[hh] = fmaxf(M[hh], __ldcg(&p0[c].m[hh]));
-        }
-      }
-#pragma unroll
-      for (int hh = 0; hh < 8; ++hh) M[hh] = warp_max(M[hh]);
-      for (int c0 = 0; c0 < nitems; c0 += 32) {
-        const int c = c0 + lane;
-        if (c < nitems) {
-#pragma unroll
-          for (int hh = 0; hh < 8; ++hh)
-            L[hh] = fmaf(__ldcg(&p0[c].l[hh]), fast_exp2(__ldcg(&p0[c].m[hh]) - M[hh]), L[hh]);
-          hbsum += __ldcg(&p0[c].hb);
-        }
-      }
-#pragma unroll
-      for (int hh = 0; hh < 8; ++hh) L[hh] = warp_sum(L[hh]);
-      hbsum = warp_sum(hbsum);
-      float4 acc[8];
-#pragma unroll
-      for (int hh = 0; hh < 8; ++hh) acc[hh] = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 2
-      for (int c = 0; c < nitems; ++c) {
-        float f[8];
-        float4 v[8];
-#pragma unroll
-        for (int hh = 0; hh < 8; ++hh) {
-          f[hh] = __ldcg(&p0[c].m[hh]);
-          v[hh] = __ldcg(reinterpret_cast<const float4*>(&p0[c].o[hh][4 * lane]));
-        }
-#pragma unroll
-        for (int hh = 0; hh < 8; ++hh) {
-          const float ff = (use_base && hh == 7) ? 1.f : fast_exp2(f[hh] - M[hh]);
-          acc[hh].x = fmaf(v[hh].x, ff, acc[hh].x);
-          acc[hh].y = fmaf(v[hh].y, ff, acc[hh].y);
-          acc[hh].z = fmaf(v[hh].z, ff, acc[hh].z);
-          acc[hh].w = fmaf(v[hh].w, ff, acc[hh].w);
-        }
-      }
-      const float Htot = (softmax_counted ? (float)G : 0.f) + (use_base ? hbsum : 0.f);
-      FinalRec* fr = pl.fin + unit;
-      float4 xs = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-      for (int hh = 0; hh < 8; ++hh) {
-        const bool brow = use_base && hh == 7;
-        float mo = 0.f, il = 0.f;
-        if (brow) {
-          xs.x += acc[hh].x; xs.y += acc[hh].y; xs.z += acc[hh].z; xs.w += acc[hh].w;
-        } else if (hh < G) {
-          mo = M[hh];
-          il = 1.f / L[hh];
-          const float4 on = make_float4(acc[hh].x * il, acc[hh].y * il, acc[hh].z * il, acc[hh].w * il);
-          *reinterpret_cast<float4*>(o + ((size_t)b * dm.Hq + h * G + hh) * kD + 4 * lane) = on;
-          if (softmax_counted) { xs.x += on.x; xs.y += on.y; xs.z += on.z; xs.w += on.w; }
-        }
-        if (lane == 0) { fr->m[hh] = mo; fr->inv_l[hh] = il; }
-      }
-      const float inv_h = (Htot > 0.f) ? 1.f / Htot : 0.f;
-      const float4 X = make_float4(xs.x * inv_h, xs.y * inv_h, xs.z * inv_h, xs.w * inv_h);
-      *reinterpret_cast<float4*>(&fr->X[4 * lane]) = X;
-      const float xx = warp_sum(fmaf(X.x, X.x, X.y * X.y) + fmaf(X.z, X.z, X.w * X.w));
-      if (lane == 0) { fr->H = Htot; fr->XX = xx; }
-      // ---------- publish the unit's B items ----------
-      __syncwarp();
-      int first = 0;
-      if (lane == 0) first = atomicAdd(&pl.ctr[2], nitems);
-      first = __shfl_sync(0xffffffffu, first, 0);
-      __threadfence();
-      for (int k = lane; k < nitems; k += 32)
-        st_release64(&pl.bq[first + k], ((unsigned long long)(unsigned)unit << 32) | (unsigned)(item0 + k + 1));
-    }
   } else {
     // ================================ consumer warps ================================
-    // Each warp is on its own: it owns tokens [16 warp, 16 warp + 16) of every tile, keeps its own
-    // softmax reference and its own full-width output accumulator, and never waits for a sibling
-    // except where the item's eight partial results are merged.
     const int head = lane >> 2, quad = lane & 3;
-    const int t0 = 16 * warp + 2 * quad;  // this thread's tokens in a tile: t0, t0 + 1, t0 + 8, t0 + 9
-    const int mi = lane >> 3, mr = lane & 7;
-    bool alive = true;
-    int items_done = 0;  // A items this warp has finished (selects the staging copy)
-    int s = 0;
-    Desc d;
-    auto next_slot = [&]() -> bool {
-      s = consumed % kSlots;
-      if (!warp_mbar_wait(&full[s], (consumed / kSlots) & 1, &ctl[0], lane)) return false;
-      d = desc[s];
-      return true;
-    };
-    auto release = [&]() {
-      __syncwarp();
-      fence_async_smem();
-      if (lane == 0) mbar_arrive(&empty[s]);
-      ++consumed;
-    };
+    const int t0 = 16 * warp + 2 * quad;  // this thread's tokens: t0, t0 + 1, t0 + 8, t0 + 9
+    uint32_t qa[8][2];
+    float m_run = -INFINITY, l_priv = 0.f, hb_priv = 0.f, corr = 0.f;
+    float o0[4] = {0.f, 0.f, 0.f, 0.f}, o1[4] = {0.f, 0.f, 0.f, 0.f};
+    int tile_par = 0;
 
-    while (alive) {
-      if (!next_slot()) { alive = false; break; }
+    for (;; ++consumed) {
+      const int s = consumed % kSlots;
+      char* sl = tiles + s * kTileBytes;
+      float* side = reinterpret_cast<float*>(sides + s * kSideBytes);  // [8][kT], then a FinalRec
+      const bool got = warp_mbar_wait(&full[s], (consumed / kSlots) & 1, &ctl[0], lane);
+      if (consumer_any(!got)) {  // uniform: either every consumer thread leaves here or none does
+        if (tid == 0 && !ctl[0]) {
+          set_status(status, CAOTE_ERR_TIMEOUT);
+          ctl[0] = 1;
+        }
+        break;
+      }
+      const Desc d = desc[s];
       if (d.type == kSlotStop) { ++consumed; break; }
+      const int b = d.unit / dm.Hkv, h = d.unit % dm.Hkv;
 
       if (d.type == kSlotKA) {
-        // =============================== one A item ===============================
-        const bool base_row = use_base && head == 7;
-        uint32_t qa[8][2];
-        float oacc[16][4];
-        float m_ref = base_row ? 0.f : -INFINITY, l_priv = 0.f, hb_priv = 0.f;
-#pragma unroll
-        for (int j = 0; j < 16; ++j) { oacc[j][0] = 0.f; oacc[j][1] = 0.f; oacc[j][2] = 0.f; oacc[j][3] = 0.f; }
-        {
+        // ===================== logits and softmax numerators of one tile =====================
+        if (d.flags & kFlagFirst) {
           // Q fragments: row = lane / 4 (rows 8..15 duplicate rows 0..7), zero for heads >= G
-          const __nv_bfloat16* qrow = reinterpret_cast<const __nv_bfloat16*>(sides + s * kSideBytes) +
-                                      (head < G ? head : 0) * kD + 2 * quad;
+          const __nv_bfloat16* qrow = reinterpret_cast<const __nv_bfloat16*>(side) + (head < G ? head : 0) * kD + 2 * quad;
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks) {
             qa[ks][0] = (head < G) ? *reinterpret_cast<const uint32_t*>(qrow + 16 * ks) : 0u;
             qa[ks][1] = (head < G) ? *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 8) : 0u;
           }
+          m_run = -INFINITY;
+          l_priv = 0.f;
+          hb_priv = 0.f;
+#pragma unroll
+          for (int i = 0; i < 4; ++i) { o0[i] = 0.f; o1[i] = 0.f; }
         }
-        for (;;) {
-          // ---------------- K tile: logits, softmax numerators ----------------
-          if (d.type != kSlotKA) { alive = false; break; }
-          uint4 frag;  // P as an A fragment: a0 = hi(tokens 0..7), a1 = lo(0..7), a2 = hi(8..15), a3 = lo(8..15)
-          {
-            const uint32_t kaddr = smem_u32(tiles + s * kTileBytes);
-            const float* side = reinterpret_cast<const float*>(sides + s * kSideBytes);
-            uint32_t kb[8][4];
-            const int tok = 16 * warp + 8 * (mi >> 1) + mr;
+        const uint32_t kaddr = smem_u32(sl);
+        float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+        {
+          const int mi = lane >> 3, r = lane & 7;
+          const int tok = 16 * warp + 8 * (mi >> 1) + r;
 #pragma unroll
-            for (int ks = 0; ks < 8; ++ks)
-              ldmatrix_x4(kaddr + tile_off(tok, 2 * ks + (mi & 1)), kb[ks][0], kb[ks][1], kb[ks][2], kb[ks][3]);
-            float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {
-              mma_bf16(s0, qa[ks][0], qa[ks][0], qa[ks][1], qa[ks][1], kb[ks][0], kb[ks][1]);
-              mma_bf16(s1, qa[ks][0], qa[ks][0], qa[ks][1], qa[ks][1], kb[ks][2], kb[ks][3]);
-            }
-            const bool v0 = t0 < d.n_valid, v1 = t0 + 1 < d.n_valid, v2 = t0 + 8 < d.n_valid, v3 = t0 + 9 < d.n_valid;
-            float bv[4] = {0.f, 0.f, 0.f, 0.f};
-            if (base_row) {
-              const float* Bb = side + 7 * kT;
-              bv[0] = v0 ? Bb[t0] : 0.f;
-              bv[1] = v1 ? Bb[t0 + 1] : 0.f;
-              bv[2] = v2 ? Bb[t0 + 8] : 0.f;
-              bv[3] = v3 ? Bb[t0 + 9] : 0.f;
-              hb_priv += (bv[0] + bv[1]) + (bv[2] + bv[3]);
-            }
-            const int tile = d.tile, unit = d.unit;
-            release();  // done with the K tile and its side rows
+          for (int ks = 0; ks < 8; ++ks) {
+            uint32_t b0, b1, b2, b3;
+            ldmatrix_x4(kaddr + tile_off(tok, 2 * ks + (mi & 1)), b0, b1, b2, b3);
+            mma_bf16(s0, qa[ks][0], qa[ks][0], qa[ks][1], qa[ks][1], b0, b1);
+            mma_bf16(s1, qa[ks][0], qa[ks][0], qa[ks][1], qa[ks][1], b2, b3);
+          }
+        }
+        const bool v0 = t0 < d.n_valid, v1 = t0 + 1 < d.n_valid, v2 = t0 + 8 < d.n_valid, v3 = t0 + 9 < d.n_valid;
+        float bv[4] = {0.f, 0.f, 0.f, 0.f};
+        if (use_base && head == 7) {
+          const float* Bb = side + 7 * kT;
+          bv[0] = v0 ? Bb[t0] : 0.f;
+          bv[1] = v1 ? Bb[t0 + 1] : 0.f;
+          bv[2] = v2 ? Bb[t0 + 8] : 0.f;
+          bv[3] = v3 ? Bb[t0 + 9] : 0.f;
+          hb_priv += (bv[0] + bv[1]) + (bv[2] + bv[3]);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&empty[s]);  // this warp is done with the K tile and its base row
 
-            float sv[4];
-            sv[0] = v0 ? s0[0] * scale2 : -INFINITY;
-            sv[1] = v1 ? s0[1] * scale2 : -INFINITY;
-            sv[2] = v2 ? s1[0] * scale2 : -INFINITY;
-            sv[3] = v3 ? s1[1] * scale2 : -INFINITY;
-            if (softmax_counted && head < G) {
-              float* Sg = pl.S + ((size_t)unit * G + head) * pl.capS + (size_t)tile * kT + t0;
-              __stcg(reinterpret_cast<float2*>(Sg), make_float2(sv[0], sv[1]));
-              __stcg(reinterpret_cast<float2*>(Sg + 8), make_float2(sv[2], sv[3]));
-            }
-            float mx = fmaxf(fmaxf(sv[0], sv[1]), fmaxf(sv[2], sv[3]));
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-            // The reference moves only when a logit exceeds it by more than 8 (p stays <= 256), so
-            // the 64 accumulator registers are rescaled a handful of times per item, not every tile.
-            const bool need = !base_row && mx > m_ref + 8.f;  // also true for the first finite maximum
-            if (__any_sync(0xffffffffu, need)) {
-              const float corr = need ? fast_exp2(m_ref - mx) : 1.f;
-              if (need) m_ref = mx;
-              l_priv *= corr;
-#pragma unroll
-              for (int j = 0; j < 16; ++j) { oacc[j][0] *= corr; oacc[j][1] *= corr; oacc[j][2] *= corr; oacc[j][3] *= corr; }
-            }
-            float p[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) p[i] = (sv[i] == -INFINITY) ? 0.f : fast_exp2(sv[i] - m_ref);
-            l_priv += (p[0] + p[1]) + (p[2] + p[3]);
-            if (head >= G) { p[0] = p[1] = p[2] = p[3] = 0.f; }
-            if (base_row) { p[0] = bv[0]; p[1] = bv[1]; p[2] = bv[2]; p[3] = bv[3]; }
-            split_pair(p[0], p[1], frag.x, frag.y);
-            split_pair(p[2], p[3], frag.z, frag.w);
-          }
-          // ---------------- V tile: partial output of this warp's 16 tokens ----------------
-          if (!next_slot() || d.type != kSlotVA) { alive = false; break; }
-          {
-            char* sl = tiles + s * kTileBytes;
-            if (d.n_valid < 16 * warp + 16) {
-              // rows behind the unit's length hold whatever the cache has there: clear this warp's
-              // so that a zero weight times a stray NaN cannot reach the accumulators
-#pragma unroll
-              for (int i = 0; i < 8; ++i) {
-                const int row = 16 * warp + 2 * i + (lane >> 4), c = lane & 15;
-                if (row >= d.n_valid) *reinterpret_cast<uint4*>(sl + tile_off(row, c)) = make_uint4(0u, 0u, 0u, 0u);
-              }
-              __syncwarp();
-            }
-            const uint32_t vaddr = smem_u32(sl);
-            const int vrow = 16 * warp + 8 * (mi & 1) + mr;
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
-              uint32_t vb[4][4];
-#pragma unroll
-              for (int jj = 0; jj < 4; ++jj)
-                ldmatrix_x4_trans(vaddr + tile_off(vrow, 2 * (4 * half + jj) + (mi >> 1)), vb[jj][0], vb[jj][1], vb[jj][2], vb[jj][3]);
-#pragma unroll
-              for (int jj = 0; jj < 4; ++jj) {
-                mma_bf16(oacc[2 * (4 * half + jj)], frag.x, frag.y, frag.z, frag.w, vb[jj][0], vb[jj][1]);
-                mma_bf16(oacc[2 * (4 * half + jj) + 1], frag.x, frag.y, frag.z, frag.w, vb[jj][2], vb[jj][3]);
-              }
-            }
-          }
-          const bool last_tile = (d.flags & kFlagLast) != 0;
-          const int unit = d.unit, item = d.item, item0 = d.item0, nitems = d.nitems;
-          release();
-          if (!last_tile) {
-            if (!next_slot()) { alive = false; break; }
-            continue;
-          }
-          // ---------------- end of the item: merge the eight warps' partial results ----------------
-          {
-            const int buf = items_done & 1, use = items_done >> 1;
-            float* stage = reinterpret_cast<float*>(stages + buf * kStageBytes);
-            float* sm_m = stage + kConsumerWarps * 8 * kD;   // [warp][head]
-            float* sm_l = sm_m + kConsumerWarps * 8;         // [warp][head]
-            float* sm_hb = sm_l + kConsumerWarps * 8;        // [warp]
-            // the copy was last used two items ago; every warp signals when it is done reading it
-            if (use >= 1 && !warp_mbar_wait(&stage_free[buf], (use - 1) & 1, &ctl[0], lane)) { alive = false; break; }
-            float* mine = stage + (warp * 8 + head) * kD;
-#pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              const int c = (4 * j + quad) ^ (4 * (head & 3));  // float2 slot, swizzled against bank conflicts
-              *reinterpret_cast<float2*>(mine + 2 * c) = make_float2(oacc[j][0] + oacc[j][2], oacc[j][1] + oacc[j][3]);
-            }
-            float ls = l_priv;
-            ls += __shfl_xor_sync(0xffffffffu, ls, 1);
-            ls += __shfl_xor_sync(0xffffffffu, ls, 2);
-            float hs = hb_priv;
-            hs += __shfl_xor_sync(0xffffffffu, hs, 1);
-            hs += __shfl_xor_sync(0xffffffffu, hs, 2);
-            if (quad == 0) {
-              sm_m[warp * 8 + head] = m_ref;
-              sm_l[warp * 8 + head] = ls;
-              if (head == 7) sm_hb[warp] = hs;
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&stage_full[buf]);
-            if (!warp_mbar_wait(&stage_full[buf], use & 1, &ctl[0], lane)) { alive = false; break; }
-            // this warp merges head `warp`; lane = 4 channels
-            {
-              PartialRec* pr = pl.part + item;
-              const int hh = warp;
-              const bool brow = use_base && hh == 7;
-              float mw[kConsumerWarps], M = -INFINITY;
-#pragma unroll
-              for (int w = 0; w < kConsumerWarps; ++w) { mw[w] = sm_m[w * 8 + hh]; M = fmaxf(M, mw[w]); }
-              float L = 0.f;
-              float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-              for (int w = 0; w < kConsumerWarps; ++w) {
-                const float f = brow ? 1.f : fast_exp2(mw[w] - M);
-                L = fmaf(sm_l[w * 8 + hh], f, L);
-                const float4 v = *reinterpret_cast<const float4*>(stage + (w * 8 + hh) * kD + 2 * ((2 * lane) ^ (4 * (hh & 3))));
-                acc.x = fmaf(v.x, f, acc.x);
-                acc.y = fmaf(v.y, f, acc.y);
-                acc.z = fmaf(v.z, f, acc.z);
-                acc.w = fmaf(v.w, f, acc.w);
-              }
-              *reinterpret_cast<float4*>(&pr->o[hh][4 * lane]) = acc;
-              if (lane == 0) { pr->m[hh] = M; pr->l[hh] = L; }
-              if (hh == 7 && lane == 0) {
-                float hb_tot = 0.f;
-#pragma unroll
-                for (int w = 0; w < kConsumerWarps; ++w) hb_tot += sm_hb[w];
-                pr->hb = use_base ? hb_tot : 0.f;
-              }
-            }
-            __syncwarp();
-            int last_warp = 0;
-            if (lane == 0) {
-              mbar_arrive(&stage_free[buf]);
-              __threadfence_block();
-              last_warp = (atomicAdd_block(const_cast<int*>(&ctl[6 + buf]), 1) == kConsumerWarps - 1) ? 1 : 0;
-              __threadfence_block();
-              if (last_warp) {
-                // the record is complete: hand it to the merge warp
-                ctl[6 + buf] = 0;
-                const long long t0c = clock64();
-                while (items_done - lds_acquire(&ctl[3]) >= kJobs) {
-                  if (ctl[0] || clock64() - t0c > kWaitCycles) { last_warp = -1; break; }
-                  __nanosleep(64);
-                }
-                if (last_warp > 0) {
-                  Job* jb = &jobs[items_done % kJobs];
-                  jb->unit = unit;
-                  jb->item0 = item0;
-                  jb->nitems = nitems;
-                  sts_release(&jb->seq, items_done + 1);
-                }
-              }
-            }
-            last_warp = __shfl_sync(0xffffffffu, last_warp, 0);
-            if (last_warp < 0) { alive = false; break; }
-            ++items_done;
-          }
-          break;
+        float sv[4];
+        sv[0] = v0 ? s0[0] * scale2 : -INFINITY;
+        sv[1] = v1 ? s0[1] * scale2 : -INFINITY;
+        sv[2] = v2 ? s1[0] * scale2 : -INFINITY;
+        sv[3] = v3 ? s1[1] * scale2 : -INFINITY;
+        if (softmax_counted && head < G) {
+          float* Sg = pl.S + ((size_t)d.unit * G + head) * pl.capS + (size_t)d.tile * kT + t0;
+          __stcg(reinterpret_cast<float2*>(Sg), make_float2(sv[0], sv[1]));
+          __stcg(reinterpret_cast<float2*>(Sg + 8), make_float2(sv[2], sv[3]));
         }
-      } else if (d.type == kSlotVB) {
-        // =============================== one B item ===============================
-        for (;;) {
-          if (d.type != kSlotVB) { alive = false; break; }
-          // ||X - v_j||^2 = ||v_j||^2 - 2 <v_j, X> + ||X||^2 for this warp's 16 tokens on the tensor
-          // cores: the V rows are the A operand; used again as the B operand they give the Gram
-          // blocks whose diagonals are ||v_j||^2; X, split into bf16 hi + lo columns, gives <v_j, X>.
-          // Tokens for which that difference cancels (v_j close to X) or that hold most of the weight
-          // are redone below by plain subtraction, so v_j = X still scores exactly 0.
-          const char* sl = tiles + s * kTileBytes;
-          const float* side = reinterpret_cast<const float*>(sides + s * kSideBytes);
-          const FinalRec* fr = reinterpret_cast<const FinalRec*>(side + 8 * kT);
-          float ca[4] = {0.f, 0.f, 0.f, 0.f}, cb[4] = {0.f, 0.f, 0.f, 0.f}, cx[4] = {0.f, 0.f, 0.f, 0.f};
+        float mx = fmaxf(fmaxf(sv[0], sv[1]), fmaxf(sv[2], sv[3]));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+        float* wmx = wmax + tile_par * kConsumerWarps * 8;
+        if (quad == 0) wmx[warp * 8 + head] = mx;
+        consumer_sync();
+        float m_new = m_run;
+#pragma unroll
+        for (int w = 0; w < kConsumerWarps; ++w) m_new = fmaxf(m_new, wmx[w * 8 + head]);
+        tile_par ^= 1;
+        corr = fast_exp2(m_run - m_new);  // m_new is finite (a tile holds a valid token); 2^-inf = 0
+        m_run = m_new;
+        float p[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) p[i] = fast_exp2(sv[i] - m_new);
+        l_priv = fmaf(l_priv, corr, (p[0] + p[1]) + (p[2] + p[3]));
+        if (head >= G) { p[0] = p[1] = p[2] = p[3] = 0.f; }
+        if (use_base && head == 7) {
+          p[0] = bv[0]; p[1] = bv[1]; p[2] = bv[2]; p[3] = bv[3];
+          corr = 1.f;
+        }
+        uint4 frag;  // a0 = hi(n-tile 0), a1 = lo(n-tile 0), a2 = hi(n-tile 1), a3 = lo(n-tile 1)
+        split_pair(p[0], p[1], frag.x, frag.y);
+        split_pair(p[2], p[3], frag.z, frag.w);
+        // the P fragments wait in the side area of the next slot, which will hold this tile's V
+        uint4* Pbuf = reinterpret_cast<uint4*>(sides + ((consumed + 1) % kSlots) * kSideBytes);
+        Pbuf[warp * 32 + lane] = frag;
+      } else if (d.type == kSlotVA) {
+        // ===================== partial output of one tile =====================
+        const uint4* Pbuf = reinterpret_cast<const uint4*>(side);
+        if (d.n_valid < kT) {
+          // rows behind the unit's length hold whatever the cache has there: clear them so that a
+          // zero weight times a stray NaN cannot reach the accumulators
+          const int rows = kT - d.n_valid;
+          for (int i = tid; i < rows * 16; i += kConsumers) {
+            const int row = d.n_valid + (i >> 4), c = i & 15;
+            *reinterpret_cast<uint4*>(sl + tile_off(row, c)) = make_uint4(0u, 0u, 0u, 0u);
+          }
+          consumer_sync();
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { o0[i] *= corr; o1[i] *= corr; }
+        const uint32_t vaddr = smem_u32(sl);
+        {
+          const int mi = lane >> 3, r = lane & 7;
+#pragma unroll
+          for (int kk = 0; kk < kT / 16; ++kk) {
+            const uint4 a = Pbuf[kk * 32 + lane];
+            uint32_t b0, b1, b2, b3;
+            ldmatrix_x4_trans(vaddr + tile_off(16 * kk + 8 * (mi & 1) + r, 2 * warp + (mi >> 1)), b0, b1, b2, b3);
+            mma_bf16(o0, a.x, a.y, a.z, a.w, b0, b1);
+            mma_bf16(o1, a.x, a.y, a.z, a.w, b2, b3);
+          }
+        }
+        __syncwarp();
+        fence_async_smem();
+        if (lane == 0) mbar_arrive(&empty[s]);
+
+        if (d.flags & kFlagLast) {
+          // ---------- the item's record ----------
+          PartialRec* pr = pl.part + d.item;
           {
-            const uint32_t vaddr = smem_u32(sl);
-            const int tok = 16 * warp + 8 * (mi & 1) + mr;
-            uint32_t va[8][4], xb[8][2];
-#pragma unroll
-            for (int ks = 0; ks < 8; ++ks)
-              ldmatrix_x4(vaddr + tile_off(tok, 2 * ks + (mi >> 1)), va[ks][0], va[ks][1], va[ks][2], va[ks][3]);
-#pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {
-              // B operand for <v, X>: column 0 = bf16 hi part of X, column 1 = lo part, the rest zero
-              const float2 f0 = *reinterpret_cast<const float2*>(fr->X + 16 * ks + 2 * quad);
-              const float2 f1 = *reinterpret_cast<const float2*>(fr->X + 16 * ks + 8 + 2 * quad);
-              uint32_t h0, l0, h1, l1;
-              split_pair(f0.x, f0.y, h0, l0);
-              split_pair(f1.x, f1.y, h1, l1);
-              xb[ks][0] = head == 0 ? h0 : (head == 1 ? l0 : 0u);
-              xb[ks][1] = head == 0 ? h1 : (head == 1 ? l1 : 0u);
+            const int c0 = 16 * warp + 2 * quad;
+            *reinterpret_cast<float2*>(&pr->o[head][c0]) = make_float2(o0[0] + o0[2], o0[1] + o0[3]);
+            *reinterpret_cast<float2*>(&pr->o[head][c0 + 8]) = make_float2(o1[0] + o1[2], o1[1] + o1[3]);
+          }
+          float ls = l_priv;
+          ls += __shfl_xor_sync(0xffffffffu, ls, 1);
+          ls += __shfl_xor_sync(0xffffffffu, ls, 2);
+          float hs = hb_priv;
+          hs += __shfl_xor_sync(0xffffffffu, hs, 1);
+          hs += __shfl_xor_sync(0xffffffffu, hs, 2);
+          if (quad == 0) {
+            wl[warp * 8 + head] = ls;
+            if (head == 7) whb[warp] = hs;
+            if (warp == 0) wm[head] = m_run;
+          }
+          consumer_sync();
+          if (warp == 0) {
+            if (lane < 8) {
+              float ll = 0.f;
+              for (int w = 0; w < kConsumerWarps; ++w) ll += wl[w * 8 + lane];
+              pr->m[lane] = wm[lane];
+              pr->l[lane] = ll;
             }
-#pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {
-              mma_bf16(ca, va[ks][0], va[ks][1], va[ks][2], va[ks][3], va[ks][0], va[ks][2]);  // x tokens 0..7
-              mma_bf16(cb, va[ks][0], va[ks][1], va[ks][2], va[ks][3], va[ks][1], va[ks][3]);  // x tokens 8..15
-              mma_bf16(cx, va[ks][0], va[ks][1], va[ks][2], va[ks][3], xb[ks][0], xb[ks][1]);
+            if (lane == 8) {
+              float hb = 0.f;
+              for (int w = 0; w < kConsumerWarps; ++w) hb += whb[w];
+              pr->hb = use_base ? hb : 0.f;
             }
           }
-          // lane (head, quad): token `head` of the warp if quad == 0, token head + 8 if quad == 1
-          const int src = (lane & ~3) | (head >> 1);
-          const float vva = __shfl_sync(0xffffffffu, (head & 1) ? ca[1] : ca[0], src);
-          const float vvb = __shfl_sync(0xffffffffu, (head & 1) ? cb[3] : cb[2], src);
-          const float vxa = __shfl_sync(0xffffffffu, cx[0] + cx[1], lane & ~3);
-          const float vxb = __shfl_sync(0xffffffffu, cx[2] + cx[3], lane & ~3);
-          // base score: heads quad and quad + 4 of both tokens, then a sum over the quad
-          const int ra = 16 * warp + head, rb = ra + 8;
-          float ha = 0.f, hbv = 0.f;
-          if (softmax_counted) {
-#pragma unroll
-            for (int gg = 0; gg < 2; ++gg) {
-              const int g = quad + 4 * gg;
-              if (g < G) {
-                const float mg = fr->m[g], il = fr->inv_l[g];
-                ha = fmaf(fast_exp2(side[g * kT + ra] - mg), il, ha);
-                hbv = fmaf(fast_exp2(side[g * kT + rb] - mg), il, hbv);
+          consumer_sync();
+          if (tid == 0) {
+            __threadfence();
+            const int old = atomicAdd(&pl.counter[d.unit], 1);
+            ctl[1] = (old == d.nitems - 1);
+          }
+          consumer_sync();
+          if (ctl[1]) {
+            // ---------- last arriver: merge the unit's records ----------
+            __threadfence();
+            const PartialRec* p0 = pl.part + d.item0;
+            const int hd = tid >> 5, c4 = (tid & 31) * 4;
+            const bool base_row = use_base && hd == 7;
+            float mfin = -INFINITY;
+            for (int c = 0; c < d.nitems; ++c) mfin = fmaxf(mfin, __ldcg(&p0[c].m[hd]));
+            float lfin = 0.f, hbsum = 0.f;
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+            for (int c = 0; c < d.nitems; ++c) {
+              const float f = base_row ? 1.f : exp2f(__ldcg(&p0[c].m[hd]) - mfin);
+              lfin = fmaf(__ldcg(&p0[c].l[hd]), f, lfin);
+              const float4 v = __ldcg(reinterpret_cast<const float4*>(&p0[c].o[hd][c4]));
+              acc.x = fmaf(v.x, f, acc.x);
+              acc.y = fmaf(v.y, f, acc.y);
+              acc.z = fmaf(v.z, f, acc.z);
+              acc.w = fmaf(v.w, f, acc.w);
+              hbsum += __ldcg(&p0[c].hb);
+            }
+            const float inv_l = (hd < G) ? 1.f / lfin : 0.f;
+            FinalRec* fr = pl.fin + d.unit;
+            float4 contrib = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (hd < G) {
+              const float4 on = make_float4(acc.x * inv_l, acc.y * inv_l, acc.z * inv_l, acc.w * inv_l);
+              *reinterpret_cast<float4*>(o + ((size_t)b * dm.Hq + h * G + hd) * kD + c4) = on;
+              if (softmax_counted) contrib = on;
+            } else if (base_row) {
+              contrib = acc;
+            }
+            const float Htot = (softmax_counted ? (float)G : 0.f) + (use_base ? hbsum : 0.f);
+            // X = (sum of the 8 rows of contrib) / Htot; row hd lives in warp hd, so the warps add
+            // their rows one after the other (fixed order: bit-reproducible)
+            for (int r = 0; r < 8; ++r) {
+              if (hd == r) {
+                float4* xp = reinterpret_cast<float4*>(&xrow[c4]);
+                float4 t = (r == 0) ? make_float4(0.f, 0.f, 0.f, 0.f) : *xp;
+                t.x += contrib.x; t.y += contrib.y; t.z += contrib.z; t.w += contrib.w;
+                *xp = t;
               }
+              consumer_sync();
             }
-            ha += __shfl_xor_sync(0xffffffffu, ha, 1);
-            ha += __shfl_xor_sync(0xffffffffu, ha, 2);
-            hbv += __shfl_xor_sync(0xffffffffu, hbv, 1);
-            hbv += __shfl_xor_sync(0xffffffffu, hbv, 2);
-          }
-          const int row = quad == 0 ? ra : rb;
-          const bool mine = quad < 2 && row < d.n_valid;
-          float hj = quad == 0 ? ha : hbv;
-          const float vv = quad == 0 ? vva : vvb, vx = quad == 0 ? vxa : vxb;
-          const size_t slot = (size_t)d.unit * dm.cap + (size_t)d.tile * kT + row;
-          if (mine) {
-            if (mode == CAOTE_BASE_ACCUM) {
-              hj += side[7 * kT + row];
-              base[slot] = hj;
-            } else if (mode == CAOTE_BASE_EXTERNAL) {
-              hj = side[7 * kT + row];
+            if ((tid & 31) == 0) { fr->m[hd] = mfin; fr->inv_l[hd] = inv_l; }
+            if (tid == 0) fr->H = Htot;
+            if (tid < kD) {
+              const float xv = (Htot > 0.f) ? xrow[tid] / Htot : 0.f;
+              fr->X[tid] = xv;
+              float xx = warp_sum(xv * xv);
+              if (lane == 0) wl[warp] = xx;  // warps 0..3
+            }
+            consumer_sync();
+            if (tid == 0) fr->XX = (wl[0] + wl[1]) + (wl[2] + wl[3]);
+            if (tid == 0) {
+              __threadfence();
+              st_release(&pl.ready[d.unit], 1);
             }
           }
-          const float Htot = fr->H, XX = fr->XX;
-          float n2 = fmaxf(vv - 2.f * vx + XX, 0.f);
-          const bool redo = mine && (n2 < 2e-3f * (vv + XX) || 2.f * hj > Htot);
-          unsigned todo = __ballot_sync(0xffffffffu, redo);
-          while (todo) {
-            const int l = __ffs((int)todo) - 1;
-            todo &= todo - 1;
-            const int rr = 16 * warp + (l >> 2) + 8 * (l & 3);  // the row lane l is responsible for
-            const uint2 raw = *reinterpret_cast<const uint2*>(sl + tile_off(rr, lane >> 1) + (lane & 1) * 8);
-            const float4 xv = *reinterpret_cast<const float4*>(fr->X + 4 * lane);
-            const float2 f0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
-            const float2 f1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
-            const float d0 = xv.x - f0.x, d1 = xv.y - f0.y, d2 = xv.z - f1.x, d3 = xv.w - f1.y;
-            const float exact = warp_sum(fmaf(d0, d0, d1 * d1) + fmaf(d2, d2, d3 * d3));
-            if (lane == l) n2 = exact;
-          }
-          if (mine) {
-            float ratio = 0.f;
-            if (Htot > 0.f) {
-              const float rest = Htot - hj;
-              ratio = (rest > 0.f) ? hj / rest : INFINITY;
-            }
-            scores[slot] = (ratio == 0.f) ? 0.f : ((ratio == INFINITY) ? INFINITY : ratio * sqrtf(n2));
-          }
-          const bool last = (d.flags & kFlagLast) != 0;
-          release();
-          if (last) break;
-          if (!next_slot()) { alive = false; break; }
         }
       } else {
-        alive = false;
+        // ===================== score pass of one tile =====================
+        // ||X - v_j||^2 = ||v_j||^2 - 2 <v_j, X> + ||X||^2 for this warp's 16 tokens on the tensor
+        // cores: the V rows are the A operand; used again as the B operand they give the Gram
+        // blocks whose diagonals are ||v_j||^2; X, split into bf16 hi + lo columns, gives <v_j, X>.
+        // Tokens for which that difference cancels (v_j close to X) or that hold most of the weight
+        // are redone below by plain subtraction, so v_j = X still scores exactly 0.
+        const FinalRec* fr = reinterpret_cast<const FinalRec*>(side + 8 * kT);
+        uint32_t xb[8][2];
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          xb[ks][0] = 0u;
+          xb[ks][1] = 0u;
+          if (head < 2) {
+            const float2 x0 = *reinterpret_cast<const float2*>(fr->X + 16 * ks + 2 * quad);
+            const float2 x1 = *reinterpret_cast<const float2*>(fr->X + 16 * ks + 8 + 2 * quad);
+            uint32_t h0, l0, h1, l1;
+            split_pair(x0.x, x0.y, h0, l0);
+            split_pair(x1.x, x1.y, h1, l1);
+            xb[ks][0] = head == 0 ? h0 : l0;
+            xb[ks][1] = head == 0 ? h1 : l1;
+          }
+        }
+        float ca[4] = {0.f, 0.f, 0.f, 0.f}, cb[4] = {0.f, 0.f, 0.f, 0.f}, cx[4] = {0.f, 0.f, 0.f, 0.f};
+        {
+          const uint32_t vaddr = smem_u32(sl);
+          const int mi = lane >> 3, r = lane & 7;
+          const int tok = 16 * warp + 8 * (mi & 1) + r;
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks) {
+            uint32_t a0, a1, a2, a3;
+            ldmatrix_x4(vaddr + tile_off(tok, 2 * ks + (mi >> 1)), a0, a1, a2, a3);
+            mma_bf16(ca, a0, a1, a2, a3, a0, a2);  // rows x tokens 0..7 of the warp
+            mma_bf16(cb, a0, a1, a2, a3, a1, a3);  // rows x tokens 8..15
+            mma_bf16(cx, a0, a1, a2, a3, xb[ks][0], xb[ks][1]);
+          }
+        }
+        // lane (head, quad): token `head` of the warp if quad == 0, token head + 8 if quad == 1
+        const int src = (lane & ~3) | (head >> 1);
+        const float vva = __shfl_sync(0xffffffffu, (head & 1) ? ca[1] : ca[0], src);
+        const float vvb = __shfl_sync(0xffffffffu, (head & 1) ? cb[3] : cb[2], src);
+        const float vxa = __shfl_sync(0xffffffffu, cx[0] + cx[1], lane & ~3);
+        const float vxb = __shfl_sync(0xffffffffu, cx[2] + cx[3], lane & ~3);
+        // base score: heads quad and quad + 4 of both tokens, then a sum over the quad
+        const int ra = 16 * warp + head, rb = ra + 8;
+        float ha = 0.f, hbv = 0.f;
+        if (softmax_counted) {
+#pragma unroll
+          for (int gg = 0; gg < 2; ++gg) {
+            const int g = quad + 4 * gg;
+            if (g < G) {
+              const float mg = fr->m[g], il = fr->inv_l[g];
+              ha = fmaf(fast_exp2(side[g * kT + ra] - mg), il, ha);
+              hbv = fmaf(fast_exp2(side[g * kT + rb] - mg), il, hbv);
+            }
+          }
+          ha += __shfl_xor_sync(0xffffffffu, ha, 1);
+          ha += __shfl_xor_sync(0xffffffffu, ha, 2);
+          hbv += __shfl_xor_sync(0xffffffffu, hbv, 1);
+          hbv += __shfl_xor_sync(0xffffffffu, hbv, 2);
+        }
+        const int row = quad == 0 ? ra : rb;
+        const bool mine = quad < 2 && row < d.n_valid;
+        float hj = quad == 0 ? ha : hbv;
+        const float vv = quad == 0 ? vva : vvb, vx = quad == 0 ? vxa : vxb;
+        const size_t slot = (size_t)d.unit * dm.cap + (size_t)d.tile * kT + row;
+        if (mine) {
+          if (mode == CAOTE_BASE_ACCUM) {
+            hj += side[7 * kT + row];
+            base[slot] = hj;
+          } else if (mode == CAOTE_BASE_EXTERNAL) {
+            hj = side[7 * kT + row];
+          }
+        }
+        const float Htot = fr->H, XX = fr->XX;
+        float n2 = fmaxf(vv - 2.f * vx + XX, 0.f);
+        const bool redo = mine && (n2 < 2e-3f * (vv + XX) || 2.f * hj > Htot);
+        unsigned todo = __ballot_sync(0xffffffffu, redo);
+        while (todo) {
+          const int l = __ffs((int)todo) - 1;
+          todo &= todo - 1;
+          const int rr = 16 * warp + (l >> 2) + 8 * (l & 3);  // the row lane l is responsible for
+          const uint2 raw = *reinterpret_cast<const uint2*>(sl + tile_off(rr, lane >> 1) + (lane & 1) * 8);
+          const float4 xv = *reinterpret_cast<const float4*>(fr->X + 4 * lane);
+          const float2 f0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
+          const float2 f1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
+          const float d0 = xv.x - f0.x, d1 = xv.y - f0.y, d2 = xv.z - f1.x, d3 = xv.w - f1.y;
+          const float exact = warp_sum(fmaf(d0, d0, d1 * d1) + fmaf(d2, d2, d3 * d3));
+          if (lane == l) n2 = exact;
+        }
+        if (mine) {
+          float ratio = 0.f;
+          if (Htot > 0.f) {
+            const float rest = Htot - hj;
+            ratio = (rest > 0.f) ? hj / rest : INFINITY;
+          }
+          scores[slot] = (ratio == 0.f) ? 0.f : ((ratio == INFINITY) ? INFINITY : ratio * sqrtf(n2));
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&empty[s]);
       }
-    }
-    if (lane == 0) {
-      if (!alive && !ctl[0]) {
-        set_status(status, CAOTE_ERR_TIMEOUT);
-        ctl[0] = 1;
-      }
-      if (warp == 0) ctl[5] = items_done;
-      __threadfence_block();
-      atomicAdd_block(const_cast<int*>(&ctl[4]), 1);
     }
   }
 
