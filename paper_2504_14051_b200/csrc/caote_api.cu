@@ -9,6 +9,7 @@
 #include "common.cuh"
 #include "decode_stream.cuh"
 #include "generic_score.cuh"
+#include "prefill_tc.cuh"
 #include "select_compact.cuh"
 
 namespace caote {
@@ -258,12 +259,72 @@ static int launch_decode_score(const Dims& dm, const void* q, const void* K, con
   return CAOTE_OK;
 }
 
+// Shapes the tensor-core prefill kernels cover.
+static bool prefill_shape_ok(const caote_params_t* p) {
+  const int G = p->n_q_heads / p->n_kv_heads;
+  return p->dtype == CAOTE_BF16 && p->head_dim == 128 && p->base_mode == CAOTE_BASE_CHUNK_SUM && p->n_new >= 16 &&
+         (long long)G * p->n_new >= 64 && (long long)p->batch * p->n_kv_heads * p->capacity < (1LL << 31) &&
+         (long long)p->batch * p->n_q_heads * p->n_new < (1LL << 31);
+}
+
+static int encode_rows_map(CUtensorMap* tm, const void* ptr, unsigned long long rows, TensorMapEncodeFn encode) {
+  const cuuint64_t gdim[2] = {128, (cuuint64_t)rows};
+  const cuuint64_t gstride[1] = {256};
+  const cuuint32_t box[2] = {64, 128};
+  const cuuint32_t estride[2] = {1, 1};
+  CUresult r = encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), gdim, gstride, box, estride,
+                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    snprintf(g_cuda_error, sizeof(g_cuda_error), "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+    return CAOTE_ERR_CUDA;
+  }
+  return CAOTE_OK;
+}
+
+static int launch_prefill_score(const Dims& dm, const void* q, const void* K, const void* V, const int* len, float* o,
+                                float* scores, char* ws, cudaStream_t st, bool* used) {
+  *used = false;
+  TensorMapEncodeFn encode = tensor_map_encoder();
+  if (!encode) return CAOTE_OK;
+  prefill::Scratch sc;
+  prefill::carve(dm, ws + kHeaderBytes, &sc);
+  int* status = reinterpret_cast<int*>(ws);
+  CUtensorMap tmQ, tmK, tmV;
+  int rc = encode_rows_map(&tmQ, q, (unsigned long long)dm.B * dm.Hq * dm.m, encode);
+  if (!rc) rc = encode_rows_map(&tmK, K, (unsigned long long)dm.units * dm.cap, encode);
+  if (!rc) rc = encode_rows_map(&tmV, V, (unsigned long long)dm.units * dm.cap, encode);
+  if (rc) return rc;
+  rc = allow_smem(prefill::attn_kernel, prefill::attn_smem_bytes());
+  if (!rc) rc = allow_smem(prefill::score_kernel, prefill::score_smem_bytes());
+  if (rc) return rc;
+  {
+    dim3 grid((dm.R + prefill::kTile - 1) / prefill::kTile, dm.units);
+    CAOTE_LAUNCH("prefill_attn_kernel", st,
+                 prefill::attn_kernel<<<grid, prefill::kThreads, prefill::attn_smem_bytes(), st>>>(tmQ, tmK, tmV, dm, len,
+                                                                                                    sc, o, status));
+  }
+  CAOTE_LAUNCH("prefill_xsum_kernel", st, prefill::xsum_kernel<<<dm.units, prefill::kD, 0, st>>>(dm, len, o, sc));
+  {
+    dim3 grid((dm.cap + prefill::kTile - 1) / prefill::kTile, dm.units);
+    CAOTE_LAUNCH("prefill_score_kernel", st,
+                 prefill::score_kernel<<<grid, prefill::kThreads, prefill::score_smem_bytes(), st>>>(
+                     tmQ, tmK, dm, (const __nv_bfloat16*)V, len, sc, scores, status));
+  }
+  *used = true;
+  return CAOTE_OK;
+}
+
 static size_t workspace_bytes(const caote_params_t* p) {
   const Dims dm = make_dims(p);
   size_t need = generic::carve(dm, nullptr, nullptr);
   if (decode_shape_ok(p)) {
     const size_t need2 = decode::carve(dm, nullptr, nullptr, 0);
     if (need2 > need) need = need2;
+  }
+  if (prefill_shape_ok(p)) {
+    const size_t need3 = prefill::carve(dm, nullptr, nullptr);
+    if (need3 > need) need = need3;
   }
   return kHeaderBytes + need;
 }
@@ -339,6 +400,11 @@ int caote_score(const caote_params_t* p, const void* q, const void* K, const voi
   if (decode_shape_ok(p) && !(p->flags & 0)) {
     bool used = false;
     rc = launch_decode_score(dm, q, K, V, len, base, o, scores, ws, st, &used);
+    if (rc || used) return rc;
+  }
+  if (prefill_shape_ok(p)) {
+    bool used = false;
+    rc = launch_prefill_score(dm, q, K, V, len, o, scores, ws, st, &used);
     if (rc || used) return rc;
   }
   if (p->dtype == CAOTE_BF16) {

@@ -1,0 +1,519 @@
+// Chunked-prefill scoring path on the 5th-generation tensor cores (tcgen05 + TMEM) for bf16,
+// head_dim 128, base mode CHUNK_SUM: a block of m new queries per sequence, M = G * m query rows per
+// (sequence, KV head) unit against its n cached keys.
+//
+//   attn_kernel   rows x keys. One CTA owns 128 query rows of a unit and walks the unit's keys in
+//                 tiles of 128: S = Q K^T (tcgen05.mma, fp32 accumulator in TMEM), per-row online
+//                 softmax (one thread per row, straight out of TMEM), P in bf16 back to shared memory,
+//                 O += P V (second tcgen05.mma; V is the MN-major operand). Writes o and the per-row
+//                 softmax statistics (reference, sum).
+//   xsum_kernel   X = mean of the unit's M output rows (the weights of CHUNK_SUM are the column sums
+//                 of the attention matrix divided by M, so sum_j w_j v_j is the mean output row).
+//   score_kernel  keys x rows. One CTA owns 128 keys of a unit and walks the unit's rows in blocks of
+//                 128: S^T = K Q^T lands in TMEM with one key per lane, so each thread sums
+//                 exp2(s - ref_r) / sum_r over the rows of its own key without any exchange:
+//                 h_j = sum_r alpha_{r,j}. Then c_j = w_j / (1 - w_j) * ||X - v_j||, w_j = h_j / M.
+//
+// Operands are staged by TMA as 64-channel boxes of 128 rows with the 128-byte swizzle, which is the
+// canonical K-major UMMA layout (8-row groups 1024 bytes apart); V in the second product is read
+// through an MN-major descriptor of the same bytes. Every mbarrier wait is bounded by a clock limit;
+// a wait that runs out records CAOTE_ERR_TIMEOUT and the CTA carries on with whatever is in its
+// buffers (all indices stay in bounds), so that no thread is left behind at a barrier.
+#pragma once
+
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace caote {
+namespace prefill {
+
+constexpr int kD = 128;
+constexpr int kTile = 128;                  // rows / keys per tile
+constexpr int kHalfBytes = kTile * 128;     // one 64-channel box
+constexpr int kTileBytes = 2 * kHalfBytes;  // 32 KB
+constexpr int kThreads = 128;
+constexpr long long kWaitCycles = 2000000000LL;
+
+struct Scratch {
+  float* stats;  // [units][Mpad][2]: log2-domain softmax reference, sum of 2^(s - ref)
+  float* X;      // [units][kD]
+  int Mpad;      // M rounded up to a multiple of kTile
+};
+
+inline size_t carve(const Dims& dm, char* base, Scratch* out) {
+  Scratch s;
+  s.Mpad = (dm.R + kTile - 1) / kTile * kTile;
+  size_t off = 0;
+  s.stats = reinterpret_cast<float*>(base + off);
+  off = align_up(off + sizeof(float) * 2 * (size_t)dm.units * s.Mpad, 256);
+  s.X = reinterpret_cast<float*>(base + off);
+  off = align_up(off + sizeof(float) * (size_t)dm.units * kD, 256);
+  if (out) *out = s;
+  return off;
+}
+
+// ---- PTX wrappers ---------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait. On expiry the error is recorded and the caller carries on (see the file comment).
+__device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, int* status) {
+  if (mbar_try_wait(bar, parity)) return;
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity)) {
+    if (clock64() - t0 > kWaitCycles) {
+      set_status(status, CAOTE_ERR_TIMEOUT);
+      return;
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// TMEM: `cols` columns (a power of two >= 32) for this CTA; one warp allocates, the same warp frees.
+__device__ __forceinline__ void tmem_alloc(uint32_t* slot_in_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot_in_smem)), "r"(cols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+
+// Shared-memory matrix descriptor (bf16 tiles staged as 128-byte rows with the 128-byte swizzle).
+//   bits [0,14)  start address >> 4        bits [16,30) leading byte offset >> 4
+//   bits [32,46) stride byte offset >> 4   bits [46,48) descriptor version (1 on sm_100)
+//   bits [61,64) layout type (2 = 128-byte swizzle)
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return (uint64_t)((addr & 0x3ffffu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
+         (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor of tcgen05.mma.kind::f16: bf16 x bf16 -> fp32, M = 128, N = 128.
+//   bits [4,6) D format (1 = f32), [7,10) A format (1 = bf16), [10,13) B format (1 = bf16),
+//   bit 15 A major, bit 16 B major (0 = K-major, 1 = MN-major), [17,23) N >> 3, [24,29) M >> 4.
+__host__ __device__ constexpr uint32_t instr_desc(bool b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+}
+// D[tmem] (+)= A[smem] * B[smem]; issued by one thread.
+__device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, bool accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.u32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"((uint32_t)accumulate) : "memory");
+}
+// The mbarrier gets one arrival once every tcgen05.mma issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// 32 consecutive fp32 columns of this thread's TMEM lane (lane = 32 * (warp % 4) + lane id).
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
+        "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])),
+        "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])),
+        "r"(__float_as_uint(v[11])), "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])),
+        "r"(__float_as_uint(v[15])), "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])),
+        "r"(__float_as_uint(v[19])), "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])),
+        "r"(__float_as_uint(v[23])), "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])),
+        "r"(__float_as_uint(v[27])), "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])),
+        "r"(__float_as_uint(v[31])) : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float x0, float x1) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(x1), "f"(x0));
+  return r;
+}
+// Byte offset of 16-byte chunk `chunk16` (0..15 along 128 bf16) of row `row` in a staged tile.
+__device__ __forceinline__ uint32_t tile_off(int row, int chunk16) {
+  return (uint32_t)((chunk16 >> 3) * kHalfBytes + row * 128 + (((chunk16 & 7) ^ (row & 7)) << 4));
+}
+// Descriptors of k-step ks (16 of the 128 contraction elements) of a staged tile.
+//   K-major: contraction along the 128-byte rows: 32 bytes per step inside a box, second box after 4.
+//   MN-major: contraction along the rows of the tile (16 rows = 2 groups of 8 = 2048 bytes per
+//   step); the two 64-element boxes along MN are kHalfBytes apart (leading byte offset).
+__device__ __forceinline__ uint64_t desc_k_major(uint32_t tile_addr, int ks) {
+  return smem_desc(tile_addr + (ks >> 2) * kHalfBytes + (ks & 3) * 32, 16, 1024);
+}
+__device__ __forceinline__ uint64_t desc_mn_major(uint32_t tile_addr, int ks) {
+  return smem_desc(tile_addr + ks * 2048, kHalfBytes, 1024);
+}
+
+
+inline size_t attn_smem_bytes() { return 1024 + 7 * (size_t)kTileBytes + 256; }
+
+// o and row statistics of 128 query rows of one unit. grid = (row blocks, units), 128 threads.
+__global__ void __launch_bounds__(kThreads, 1)
+attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+            const __grid_constant__ CUtensorMap tmV, Dims dm, const int* __restrict__ len, Scratch sc,
+            float* __restrict__ o, int* status) {
+  extern __shared__ char smem_raw[];
+  char* sm = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  char* Qs = sm;
+  char* Ks = Qs + kTileBytes;       // [2]
+  char* Vs = Ks + 2 * kTileBytes;   // [2]
+  char* Ps = Vs + 2 * kTileBytes;   // [2]: bf16 hi part of P, bf16 lo part (P ~= hi + lo to ~16 bits)
+  uint64_t* bars = reinterpret_cast<uint64_t*>(Ps + 2 * kTileBytes);  // q, kv[2], s, o
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
+
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int unit = blockIdx.y, row0 = blockIdx.x * kTile;
+  const int b = unit / dm.Hkv;
+  const int n = len[b], M = dm.R, m = dm.m;
+  if (n == 0) return;
+  if (n < m || n > dm.cap) {
+    if (tid == 0) set_status(status, CAOTE_ERR_BAD_LENGTH);
+    return;
+  }
+  const int ntiles = (n + kTile - 1) / kTile;
+  const int R = row0 + tid;
+  const int nvis = (R < M) ? n - m + (R % m) + 1 : n;  // keys this row sees (causal inside the block)
+  const float scale2 = dm.scale * 1.4426950408889634f;
+
+  if (tid == 0) {
+    for (int i = 0; i < 5; ++i) mbar_init(&bars[i], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) tmem_alloc(tmem_slot, 256);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t t_s = tmem + ((uint32_t)(warp * 32) << 16);  // this thread's lane, S columns
+  const uint32_t t_o = t_s + 128;                             // O columns
+  uint64_t *q_bar = &bars[0], *kv_bar = &bars[1], *s_bar = &bars[3], *o_bar = &bars[4];
+
+  auto issue_kv = [&](int kt) {  // tid 0
+    const int buf = kt & 1, row = unit * dm.cap + kt * kTile;
+    mbar_expect_tx(&kv_bar[buf], 2 * kTileBytes);
+    tma_load_2d(Ks + buf * kTileBytes, &tmK, 0, row, &kv_bar[buf]);
+    tma_load_2d(Ks + buf * kTileBytes + kHalfBytes, &tmK, 64, row, &kv_bar[buf]);
+    tma_load_2d(Vs + buf * kTileBytes, &tmV, 0, row, &kv_bar[buf]);
+    tma_load_2d(Vs + buf * kTileBytes + kHalfBytes, &tmV, 64, row, &kv_bar[buf]);
+  };
+  if (tid == 0) {
+    mbar_expect_tx(q_bar, kTileBytes);
+    tma_load_2d(Qs, &tmQ, 0, unit * M + row0, q_bar);
+    tma_load_2d(Qs + kHalfBytes, &tmQ, 64, unit * M + row0, q_bar);
+    issue_kv(0);
+  }
+  constexpr uint32_t kIdescKK = instr_desc(false), kIdescKMN = instr_desc(true);
+  const uint32_t q_addr = smem_u32(Qs), p_addr = smem_u32(Ps);
+  float m_ref = -INFINITY, l = 0.f;
+
+  for (int kt = 0; kt < ntiles; ++kt) {
+    const int buf = kt & 1;
+    if (tid == 0 && kt + 1 < ntiles) issue_kv(kt + 1);  // the other buffer: its products have completed
+    if (kt == 0) mbar_wait(q_bar, 0, status);
+    mbar_wait(&kv_bar[buf], (kt >> 1) & 1, status);
+    const int n_valid = min(kTile, n - kt * kTile);
+    if (tid >= n_valid) {
+      // V rows behind the unit's length: clear them so that 0 * (stray NaN) cannot reach O
+      char* vrow = Vs + buf * kTileBytes;
+#pragma unroll
+      for (int c = 0; c < 16; ++c) *reinterpret_cast<uint4*>(vrow + tile_off(tid, c)) = make_uint4(0u, 0u, 0u, 0u);
+      fence_async_smem();
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0) {
+      tc_fence_after();
+      const uint32_t k_addr = smem_u32(Ks + buf * kTileBytes);
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) umma(tmem, desc_k_major(q_addr, ks), desc_k_major(k_addr, ks), kIdescKK, ks > 0);
+      umma_commit(s_bar);
+    }
+    mbar_wait(s_bar, kt & 1, status);
+    tc_fence_after();
+
+    // ---- online softmax of this thread's row ----
+    const int j0 = kt * kTile;
+    float mx = -INFINITY;
+#pragma unroll
+    for (int cc = 0; cc < 4; ++cc) {
+      float v[32];
+      tmem_ld32(t_s + cc * 32, v);
+#pragma unroll
+      for (int i = 0; i < 32; ++i)
+        if (j0 + cc * 32 + i < nvis) mx = fmaxf(mx, v[i] * scale2);
+    }
+    // the reference moves only when a logit exceeds it by more than 8 (p <= 256 in between)
+    const bool need = mx > m_ref + 8.f;
+    if (__any_sync(0xffffffffu, need)) {
+      const float corr = need ? fast_exp2(m_ref - mx) : 1.f;
+      if (need) m_ref = mx;
+      l *= corr;
+      if (kt > 0) {
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) {
+          float v[32];
+          tmem_ld32(t_o + cc * 32, v);
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] *= corr;
+          tmem_st32(t_o + cc * 32, v);
+        }
+        tmem_st_wait();
+      }
+    }
+#pragma unroll
+    for (int cc = 0; cc < 4; ++cc) {
+      float v[32];
+      tmem_ld32(t_s + cc * 32, v);
+      uint32_t pk[16], pl[16];
+#pragma unroll
+      for (int i = 0; i < 32; i += 2) {
+        const float p0 = (j0 + cc * 32 + i < nvis) ? fast_exp2(v[i] * scale2 - m_ref) : 0.f;
+        const float p1 = (j0 + cc * 32 + i + 1 < nvis) ? fast_exp2(v[i + 1] * scale2 - m_ref) : 0.f;
+        const uint32_t hi = pack_bf16(p0, p1);
+        pk[i >> 1] = hi;
+        pl[i >> 1] = pack_bf16(p0 - __uint_as_float(hi << 16), p1 - __uint_as_float(hi & 0xffff0000u));
+        l += p0 + p1;
+      }
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        *reinterpret_cast<uint4*>(Ps + tile_off(tid, cc * 4 + c)) = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+        *reinterpret_cast<uint4*>(Ps + kTileBytes + tile_off(tid, cc * 4 + c)) = make_uint4(pl[4 * c], pl[4 * c + 1], pl[4 * c + 2], pl[4 * c + 3]);
+      }
+    }
+    fence_async_smem();
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0) {
+      tc_fence_after();
+      const uint32_t v_addr = smem_u32(Vs + buf * kTileBytes);
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) {
+        umma(tmem + 128, desc_k_major(p_addr, ks), desc_mn_major(v_addr, ks), kIdescKMN, kt > 0 || ks > 0);
+        umma(tmem + 128, desc_k_major(p_addr + kTileBytes, ks), desc_mn_major(v_addr, ks), kIdescKMN, true);
+      }
+      umma_commit(o_bar);
+    }
+    mbar_wait(o_bar, kt & 1, status);
+    tc_fence_after();
+  }
+
+  // ---- normalise and write out ----
+  const float inv_l = 1.f / l;
+  float* orow = o + ((size_t)unit * M + R) * kD;
+#pragma unroll
+  for (int cc = 0; cc < 4; ++cc) {
+    float v[32];
+    tmem_ld32(t_o + cc * 32, v);  // collective: every lane takes part, rows beyond M just do not store
+    if (R < M) {
+#pragma unroll
+      for (int i = 0; i < 32; i += 4)
+        *reinterpret_cast<float4*>(orow + cc * 32 + i) = make_float4(v[i] * inv_l, v[i + 1] * inv_l, v[i + 2] * inv_l, v[i + 3] * inv_l);
+    }
+  }
+  if (R < M) {
+    sc.stats[((size_t)unit * sc.Mpad + R) * 2] = m_ref;
+    sc.stats[((size_t)unit * sc.Mpad + R) * 2 + 1] = l;
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem, 256);
+}
+
+
+// X[unit] = mean of the unit's M rows of o. grid = units, 128 threads (one per channel).
+__global__ void __launch_bounds__(kD)
+xsum_kernel(Dims dm, const int* __restrict__ len, const float* __restrict__ o, Scratch sc) {
+  const int unit = blockIdx.x, c = threadIdx.x;
+  const int n = len[unit / dm.Hkv];
+  if (n == 0 || n < dm.m || n > dm.cap) return;
+  const float* base = o + (size_t)unit * dm.R * kD + c;
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  int r = 0;
+  for (; r + 4 <= dm.R; r += 4) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) acc[i] += base[(size_t)(r + i) * kD];
+  }
+  for (; r < dm.R; ++r) acc[0] += base[(size_t)r * kD];
+  sc.X[(size_t)unit * kD + c] = ((acc[0] + acc[1]) + (acc[2] + acc[3])) / (float)dm.R;
+}
+
+inline size_t score_smem_bytes() { return 1024 + 3 * (size_t)kTileBytes + 2 * kTile * 2 * sizeof(float) + kD * sizeof(float) + 256; }
+
+// CAOTE scores of 128 keys of one unit. grid = (key tiles, units), 128 threads (one per key).
+__global__ void __launch_bounds__(kThreads, 1)
+score_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, Dims dm,
+             const __nv_bfloat16* __restrict__ V, const int* __restrict__ len, Scratch sc,
+             float* __restrict__ scores, int* status) {
+  extern __shared__ char smem_raw[];
+  char* sm = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  char* Ks = sm;
+  char* Qs = Ks + kTileBytes;                                       // [2]
+  float* st = reinterpret_cast<float*>(Qs + 2 * kTileBytes);        // [2][kTile][2] (ref, 1 / sum)
+  float* Xs = st + 2 * kTile * 2;                                   // [kD]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(Xs + kD);            // k, q[2], s[2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
+
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int unit = blockIdx.y, j0 = blockIdx.x * kTile;
+  const int b = unit / dm.Hkv;
+  const int n = len[b], M = dm.R, m = dm.m;
+  if (n == 0 || n < m || n > dm.cap || j0 >= n) return;
+  const int nblocks = (M + kTile - 1) / kTile;
+  const int j = j0 + tid;  // this thread's key
+  const float scale2 = dm.scale * 1.4426950408889634f;
+
+  if (tid == 0) {
+    for (int i = 0; i < 5; ++i) mbar_init(&bars[i], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) tmem_alloc(tmem_slot, 256);
+  Xs[tid] = sc.X[(size_t)unit * kD + tid];
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);
+  uint64_t *k_bar = &bars[0], *q_bar = &bars[1], *s_bar = &bars[3];
+  constexpr uint32_t kIdesc = instr_desc(false);
+  const uint32_t k_addr = smem_u32(Ks);
+
+  auto issue_q = [&](int rb) {  // tid 0
+    const int buf = rb & 1;
+    mbar_expect_tx(&q_bar[buf], kTileBytes);
+    tma_load_2d(Qs + buf * kTileBytes, &tmQ, 0, unit * M + rb * kTile, &q_bar[buf]);
+    tma_load_2d(Qs + buf * kTileBytes + kHalfBytes, &tmQ, 64, unit * M + rb * kTile, &q_bar[buf]);
+  };
+  auto issue_mma = [&](int rb) {  // tid 0, after Q block rb has landed
+    const int buf = rb & 1;
+    tc_fence_after();
+    const uint32_t q_addr = smem_u32(Qs + buf * kTileBytes);
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks)
+      umma(tmem + buf * 128, desc_k_major(k_addr, ks), desc_k_major(q_addr, ks), kIdesc, ks > 0);
+    umma_commit(&s_bar[buf]);
+  };
+  if (tid == 0) {
+    mbar_expect_tx(k_bar, kTileBytes);
+    tma_load_2d(Ks, &tmK, 0, unit * dm.cap + j0, k_bar);
+    tma_load_2d(Ks + kHalfBytes, &tmK, 64, unit * dm.cap + j0, k_bar);
+    issue_q(0);
+    if (nblocks > 1) issue_q(1);
+    mbar_wait(k_bar, 0, status);
+    mbar_wait(&q_bar[0], 0, status);
+    issue_mma(0);
+  }
+
+  float h = 0.f;
+  for (int rb = 0; rb < nblocks; ++rb) {
+    const int buf = rb & 1;
+    // row statistics of this block (plain loads; rows beyond M get a zero weight)
+    {
+      const int R = rb * kTile + tid;
+      float ref = 0.f, il = 0.f;
+      if (R < M) {
+        ref = sc.stats[((size_t)unit * sc.Mpad + R) * 2];
+        il = 1.f / sc.stats[((size_t)unit * sc.Mpad + R) * 2 + 1];
+      }
+      st[(buf * kTile + tid) * 2] = ref;
+      st[(buf * kTile + tid) * 2 + 1] = il;
+    }
+    // the product of the next block runs while this one is reduced
+    if (tid == 0 && rb + 1 < nblocks) {
+      mbar_wait(&q_bar[buf ^ 1], ((rb + 1) >> 1) & 1, status);
+      issue_mma(rb + 1);
+    }
+    __syncthreads();  // statistics visible
+    mbar_wait(&s_bar[buf], (rb >> 1) & 1, status);
+    tc_fence_after();
+    // only the keys of the new block itself are masked (causal inside the block), and only the last
+    // row block can have columns beyond M
+    const bool plain = (j0 + kTile - 1 < n - m + 1) && (rb * kTile + kTile <= M);
+#pragma unroll
+    for (int cc = 0; cc < 4; ++cc) {
+      float v[32];
+      tmem_ld32(t_lane + buf * 128 + cc * 32, v);
+      const float* stc = st + (buf * kTile + cc * 32) * 2;
+      if (plain) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) h = fmaf(fast_exp2(fmaf(v[i], scale2, -stc[2 * i])), stc[2 * i + 1], h);
+      } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const int R = rb * kTile + cc * 32 + i;  // query row of this column
+          // row R sees key j iff j <= n - m + (R % m)
+          const bool vis = R < M && j < n - m + (R % m) + 1;
+          const float a = fast_exp2(fmaf(v[i], scale2, -stc[2 * i])) * stc[2 * i + 1];
+          h += vis ? a : 0.f;
+        }
+      }
+    }
+    tc_fence_before();
+    __syncthreads();  // everyone is done with S[buf], Q[buf] and the statistics
+    if (tid == 0 && rb + 2 < nblocks) issue_q(rb + 2);
+  }
+
+  // ---- c_j = w_j / (1 - w_j) * ||X - v_j||, w_j = h_j / M ----
+  if (j < n) {
+    const __nv_bfloat16* vrow = V + ((size_t)unit * dm.cap + j) * kD;
+    float acc = 0.f;
+#pragma unroll
+    for (int c = 0; c < kD; c += 8) {
+      float f[8];
+      load8(vrow + c, f);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const float d0 = Xs[c + e] - f[e];
+        acc = fmaf(d0, d0, acc);
+      }
+    }
+    const float Htot = (float)M;
+    const float rest = Htot - h;
+    const float ratio = (rest > 0.f) ? h / rest : INFINITY;
+    scores[(size_t)unit * dm.cap + j] = (ratio == 0.f) ? 0.f : ((ratio == INFINITY) ? INFINITY : ratio * sqrtf(acc));
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem, 256);
+}
+
+}  // namespace prefill
+}  // namespace caote
