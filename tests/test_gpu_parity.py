@@ -54,6 +54,12 @@ SHAPES = [
     (40, 8, 8, 128, 704, 1, [704 - 13 * (i % 7) for i in range(40)]),
     (1, 8, 1, 128, 16400, 1, [16385]),
     (2, 6, 2, 128, 384, 1, [384, 256]),
+    # blocks of queries on the tensor-core prefill path: several row blocks and key tiles, ragged tails,
+    # a sequence shorter than two tiles, a group size that does not fill a row block
+    (2, 16, 2, 128, 1200, 128, [1200, 777]),
+    (1, 8, 1, 128, 700, 512, [699]),
+    (2, 14, 2, 128, 300, 16, [16, 259]),
+    (1, 24, 8, 128, 2200, 32, [2177]),
 ]
 
 
