@@ -152,6 +152,18 @@ def useful_flops(w, caches) -> float:
     return tot
 
 
+def aggregate_over_ranks(ms: float, units_this_rank: float, world: int, device):
+    """Whole-job figures from one rank's: the step time is the MAX over ranks, the work is the SUM over ranks
+    (replicas share nothing, so these two reductions are the only collectives of a multi-GPU run)."""
+    if world <= 1:
+        return float(ms), float(units_this_rank)
+    t_all = torch.tensor([ms], device=device, dtype=torch.float64)
+    torch.distributed.all_reduce(t_all, op=torch.distributed.ReduceOp.MAX)
+    th_all = torch.tensor([units_this_rank], device=device, dtype=torch.float64)
+    torch.distributed.all_reduce(th_all, op=torch.distributed.ReduceOp.SUM)
+    return float(t_all.item()), float(th_all.item())
+
+
 def run_ours(args, w0, rank, world, device):
     import paper_2504_14051_b200 as P
 
@@ -191,15 +203,7 @@ def run_ours(args, w0, rank, world, device):
     status = max(abs(c.status()) for c in caches)
     if status != 0:
         raise RuntimeError(f"device status word = -{status} after the timed region")
-    if world > 1:
-        t_all = torch.tensor([ms], device=device, dtype=torch.float64)
-        torch.distributed.all_reduce(t_all, op=torch.distributed.ReduceOp.MAX)
-        ms = float(t_all.item())
-        th_all = torch.tensor([th_per_step], device=device, dtype=torch.float64)
-        torch.distributed.all_reduce(th_all, op=torch.distributed.ReduceOp.SUM)
-        th_total = float(th_all.item())
-    else:
-        th_total = float(th_per_step)
+    ms, th_total = aggregate_over_ranks(ms, th_per_step, world, device)
     ms_per_step = ms / steps
     value = th_total / (ms_per_step * 1e-3)
 
@@ -265,10 +269,7 @@ def run_ours(args, w0, rank, world, device):
     e1.record(stream)
     barrier()
     e2e_ms = e0.elapsed_time(e1)
-    if world > 1:
-        t_all = torch.tensor([e2e_ms], device=device, dtype=torch.float64)
-        torch.distributed.all_reduce(t_all, op=torch.distributed.ReduceOp.MAX)
-        e2e_ms = float(t_all.item())
+    e2e_ms, _ = aggregate_over_ranks(e2e_ms, th_per_step, world, device)
     e2e_value = th_total / (e2e_ms / e2e_steps * 1e-3)
 
     out = {
