@@ -262,15 +262,16 @@ static int launch_decode_score(const Dims& dm, const void* q, const void* K, con
 // Shapes the tensor-core prefill kernels cover.
 static bool prefill_shape_ok(const caote_params_t* p) {
   const int G = p->n_q_heads / p->n_kv_heads;
-  return p->dtype == CAOTE_BF16 && p->head_dim == 128 && p->base_mode == CAOTE_BASE_CHUNK_SUM && p->n_new >= 16 &&
+  return p->dtype == CAOTE_BF16 && p->head_dim == 128 && p->base_mode == CAOTE_BASE_CHUNK_SUM && p->n_new >= 16 && p->scale > 0.f &&
          (long long)G * p->n_new >= 64 && (long long)p->batch * p->n_kv_heads * p->capacity < (1LL << 31) &&
          (long long)p->batch * p->n_q_heads * p->n_new < (1LL << 31);
 }
 
-static int encode_rows_map(CUtensorMap* tm, const void* ptr, unsigned long long rows, TensorMapEncodeFn encode) {
+static int encode_rows_map(CUtensorMap* tm, const void* ptr, unsigned long long rows, TensorMapEncodeFn encode,
+                           unsigned box_rows = 128) {
   const cuuint64_t gdim[2] = {128, (cuuint64_t)rows};
   const cuuint64_t gstride[1] = {256};
-  const cuuint32_t box[2] = {64, 128};
+  const cuuint32_t box[2] = {64, box_rows};
   const cuuint32_t estride[2] = {1, 1};
   CUresult r = encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), gdim, gstride, box, estride,
                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -290,10 +291,11 @@ static int launch_prefill_score(const Dims& dm, const void* q, const void* K, co
   prefill::Scratch sc;
   prefill::carve(dm, ws + kHeaderBytes, &sc);
   int* status = reinterpret_cast<int*>(ws);
-  CUtensorMap tmQ, tmK, tmV;
+  CUtensorMap tmQ, tmK, tmK64, tmV64;
   int rc = encode_rows_map(&tmQ, q, (unsigned long long)dm.B * dm.Hq * dm.m, encode);
   if (!rc) rc = encode_rows_map(&tmK, K, (unsigned long long)dm.units * dm.cap, encode);
-  if (!rc) rc = encode_rows_map(&tmV, V, (unsigned long long)dm.units * dm.cap, encode);
+  if (!rc) rc = encode_rows_map(&tmK64, K, (unsigned long long)dm.units * dm.cap, encode, prefill::kKeys);
+  if (!rc) rc = encode_rows_map(&tmV64, V, (unsigned long long)dm.units * dm.cap, encode, prefill::kKeys);
   if (rc) return rc;
   rc = allow_smem(prefill::attn_kernel, prefill::attn_smem_bytes());
   if (!rc) rc = allow_smem(prefill::score_kernel, prefill::score_smem_bytes());
@@ -301,7 +303,7 @@ static int launch_prefill_score(const Dims& dm, const void* q, const void* K, co
   {
     dim3 grid((dm.R + prefill::kTile - 1) / prefill::kTile, dm.units);
     CAOTE_LAUNCH("prefill_attn_kernel", st,
-                 prefill::attn_kernel<<<grid, prefill::kThreads, prefill::attn_smem_bytes(), st>>>(tmQ, tmK, tmV, dm, len,
+                 prefill::attn_kernel<<<grid, prefill::kThreads, prefill::attn_smem_bytes(), st>>>(tmQ, tmK64, tmV64, dm, len,
                                                                                                     sc, o, status));
   }
   CAOTE_LAUNCH("prefill_xsum_kernel", st, prefill::xsum_kernel<<<dm.units, prefill::kD, 0, st>>>(dm, len, o, sc));

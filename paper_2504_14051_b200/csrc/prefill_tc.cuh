@@ -184,20 +184,45 @@ __device__ __forceinline__ uint64_t desc_mn_major(uint32_t tile_addr, int ks) {
 }
 
 
-inline size_t attn_smem_bytes() { return 1024 + 7 * (size_t)kTileBytes + 256; }
+// ---- attention pass ---------------------------------------------------------------------------------
+// Keys are walked in tiles of 64 so that three K/V stages, two P buffers (bf16 hi and lo parts each) and
+// the Q block fit in shared memory together; the tensor pipe then always has the next S = Q K^T queued
+// while the threads are busy with the softmax of the current tile:
+//   tensor pipe:  QK(t+1)  PV(t)  QK(t+2)  PV(t+1) ...
+//   threads:      softmax(t) ............ softmax(t+1) ...
+constexpr int kKeys = 64;                    // keys per tile of the attention pass
+constexpr int kKvHalf = kKeys * 128;         // one 64-channel box of 64 keys: 8 KB
+constexpr int kKvTile = 2 * kKvHalf;         // K or V tile: 16 KB
+constexpr int kPTile = kTile * 128;          // P part: 128 rows x 64 keys bf16 = 16 KB
+constexpr int kStages = 3;
+
+inline size_t attn_smem_bytes() {
+  return 1024 + kTileBytes + (size_t)kStages * 2 * kKvTile + 2 * 2 * (size_t)kPTile + 256;
+}
+
+// K-major / MN-major descriptors of k-step ks of a 64-key tile (boxes of 64 rows: kKvHalf apart).
+__device__ __forceinline__ uint64_t desc_k_major64(uint32_t tile_addr, int ks) {
+  return smem_desc(tile_addr + (ks >> 2) * kKvHalf + (ks & 3) * 32, 16, 1024);
+}
+__device__ __forceinline__ uint64_t desc_mn_major64(uint32_t tile_addr, int ks) {
+  return smem_desc(tile_addr + ks * 2048, kKvHalf, 1024);
+}
+__host__ __device__ constexpr uint32_t instr_desc_n(bool b_mn_major, uint32_t n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((n >> 3) << 17) | ((128u >> 4) << 24);
+}
 
 // o and row statistics of 128 query rows of one unit. grid = (row blocks, units), 128 threads.
+// tmK64 / tmV64: tensor maps of K and V with boxes of 64 channels x 64 rows.
 __global__ void __launch_bounds__(kThreads, 1)
-attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-            const __grid_constant__ CUtensorMap tmV, Dims dm, const int* __restrict__ len, Scratch sc,
+attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK64,
+            const __grid_constant__ CUtensorMap tmV64, Dims dm, const int* __restrict__ len, Scratch sc,
             float* __restrict__ o, int* status) {
   extern __shared__ char smem_raw[];
   char* sm = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   char* Qs = sm;
-  char* Ks = Qs + kTileBytes;       // [2]
-  char* Vs = Ks + 2 * kTileBytes;   // [2]
-  char* Ps = Vs + 2 * kTileBytes;   // [2]: bf16 hi part of P, bf16 lo part (P ~= hi + lo to ~16 bits)
-  uint64_t* bars = reinterpret_cast<uint64_t*>(Ps + 2 * kTileBytes);  // q, kv[2], s, o
+  char* KVs = Qs + kTileBytes;                 // [kStages][K tile, V tile]
+  char* Ps = KVs + kStages * 2 * kKvTile;      // [2][hi part, lo part]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(Ps + 2 * 2 * kPTile);  // q, kv[3], s[2], o[2]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
 
   const int tid = threadIdx.x, warp = tid >> 5;
@@ -209,13 +234,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     if (tid == 0) set_status(status, CAOTE_ERR_BAD_LENGTH);
     return;
   }
-  const int ntiles = (n + kTile - 1) / kTile;
+  const int ntiles = (n + kKeys - 1) / kKeys;
   const int R = row0 + tid;
   const int nvis = (R < M) ? n - m + (R % m) + 1 : n;  // keys this row sees (causal inside the block)
   const float scale2 = dm.scale * 1.4426950408889634f;
 
   if (tid == 0) {
-    for (int i = 0; i < 5; ++i) mbar_init(&bars[i], 1);
+    for (int i = 0; i < 8; ++i) mbar_init(&bars[i], 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) tmem_alloc(tmem_slot, 256);
@@ -223,63 +248,69 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t t_s = tmem + ((uint32_t)(warp * 32) << 16);  // this thread's lane, S columns
-  const uint32_t t_o = t_s + 128;                             // O columns
-  uint64_t *q_bar = &bars[0], *kv_bar = &bars[1], *s_bar = &bars[3], *o_bar = &bars[4];
+  const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);  // this thread's lane; S0 [0,64), S1 [64,128)
+  const uint32_t t_o = t_lane + 128;                              // O columns [128,256)
+  uint64_t *q_bar = &bars[0], *kv_bar = &bars[1], *s_bar = &bars[4], *o_bar = &bars[6];
+  constexpr uint32_t kIdescS = instr_desc_n(false, kKeys), kIdescO = instr_desc_n(true, kD);
+  const uint32_t q_addr = smem_u32(Qs);
 
   auto issue_kv = [&](int kt) {  // tid 0
-    const int buf = kt & 1, row = unit * dm.cap + kt * kTile;
-    mbar_expect_tx(&kv_bar[buf], 2 * kTileBytes);
-    tma_load_2d(Ks + buf * kTileBytes, &tmK, 0, row, &kv_bar[buf]);
-    tma_load_2d(Ks + buf * kTileBytes + kHalfBytes, &tmK, 64, row, &kv_bar[buf]);
-    tma_load_2d(Vs + buf * kTileBytes, &tmV, 0, row, &kv_bar[buf]);
-    tma_load_2d(Vs + buf * kTileBytes + kHalfBytes, &tmV, 64, row, &kv_bar[buf]);
+    const int st = kt % kStages, row = unit * dm.cap + kt * kKeys;
+    char* kd = KVs + st * 2 * kKvTile;
+    mbar_expect_tx(&kv_bar[st], 2 * kKvTile);
+    tma_load_2d(kd, &tmK64, 0, row, &kv_bar[st]);
+    tma_load_2d(kd + kKvHalf, &tmK64, 64, row, &kv_bar[st]);
+    tma_load_2d(kd + kKvTile, &tmV64, 0, row, &kv_bar[st]);
+    tma_load_2d(kd + kKvTile + kKvHalf, &tmV64, 64, row, &kv_bar[st]);
+  };
+  auto issue_qk = [&](int kt) {  // tid 0; K of tile kt has landed
+    tc_fence_after();
+    const uint32_t k_addr = smem_u32(KVs + (kt % kStages) * 2 * kKvTile);
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks)
+      umma(tmem + (kt & 1) * kKeys, desc_k_major(q_addr, ks), desc_k_major64(k_addr, ks), kIdescS, ks > 0);
+    umma_commit(&s_bar[kt & 1]);
   };
   if (tid == 0) {
     mbar_expect_tx(q_bar, kTileBytes);
     tma_load_2d(Qs, &tmQ, 0, unit * M + row0, q_bar);
     tma_load_2d(Qs + kHalfBytes, &tmQ, 64, unit * M + row0, q_bar);
     issue_kv(0);
+    if (ntiles > 1) issue_kv(1);
+    mbar_wait(q_bar, 0, status);
+    mbar_wait(&kv_bar[0], 0, status);
+    issue_qk(0);
   }
-  constexpr uint32_t kIdescKK = instr_desc(false), kIdescKMN = instr_desc(true);
-  const uint32_t q_addr = smem_u32(Qs), p_addr = smem_u32(Ps);
   float m_ref = -INFINITY, l = 0.f;
 
   for (int kt = 0; kt < ntiles; ++kt) {
-    const int buf = kt & 1;
-    if (tid == 0 && kt + 1 < ntiles) issue_kv(kt + 1);  // the other buffer: its products have completed
-    if (kt == 0) mbar_wait(q_bar, 0, status);
-    mbar_wait(&kv_bar[buf], (kt >> 1) & 1, status);
-    const int n_valid = min(kTile, n - kt * kTile);
-    if (tid >= n_valid) {
-      // V rows behind the unit's length: clear them so that 0 * (stray NaN) cannot reach O
-      char* vrow = Vs + buf * kTileBytes;
-#pragma unroll
-      for (int c = 0; c < 16; ++c) *reinterpret_cast<uint4*>(vrow + tile_off(tid, c)) = make_uint4(0u, 0u, 0u, 0u);
-      fence_async_smem();
+    const int st = kt % kStages;
+    // (a) queue the next S product behind whatever the tensor pipe is doing
+    if (tid == 0 && kt + 1 < ntiles) {
+      mbar_wait(&kv_bar[(kt + 1) % kStages], ((kt + 1) / kStages) & 1, status);
+      issue_qk(kt + 1);
     }
-    tc_fence_before();
-    __syncthreads();
-    if (tid == 0) {
-      tc_fence_after();
-      const uint32_t k_addr = smem_u32(Ks + buf * kTileBytes);
-#pragma unroll
-      for (int ks = 0; ks < 8; ++ks) umma(tmem, desc_k_major(q_addr, ks), desc_k_major(k_addr, ks), kIdescKK, ks > 0);
-      umma_commit(s_bar);
-    }
-    mbar_wait(s_bar, kt & 1, status);
+    // (b) online softmax of this thread's row over the tile's 64 keys
+    mbar_wait(&s_bar[kt & 1], (kt >> 1) & 1, status);
+    if (tid != 0) mbar_wait(&kv_bar[st], (kt / kStages) & 1, status);  // V of this tile (tid 0 saw it before QK)
     tc_fence_after();
-
-    // ---- online softmax of this thread's row ----
-    const int j0 = kt * kTile;
-    float mx = -INFINITY;
+    const int j0 = kt * kKeys;
+    const uint32_t t_s = t_lane + (kt & 1) * kKeys;
+    float sv[64];  // raw products; masked keys become -inf
+    tmem_ld32(t_s, *reinterpret_cast<float(*)[32]>(&sv[0]));
+    tmem_ld32(t_s + 32, *reinterpret_cast<float(*)[32]>(&sv[32]));
+    if (j0 + kKeys > n - m + 1) {  // only tiles that reach into the new block (or past the length) need the mask
 #pragma unroll
-    for (int cc = 0; cc < 4; ++cc) {
-      float v[32];
-      tmem_ld32(t_s + cc * 32, v);
+      for (int i = 0; i < 64; ++i) sv[i] = (j0 + i < nvis) ? sv[i] : -INFINITY;
+    }
+    float mx;
+    {
+      float pm[8];
 #pragma unroll
-      for (int i = 0; i < 32; ++i)
-        if (j0 + cc * 32 + i < nvis) mx = fmaxf(mx, v[i] * scale2);
+      for (int i = 0; i < 8; ++i) pm[i] = sv[i] * scale2;
+#pragma unroll
+      for (int i = 8; i < 64; ++i) pm[i & 7] = fmaxf(pm[i & 7], sv[i] * scale2);
+      mx = fmaxf(fmaxf(fmaxf(pm[0], pm[1]), fmaxf(pm[2], pm[3])), fmaxf(fmaxf(pm[4], pm[5]), fmaxf(pm[6], pm[7])));
     }
     // the reference moves only when a logit exceeds it by more than 8 (p <= 256 in between)
     const bool need = mx > m_ref + 8.f;
@@ -288,6 +319,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
       if (need) m_ref = mx;
       l *= corr;
       if (kt > 0) {
+        mbar_wait(&o_bar[(kt - 1) & 1], ((kt - 1) >> 1) & 1, status);  // O += P V of the previous tile is done
+        tc_fence_after();
 #pragma unroll
         for (int cc = 0; cc < 4; ++cc) {
           float v[32];
@@ -299,42 +332,64 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         tmem_st_wait();
       }
     }
+    // this tile's P buffer was last read by the product of tile kt - 2
+    if (kt >= 2) mbar_wait(&o_bar[kt & 1], ((kt - 2) >> 1) & 1, status);
+    {
+      char* ph = Ps + (kt & 1) * 2 * kPTile;
+      char* pl = ph + kPTile;
+      const float neg_ref = -m_ref;
+      float ls[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-    for (int cc = 0; cc < 4; ++cc) {
-      float v[32];
-      tmem_ld32(t_s + cc * 32, v);
-      uint32_t pk[16], pl[16];
+      for (int c = 0; c < 8; ++c) {  // 16-byte chunk c = keys 8c .. 8c + 7 of this row
+        uint32_t hi[4], lo[4];
 #pragma unroll
-      for (int i = 0; i < 32; i += 2) {
-        const float p0 = (j0 + cc * 32 + i < nvis) ? fast_exp2(v[i] * scale2 - m_ref) : 0.f;
-        const float p1 = (j0 + cc * 32 + i + 1 < nvis) ? fast_exp2(v[i + 1] * scale2 - m_ref) : 0.f;
-        const uint32_t hi = pack_bf16(p0, p1);
-        pk[i >> 1] = hi;
-        pl[i >> 1] = pack_bf16(p0 - __uint_as_float(hi << 16), p1 - __uint_as_float(hi & 0xffff0000u));
-        l += p0 + p1;
+        for (int e = 0; e < 4; ++e) {
+          // P = hi + lo, hi truncated and lo rounded to bf16 (16 significant bits together); plain bit
+          // operations, so the conversion unit is left to the exponentials
+          const float p0 = fast_exp2(fmaf(sv[8 * c + 2 * e], scale2, neg_ref));
+          const float p1 = fast_exp2(fmaf(sv[8 * c + 2 * e + 1], scale2, neg_ref));
+          const uint32_t b0 = __float_as_uint(p0), b1 = __float_as_uint(p1);
+          hi[e] = __byte_perm(b0, b1, 0x7632);
+          const float r0 = p0 - __uint_as_float(b0 & 0xffff0000u), r1 = p1 - __uint_as_float(b1 & 0xffff0000u);
+          lo[e] = __byte_perm(__float_as_uint(r0) + 0x8000u, __float_as_uint(r1) + 0x8000u, 0x7632);  // rounded
+          ls[e] += p0 + p1;
+        }
+        const uint32_t off = (uint32_t)(tid * 128 + ((c ^ (tid & 7)) << 4));
+        *reinterpret_cast<uint4*>(ph + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+        *reinterpret_cast<uint4*>(pl + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
       }
+      l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
+    }
+    const int n_valid = min(kKeys, n - j0);
+    if (tid < kKeys && tid >= n_valid) {
+      // V rows behind the unit's length: clear them so that 0 * (stray NaN) cannot reach O
+      char* vt = KVs + st * 2 * kKvTile + kKvTile;
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        *reinterpret_cast<uint4*>(Ps + tile_off(tid, cc * 4 + c)) = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-        *reinterpret_cast<uint4*>(Ps + kTileBytes + tile_off(tid, cc * 4 + c)) = make_uint4(pl[4 * c], pl[4 * c + 1], pl[4 * c + 2], pl[4 * c + 3]);
-      }
+      for (int c = 0; c < 16; ++c)
+        *reinterpret_cast<uint4*>(vt + (c >> 3) * kKvHalf + tid * 128 + (((c & 7) ^ (tid & 7)) << 4)) = make_uint4(0u, 0u, 0u, 0u);
     }
     fence_async_smem();
     tc_fence_before();
     __syncthreads();
+    // (c) O += P V, (d) refill the stage that the previous tile's product has released
     if (tid == 0) {
       tc_fence_after();
-      const uint32_t v_addr = smem_u32(Vs + buf * kTileBytes);
+      const uint32_t v_addr = smem_u32(KVs + st * 2 * kKvTile + kKvTile);
+      const uint32_t p_addr = smem_u32(Ps + (kt & 1) * 2 * kPTile);
 #pragma unroll
-      for (int ks = 0; ks < 8; ++ks) {
-        umma(tmem + 128, desc_k_major(p_addr, ks), desc_mn_major(v_addr, ks), kIdescKMN, kt > 0 || ks > 0);
-        umma(tmem + 128, desc_k_major(p_addr + kTileBytes, ks), desc_mn_major(v_addr, ks), kIdescKMN, true);
+      for (int ks = 0; ks < 4; ++ks) {
+        umma(tmem + 128, smem_desc(p_addr + ks * 32, 16, 1024), desc_mn_major64(v_addr, ks), kIdescO, kt > 0 || ks > 0);
+        umma(tmem + 128, smem_desc(p_addr + kPTile + ks * 32, 16, 1024), desc_mn_major64(v_addr, ks), kIdescO, true);
       }
-      umma_commit(o_bar);
+      umma_commit(&o_bar[kt & 1]);
+      if (kt + 2 < ntiles) {
+        if (kt >= 1) mbar_wait(&o_bar[(kt - 1) & 1], ((kt - 1) >> 1) & 1, status);
+        issue_kv(kt + 2);
+      }
     }
-    mbar_wait(o_bar, kt & 1, status);
-    tc_fence_after();
   }
+  mbar_wait(&o_bar[(ntiles - 1) & 1], ((ntiles - 1) >> 1) & 1, status);
+  tc_fence_after();
 
   // ---- normalise and write out ----
   const float inv_l = 1.f / l;
@@ -357,7 +412,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem, 256);
 }
-
 
 // X[unit] = mean of the unit's M rows of o. grid = units, 128 threads (one per channel).
 __global__ void __launch_bounds__(kD)
