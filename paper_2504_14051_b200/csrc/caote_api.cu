@@ -303,7 +303,7 @@ static int launch_prefill_score(const Dims& dm, const void* q, const void* K, co
   {
     dim3 grid((dm.R + prefill::kTile - 1) / prefill::kTile, dm.units);
     CAOTE_LAUNCH("prefill_attn_kernel", st,
-                 prefill::attn_kernel<<<grid, prefill::kThreads, prefill::attn_smem_bytes(), st>>>(tmQ, tmK64, tmV64, dm, len,
+                 prefill::attn_kernel<<<grid, prefill::kAttnThreads, prefill::attn_smem_bytes(), st>>>(tmQ, tmK64, tmV64, dm, len,
                                                                                                     sc, o, status));
   }
   CAOTE_LAUNCH("prefill_xsum_kernel", st, prefill::xsum_kernel<<<dm.units, prefill::kD, 0, st>>>(dm, len, o, sc));

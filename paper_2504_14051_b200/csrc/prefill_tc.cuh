@@ -194,10 +194,12 @@ constexpr int kKeys = 64;                    // keys per tile of the attention p
 constexpr int kKvHalf = kKeys * 128;         // one 64-channel box of 64 keys: 8 KB
 constexpr int kKvTile = 2 * kKvHalf;         // K or V tile: 16 KB
 constexpr int kPTile = kTile * 128;          // P part: 128 rows x 64 keys bf16 = 16 KB
-constexpr int kStages = 3;
+constexpr int kKStages = 4;                  // K runs well ahead: its stage is free as soon as S is formed
+constexpr int kVStages = 3;
+constexpr int kAttnThreads = kThreads + 32;  // 128 softmax threads (one per row) + one warp that issues
 
 inline size_t attn_smem_bytes() {
-  return 1024 + kTileBytes + (size_t)kStages * 2 * kKvTile + 2 * 2 * (size_t)kPTile + 256;
+  return 1024 + kTileBytes + (size_t)(kKStages + kVStages) * kKvTile + 2 * 2 * (size_t)kPTile + 256;
 }
 
 // K-major / MN-major descriptors of k-step ks of a 64-key tile (boxes of 64 rows: kKvHalf apart).
@@ -210,20 +212,27 @@ __device__ __forceinline__ uint64_t desc_mn_major64(uint32_t tile_addr, int ks) 
 __host__ __device__ constexpr uint32_t instr_desc_n(bool b_mn_major, uint32_t n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((n >> 3) << 17) | ((128u >> 4) << 24);
 }
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
 
-// o and row statistics of 128 query rows of one unit. grid = (row blocks, units), 128 threads.
+// o and row statistics of 128 query rows of one unit. grid = (row blocks, units), 160 threads:
+// warps 0..3 own one query row per thread, warp 4 issues every copy and every product.
 // tmK64 / tmV64: tensor maps of K and V with boxes of 64 channels x 64 rows.
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kAttnThreads, 1)
 attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK64,
             const __grid_constant__ CUtensorMap tmV64, Dims dm, const int* __restrict__ len, Scratch sc,
             float* __restrict__ o, int* status) {
   extern __shared__ char smem_raw[];
   char* sm = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   char* Qs = sm;
-  char* KVs = Qs + kTileBytes;                 // [kStages][K tile, V tile]
-  char* Ps = KVs + kStages * 2 * kKvTile;      // [2][hi part, lo part]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(Ps + 2 * 2 * kPTile);  // q, kv[3], s[2], o[2]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
+  char* Ksm = Qs + kTileBytes;                 // [kKStages]
+  char* Vsm = Ksm + kKStages * kKvTile;        // [kVStages]
+  char* Ps = Vsm + kVStages * kKvTile;         // [2][hi part, lo part]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(Ps + 2 * 2 * kPTile);
+  uint64_t *q_bar = &bars[0], *k_bar = &bars[1], *v_bar = &bars[5], *s_bar = &bars[8], *o_bar = &bars[10],
+           *p_bar = &bars[12];                 // 1 + 4 + 3 + 2 + 2 + 2 = 14 barriers
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
 
   const int tid = threadIdx.x, warp = tid >> 5;
   const int unit = blockIdx.y, row0 = blockIdx.x * kTile;
@@ -235,178 +244,193 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     return;
   }
   const int ntiles = (n + kKeys - 1) / kKeys;
-  const int R = row0 + tid;
-  const int nvis = (R < M) ? n - m + (R % m) + 1 : n;  // keys this row sees (causal inside the block)
-  const float scale2 = dm.scale * 1.4426950408889634f;
 
   if (tid == 0) {
-    for (int i = 0; i < 8; ++i) mbar_init(&bars[i], 1);
+    for (int i = 0; i < 12; ++i) mbar_init(&bars[i], 1);
+    mbar_init(&p_bar[0], kThreads);
+    mbar_init(&p_bar[1], kThreads);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) tmem_alloc(tmem_slot, 256);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem = *tmem_slot;
-  const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);  // this thread's lane; S0 [0,64), S1 [64,128)
-  const uint32_t t_o = t_lane + 128;                              // O columns [128,256)
-  uint64_t *q_bar = &bars[0], *kv_bar = &bars[1], *s_bar = &bars[4], *o_bar = &bars[6];
-  constexpr uint32_t kIdescS = instr_desc_n(false, kKeys), kIdescO = instr_desc_n(true, kD);
-  const uint32_t q_addr = smem_u32(Qs);
+  const uint32_t tmem = *tmem_slot;  // S0 columns [0,64), S1 [64,128), O [128,256)
 
-  auto issue_kv = [&](int kt) {  // tid 0
-    const int st = kt % kStages, row = unit * dm.cap + kt * kKeys;
-    char* kd = KVs + st * 2 * kKvTile;
-    mbar_expect_tx(&kv_bar[st], 2 * kKvTile);
-    tma_load_2d(kd, &tmK64, 0, row, &kv_bar[st]);
-    tma_load_2d(kd + kKvHalf, &tmK64, 64, row, &kv_bar[st]);
-    tma_load_2d(kd + kKvTile, &tmV64, 0, row, &kv_bar[st]);
-    tma_load_2d(kd + kKvTile + kKvHalf, &tmV64, 64, row, &kv_bar[st]);
-  };
-  auto issue_qk = [&](int kt) {  // tid 0; K of tile kt has landed
-    tc_fence_after();
-    const uint32_t k_addr = smem_u32(KVs + (kt % kStages) * 2 * kKvTile);
-#pragma unroll
-    for (int ks = 0; ks < 8; ++ks)
-      umma(tmem + (kt & 1) * kKeys, desc_k_major(q_addr, ks), desc_k_major64(k_addr, ks), kIdescS, ks > 0);
-    umma_commit(&s_bar[kt & 1]);
-  };
-  if (tid == 0) {
-    mbar_expect_tx(q_bar, kTileBytes);
-    tma_load_2d(Qs, &tmQ, 0, unit * M + row0, q_bar);
-    tma_load_2d(Qs + kHalfBytes, &tmQ, 64, unit * M + row0, q_bar);
-    issue_kv(0);
-    if (ntiles > 1) issue_kv(1);
-    mbar_wait(q_bar, 0, status);
-    mbar_wait(&kv_bar[0], 0, status);
-    issue_qk(0);
-  }
-  float m_ref = -INFINITY, l = 0.f;
-
-  for (int kt = 0; kt < ntiles; ++kt) {
-    const int st = kt % kStages;
-    // (a) queue the next S product behind whatever the tensor pipe is doing
-    if (tid == 0 && kt + 1 < ntiles) {
-      mbar_wait(&kv_bar[(kt + 1) % kStages], ((kt + 1) / kStages) & 1, status);
-      issue_qk(kt + 1);
-    }
-    // (b) online softmax of this thread's row over the tile's 64 keys
-    mbar_wait(&s_bar[kt & 1], (kt >> 1) & 1, status);
-    if (tid != 0) mbar_wait(&kv_bar[st], (kt / kStages) & 1, status);  // V of this tile (tid 0 saw it before QK)
-    tc_fence_after();
-    const int j0 = kt * kKeys;
-    const uint32_t t_s = t_lane + (kt & 1) * kKeys;
-    float sv[64];  // raw products; masked keys become -inf
-    tmem_ld32(t_s, *reinterpret_cast<float(*)[32]>(&sv[0]));
-    tmem_ld32(t_s + 32, *reinterpret_cast<float(*)[32]>(&sv[32]));
-    if (j0 + kKeys > n - m + 1) {  // only tiles that reach into the new block (or past the length) need the mask
-#pragma unroll
-      for (int i = 0; i < 64; ++i) sv[i] = (j0 + i < nvis) ? sv[i] : -INFINITY;
-    }
-    float mx;
-    {
-      float pm[8];
-#pragma unroll
-      for (int i = 0; i < 8; ++i) pm[i] = sv[i] * scale2;
-#pragma unroll
-      for (int i = 8; i < 64; ++i) pm[i & 7] = fmaxf(pm[i & 7], sv[i] * scale2);
-      mx = fmaxf(fmaxf(fmaxf(pm[0], pm[1]), fmaxf(pm[2], pm[3])), fmaxf(fmaxf(pm[4], pm[5]), fmaxf(pm[6], pm[7])));
-    }
-    // the reference moves only when a logit exceeds it by more than 8 (p <= 256 in between)
-    const bool need = mx > m_ref + 8.f;
-    if (__any_sync(0xffffffffu, need)) {
-      const float corr = need ? fast_exp2(m_ref - mx) : 1.f;
-      if (need) m_ref = mx;
-      l *= corr;
-      if (kt > 0) {
-        mbar_wait(&o_bar[(kt - 1) & 1], ((kt - 1) >> 1) & 1, status);  // O += P V of the previous tile is done
+  if (warp == 4) {
+    // =============================== issuing warp (one lane) ===============================
+    if (tid == kThreads) {
+      constexpr uint32_t kIdescS = instr_desc_n(false, kKeys), kIdescO = instr_desc_n(true, kD);
+      const uint32_t q_addr = smem_u32(Qs);
+      auto load_k = [&](int kt) {
+        const int st = kt % kKStages, row = unit * dm.cap + kt * kKeys;
+        mbar_expect_tx(&k_bar[st], kKvTile);
+        tma_load_2d(Ksm + st * kKvTile, &tmK64, 0, row, &k_bar[st]);
+        tma_load_2d(Ksm + st * kKvTile + kKvHalf, &tmK64, 64, row, &k_bar[st]);
+      };
+      auto load_v = [&](int kt) {
+        const int st = kt % kVStages, row = unit * dm.cap + kt * kKeys;
+        mbar_expect_tx(&v_bar[st], kKvTile);
+        tma_load_2d(Vsm + st * kKvTile, &tmV64, 0, row, &v_bar[st]);
+        tma_load_2d(Vsm + st * kKvTile + kKvHalf, &tmV64, 64, row, &v_bar[st]);
+      };
+      auto issue_qk = [&](int kt) {
+        mbar_wait(&k_bar[kt % kKStages], (kt / kKStages) & 1, status);
         tc_fence_after();
+        const uint32_t k_addr = smem_u32(Ksm + (kt % kKStages) * kKvTile);
 #pragma unroll
-        for (int cc = 0; cc < 4; ++cc) {
-          float v[32];
-          tmem_ld32(t_o + cc * 32, v);
-#pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] *= corr;
-          tmem_st32(t_o + cc * 32, v);
+        for (int ks = 0; ks < 8; ++ks)
+          umma(tmem + (kt & 1) * kKeys, desc_k_major(q_addr, ks), desc_k_major64(k_addr, ks), kIdescS, ks > 0);
+        umma_commit(&s_bar[kt & 1]);
+      };
+      mbar_expect_tx(q_bar, kTileBytes);
+      tma_load_2d(Qs, &tmQ, 0, unit * M + row0, q_bar);
+      tma_load_2d(Qs + kHalfBytes, &tmQ, 64, unit * M + row0, q_bar);
+      for (int kt = 0; kt < kKStages - 1 && kt < ntiles; ++kt) load_k(kt);
+      for (int kt = 0; kt < kVStages - 1 && kt < ntiles; ++kt) load_v(kt);
+      mbar_wait(q_bar, 0, status);
+      issue_qk(0);
+      for (int kt = 0; kt < ntiles; ++kt) {
+        // S of tile kt is formed (or about to be): its K stage's predecessor is free for tile kt + 3
+        if (kt + kKStages - 1 < ntiles) {
+          if (kt >= 1) mbar_wait(&s_bar[(kt - 1) & 1], ((kt - 1) >> 1) & 1, status);  // QK(kt - 1) has read its K
+          load_k(kt + kKStages - 1);
         }
-        tmem_st_wait();
-      }
-    }
-    // this tile's P buffer was last read by the product of tile kt - 2
-    if (kt >= 2) mbar_wait(&o_bar[kt & 1], ((kt - 2) >> 1) & 1, status);
-    {
-      char* ph = Ps + (kt & 1) * 2 * kPTile;
-      char* pl = ph + kPTile;
-      const float neg_ref = -m_ref;
-      float ls[4] = {0.f, 0.f, 0.f, 0.f};
+        // queue S of the next tile: its buffer was read by the softmax of tile kt - 1, which has
+        // arrived on p_bar before PV(kt - 1) was issued
+        if (kt + 1 < ntiles) issue_qk(kt + 1);
+        // O += P V once the rows have written P of this tile
+        mbar_wait(&p_bar[kt & 1], (kt >> 1) & 1, status);
+        mbar_wait(&v_bar[kt % kVStages], (kt / kVStages) & 1, status);
+        tc_fence_after();
+        const uint32_t v_addr = smem_u32(Vsm + (kt % kVStages) * kKvTile);
+        const uint32_t p_addr = smem_u32(Ps + (kt & 1) * 2 * kPTile);
 #pragma unroll
-      for (int c = 0; c < 8; ++c) {  // 16-byte chunk c = keys 8c .. 8c + 7 of this row
-        uint32_t hi[4], lo[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          // P = hi + lo, hi truncated and lo rounded to bf16 (16 significant bits together); plain bit
-          // operations, so the conversion unit is left to the exponentials
-          const float p0 = fast_exp2(fmaf(sv[8 * c + 2 * e], scale2, neg_ref));
-          const float p1 = fast_exp2(fmaf(sv[8 * c + 2 * e + 1], scale2, neg_ref));
-          const uint32_t b0 = __float_as_uint(p0), b1 = __float_as_uint(p1);
-          hi[e] = __byte_perm(b0, b1, 0x7632);
-          const float r0 = p0 - __uint_as_float(b0 & 0xffff0000u), r1 = p1 - __uint_as_float(b1 & 0xffff0000u);
-          lo[e] = __byte_perm(__float_as_uint(r0) + 0x8000u, __float_as_uint(r1) + 0x8000u, 0x7632);  // rounded
-          ls[e] += p0 + p1;
+        for (int ks = 0; ks < 4; ++ks) {
+          umma(tmem + 128, smem_desc(p_addr + ks * 32, 16, 1024), desc_mn_major64(v_addr, ks), kIdescO, kt > 0 || ks > 0);
+          umma(tmem + 128, smem_desc(p_addr + kPTile + ks * 32, 16, 1024), desc_mn_major64(v_addr, ks), kIdescO, true);
         }
-        const uint32_t off = (uint32_t)(tid * 128 + ((c ^ (tid & 7)) << 4));
-        *reinterpret_cast<uint4*>(ph + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-        *reinterpret_cast<uint4*>(pl + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-      }
-      l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
-    }
-    const int n_valid = min(kKeys, n - j0);
-    if (tid < kKeys && tid >= n_valid) {
-      // V rows behind the unit's length: clear them so that 0 * (stray NaN) cannot reach O
-      char* vt = KVs + st * 2 * kKvTile + kKvTile;
-#pragma unroll
-      for (int c = 0; c < 16; ++c)
-        *reinterpret_cast<uint4*>(vt + (c >> 3) * kKvHalf + tid * 128 + (((c & 7) ^ (tid & 7)) << 4)) = make_uint4(0u, 0u, 0u, 0u);
-    }
-    fence_async_smem();
-    tc_fence_before();
-    __syncthreads();
-    // (c) O += P V, (d) refill the stage that the previous tile's product has released
-    if (tid == 0) {
-      tc_fence_after();
-      const uint32_t v_addr = smem_u32(KVs + st * 2 * kKvTile + kKvTile);
-      const uint32_t p_addr = smem_u32(Ps + (kt & 1) * 2 * kPTile);
-#pragma unroll
-      for (int ks = 0; ks < 4; ++ks) {
-        umma(tmem + 128, smem_desc(p_addr + ks * 32, 16, 1024), desc_mn_major64(v_addr, ks), kIdescO, kt > 0 || ks > 0);
-        umma(tmem + 128, smem_desc(p_addr + kPTile + ks * 32, 16, 1024), desc_mn_major64(v_addr, ks), kIdescO, true);
-      }
-      umma_commit(&o_bar[kt & 1]);
-      if (kt + 2 < ntiles) {
-        if (kt >= 1) mbar_wait(&o_bar[(kt - 1) & 1], ((kt - 1) >> 1) & 1, status);
-        issue_kv(kt + 2);
+        umma_commit(&o_bar[kt & 1]);
+        // the V stage of tile kt - 1 is free once its product is done
+        if (kt + kVStages - 1 < ntiles) {
+          if (kt >= 1) mbar_wait(&o_bar[(kt - 1) & 1], ((kt - 1) >> 1) & 1, status);
+          load_v(kt + kVStages - 1);
+        }
       }
     }
-  }
-  mbar_wait(&o_bar[(ntiles - 1) & 1], ((ntiles - 1) >> 1) & 1, status);
-  tc_fence_after();
+  } else {
+    // =============================== one query row per thread ===============================
+    const int R = row0 + tid;
+    const int nvis = (R < M) ? n - m + (R % m) + 1 : n;  // keys this row sees (causal inside the block)
+    const float scale2 = dm.scale * 1.4426950408889634f;
+    const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);
+    const uint32_t t_o = t_lane + 128;
+    float m_ref = -INFINITY, l = 0.f;
 
-  // ---- normalise and write out ----
-  const float inv_l = 1.f / l;
-  float* orow = o + ((size_t)unit * M + R) * kD;
+    for (int kt = 0; kt < ntiles; ++kt) {
+      mbar_wait(&s_bar[kt & 1], (kt >> 1) & 1, status);
+      tc_fence_after();
+      const int j0 = kt * kKeys;
+      const uint32_t t_s = t_lane + (kt & 1) * kKeys;
+      float sv[64];  // raw products; masked keys become -inf
+      tmem_ld32(t_s, *reinterpret_cast<float(*)[32]>(&sv[0]));
+      tmem_ld32(t_s + 32, *reinterpret_cast<float(*)[32]>(&sv[32]));
+      if (j0 + kKeys > n - m + 1) {  // only tiles that reach into the new block (or past the length) need the mask
 #pragma unroll
-  for (int cc = 0; cc < 4; ++cc) {
-    float v[32];
-    tmem_ld32(t_o + cc * 32, v);  // collective: every lane takes part, rows beyond M just do not store
-    if (R < M) {
+        for (int i = 0; i < 64; ++i) sv[i] = (j0 + i < nvis) ? sv[i] : -INFINITY;
+      }
+      float mx;
+      {
+        float pm[8];
 #pragma unroll
-      for (int i = 0; i < 32; i += 4)
-        *reinterpret_cast<float4*>(orow + cc * 32 + i) = make_float4(v[i] * inv_l, v[i + 1] * inv_l, v[i + 2] * inv_l, v[i + 3] * inv_l);
+        for (int i = 0; i < 8; ++i) pm[i] = sv[i] * scale2;
+#pragma unroll
+        for (int i = 8; i < 64; ++i) pm[i & 7] = fmaxf(pm[i & 7], sv[i] * scale2);
+        mx = fmaxf(fmaxf(fmaxf(pm[0], pm[1]), fmaxf(pm[2], pm[3])), fmaxf(fmaxf(pm[4], pm[5]), fmaxf(pm[6], pm[7])));
+      }
+      // the reference moves only when a logit exceeds it by more than 8 (p <= 256 in between)
+      const bool need = mx > m_ref + 8.f;
+      if (__any_sync(0xffffffffu, need)) {
+        const float corr = need ? fast_exp2(m_ref - mx) : 1.f;
+        if (need) m_ref = mx;
+        l *= corr;
+        if (kt > 0) {
+          mbar_wait(&o_bar[(kt - 1) & 1], ((kt - 1) >> 1) & 1, status);  // O += P V of the previous tile is done
+          tc_fence_after();
+#pragma unroll
+          for (int cc = 0; cc < 4; ++cc) {
+            float v[32];
+            tmem_ld32(t_o + cc * 32, v);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] *= corr;
+            tmem_st32(t_o + cc * 32, v);
+          }
+          tmem_st_wait();
+        }
+      }
+      // this tile's P buffer was last read by the product of tile kt - 2
+      if (kt >= 2) mbar_wait(&o_bar[kt & 1], ((kt - 2) >> 1) & 1, status);
+      {
+        char* ph = Ps + (kt & 1) * 2 * kPTile;
+        char* pl = ph + kPTile;
+        const float neg_ref = -m_ref;
+        float ls[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {  // 16-byte chunk c = keys 8c .. 8c + 7 of this row
+          uint32_t hi[4], lo[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            // P = hi + lo, hi truncated and lo rounded to bf16 (16 significant bits together); plain bit
+            // operations, so the conversion unit is left to the exponentials
+            const float p0 = fast_exp2(fmaf(sv[8 * c + 2 * e], scale2, neg_ref));
+            const float p1 = fast_exp2(fmaf(sv[8 * c + 2 * e + 1], scale2, neg_ref));
+            const uint32_t b0 = __float_as_uint(p0), b1 = __float_as_uint(p1);
+            hi[e] = __byte_perm(b0, b1, 0x7632);
+            const float r0 = p0 - __uint_as_float(b0 & 0xffff0000u), r1 = p1 - __uint_as_float(b1 & 0xffff0000u);
+            lo[e] = __byte_perm(__float_as_uint(r0) + 0x8000u, __float_as_uint(r1) + 0x8000u, 0x7632);  // rounded
+            ls[e] += p0 + p1;
+          }
+          const uint32_t off = (uint32_t)(tid * 128 + ((c ^ (tid & 7)) << 4));
+          *reinterpret_cast<uint4*>(ph + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+          *reinterpret_cast<uint4*>(pl + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        }
+        l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
+      }
+      const int n_valid = min(kKeys, n - j0);
+      if (n_valid < kKeys) {
+        // V rows behind the unit's length: clear them so that 0 * (stray NaN) cannot reach O
+        mbar_wait(&v_bar[kt % kVStages], (kt / kVStages) & 1, status);
+        if (tid < kKeys && tid >= n_valid) {
+          char* vt = Vsm + (kt % kVStages) * kKvTile;
+#pragma unroll
+          for (int c = 0; c < 16; ++c)
+            *reinterpret_cast<uint4*>(vt + (c >> 3) * kKvHalf + tid * 128 + (((c & 7) ^ (tid & 7)) << 4)) = make_uint4(0u, 0u, 0u, 0u);
+        }
+      }
+      fence_async_smem();
+      tc_fence_before();
+      mbar_arrive(&p_bar[kt & 1]);
     }
-  }
-  if (R < M) {
-    sc.stats[((size_t)unit * sc.Mpad + R) * 2] = m_ref;
-    sc.stats[((size_t)unit * sc.Mpad + R) * 2 + 1] = l;
+    mbar_wait(&o_bar[(ntiles - 1) & 1], ((ntiles - 1) >> 1) & 1, status);
+    tc_fence_after();
+
+    // ---- normalise and write out ----
+    const float inv_l = 1.f / l;
+    float* orow = o + ((size_t)unit * M + R) * kD;
+#pragma unroll
+    for (int cc = 0; cc < 4; ++cc) {
+      float v[32];
+      tmem_ld32(t_o + cc * 32, v);  // collective: every lane takes part, rows beyond M just do not store
+      if (R < M) {
+#pragma unroll
+        for (int i = 0; i < 32; i += 4)
+          *reinterpret_cast<float4*>(orow + cc * 32 + i) = make_float4(v[i] * inv_l, v[i + 1] * inv_l, v[i + 2] * inv_l, v[i + 3] * inv_l);
+      }
+    }
+    if (R < M) {
+      sc.stats[((size_t)unit * sc.Mpad + R) * 2] = m_ref;
+      sc.stats[((size_t)unit * sc.Mpad + R) * 2 + 1] = l;
+    }
   }
   tc_fence_before();
   __syncthreads();
