@@ -156,6 +156,24 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) 
         "r"(__float_as_uint(v[27])), "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])),
         "r"(__float_as_uint(v[31])) : "memory");
 }
+__device__ __forceinline__ void tmem_st32u(uint32_t taddr, const uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
+        "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(v[16]), "r"(v[17]),
+        "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]),
+        "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31]) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]: the A operand (K-major, two bf16 per 32-bit column) comes from TMEM.
+__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, bool accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.u32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"((uint32_t)accumulate) : "memory");
+}
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 __device__ __forceinline__ float fast_exp2(float x) {
@@ -193,13 +211,12 @@ __device__ __forceinline__ uint64_t desc_mn_major(uint32_t tile_addr, int ks) {
 constexpr int kKeys = 64;                    // keys per tile of the attention pass
 constexpr int kKvHalf = kKeys * 128;         // one 64-channel box of 64 keys: 8 KB
 constexpr int kKvTile = 2 * kKvHalf;         // K or V tile: 16 KB
-constexpr int kPTile = kTile * 128;          // P part: 128 rows x 64 keys bf16 = 16 KB
-constexpr int kKStages = 4;                  // K runs well ahead: its stage is free as soon as S is formed
-constexpr int kVStages = 3;
+constexpr int kKStages = 6;                  // K runs well ahead: its stage is free as soon as S is formed
+constexpr int kVStages = 5;
 constexpr int kAttnThreads = kThreads + 32;  // 128 softmax threads (one per row) + one warp that issues
 
 inline size_t attn_smem_bytes() {
-  return 1024 + kTileBytes + (size_t)(kKStages + kVStages) * kKvTile + 2 * 2 * (size_t)kPTile + 256;
+  return 1024 + kTileBytes + (size_t)(kKStages + kVStages) * kKvTile + 256;
 }
 
 // K-major / MN-major descriptors of k-step ks of a 64-key tile (boxes of 64 rows: kKvHalf apart).
@@ -228,11 +245,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
   char* Qs = sm;
   char* Ksm = Qs + kTileBytes;                 // [kKStages]
   char* Vsm = Ksm + kKStages * kKvTile;        // [kVStages]
-  char* Ps = Vsm + kVStages * kKvTile;         // [2][hi part, lo part]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(Ps + 2 * 2 * kPTile);
-  uint64_t *q_bar = &bars[0], *k_bar = &bars[1], *v_bar = &bars[5], *s_bar = &bars[8], *o_bar = &bars[10],
-           *p_bar = &bars[12];                 // 1 + 4 + 3 + 2 + 2 + 2 = 14 barriers
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(Vsm + kVStages * kKvTile);
+  uint64_t *q_bar = &bars[0], *k_bar = &bars[1], *v_bar = k_bar + kKStages, *s_bar = v_bar + kVStages, *o_bar = s_bar + 2,
+           *p_bar = o_bar + 2;
+  constexpr int kBars = 1 + kKStages + kVStages + 6;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kBars);
 
   const int tid = threadIdx.x, warp = tid >> 5;
   const int unit = blockIdx.y, row0 = blockIdx.x * kTile;
@@ -246,16 +263,17 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
   const int ntiles = (n + kKeys - 1) / kKeys;
 
   if (tid == 0) {
-    for (int i = 0; i < 12; ++i) mbar_init(&bars[i], 1);
+    for (int i = 0; i < kBars - 2; ++i) mbar_init(&bars[i], 1);
     mbar_init(&p_bar[0], kThreads);
     mbar_init(&p_bar[1], kThreads);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 0) tmem_alloc(tmem_slot, 256);
+  if (warp == 0) tmem_alloc(tmem_slot, 512);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem = *tmem_slot;  // S0 columns [0,64), S1 [64,128), O [128,256)
+  // columns: S0 [0,64), S1 [64,128), O [128,256), P0 hi [256,288) lo [288,320), P1 hi [320,352) lo [352,384)
+  const uint32_t tmem = *tmem_slot;
 
   if (warp == 4) {
     // =============================== issuing warp (one lane) ===============================
@@ -304,11 +322,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         mbar_wait(&v_bar[kt % kVStages], (kt / kVStages) & 1, status);
         tc_fence_after();
         const uint32_t v_addr = smem_u32(Vsm + (kt % kVStages) * kKvTile);
-        const uint32_t p_addr = smem_u32(Ps + (kt & 1) * 2 * kPTile);
+        const uint32_t p_tmem = tmem + 256 + (kt & 1) * 64;
 #pragma unroll
-        for (int ks = 0; ks < 4; ++ks) {
-          umma(tmem + 128, smem_desc(p_addr + ks * 32, 16, 1024), desc_mn_major64(v_addr, ks), kIdescO, kt > 0 || ks > 0);
-          umma(tmem + 128, smem_desc(p_addr + kPTile + ks * 32, 16, 1024), desc_mn_major64(v_addr, ks), kIdescO, true);
+        for (int ks = 0; ks < 4; ++ks) {  // 16 keys = 8 packed columns per step
+          umma_ts(tmem + 128, p_tmem + ks * 8, desc_mn_major64(v_addr, ks), kIdescO, kt > 0 || ks > 0);
+          umma_ts(tmem + 128, p_tmem + 32 + ks * 8, desc_mn_major64(v_addr, ks), kIdescO, true);
         }
         umma_commit(&o_bar[kt & 1]);
         // the V stage of tile kt - 1 is free once its product is done
@@ -371,29 +389,25 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
       // this tile's P buffer was last read by the product of tile kt - 2
       if (kt >= 2) mbar_wait(&o_bar[kt & 1], ((kt - 2) >> 1) & 1, status);
       {
-        char* ph = Ps + (kt & 1) * 2 * kPTile;
-        char* pl = ph + kPTile;
         const float neg_ref = -m_ref;
         float ls[4] = {0.f, 0.f, 0.f, 0.f};
+        uint32_t hi[32], lo[32];  // column c = keys 2c (low half) and 2c + 1
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {  // 16-byte chunk c = keys 8c .. 8c + 7 of this row
-          uint32_t hi[4], lo[4];
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            // P = hi + lo, hi truncated and lo rounded to bf16 (16 significant bits together); plain bit
-            // operations, so the conversion unit is left to the exponentials
-            const float p0 = fast_exp2(fmaf(sv[8 * c + 2 * e], scale2, neg_ref));
-            const float p1 = fast_exp2(fmaf(sv[8 * c + 2 * e + 1], scale2, neg_ref));
-            const uint32_t b0 = __float_as_uint(p0), b1 = __float_as_uint(p1);
-            hi[e] = __byte_perm(b0, b1, 0x7632);
-            const float r0 = p0 - __uint_as_float(b0 & 0xffff0000u), r1 = p1 - __uint_as_float(b1 & 0xffff0000u);
-            lo[e] = __byte_perm(__float_as_uint(r0) + 0x8000u, __float_as_uint(r1) + 0x8000u, 0x7632);  // rounded
-            ls[e] += p0 + p1;
-          }
-          const uint32_t off = (uint32_t)(tid * 128 + ((c ^ (tid & 7)) << 4));
-          *reinterpret_cast<uint4*>(ph + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-          *reinterpret_cast<uint4*>(pl + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        for (int c = 0; c < 32; ++c) {
+          // P = hi + lo, hi truncated and lo rounded to bf16 (16 significant bits together); plain bit
+          // operations, so the conversion unit is left to the exponentials
+          const float p0 = fast_exp2(fmaf(sv[2 * c], scale2, neg_ref));
+          const float p1 = fast_exp2(fmaf(sv[2 * c + 1], scale2, neg_ref));
+          const uint32_t b0 = __float_as_uint(p0), b1 = __float_as_uint(p1);
+          hi[c] = __byte_perm(b0, b1, 0x7632);
+          const float r0 = p0 - __uint_as_float(b0 & 0xffff0000u), r1 = p1 - __uint_as_float(b1 & 0xffff0000u);
+          lo[c] = __byte_perm(__float_as_uint(r0) + 0x8000u, __float_as_uint(r1) + 0x8000u, 0x7632);  // rounded
+          ls[c & 3] += p0 + p1;
         }
+        const uint32_t t_p = t_lane + 256 + (kt & 1) * 64;
+        tmem_st32u(t_p, hi);
+        tmem_st32u(t_p + 32, lo);
+        tmem_st_wait();
         l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
       }
       const int n_valid = min(kKeys, n - j0);
@@ -434,7 +448,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) tmem_dealloc(tmem, 256);
+  if (warp == 0) tmem_dealloc(tmem, 512);
 }
 
 // X[unit] = mean of the unit's M rows of o. grid = units, 128 threads (one per channel).
