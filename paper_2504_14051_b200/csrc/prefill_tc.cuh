@@ -213,7 +213,7 @@ constexpr int kKvHalf = kKeys * 128;         // one 64-channel box of 64 keys: 8
 constexpr int kKvTile = 2 * kKvHalf;         // K or V tile: 16 KB
 constexpr int kKStages = 6;                  // K runs well ahead: its stage is free as soon as S is formed
 constexpr int kVStages = 5;
-constexpr int kAttnThreads = kThreads + 32;  // 128 softmax threads (one per row) + one warp that issues
+constexpr int kAttnThreads = kThreads + 96;  // 128 softmax threads (one per row) + MMA, K-load and V-load warps
 
 inline size_t attn_smem_bytes() {
   return 1024 + kTileBytes + (size_t)(kKStages + kVStages) * kKvTile + 256;
@@ -233,8 +233,9 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
-// o and row statistics of 128 query rows of one unit. grid = (row blocks, units), 160 threads:
-// warps 0..3 own one query row per thread, warp 4 issues every copy and every product.
+// o and row statistics of 128 query rows of one unit. grid = (row blocks, units), 224 threads:
+// warps 0..3 own one query row per thread; one lane each of warps 4, 5, 6 issues the products, the K
+// copies and the V copies.
 // tmK64 / tmV64: tensor maps of K and V with boxes of 64 channels x 64 rows.
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK64,
@@ -247,8 +248,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
   char* Vsm = Ksm + kKStages * kKvTile;        // [kVStages]
   uint64_t* bars = reinterpret_cast<uint64_t*>(Vsm + kVStages * kKvTile);
   uint64_t *q_bar = &bars[0], *k_bar = &bars[1], *v_bar = k_bar + kKStages, *s_bar = v_bar + kVStages, *o_bar = s_bar + 2,
-           *p_bar = o_bar + 2;
-  constexpr int kBars = 1 + kKStages + kVStages + 6;
+           *p_bar = o_bar + 2, *k_free = p_bar + 2, *v_free = k_free + kKStages;
+  constexpr int kBars = 1 + 2 * (kKStages + kVStages) + 6;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kBars);
 
   const int tid = threadIdx.x, warp = tid >> 5;
@@ -263,7 +264,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
   const int ntiles = (n + kKeys - 1) / kKeys;
 
   if (tid == 0) {
-    for (int i = 0; i < kBars - 2; ++i) mbar_init(&bars[i], 1);
+    for (int i = 0; i < kBars; ++i) mbar_init(&bars[i], 1);
     mbar_init(&p_bar[0], kThreads);
     mbar_init(&p_bar[1], kThreads);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -275,23 +276,36 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
   // columns: S0 [0,64), S1 [64,128), O [128,256), P0 hi [256,288) lo [288,320), P1 hi [320,352) lo [352,384)
   const uint32_t tmem = *tmem_slot;
 
-  if (warp == 4) {
-    // =============================== issuing warp (one lane) ===============================
-    if (tid == kThreads) {
-      constexpr uint32_t kIdescS = instr_desc_n(false, kKeys), kIdescO = instr_desc_n(true, kD);
-      const uint32_t q_addr = smem_u32(Qs);
-      auto load_k = [&](int kt) {
+  if (warp == 5) {
+    // =============================== K loads (one lane) ===============================
+    if (tid == kThreads + 32) {
+      mbar_expect_tx(q_bar, kTileBytes);
+      tma_load_2d(Qs, &tmQ, 0, unit * M + row0, q_bar);
+      tma_load_2d(Qs + kHalfBytes, &tmQ, 64, unit * M + row0, q_bar);
+      for (int kt = 0; kt < ntiles; ++kt) {
         const int st = kt % kKStages, row = unit * dm.cap + kt * kKeys;
+        if (kt >= kKStages) mbar_wait(&k_free[st], ((kt / kKStages) - 1) & 1, status);  // S of tile kt - 6 is formed
         mbar_expect_tx(&k_bar[st], kKvTile);
         tma_load_2d(Ksm + st * kKvTile, &tmK64, 0, row, &k_bar[st]);
         tma_load_2d(Ksm + st * kKvTile + kKvHalf, &tmK64, 64, row, &k_bar[st]);
-      };
-      auto load_v = [&](int kt) {
+      }
+    }
+  } else if (warp == 6) {
+    // =============================== V loads (one lane) ===============================
+    if (tid == kThreads + 64) {
+      for (int kt = 0; kt < ntiles; ++kt) {
         const int st = kt % kVStages, row = unit * dm.cap + kt * kKeys;
+        if (kt >= kVStages) mbar_wait(&v_free[st], ((kt / kVStages) - 1) & 1, status);  // O += P V of tile kt - 5 is done
         mbar_expect_tx(&v_bar[st], kKvTile);
         tma_load_2d(Vsm + st * kKvTile, &tmV64, 0, row, &v_bar[st]);
         tma_load_2d(Vsm + st * kKvTile + kKvHalf, &tmV64, 64, row, &v_bar[st]);
-      };
+      }
+    }
+  } else if (warp == 4) {
+    // =============================== products (one lane) ===============================
+    if (tid == kThreads) {
+      constexpr uint32_t kIdescS = instr_desc_n(false, kKeys), kIdescO = instr_desc_n(true, kD);
+      const uint32_t q_addr = smem_u32(Qs);
       auto issue_qk = [&](int kt) {
         mbar_wait(&k_bar[kt % kKStages], (kt / kKStages) & 1, status);
         tc_fence_after();
@@ -300,20 +314,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         for (int ks = 0; ks < 8; ++ks)
           umma(tmem + (kt & 1) * kKeys, desc_k_major(q_addr, ks), desc_k_major64(k_addr, ks), kIdescS, ks > 0);
         umma_commit(&s_bar[kt & 1]);
+        umma_commit(&k_free[kt % kKStages]);
       };
-      mbar_expect_tx(q_bar, kTileBytes);
-      tma_load_2d(Qs, &tmQ, 0, unit * M + row0, q_bar);
-      tma_load_2d(Qs + kHalfBytes, &tmQ, 64, unit * M + row0, q_bar);
-      for (int kt = 0; kt < kKStages - 1 && kt < ntiles; ++kt) load_k(kt);
-      for (int kt = 0; kt < kVStages - 1 && kt < ntiles; ++kt) load_v(kt);
       mbar_wait(q_bar, 0, status);
       issue_qk(0);
       for (int kt = 0; kt < ntiles; ++kt) {
-        // S of tile kt is formed (or about to be): its K stage's predecessor is free for tile kt + 3
-        if (kt + kKStages - 1 < ntiles) {
-          if (kt >= 1) mbar_wait(&s_bar[(kt - 1) & 1], ((kt - 1) >> 1) & 1, status);  // QK(kt - 1) has read its K
-          load_k(kt + kKStages - 1);
-        }
         // queue S of the next tile: its buffer was read by the softmax of tile kt - 1, which has
         // arrived on p_bar before PV(kt - 1) was issued
         if (kt + 1 < ntiles) issue_qk(kt + 1);
@@ -329,11 +334,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
           umma_ts(tmem + 128, p_tmem + 32 + ks * 8, desc_mn_major64(v_addr, ks), kIdescO, true);
         }
         umma_commit(&o_bar[kt & 1]);
-        // the V stage of tile kt - 1 is free once its product is done
-        if (kt + kVStages - 1 < ntiles) {
-          if (kt >= 1) mbar_wait(&o_bar[(kt - 1) & 1], ((kt - 1) >> 1) & 1, status);
-          load_v(kt + kVStages - 1);
-        }
+        umma_commit(&v_free[kt % kVStages]);
       }
     }
   } else {
