@@ -310,7 +310,7 @@ static int launch_prefill_score(const Dims& dm, const void* q, const void* K, co
   {
     dim3 grid((dm.cap + prefill::kTile - 1) / prefill::kTile, dm.units);
     CAOTE_LAUNCH("prefill_score_kernel", st,
-                 prefill::score_kernel<<<grid, prefill::kThreads, prefill::score_smem_bytes(), st>>>(
+                 prefill::score_kernel<<<grid, prefill::kScoreThreads, prefill::score_smem_bytes(), st>>>(
                      tmQ, tmK, dm, (const __nv_bfloat16*)V, len, sc, scores, status));
   }
   *used = true;

@@ -36,7 +36,7 @@ constexpr int kThreads = 128;
 constexpr long long kWaitCycles = 2000000000LL;
 
 struct Scratch {
-  float* stats;  // [units][Mpad][2]: log2-domain softmax reference, sum of 2^(s - ref)
+  float* stats;  // [units][Mpad][2]: log2-domain softmax reference, 1 / sum of 2^(s - ref)
   float* X;      // [units][kD]
   int Mpad;      // M rounded up to a multiple of kTile
 };
@@ -444,7 +444,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     }
     if (R < M) {
       sc.stats[((size_t)unit * sc.Mpad + R) * 2] = m_ref;
-      sc.stats[((size_t)unit * sc.Mpad + R) * 2 + 1] = l;
+      sc.stats[((size_t)unit * sc.Mpad + R) * 2 + 1] = inv_l;
     }
   }
   tc_fence_before();
@@ -469,20 +469,30 @@ xsum_kernel(Dims dm, const int* __restrict__ len, const float* __restrict__ o, S
   sc.X[(size_t)unit * kD + c] = ((acc[0] + acc[1]) + (acc[2] + acc[3])) / (float)dm.R;
 }
 
-inline size_t score_smem_bytes() { return 1024 + 3 * (size_t)kTileBytes + 2 * kTile * 2 * sizeof(float) + kD * sizeof(float) + 256; }
+constexpr int kScoreThreads = kThreads + 64;  // 128 key threads + a warp for the products + a warp for the copies
+constexpr int kStatBytes = kTile * 2 * 4;     // (reference, 1 / sum) of the 128 rows of a block
+constexpr int kQStage = kTileBytes + kStatBytes;
 
-// CAOTE scores of 128 keys of one unit. grid = (key tiles, units), 128 threads (one per key).
-__global__ void __launch_bounds__(kThreads, 1)
+inline size_t score_smem_bytes() { return 1024 + kTileBytes + 2 * (size_t)kQStage + kD * sizeof(float) + 256; }
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+      ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+
+// CAOTE scores of 128 keys of one unit. grid = (key tiles, units), 192 threads: warps 0..3 own one key
+// per thread, one lane of warp 4 issues the products, one lane of warp 5 the copies.
+__global__ void __launch_bounds__(kScoreThreads, 2)
 score_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, Dims dm,
              const __nv_bfloat16* __restrict__ V, const int* __restrict__ len, Scratch sc,
              float* __restrict__ scores, int* status) {
   extern __shared__ char smem_raw[];
   char* sm = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   char* Ks = sm;
-  char* Qs = Ks + kTileBytes;                                       // [2]
-  float* st = reinterpret_cast<float*>(Qs + 2 * kTileBytes);        // [2][kTile][2] (ref, 1 / sum)
-  float* Xs = st + 2 * kTile * 2;                                   // [kD]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(Xs + kD);            // k, q[2], s[2]
+  char* Qst = Ks + kTileBytes;                                       // [2][Q block, row statistics]
+  float* Xs = reinterpret_cast<float*>(Qst + 2 * kQStage);           // [kD]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(Xs + kD);             // k, q[2], s[2], c[2]
+  uint64_t *k_bar = &bars[0], *q_bar = &bars[1], *s_bar = &bars[3], *c_bar = &bars[5];
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
 
   const int tid = threadIdx.x, warp = tid >> 5;
@@ -491,101 +501,100 @@ score_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
   const int n = len[b], M = dm.R, m = dm.m;
   if (n == 0 || n < m || n > dm.cap || j0 >= n) return;
   const int nblocks = (M + kTile - 1) / kTile;
-  const int j = j0 + tid;  // this thread's key
-  const float scale2 = dm.scale * 1.4426950408889634f;
 
   if (tid == 0) {
     for (int i = 0; i < 5; ++i) mbar_init(&bars[i], 1);
+    mbar_init(&c_bar[0], kThreads);
+    mbar_init(&c_bar[1], kThreads);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) tmem_alloc(tmem_slot, 256);
-  Xs[tid] = sc.X[(size_t)unit * kD + tid];
+  if (tid < kD) Xs[tid] = sc.X[(size_t)unit * kD + tid];
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);
-  uint64_t *k_bar = &bars[0], *q_bar = &bars[1], *s_bar = &bars[3];
-  constexpr uint32_t kIdesc = instr_desc(false);
-  const uint32_t k_addr = smem_u32(Ks);
-
-  auto issue_q = [&](int rb) {  // tid 0
-    const int buf = rb & 1;
-    mbar_expect_tx(&q_bar[buf], kTileBytes);
-    tma_load_2d(Qs + buf * kTileBytes, &tmQ, 0, unit * M + rb * kTile, &q_bar[buf]);
-    tma_load_2d(Qs + buf * kTileBytes + kHalfBytes, &tmQ, 64, unit * M + rb * kTile, &q_bar[buf]);
-  };
-  auto issue_mma = [&](int rb) {  // tid 0, after Q block rb has landed
-    const int buf = rb & 1;
-    tc_fence_after();
-    const uint32_t q_addr = smem_u32(Qs + buf * kTileBytes);
-#pragma unroll
-    for (int ks = 0; ks < 8; ++ks)
-      umma(tmem + buf * 128, desc_k_major(k_addr, ks), desc_k_major(q_addr, ks), kIdesc, ks > 0);
-    umma_commit(&s_bar[buf]);
-  };
-  if (tid == 0) {
-    mbar_expect_tx(k_bar, kTileBytes);
-    tma_load_2d(Ks, &tmK, 0, unit * dm.cap + j0, k_bar);
-    tma_load_2d(Ks + kHalfBytes, &tmK, 64, unit * dm.cap + j0, k_bar);
-    issue_q(0);
-    if (nblocks > 1) issue_q(1);
-    mbar_wait(k_bar, 0, status);
-    mbar_wait(&q_bar[0], 0, status);
-    issue_mma(0);
-  }
-
   float h = 0.f;
-  for (int rb = 0; rb < nblocks; ++rb) {
-    const int buf = rb & 1;
-    // row statistics of this block (plain loads; rows beyond M get a zero weight)
-    {
-      const int R = rb * kTile + tid;
-      float ref = 0.f, il = 0.f;
-      if (R < M) {
-        ref = sc.stats[((size_t)unit * sc.Mpad + R) * 2];
-        il = 1.f / sc.stats[((size_t)unit * sc.Mpad + R) * 2 + 1];
+  const int j = j0 + tid;  // key threads: this thread's key
+
+  if (warp == 5) {
+    // =============================== copies (one lane) ===============================
+    if (tid == kThreads + 32) {
+      mbar_expect_tx(k_bar, kTileBytes);
+      tma_load_2d(Ks, &tmK, 0, unit * dm.cap + j0, k_bar);
+      tma_load_2d(Ks + kHalfBytes, &tmK, 64, unit * dm.cap + j0, k_bar);
+      for (int rb = 0; rb < nblocks; ++rb) {
+        const int buf = rb & 1;
+        if (rb >= 2) mbar_wait(&c_bar[buf], ((rb - 2) >> 1) & 1, status);  // block rb - 2 is reduced
+        char* qd = Qst + buf * kQStage;
+        mbar_expect_tx(&q_bar[buf], kQStage);
+        tma_load_2d(qd, &tmQ, 0, unit * M + rb * kTile, &q_bar[buf]);
+        tma_load_2d(qd + kHalfBytes, &tmQ, 64, unit * M + rb * kTile, &q_bar[buf]);
+        bulk_load(qd + kTileBytes, sc.stats + ((size_t)unit * sc.Mpad + (size_t)rb * kTile) * 2, kStatBytes, &q_bar[buf]);
       }
-      st[(buf * kTile + tid) * 2] = ref;
-      st[(buf * kTile + tid) * 2 + 1] = il;
     }
-    // the product of the next block runs while this one is reduced
-    if (tid == 0 && rb + 1 < nblocks) {
-      mbar_wait(&q_bar[buf ^ 1], ((rb + 1) >> 1) & 1, status);
-      issue_mma(rb + 1);
+  } else if (warp == 4) {
+    // =============================== products (one lane) ===============================
+    if (tid == kThreads) {
+      constexpr uint32_t kIdesc = instr_desc(false);
+      const uint32_t k_addr = smem_u32(Ks);
+      mbar_wait(k_bar, 0, status);
+      for (int rb = 0; rb < nblocks; ++rb) {
+        const int buf = rb & 1;
+        mbar_wait(&q_bar[buf], (rb >> 1) & 1, status);
+        if (rb >= 2) mbar_wait(&c_bar[buf], ((rb - 2) >> 1) & 1, status);  // its S buffer has been read
+        tc_fence_after();
+        const uint32_t q_addr = smem_u32(Qst + buf * kQStage);
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks)
+          umma(tmem + buf * 128, desc_k_major(k_addr, ks), desc_k_major(q_addr, ks), kIdesc, ks > 0);
+        umma_commit(&s_bar[buf]);
+      }
     }
-    __syncthreads();  // statistics visible
-    mbar_wait(&s_bar[buf], (rb >> 1) & 1, status);
-    tc_fence_after();
-    // only the keys of the new block itself are masked (causal inside the block), and only the last
-    // row block can have columns beyond M
-    const bool plain = (j0 + kTile - 1 < n - m + 1) && (rb * kTile + kTile <= M);
+  } else {
+    // =============================== one key per thread ===============================
+    const float scale2 = dm.scale * 1.4426950408889634f;
+    const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);
+    for (int rb = 0; rb < nblocks; ++rb) {
+      const int buf = rb & 1;
+      mbar_wait(&q_bar[buf], (rb >> 1) & 1, status);  // the row statistics have landed
+      mbar_wait(&s_bar[buf], (rb >> 1) & 1, status);
+      tc_fence_after();
+      const float* st = reinterpret_cast<const float*>(Qst + buf * kQStage + kTileBytes);
+      // only the keys of the new block itself are masked (causal inside the block), and only the last
+      // row block can have columns beyond M
+      const bool plain = (j0 + kTile - 1 < n - m + 1) && (rb * kTile + kTile <= M);
 #pragma unroll
-    for (int cc = 0; cc < 4; ++cc) {
-      float v[32];
-      tmem_ld32(t_lane + buf * 128 + cc * 32, v);
-      const float* stc = st + (buf * kTile + cc * 32) * 2;
-      if (plain) {
+      for (int cc = 0; cc < 4; ++cc) {
+        float v[32];
+        tmem_ld32(t_lane + buf * 128 + cc * 32, v);
+        const float* stc = st + cc * 32 * 2;
+        if (plain) {
+          float h4[4] = {0.f, 0.f, 0.f, 0.f};  // independent partial sums
 #pragma unroll
-        for (int i = 0; i < 32; ++i) h = fmaf(fast_exp2(fmaf(v[i], scale2, -stc[2 * i])), stc[2 * i + 1], h);
-      } else {
+          for (int i = 0; i < 32; ++i) {
+            const float2 rs = *reinterpret_cast<const float2*>(stc + 2 * i);  // (reference, 1 / sum) of the row
+            h4[i & 3] = fmaf(fast_exp2(fmaf(v[i], scale2, -rs.x)), rs.y, h4[i & 3]);
+          }
+          h += (h4[0] + h4[1]) + (h4[2] + h4[3]);
+        } else {
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const int R = rb * kTile + cc * 32 + i;  // query row of this column
-          // row R sees key j iff j <= n - m + (R % m)
-          const bool vis = R < M && j < n - m + (R % m) + 1;
-          const float a = fast_exp2(fmaf(v[i], scale2, -stc[2 * i])) * stc[2 * i + 1];
-          h += vis ? a : 0.f;
+          for (int i = 0; i < 32; ++i) {
+            const int R = rb * kTile + cc * 32 + i;  // query row of this column
+            // row R sees key j iff j <= n - m + (R % m)
+            const bool vis = R < M && j < n - m + (R % m) + 1;
+            const float a = fast_exp2(fmaf(v[i], scale2, -stc[2 * i])) * stc[2 * i + 1];
+            h += vis ? a : 0.f;
+          }
         }
       }
+      tc_fence_before();
+      mbar_arrive(&c_bar[buf]);
     }
-    tc_fence_before();
-    __syncthreads();  // everyone is done with S[buf], Q[buf] and the statistics
-    if (tid == 0 && rb + 2 < nblocks) issue_q(rb + 2);
   }
 
   // ---- c_j = w_j / (1 - w_j) * ||X - v_j||, w_j = h_j / M ----
-  if (j < n) {
+  if (tid < kThreads && j < n) {
     const __nv_bfloat16* vrow = V + ((size_t)unit * dm.cap + j) * kD;
     float acc = 0.f;
 #pragma unroll
