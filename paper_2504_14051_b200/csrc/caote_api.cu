@@ -308,7 +308,7 @@ static int launch_prefill_score(const Dims& dm, const void* q, const void* K, co
   }
   CAOTE_LAUNCH("prefill_xsum_kernel", st, prefill::xsum_kernel<<<dm.units, prefill::kD, 0, st>>>(dm, len, o, sc));
   {
-    dim3 grid((dm.cap + prefill::kTile - 1) / prefill::kTile, dm.units);
+    dim3 grid((dm.cap + prefill::kScoreKeys - 1) / prefill::kScoreKeys, dm.units);
     CAOTE_LAUNCH("prefill_score_kernel", st,
                  prefill::score_kernel<<<grid, prefill::kScoreThreads, prefill::score_smem_bytes(), st>>>(
                      tmQ, tmK, dm, (const __nv_bfloat16*)V, len, sc, scores, status));

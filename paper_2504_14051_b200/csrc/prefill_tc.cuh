@@ -469,106 +469,116 @@ xsum_kernel(Dims dm, const int* __restrict__ len, const float* __restrict__ o, S
   sc.X[(size_t)unit * kD + c] = ((acc[0] + acc[1]) + (acc[2] + acc[3])) / (float)dm.R;
 }
 
-constexpr int kScoreThreads = kThreads + 64;  // 128 key threads + a warp for the products + a warp for the copies
-constexpr int kStatBytes = kTile * 2 * 4;     // (reference, 1 / sum) of the 128 rows of a block
+constexpr int kScoreKeys = 2 * kTile;            // keys per CTA: two key tiles share every Q block
+constexpr int kScoreThreads = kScoreKeys + 64;    // 256 key threads + a warp for the products + a warp for the copies
+constexpr int kStatBytes = kTile * 2 * 4;         // (reference, 1 / sum) of the 128 rows of a block
 constexpr int kQStage = kTileBytes + kStatBytes;
+constexpr int kQStages = 3;
 
-inline size_t score_smem_bytes() { return 1024 + kTileBytes + 2 * (size_t)kQStage + kD * sizeof(float) + 256; }
+inline size_t score_smem_bytes() { return 1024 + 2 * kTileBytes + kQStages * (size_t)kQStage + kD * sizeof(float) + 256; }
 __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
   asm volatile(
       "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
       ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 
-// CAOTE scores of 128 keys of one unit. grid = (key tiles, units), 192 threads: warps 0..3 own one key
-// per thread, one lane of warp 4 issues the products, one lane of warp 5 the copies.
-__global__ void __launch_bounds__(kScoreThreads, 2)
+// CAOTE scores of 256 keys of one unit. grid = (key tile pairs, units), 320 threads: warps 0..7 own one
+// key per thread (warps 0..3 the first key tile, 4..7 the second), one lane of warp 8 issues the products,
+// one lane of warp 9 the copies.
+__global__ void __launch_bounds__(kScoreThreads, 1)
 score_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, Dims dm,
              const __nv_bfloat16* __restrict__ V, const int* __restrict__ len, Scratch sc,
              float* __restrict__ scores, int* status) {
   extern __shared__ char smem_raw[];
   char* sm = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  char* Ks = sm;
-  char* Qst = Ks + kTileBytes;                                       // [2][Q block, row statistics]
-  float* Xs = reinterpret_cast<float*>(Qst + 2 * kQStage);           // [kD]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(Xs + kD);             // k, q[2], s[2], c[2]
-  uint64_t *k_bar = &bars[0], *q_bar = &bars[1], *s_bar = &bars[3], *c_bar = &bars[5];
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
+  char* Ks = sm;                                                     // [2] key tiles
+  char* Qst = Ks + 2 * kTileBytes;                                   // [kQStages][Q block, row statistics]
+  float* Xs = reinterpret_cast<float*>(Qst + kQStages * kQStage);    // [kD]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(Xs + kD);
+  uint64_t *k_bar = &bars[0], *q_bar = &bars[1], *s_bar = q_bar + kQStages, *c_bar = s_bar + 2, *q_free = c_bar + 2;
+  constexpr int kBars = 1 + kQStages + 2 + 2 + kQStages;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kBars);
 
   const int tid = threadIdx.x, warp = tid >> 5;
-  const int unit = blockIdx.y, j0 = blockIdx.x * kTile;
+  const int unit = blockIdx.y, j0 = blockIdx.x * kScoreKeys;
   const int b = unit / dm.Hkv;
   const int n = len[b], M = dm.R, m = dm.m;
   if (n == 0 || n < m || n > dm.cap || j0 >= n) return;
   const int nblocks = (M + kTile - 1) / kTile;
 
   if (tid == 0) {
-    for (int i = 0; i < 5; ++i) mbar_init(&bars[i], 1);
-    mbar_init(&c_bar[0], kThreads);
-    mbar_init(&c_bar[1], kThreads);
+    for (int i = 0; i < 1 + kQStages + 2; ++i) mbar_init(&bars[i], 1);
+    for (int i = 0; i < 2; ++i) mbar_init(&c_bar[i], kScoreKeys);
+    for (int i = 0; i < kQStages; ++i) mbar_init(&q_free[i], kScoreKeys);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 0) tmem_alloc(tmem_slot, 256);
+  if (warp == 0) tmem_alloc(tmem_slot, 512);
   if (tid < kD) Xs[tid] = sc.X[(size_t)unit * kD + tid];
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem = *tmem_slot;
+  const uint32_t tmem = *tmem_slot;  // key tile kk, buffer buf: columns [kk * 256 + buf * 128, + 128)
   float h = 0.f;
   const int j = j0 + tid;  // key threads: this thread's key
 
-  if (warp == 5) {
+  if (warp == 9) {
     // =============================== copies (one lane) ===============================
-    if (tid == kThreads + 32) {
-      mbar_expect_tx(k_bar, kTileBytes);
-      tma_load_2d(Ks, &tmK, 0, unit * dm.cap + j0, k_bar);
-      tma_load_2d(Ks + kHalfBytes, &tmK, 64, unit * dm.cap + j0, k_bar);
+    if (tid == kScoreKeys + 32) {
+      mbar_expect_tx(k_bar, 2 * kTileBytes);
+      for (int kk = 0; kk < 2; ++kk) {
+        tma_load_2d(Ks + kk * kTileBytes, &tmK, 0, unit * dm.cap + j0 + kk * kTile, k_bar);
+        tma_load_2d(Ks + kk * kTileBytes + kHalfBytes, &tmK, 64, unit * dm.cap + j0 + kk * kTile, k_bar);
+      }
       for (int rb = 0; rb < nblocks; ++rb) {
-        const int buf = rb & 1;
-        if (rb >= 2) mbar_wait(&c_bar[buf], ((rb - 2) >> 1) & 1, status);  // block rb - 2 is reduced
-        char* qd = Qst + buf * kQStage;
-        mbar_expect_tx(&q_bar[buf], kQStage);
-        tma_load_2d(qd, &tmQ, 0, unit * M + rb * kTile, &q_bar[buf]);
-        tma_load_2d(qd + kHalfBytes, &tmQ, 64, unit * M + rb * kTile, &q_bar[buf]);
-        bulk_load(qd + kTileBytes, sc.stats + ((size_t)unit * sc.Mpad + (size_t)rb * kTile) * 2, kStatBytes, &q_bar[buf]);
+        const int st = rb % kQStages;
+        if (rb >= kQStages) mbar_wait(&q_free[st], ((rb / kQStages) - 1) & 1, status);  // block rb - 3 is reduced
+        char* qd = Qst + st * kQStage;
+        mbar_expect_tx(&q_bar[st], kQStage);
+        tma_load_2d(qd, &tmQ, 0, unit * M + rb * kTile, &q_bar[st]);
+        tma_load_2d(qd + kHalfBytes, &tmQ, 64, unit * M + rb * kTile, &q_bar[st]);
+        bulk_load(qd + kTileBytes, sc.stats + ((size_t)unit * sc.Mpad + (size_t)rb * kTile) * 2, kStatBytes, &q_bar[st]);
       }
     }
-  } else if (warp == 4) {
+  } else if (warp == 8) {
     // =============================== products (one lane) ===============================
-    if (tid == kThreads) {
+    if (tid == kScoreKeys) {
       constexpr uint32_t kIdesc = instr_desc(false);
       const uint32_t k_addr = smem_u32(Ks);
       mbar_wait(k_bar, 0, status);
       for (int rb = 0; rb < nblocks; ++rb) {
-        const int buf = rb & 1;
-        mbar_wait(&q_bar[buf], (rb >> 1) & 1, status);
-        if (rb >= 2) mbar_wait(&c_bar[buf], ((rb - 2) >> 1) & 1, status);  // its S buffer has been read
+        const int buf = rb & 1, st = rb % kQStages;
+        mbar_wait(&q_bar[st], (rb / kQStages) & 1, status);
+        if (rb >= 2) mbar_wait(&c_bar[buf], ((rb - 2) >> 1) & 1, status);  // its S buffers have been read
         tc_fence_after();
-        const uint32_t q_addr = smem_u32(Qst + buf * kQStage);
+        const uint32_t q_addr = smem_u32(Qst + st * kQStage);
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks)
-          umma(tmem + buf * 128, desc_k_major(k_addr, ks), desc_k_major(q_addr, ks), kIdesc, ks > 0);
+        for (int kk = 0; kk < 2; ++kk) {
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks)
+            umma(tmem + kk * 256 + buf * 128, desc_k_major(k_addr + kk * kTileBytes, ks), desc_k_major(q_addr, ks), kIdesc, ks > 0);
+        }
         umma_commit(&s_bar[buf]);
       }
     }
   } else {
     // =============================== one key per thread ===============================
     const float scale2 = dm.scale * 1.4426950408889634f;
-    const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);
+    const int kk = warp >> 2;
+    const uint32_t t_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16) + kk * 256;
     for (int rb = 0; rb < nblocks; ++rb) {
-      const int buf = rb & 1;
-      mbar_wait(&q_bar[buf], (rb >> 1) & 1, status);  // the row statistics have landed
+      const int buf = rb & 1, st = rb % kQStages;
+      mbar_wait(&q_bar[st], (rb / kQStages) & 1, status);  // the row statistics have landed
       mbar_wait(&s_bar[buf], (rb >> 1) & 1, status);
       tc_fence_after();
-      const float* st = reinterpret_cast<const float*>(Qst + buf * kQStage + kTileBytes);
+      const float* stt = reinterpret_cast<const float*>(Qst + st * kQStage + kTileBytes);
       // only the keys of the new block itself are masked (causal inside the block), and only the last
       // row block can have columns beyond M
-      const bool plain = (j0 + kTile - 1 < n - m + 1) && (rb * kTile + kTile <= M);
+      const bool plain = (j0 + kScoreKeys - 1 < n - m + 1) && (rb * kTile + kTile <= M);
 #pragma unroll
       for (int cc = 0; cc < 4; ++cc) {
         float v[32];
         tmem_ld32(t_lane + buf * 128 + cc * 32, v);
-        const float* stc = st + cc * 32 * 2;
+        const float* stc = stt + cc * 32 * 2;
         if (plain) {
           float h4[4] = {0.f, 0.f, 0.f, 0.f};  // independent partial sums
 #pragma unroll
@@ -590,11 +600,12 @@ score_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       }
       tc_fence_before();
       mbar_arrive(&c_bar[buf]);
+      mbar_arrive(&q_free[st]);
     }
   }
 
   // ---- c_j = w_j / (1 - w_j) * ||X - v_j||, w_j = h_j / M ----
-  if (tid < kThreads && j < n) {
+  if (tid < kScoreKeys && j < n) {
     const __nv_bfloat16* vrow = V + ((size_t)unit * dm.cap + j) * kD;
     float acc = 0.f;
 #pragma unroll
@@ -614,7 +625,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) tmem_dealloc(tmem, 256);
+  if (warp == 0) tmem_dealloc(tmem, 512);
 }
 
 }  // namespace prefill
