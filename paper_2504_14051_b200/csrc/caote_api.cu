@@ -488,6 +488,19 @@ int caote_step(const caote_params_t* p, const void* q, const void* k_new, const 
   }
   rc = caote_score(p, q, K, V, len, base, o, scores, workspace, workspace_bytes_, stream);
   if (rc) return rc;
+  if (compact_mode == CAOTE_COMPACT_FILL) {
+    // selection, compaction and the length update in one launch (same results as the two calls below)
+    if (!budget || !evict_idx || !n_evict || max_evict < 1) return CAOTE_ERR_INVALID_ARG;
+    const Dims dm = make_dims(p);
+    const int row_bytes = dm.D * (p->dtype == CAOTE_BF16 ? 2 : 4);
+    cudaStream_t st = (cudaStream_t)stream;
+    int* hdr = reinterpret_cast<int*>(workspace);
+    CAOTE_LAUNCH("select_compact_kernel", st,
+                 sel::select_compact_kernel<<<dm.units, sel::kSelThreads, 0, st>>>(
+                     dm.B, dm.Hkv, dm.cap, row_bytes, scores, (char*)K, (char*)V, base, pos, len, budget, evict_idx,
+                     max_evict, n_evict, hdr, hdr + 4));
+    return CAOTE_OK;
+  }
   rc = caote_select_evict(p, scores, len, budget, pos, evict_idx, max_evict, n_evict, workspace,
                           workspace_bytes_, stream);
   if (rc) return rc;

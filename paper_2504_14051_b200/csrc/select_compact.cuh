@@ -20,10 +20,11 @@ __device__ __forceinline__ unsigned long long make_key(float score, int pos) {
 // One CTA per unit. k = max(0, n - budget). Finds the k-th smallest key by 8 passes of an 8-bit
 // radix histogram (most significant digit first), then writes the slots whose key is <= that key in
 // ascending slot order with a block-wide ordered compaction.
-__global__ void __launch_bounds__(kSelThreads)
-select_kernel(int Hkv, int cap, const float* __restrict__ scores, const int* __restrict__ len,
-              const int* __restrict__ budget, const int* __restrict__ pos, int* __restrict__ evict_idx,
-              int max_evict, int* __restrict__ n_evict, int* status) {
+// Returns k, the number of slots the unit evicts (the same value in every thread of the CTA).
+__device__ __forceinline__ int select_unit(int unit, int Hkv, int cap, const float* __restrict__ scores,
+                                           const int* __restrict__ len, const int* __restrict__ budget,
+                                           const int* __restrict__ pos, int* __restrict__ evict_idx, int max_evict,
+                                           int* __restrict__ n_evict, int* status) {
   __shared__ unsigned int hist[256];
   __shared__ unsigned long long s_prefix;
   __shared__ int s_remaining;
@@ -31,7 +32,7 @@ select_kernel(int Hkv, int cap, const float* __restrict__ scores, const int* __r
   __shared__ int s_running;
   __shared__ unsigned long long s_min[kSelThreads / 32];
 
-  const int unit = blockIdx.x, b = unit / Hkv, h = unit % Hkv;
+  const int b = unit / Hkv, h = unit % Hkv;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n = len[b];
   int bud = budget[b];
@@ -44,7 +45,7 @@ select_kernel(int Hkv, int cap, const float* __restrict__ scores, const int* __r
     k = 0;
   }
   if (h == 0 && tid == 0) n_evict[b] = k;
-  if (k == 0) return;
+  if (k == 0) return 0;
   const float* sc = scores + (size_t)unit * cap;
   const int* ps = pos ? pos + (size_t)unit * cap : nullptr;
   int* out = evict_idx + (size_t)unit * max_evict;
@@ -76,7 +77,7 @@ select_kernel(int Hkv, int cap, const float* __restrict__ scores, const int* __r
       }
       if (lane == 0) out[0] = best_slot;
     }
-    return;
+    return 1;
   }
 
   if (tid == 0) { s_prefix = 0ull; s_remaining = k; }
@@ -127,6 +128,14 @@ select_kernel(int Hkv, int cap, const float* __restrict__ scores, const int* __r
     }
     __syncthreads();
   }
+  return k;
+}
+
+__global__ void __launch_bounds__(kSelThreads)
+select_kernel(int Hkv, int cap, const float* __restrict__ scores, const int* __restrict__ len,
+              const int* __restrict__ budget, const int* __restrict__ pos, int* __restrict__ evict_idx,
+              int max_evict, int* __restrict__ n_evict, int* status) {
+  select_unit(blockIdx.x, Hkv, cap, scores, len, budget, pos, evict_idx, max_evict, n_evict, status);
 }
 
 // Copy one row of `bytes` bytes (a multiple of 16, 16-byte aligned on both sides) with one warp.
@@ -148,12 +157,11 @@ __device__ __forceinline__ int lower_bound(const int* a, int n, int x) {
 // FILL compaction, one CTA per unit. With n' = n - k, the evicted slots below n' are holes, and the
 // k slots [n', n) hold exactly as many survivors; the i-th surviving tail slot moves into the i-th
 // hole. Sources lie in [n', n) and destinations in [0, n'), so no move can clobber another's source.
-__global__ void __launch_bounds__(256)
-compact_fill_kernel(int Hkv, int cap, int row_bytes, char* __restrict__ K, char* __restrict__ V,
-                    float* __restrict__ base, int* __restrict__ pos, const int* __restrict__ len,
-                    const int* __restrict__ evict_idx, int max_evict, const int* __restrict__ n_evict) {
-  const int unit = blockIdx.x, b = unit / Hkv;
-  const int k = n_evict[b];
+__device__ __forceinline__ void compact_fill_unit(int unit, int k, int Hkv, int cap, int row_bytes, char* __restrict__ K,
+                                                  char* __restrict__ V, float* __restrict__ base, int* __restrict__ pos,
+                                                  const int* __restrict__ len, const int* __restrict__ evict_idx,
+                                                  int max_evict) {
+  const int b = unit / Hkv;
   if (k <= 0) return;
   const int n = len[b], n_new = n - k;
   const int* E = evict_idx + (size_t)unit * max_evict;
@@ -172,6 +180,39 @@ compact_fill_kernel(int Hkv, int cap, int row_bytes, char* __restrict__ K, char*
       if (base) base[dof] = base[so];
       if (pos) pos[dof] = pos[so];
     }
+  }
+}
+
+__global__ void __launch_bounds__(256)
+compact_fill_kernel(int Hkv, int cap, int row_bytes, char* __restrict__ K, char* __restrict__ V,
+                    float* __restrict__ base, int* __restrict__ pos, const int* __restrict__ len,
+                    const int* __restrict__ evict_idx, int max_evict, const int* __restrict__ n_evict) {
+  compact_fill_unit(blockIdx.x, n_evict[blockIdx.x / Hkv], Hkv, cap, row_bytes, K, V, base, pos, len, evict_idx, max_evict);
+}
+
+// Selection and FILL compaction of one unit per CTA in one launch, and the length update by whichever
+// CTA finishes last (a ticket counter in the workspace header, which that CTA also resets). Same results
+// as select_kernel + compact_fill_kernel + update_len_kernel.
+__global__ void __launch_bounds__(kSelThreads)
+select_compact_kernel(int B, int Hkv, int cap, int row_bytes, const float* __restrict__ scores, char* __restrict__ K,
+                      char* __restrict__ V, float* __restrict__ base, int* __restrict__ pos, int* __restrict__ len,
+                      const int* __restrict__ budget, int* __restrict__ evict_idx, int max_evict,
+                      int* __restrict__ n_evict, int* status, int* ticket) {
+  __shared__ int s_last;
+  const int unit = blockIdx.x;
+  const int k = select_unit(unit, Hkv, cap, scores, len, budget, pos, evict_idx, max_evict, n_evict, status);
+  __syncthreads();  // evict_idx of this unit is written
+  compact_fill_unit(unit, k, Hkv, cap, row_bytes, K, V, base, pos, len, evict_idx, max_evict);
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    s_last = (atomicAdd(ticket, 1) == (int)gridDim.x - 1);
+  }
+  __syncthreads();
+  if (s_last) {
+    __threadfence();
+    for (int b = threadIdx.x; b < B; b += blockDim.x) len[b] -= __ldcg(&n_evict[b]);
+    if (threadIdx.x == 0) *ticket = 0;
   }
 }
 
