@@ -107,7 +107,8 @@ typedef struct {
 
 /* Bytes of scratch that caote_score / caote_select_evict / caote_compact / caote_append need for these
  * parameters (the maximum over the four; one buffer serves all). Returns 0 if params is invalid.
- * The first 256 bytes hold the status word; zero them once (cudaMemsetAsync) before first use. */
+ * The first 256 bytes hold the status word and the library's own counters; zero them once
+ * (cudaMemsetAsync) before first use and leave them alone afterwards. */
 CAOTE_API size_t caote_workspace_bytes(const caote_params_t* params);
 
 /* Append the m = n_new newest tokens of every sequence to its cache (Sec. 2: the block

@@ -380,8 +380,7 @@ int caote_append(const caote_params_t* p, void* K, void* V, float* base, int32_t
   cudaStream_t st = (cudaStream_t)stream;
   CAOTE_LAUNCH("append_kernel", st, sel::append_kernel<<<dm.units, 256, 0, st>>>(dm.Hkv, dm.cap, dm.m, row_bytes, (char*)K, (char*)V, base, pos,
                                                len, n_seen, (const char*)k_new, (const char*)v_new,
-                                               (int*)workspace));
-  CAOTE_LAUNCH("bump_len_kernel", st, sel::bump_len_kernel<<<(dm.B + 127) / 128, 128, 0, st>>>(dm.B, dm.cap, dm.m, len, n_seen));
+                                               (int*)workspace, dm.B, (int*)workspace + 4));
   return CAOTE_OK;
 }
 

@@ -278,18 +278,16 @@ __global__ void update_len_kernel(int B, int* __restrict__ len, const int* __res
 // Append m new rows per unit: one CTA per unit, one warp per row.
 __global__ void __launch_bounds__(256)
 append_kernel(int Hkv, int cap, int m, int row_bytes, char* __restrict__ K, char* __restrict__ V,
-              float* __restrict__ base, int* __restrict__ pos, const int* __restrict__ len,
-              const int* __restrict__ n_seen, const char* __restrict__ k_new,
-              const char* __restrict__ v_new, int* status) {
+              float* __restrict__ base, int* __restrict__ pos, int* __restrict__ len,
+              int* __restrict__ n_seen, const char* __restrict__ k_new,
+              const char* __restrict__ v_new, int* status, int B, int* ticket) {
   const int unit = blockIdx.x, b = unit / Hkv;
   const int n = len[b];
-  if (n < 0 || n + m > cap) {
-    if (threadIdx.x == 0) set_status(status, CAOTE_ERR_OVERFLOW);
-    return;
-  }
+  const bool fits = n >= 0 && n + m <= cap;
+  if (!fits && threadIdx.x == 0) set_status(status, CAOTE_ERR_OVERFLOW);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
   const int seen = n_seen ? n_seen[b] : n;
-  for (int i = warp; i < m; i += nwarps) {
+  for (int i = warp; fits && i < m; i += nwarps) {
     const size_t dst = (size_t)unit * cap + n + i, src = (size_t)unit * m + i;
     warp_copy_row(K + dst * row_bytes, k_new + src * row_bytes, row_bytes, lane);
     warp_copy_row(V + dst * row_bytes, v_new + src * row_bytes, row_bytes, lane);
@@ -298,14 +296,25 @@ append_kernel(int Hkv, int cap, int m, int row_bytes, char* __restrict__ K, char
       if (pos) pos[dst] = seen + i;
     }
   }
-}
-
-// len[b] += m and n_seen[b] += m for the sequences append_kernel did not skip.
-__global__ void bump_len_kernel(int B, int cap, int m, int* __restrict__ len, int* __restrict__ n_seen) {
-  const int b = blockIdx.x * blockDim.x + threadIdx.x;
-  if (b < B && len[b] >= 0 && len[b] + m <= cap) {
-    len[b] += m;
-    if (n_seen) n_seen[b] += m;
+  // the CTA that finishes last moves the lengths on: len[b] += m and n_seen[b] += m for the
+  // sequences that were not skipped (a ticket counter in the workspace header, reset here)
+  __shared__ int s_last;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    s_last = (atomicAdd(ticket, 1) == (int)gridDim.x - 1);
+  }
+  __syncthreads();
+  if (s_last) {
+    __threadfence();
+    for (int bb = threadIdx.x; bb < B; bb += blockDim.x) {
+      const int nb = len[bb];
+      if (nb >= 0 && nb + m <= cap) {
+        len[bb] = nb + m;
+        if (n_seen) n_seen[bb] += m;
+      }
+    }
+    if (threadIdx.x == 0) *ticket = 0;
   }
 }
 
