@@ -29,6 +29,14 @@ sys.path.insert(0, ROOT)
 
 from paper_2504_14051_b200 import workloads as wl  # noqa: E402
 
+# DRAM bytes (read + write) of one launch per unit of work, from ncu captures of reduced cases
+# (profiles/*_ncu.txt), scaled to the launch at hand by the units it processes; traffic grows in
+# proportion to them. A value is set to None when its kernel has changed since the capture.
+NCU_TRAFFIC = {
+    "decode_kernel": {"bytes_per_token_head": 288304128 / 449880, "profile": "profiles/decode_kernel_c4_batch16_ncu.txt"},
+    "prefill_attn_kernel": None,
+}
+
 METRIC = "cached tokens scored+evicted/sec"
 UNIT = "token-heads/s"
 
@@ -228,7 +236,10 @@ def run_ours(args, w0, rank, world, device):
         achieved = bytes_per_launch / (per_launch_ms * 1e-3) / 1e9
         roofline = {"bound": "hbm", "kernel": top, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "frac": achieved / peaks["hbm_gbs"], "frac_of_nominal_8000": achieved / 8000.0,
-                    "peak_source": peaks["source"] + " copy bandwidth", "traffic": None,
+                    "peak_source": peaks["source"] + " copy bandwidth",
+                    "traffic": (NCU_TRAFFIC[top]["bytes_per_token_head"] * th_per_step / launches_per_step_top
+                                if NCU_TRAFFIC.get(top) else None),
+                    "traffic_source": NCU_TRAFFIC[top]["profile"] if NCU_TRAFFIC.get(top) else None,
                     "algorithmic_bytes_per_launch": bytes_per_launch,
                     "algorithmic_bytes_per_token_head": algo["per_token_head"],
                     "step_frac": (algo["per_step"] / (ms_per_step * 1e-3) / 1e9) / peaks["hbm_gbs"]}
@@ -237,7 +248,9 @@ def run_ours(args, w0, rank, world, device):
         achieved = fl_per_launch / (per_launch_ms * 1e-3) / 1e12
         roofline = {"bound": "tensor", "kernel": top, "achieved": achieved, "peak": peaks["bf16_tflops_sustained"],
                     "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops_sustained"],
-                    "peak_source": peaks["source"] + " cuBLAS bf16 sustained", "traffic": None,
+                    "peak_source": peaks["source"] + " cuBLAS bf16 sustained",
+                    "traffic": (NCU_TRAFFIC[top]["bytes_per_unit"] * units if NCU_TRAFFIC.get(top) else None),
+                    "traffic_source": NCU_TRAFFIC[top]["profile"] if NCU_TRAFFIC.get(top) else None,
                     "useful_flops_per_launch": fl_per_launch,
                     "step_frac": (flops_per_step / (ms_per_step * 1e-3) / 1e12) / peaks["bf16_tflops_sustained"]}
 
