@@ -3,22 +3,26 @@
 // (sequence, KV head) unit against its n cached keys.
 //
 //   attn_kernel   rows x keys. One CTA owns 128 query rows of a unit and walks the unit's keys in
-//                 tiles of 128: S = Q K^T (tcgen05.mma, fp32 accumulator in TMEM), per-row online
-//                 softmax (one thread per row, straight out of TMEM), P in bf16 back to shared memory,
-//                 O += P V (second tcgen05.mma; V is the MN-major operand). Writes o and the per-row
-//                 softmax statistics (reference, sum).
+//                 tiles of 64: S = Q K^T (tcgen05.mma, fp32 accumulator in TMEM), per-row online
+//                 softmax (one thread per row, straight out of TMEM), P back into TMEM as two bf16
+//                 parts (hi + lo, 16 significant bits together), O += P V with P as the TMEM-side A
+//                 operand and V as the MN-major B operand. Writes o and the per-row softmax
+//                 statistics (reference, 1 / sum). One lane each of three extra warps issues the
+//                 products, the K copies and the V copies, so the tensor pipe always has the next
+//                 S queued while the rows are busy with the current one.
 //   xsum_kernel   X = mean of the unit's M output rows (the weights of CHUNK_SUM are the column sums
 //                 of the attention matrix divided by M, so sum_j w_j v_j is the mean output row).
-//   score_kernel  keys x rows. One CTA owns 128 keys of a unit and walks the unit's rows in blocks of
-//                 128: S^T = K Q^T lands in TMEM with one key per lane, so each thread sums
-//                 exp2(s - ref_r) / sum_r over the rows of its own key without any exchange:
-//                 h_j = sum_r alpha_{r,j}. Then c_j = w_j / (1 - w_j) * ||X - v_j||, w_j = h_j / M.
+//   score_kernel  keys x rows. One CTA owns 256 keys of a unit (two key tiles) and walks the unit's
+//                 rows in blocks of 128: S^T = K Q^T lands in TMEM with one key per lane, so each
+//                 thread sums exp2(s - ref_r) / sum_r over the rows of its own key without any
+//                 exchange: h_j = sum_r alpha_{r,j}. Then c_j = w_j / (1 - w_j) * ||X - v_j||,
+//                 w_j = h_j / M.
 //
-// Operands are staged by TMA as 64-channel boxes of 128 rows with the 128-byte swizzle, which is the
-// canonical K-major UMMA layout (8-row groups 1024 bytes apart); V in the second product is read
-// through an MN-major descriptor of the same bytes. Every mbarrier wait is bounded by a clock limit;
-// a wait that runs out records CAOTE_ERR_TIMEOUT and the CTA carries on with whatever is in its
-// buffers (all indices stay in bounds), so that no thread is left behind at a barrier.
+// Operands are staged by TMA as 64-channel boxes with the 128-byte swizzle, which is the canonical
+// K-major UMMA layout (8-row groups 1024 bytes apart); V in the second product is read through an
+// MN-major descriptor of the same bytes. Every mbarrier wait is bounded by a clock limit; a wait
+// that runs out records CAOTE_ERR_TIMEOUT and the thread carries on with whatever is in its buffers
+// (all indices stay in bounds), so that no thread is left behind at a barrier.
 #pragma once
 
 #include <cuda.h>
