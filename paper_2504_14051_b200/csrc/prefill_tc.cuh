@@ -85,6 +85,19 @@ __device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, int* s
     }
   }
 }
+// The same for the single-lane helper warps: they back off between polls so that their spinning does
+// not take issue slots from the warps that do the arithmetic on the same scheduler.
+__device__ __forceinline__ void mbar_wait_idle(uint64_t* bar, uint32_t parity, int* status) {
+  if (mbar_try_wait(bar, parity)) return;
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity)) {
+    __nanosleep(20);
+    if (clock64() - t0 > kWaitCycles) {
+      set_status(status, CAOTE_ERR_TIMEOUT);
+      return;
+    }
+  }
+}
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
@@ -288,7 +301,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
       tma_load_2d(Qs + kHalfBytes, &tmQ, 64, unit * M + row0, q_bar);
       for (int kt = 0; kt < ntiles; ++kt) {
         const int st = kt % kKStages, row = unit * dm.cap + kt * kKeys;
-        if (kt >= kKStages) mbar_wait(&k_free[st], ((kt / kKStages) - 1) & 1, status);  // S of tile kt - 6 is formed
+        if (kt >= kKStages) mbar_wait_idle(&k_free[st], ((kt / kKStages) - 1) & 1, status);  // S of tile kt - 6 is formed
         mbar_expect_tx(&k_bar[st], kKvTile);
         tma_load_2d(Ksm + st * kKvTile, &tmK64, 0, row, &k_bar[st]);
         tma_load_2d(Ksm + st * kKvTile + kKvHalf, &tmK64, 64, row, &k_bar[st]);
@@ -299,7 +312,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     if (tid == kThreads + 64) {
       for (int kt = 0; kt < ntiles; ++kt) {
         const int st = kt % kVStages, row = unit * dm.cap + kt * kKeys;
-        if (kt >= kVStages) mbar_wait(&v_free[st], ((kt / kVStages) - 1) & 1, status);  // O += P V of tile kt - 5 is done
+        if (kt >= kVStages) mbar_wait_idle(&v_free[st], ((kt / kVStages) - 1) & 1, status);  // O += P V of tile kt - 5 is done
         mbar_expect_tx(&v_bar[st], kKvTile);
         tma_load_2d(Vsm + st * kKvTile, &tmV64, 0, row, &v_bar[st]);
         tma_load_2d(Vsm + st * kKvTile + kKvHalf, &tmV64, 64, row, &v_bar[st]);
@@ -310,32 +323,46 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     if (tid == kThreads) {
       constexpr uint32_t kIdescS = instr_desc_n(false, kKeys), kIdescO = instr_desc_n(true, kD);
       const uint32_t q_addr = smem_u32(Qs);
+      // Descriptors are built once; inside the loop a product costs one 64-bit add per operand (the
+      // single issuing thread is bound by the latency of its own instruction stream, not by the pipe).
+      uint64_t qdesc[8];
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) qdesc[ks] = desc_k_major(q_addr, ks);
+      const uint64_t kdesc0 = smem_desc(smem_u32(Ksm), 16, 1024);
+      const uint64_t vdesc0 = smem_desc(smem_u32(Vsm), kKvHalf, 1024);
       auto issue_qk = [&](int kt) {
-        mbar_wait(&k_bar[kt % kKStages], (kt / kKStages) & 1, status);
+        mbar_wait_idle(&k_bar[kt % kKStages], (kt / kKStages) & 1, status);
         tc_fence_after();
-        const uint32_t k_addr = smem_u32(Ksm + (kt % kKStages) * kKvTile);
+        const uint64_t kd = kdesc0 + (uint64_t)(((kt % kKStages) * kKvTile) >> 4);
+        const uint32_t d_s = tmem + (kt & 1) * kKeys;
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks)
-          umma(tmem + (kt & 1) * kKeys, desc_k_major(q_addr, ks), desc_k_major64(k_addr, ks), kIdescS, ks > 0);
+          umma(d_s, qdesc[ks], kd + (uint64_t)((((ks >> 2) * kKvHalf) + (ks & 3) * 32) >> 4), kIdescS, ks > 0);
         umma_commit(&s_bar[kt & 1]);
         umma_commit(&k_free[kt % kKStages]);
       };
-      mbar_wait(q_bar, 0, status);
+      mbar_wait_idle(q_bar, 0, status);
       issue_qk(0);
       for (int kt = 0; kt < ntiles; ++kt) {
         // queue S of the next tile: its buffer was read by the softmax of tile kt - 1, which has
         // arrived on p_bar before PV(kt - 1) was issued
         if (kt + 1 < ntiles) issue_qk(kt + 1);
         // O += P V once the rows have written P of this tile
-        mbar_wait(&p_bar[kt & 1], (kt >> 1) & 1, status);
-        mbar_wait(&v_bar[kt % kVStages], (kt / kVStages) & 1, status);
+        mbar_wait_idle(&p_bar[kt & 1], (kt >> 1) & 1, status);
+        mbar_wait_idle(&v_bar[kt % kVStages], (kt / kVStages) & 1, status);
         tc_fence_after();
-        const uint32_t v_addr = smem_u32(Vsm + (kt % kVStages) * kKvTile);
+        const uint64_t vd = vdesc0 + (uint64_t)(((kt % kVStages) * kKvTile) >> 4);
         const uint32_t p_tmem = tmem + 256 + (kt & 1) * 64;
+        if (kt == 0) {
+          umma_ts(tmem + 128, p_tmem, vd, kIdescO, false);
+        } else {
+          umma_ts(tmem + 128, p_tmem, vd, kIdescO, true);
+        }
+        umma_ts(tmem + 128, p_tmem + 32, vd, kIdescO, true);
 #pragma unroll
-        for (int ks = 0; ks < 4; ++ks) {  // 16 keys = 8 packed columns per step
-          umma_ts(tmem + 128, p_tmem + ks * 8, desc_mn_major64(v_addr, ks), kIdescO, kt > 0 || ks > 0);
-          umma_ts(tmem + 128, p_tmem + 32 + ks * 8, desc_mn_major64(v_addr, ks), kIdescO, true);
+        for (int ks = 1; ks < 4; ++ks) {  // 16 keys = 8 packed columns per step
+          umma_ts(tmem + 128, p_tmem + ks * 8, vd + (uint64_t)((ks * 2048) >> 4), kIdescO, true);
+          umma_ts(tmem + 128, p_tmem + 32 + ks * 8, vd + (uint64_t)((ks * 2048) >> 4), kIdescO, true);
         }
         umma_commit(&o_bar[kt & 1]);
         umma_commit(&v_free[kt % kVStages]);
@@ -535,7 +562,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       }
       for (int rb = 0; rb < nblocks; ++rb) {
         const int st = rb % kQStages;
-        if (rb >= kQStages) mbar_wait(&q_free[st], ((rb / kQStages) - 1) & 1, status);  // block rb - 3 is reduced
+        if (rb >= kQStages) mbar_wait_idle(&q_free[st], ((rb / kQStages) - 1) & 1, status);  // block rb - 3 is reduced
         char* qd = Qst + st * kQStage;
         mbar_expect_tx(&q_bar[st], kQStage);
         tma_load_2d(qd, &tmQ, 0, unit * M + rb * kTile, &q_bar[st]);
@@ -548,11 +575,11 @@ score_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     if (tid == kScoreKeys) {
       constexpr uint32_t kIdesc = instr_desc(false);
       const uint32_t k_addr = smem_u32(Ks);
-      mbar_wait(k_bar, 0, status);
+      mbar_wait_idle(k_bar, 0, status);
       for (int rb = 0; rb < nblocks; ++rb) {
         const int buf = rb & 1, st = rb % kQStages;
-        mbar_wait(&q_bar[st], (rb / kQStages) & 1, status);
-        if (rb >= 2) mbar_wait(&c_bar[buf], ((rb - 2) >> 1) & 1, status);  // its S buffers have been read
+        mbar_wait_idle(&q_bar[st], (rb / kQStages) & 1, status);
+        if (rb >= 2) mbar_wait_idle(&c_bar[buf], ((rb - 2) >> 1) & 1, status);  // its S buffers have been read
         tc_fence_after();
         const uint32_t q_addr = smem_u32(Qst + st * kQStage);
 #pragma unroll
