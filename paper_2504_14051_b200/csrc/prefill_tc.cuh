@@ -225,15 +225,16 @@ __device__ __forceinline__ uint64_t desc_mn_major(uint32_t tile_addr, int ks) {
 // while the threads are busy with the softmax of the current tile:
 //   tensor pipe:  QK(t+1)  PV(t)  QK(t+2)  PV(t+1) ...
 //   threads:      softmax(t) ............ softmax(t+1) ...
-constexpr int kKeys = 64;                    // keys per tile of the attention pass
-constexpr int kKvHalf = kKeys * 128;         // one 64-channel box of 64 keys: 8 KB
-constexpr int kKvTile = 2 * kKvHalf;         // K or V tile: 16 KB
-constexpr int kKStages = 6;                  // K runs well ahead: its stage is free as soon as S is formed
-constexpr int kVStages = 5;
-constexpr int kAttnThreads = kThreads + 96;  // 128 softmax threads (one per row) + MMA, K-load and V-load warps
+constexpr int kKeys = 128;                   // keys per tile of the attention pass
+constexpr int kKvHalf = kKeys * 128;         // one 64-channel box of 128 keys: 16 KB
+constexpr int kKvTile = 2 * kKvHalf;         // K or V tile: 32 KB
+constexpr int kKStages = 3;                  // a K stage is free as soon as S is formed
+constexpr int kVStages = 2;
+constexpr int kRowThreads = 2 * kThreads;    // two threads per query row: each owns 64 of the tile's 128 keys
+constexpr int kAttnThreads = kRowThreads + 96;  // + MMA, K-load and V-load warps
 
 inline size_t attn_smem_bytes() {
-  return 1024 + kTileBytes + (size_t)(kKStages + kVStages) * kKvTile + 256;
+  return 1024 + kTileBytes + (size_t)(kKStages + kVStages) * kKvTile + 2 * kRowThreads * sizeof(float) + 256;
 }
 
 // K-major / MN-major descriptors of k-step ks of a 64-key tile (boxes of 64 rows: kKvHalf apart).
@@ -250,10 +251,10 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
-// o and row statistics of 128 query rows of one unit. grid = (row blocks, units), 224 threads:
-// warps 0..3 own one query row per thread; one lane each of warps 4, 5, 6 issues the products, the K
-// copies and the V copies.
-// tmK64 / tmV64: tensor maps of K and V with boxes of 64 channels x 64 rows.
+// o and row statistics of 128 query rows of one unit. grid = (row blocks, units), 352 threads:
+// warps 0..7 are the row threads (two per row); one lane each of warps 8, 9, 10 issues the products,
+// the K copies and the V copies.
+// tmK64 / tmV64: tensor maps of K and V with boxes of 64 channels x kKeys rows.
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK64,
             const __grid_constant__ CUtensorMap tmV64, Dims dm, const int* __restrict__ len, Scratch sc,
@@ -263,7 +264,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
   char* Qs = sm;
   char* Ksm = Qs + kTileBytes;                 // [kKStages]
   char* Vsm = Ksm + kKStages * kKvTile;        // [kVStages]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(Vsm + kVStages * kKvTile);
+  float* xch = reinterpret_cast<float*>(Vsm + kVStages * kKvTile);  // [2][kRowThreads] half-row maxima / sums
+  uint64_t* bars = reinterpret_cast<uint64_t*>(xch + 2 * kRowThreads);
   uint64_t *q_bar = &bars[0], *k_bar = &bars[1], *v_bar = k_bar + kKStages, *s_bar = v_bar + kVStages, *o_bar = s_bar + 2,
            *p_bar = o_bar + 2, *k_free = p_bar + 2, *v_free = k_free + kKStages;
   constexpr int kBars = 1 + 2 * (kKStages + kVStages) + 6;
@@ -282,45 +284,45 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
 
   if (tid == 0) {
     for (int i = 0; i < kBars; ++i) mbar_init(&bars[i], 1);
-    mbar_init(&p_bar[0], kThreads);
-    mbar_init(&p_bar[1], kThreads);
+    mbar_init(&p_bar[0], kRowThreads);
+    mbar_init(&p_bar[1], kRowThreads);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) tmem_alloc(tmem_slot, 512);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  // columns: S0 [0,64), S1 [64,128), O [128,256), P0 hi [256,288) lo [288,320), P1 hi [320,352) lo [352,384)
+  // columns: S0 [0,128), S1 [128,256), O [256,384), P hi [384,448), P lo [448,512) (two bf16 per column)
   const uint32_t tmem = *tmem_slot;
 
-  if (warp == 5) {
+  if (warp == 9) {
     // =============================== K loads (one lane) ===============================
-    if (tid == kThreads + 32) {
+    if (tid == kRowThreads + 32) {
       mbar_expect_tx(q_bar, kTileBytes);
       tma_load_2d(Qs, &tmQ, 0, unit * M + row0, q_bar);
       tma_load_2d(Qs + kHalfBytes, &tmQ, 64, unit * M + row0, q_bar);
       for (int kt = 0; kt < ntiles; ++kt) {
         const int st = kt % kKStages, row = unit * dm.cap + kt * kKeys;
-        if (kt >= kKStages) mbar_wait_idle(&k_free[st], ((kt / kKStages) - 1) & 1, status);  // S of tile kt - 6 is formed
+        if (kt >= kKStages) mbar_wait_idle(&k_free[st], ((kt / kKStages) - 1) & 1, status);  // S of tile kt - 3 is formed
         mbar_expect_tx(&k_bar[st], kKvTile);
         tma_load_2d(Ksm + st * kKvTile, &tmK64, 0, row, &k_bar[st]);
         tma_load_2d(Ksm + st * kKvTile + kKvHalf, &tmK64, 64, row, &k_bar[st]);
       }
     }
-  } else if (warp == 6) {
+  } else if (warp == 10) {
     // =============================== V loads (one lane) ===============================
-    if (tid == kThreads + 64) {
+    if (tid == kRowThreads + 64) {
       for (int kt = 0; kt < ntiles; ++kt) {
         const int st = kt % kVStages, row = unit * dm.cap + kt * kKeys;
-        if (kt >= kVStages) mbar_wait_idle(&v_free[st], ((kt / kVStages) - 1) & 1, status);  // O += P V of tile kt - 5 is done
+        if (kt >= kVStages) mbar_wait_idle(&v_free[st], ((kt / kVStages) - 1) & 1, status);  // O += P V of tile kt - 2 is done
         mbar_expect_tx(&v_bar[st], kKvTile);
         tma_load_2d(Vsm + st * kKvTile, &tmV64, 0, row, &v_bar[st]);
         tma_load_2d(Vsm + st * kKvTile + kKvHalf, &tmV64, 64, row, &v_bar[st]);
       }
     }
-  } else if (warp == 4) {
+  } else if (warp == 8) {
     // =============================== products (one lane) ===============================
-    if (tid == kThreads) {
+    if (tid == kRowThreads) {
       constexpr uint32_t kIdescS = instr_desc_n(false, kKeys), kIdescO = instr_desc_n(true, kD);
       const uint32_t q_addr = smem_u32(Qs);
       // Descriptors are built once; inside the loop a product costs one 64-bit add per operand (the
@@ -334,7 +336,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         mbar_wait_idle(&k_bar[kt % kKStages], (kt / kKStages) & 1, status);
         tc_fence_after();
         const uint64_t kd = kdesc0 + (uint64_t)(((kt % kKStages) * kKvTile) >> 4);
-        const uint32_t d_s = tmem + (kt & 1) * kKeys;
+        const uint32_t d_s = tmem + (kt & 1) * kKeys;  // S0 or S1
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks)
           umma(d_s, qdesc[ks], kd + (uint64_t)((((ks >> 2) * kKvHalf) + (ks & 3) * 32) >> 4), kIdescS, ks > 0);
@@ -352,40 +354,45 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         mbar_wait_idle(&v_bar[kt % kVStages], (kt / kVStages) & 1, status);
         tc_fence_after();
         const uint64_t vd = vdesc0 + (uint64_t)(((kt % kVStages) * kKvTile) >> 4);
-        const uint32_t p_tmem = tmem + 256 + (kt & 1) * 64;
+        const uint32_t p_tmem = tmem + 384;
         if (kt == 0) {
-          umma_ts(tmem + 128, p_tmem, vd, kIdescO, false);
+          umma_ts(tmem + 256, p_tmem, vd, kIdescO, false);
         } else {
-          umma_ts(tmem + 128, p_tmem, vd, kIdescO, true);
+          umma_ts(tmem + 256, p_tmem, vd, kIdescO, true);
         }
-        umma_ts(tmem + 128, p_tmem + 32, vd, kIdescO, true);
+        umma_ts(tmem + 256, p_tmem + 64, vd, kIdescO, true);
 #pragma unroll
-        for (int ks = 1; ks < 4; ++ks) {  // 16 keys = 8 packed columns per step
-          umma_ts(tmem + 128, p_tmem + ks * 8, vd + (uint64_t)((ks * 2048) >> 4), kIdescO, true);
-          umma_ts(tmem + 128, p_tmem + 32 + ks * 8, vd + (uint64_t)((ks * 2048) >> 4), kIdescO, true);
+        for (int ks = 1; ks < 8; ++ks) {  // 16 keys = 8 packed columns per step
+          umma_ts(tmem + 256, p_tmem + ks * 8, vd + (uint64_t)((ks * 2048) >> 4), kIdescO, true);
+          umma_ts(tmem + 256, p_tmem + 64 + ks * 8, vd + (uint64_t)((ks * 2048) >> 4), kIdescO, true);
         }
         umma_commit(&o_bar[kt & 1]);
         umma_commit(&v_free[kt % kVStages]);
       }
     }
   } else {
-    // =============================== one query row per thread ===============================
-    const int R = row0 + tid;
+    // =============================== two threads per query row ===============================
+    // Thread t and thread t + 128 share row t of the block: each owns 64 of a tile's 128 keys (and 64
+    // of the 128 output channels when O is rescaled or written out). They agree on the softmax
+    // reference through a two-float exchange in shared memory and one barrier of the row threads.
+    const int rowl = tid & (kThreads - 1), half = tid >> 7;
+    const int R = row0 + rowl;
     const int nvis = (R < M) ? n - m + (R % m) + 1 : n;  // keys this row sees (causal inside the block)
     const float scale2 = dm.scale * 1.4426950408889634f;
-    const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);
-    const uint32_t t_o = t_lane + 128;
+    const uint32_t t_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+    const uint32_t t_o = t_lane + 256 + half * 64;
+    const uint32_t t_p = t_lane + 384 + half * 32;  // this half's 64 keys = 32 packed columns (hi); lo at + 64
     float m_ref = -INFINITY, l = 0.f;
 
     for (int kt = 0; kt < ntiles; ++kt) {
       mbar_wait(&s_bar[kt & 1], (kt >> 1) & 1, status);
       tc_fence_after();
-      const int j0 = kt * kKeys;
-      const uint32_t t_s = t_lane + (kt & 1) * kKeys;
+      const int j0 = kt * kKeys + half * 64;  // first key of this thread's half
+      const uint32_t t_s = t_lane + (kt & 1) * kKeys + half * 64;
       float sv[64];  // raw products; masked keys become -inf
       tmem_ld32(t_s, *reinterpret_cast<float(*)[32]>(&sv[0]));
       tmem_ld32(t_s + 32, *reinterpret_cast<float(*)[32]>(&sv[32]));
-      if (j0 + kKeys > n - m + 1) {  // only tiles that reach into the new block (or past the length) need the mask
+      if (kt * kKeys + kKeys > n - m + 1) {  // only tiles that reach into the new block (or past the length) need the mask
 #pragma unroll
         for (int i = 0; i < 64; ++i) sv[i] = (j0 + i < nvis) ? sv[i] : -INFINITY;
       }
@@ -398,6 +405,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         for (int i = 8; i < 64; ++i) pm[i & 7] = fmaxf(pm[i & 7], sv[i] * scale2);
         mx = fmaxf(fmaxf(fmaxf(pm[0], pm[1]), fmaxf(pm[2], pm[3])), fmaxf(fmaxf(pm[4], pm[5]), fmaxf(pm[6], pm[7])));
       }
+      // the other half of the row
+      float* xm = xch + (kt & 1) * kRowThreads;
+      xm[tid] = mx;
+      asm volatile("bar.sync 1, %0;" ::"n"(kRowThreads) : "memory");
+      mx = fmaxf(mx, xm[tid ^ kThreads]);
       // the reference moves only when a logit exceeds it by more than 8 (p <= 256 in between)
       const bool need = mx > m_ref + 8.f;
       if (__any_sync(0xffffffffu, need)) {
@@ -408,7 +420,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
           mbar_wait(&o_bar[(kt - 1) & 1], ((kt - 1) >> 1) & 1, status);  // O += P V of the previous tile is done
           tc_fence_after();
 #pragma unroll
-          for (int cc = 0; cc < 4; ++cc) {
+          for (int cc = 0; cc < 2; ++cc) {
             float v[32];
             tmem_ld32(t_o + cc * 32, v);
 #pragma unroll
@@ -418,8 +430,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
           tmem_st_wait();
         }
       }
-      // this tile's P buffer was last read by the product of tile kt - 2
-      if (kt >= 2) mbar_wait(&o_bar[kt & 1], ((kt - 2) >> 1) & 1, status);
       {
         const float neg_ref = -m_ref;
         float ls[4] = {0.f, 0.f, 0.f, 0.f};
@@ -436,13 +446,14 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
           lo[c] = __byte_perm(__float_as_uint(r0) + 0x8000u, __float_as_uint(r1) + 0x8000u, 0x7632);  // rounded
           ls[c & 3] += p0 + p1;
         }
-        const uint32_t t_p = t_lane + 256 + (kt & 1) * 64;
+        // the one P buffer is still being read by the product of the previous tile until o_bar says so
+        if (kt >= 1) mbar_wait(&o_bar[(kt - 1) & 1], ((kt - 1) >> 1) & 1, status);
         tmem_st32u(t_p, hi);
-        tmem_st32u(t_p + 32, lo);
+        tmem_st32u(t_p + 64, lo);
         tmem_st_wait();
         l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
       }
-      const int n_valid = min(kKeys, n - j0);
+      const int n_valid = min(kKeys, n - kt * kKeys);
       if (n_valid < kKeys) {
         // V rows behind the unit's length: clear them so that 0 * (stray NaN) cannot reach O
         mbar_wait(&v_bar[kt % kVStages], (kt / kVStages) & 1, status);
@@ -460,11 +471,15 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     mbar_wait(&o_bar[(ntiles - 1) & 1], ((ntiles - 1) >> 1) & 1, status);
     tc_fence_after();
 
-    // ---- normalise and write out ----
+    // ---- normalise and write out: the two halves of a row add up their sums first ----
+    float* xl = xch + (ntiles & 1) * kRowThreads;  // the copy the last tile did not use
+    xl[tid] = l;
+    asm volatile("bar.sync 1, %0;" ::"n"(kRowThreads) : "memory");
+    l += xl[tid ^ kThreads];
     const float inv_l = 1.f / l;
-    float* orow = o + ((size_t)unit * M + R) * kD;
+    float* orow = o + ((size_t)unit * M + R) * kD + half * 64;
 #pragma unroll
-    for (int cc = 0; cc < 4; ++cc) {
+    for (int cc = 0; cc < 2; ++cc) {
       float v[32];
       tmem_ld32(t_o + cc * 32, v);  // collective: every lane takes part, rows beyond M just do not store
       if (R < M) {
@@ -473,7 +488,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
           *reinterpret_cast<float4*>(orow + cc * 32 + i) = make_float4(v[i] * inv_l, v[i + 1] * inv_l, v[i + 2] * inv_l, v[i + 3] * inv_l);
       }
     }
-    if (R < M) {
+    if (R < M && half == 0) {
       sc.stats[((size_t)unit * sc.Mpad + R) * 2] = m_ref;
       sc.stats[((size_t)unit * sc.Mpad + R) * 2 + 1] = inv_l;
     }
