@@ -34,7 +34,7 @@ from paper_2504_14051_b200 import workloads as wl  # noqa: E402
 # proportion to them. A value is set to None when its kernel has changed since the capture.
 NCU_TRAFFIC = {
     "decode_kernel": {"bytes_per_token_head": 288304128 / 449880, "profile": "profiles/decode_kernel_c4_batch16_ncu.txt"},
-    "prefill_attn_kernel": None,
+    "prefill_attn_kernel": {"bytes_per_unit": (155871488 + 22343680) / 16, "profile": "profiles/prefill_kernels_c5p_batch2_ncu.txt"},
 }
 
 METRIC = "cached tokens scored+evicted/sec"

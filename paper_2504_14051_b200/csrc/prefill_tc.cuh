@@ -3,13 +3,13 @@
 // (sequence, KV head) unit against its n cached keys.
 //
 //   attn_kernel   rows x keys. One CTA owns 128 query rows of a unit and walks the unit's keys in
-//                 tiles of 64: S = Q K^T (tcgen05.mma, fp32 accumulator in TMEM), per-row online
-//                 softmax (one thread per row, straight out of TMEM), P back into TMEM as two bf16
-//                 parts (hi + lo, 16 significant bits together), O += P V with P as the TMEM-side A
-//                 operand and V as the MN-major B operand. Writes o and the per-row softmax
-//                 statistics (reference, 1 / sum). One lane each of three extra warps issues the
-//                 products, the K copies and the V copies, so the tensor pipe always has the next
-//                 S queued while the rows are busy with the current one.
+//                 tiles of 128: S = Q K^T (tcgen05.mma, fp32 accumulator in TMEM), per-row online
+//                 softmax straight out of TMEM (two threads per row, 64 keys each), P back into TMEM
+//                 as two bf16 parts (hi + lo, 16 significant bits together), O += P V with P as the
+//                 TMEM-side A operand and V as the MN-major B operand. Writes o and the per-row
+//                 softmax statistics (reference, 1 / sum). One lane each of three extra warps issues
+//                 the products, the K copies and the V copies, so the tensor pipe always has the
+//                 next S queued while the rows are busy with the current one.
 //   xsum_kernel   X = mean of the unit's M output rows (the weights of CHUNK_SUM are the column sums
 //                 of the attention matrix divided by M, so sum_j w_j v_j is the mean output row).
 //   score_kernel  keys x rows. One CTA owns 256 keys of a unit (two key tiles) and walks the unit's
