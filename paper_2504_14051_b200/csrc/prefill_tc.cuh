@@ -516,21 +516,25 @@ xsum_kernel(Dims dm, const int* __restrict__ len, const float* __restrict__ o, S
 }
 
 constexpr int kScoreKeys = 2 * kTile;            // keys per CTA: two key tiles share every Q block
-constexpr int kScoreThreads = kScoreKeys + 64;    // 256 key threads + a warp for the products + a warp for the copies
+constexpr int kKeyThreads = 2 * kScoreKeys;       // two threads per key: each owns 64 of a block's 128 rows
+constexpr int kScoreThreads = kKeyThreads + 64;   // + a warp for the products + a warp for the copies
 constexpr int kStatBytes = kTile * 2 * 4;         // (reference, 1 / sum) of the 128 rows of a block
 constexpr int kQStage = kTileBytes + kStatBytes;
 constexpr int kQStages = 3;
 
-inline size_t score_smem_bytes() { return 1024 + 2 * kTileBytes + kQStages * (size_t)kQStage + kD * sizeof(float) + 256; }
+inline size_t score_smem_bytes() {
+  return 1024 + 2 * kTileBytes + kQStages * (size_t)kQStage + (kD + kScoreKeys) * sizeof(float) + 256;
+}
 __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
   asm volatile(
       "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
       ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 
-// CAOTE scores of 256 keys of one unit. grid = (key tile pairs, units), 320 threads: warps 0..7 own one
-// key per thread (warps 0..3 the first key tile, 4..7 the second), one lane of warp 8 issues the products,
-// one lane of warp 9 the copies.
+// CAOTE scores of 256 keys of one unit. grid = (key tile pairs, units), 576 threads: warps 0..15 are the
+// key threads, two per key (warps 0..3 and 8..11 the first key tile, 4..7 and 12..15 the second; the
+// lower eight take rows 0..63 of every Q block, the upper eight rows 64..127), one lane of warp 16 issues
+// the products, one lane of warp 17 the copies.
 __global__ void __launch_bounds__(kScoreThreads, 1)
 score_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, Dims dm,
              const __nv_bfloat16* __restrict__ V, const int* __restrict__ len, Scratch sc,
@@ -540,7 +544,8 @@ score_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
   char* Ks = sm;                                                     // [2] key tiles
   char* Qst = Ks + 2 * kTileBytes;                                   // [kQStages][Q block, row statistics]
   float* Xs = reinterpret_cast<float*>(Qst + kQStages * kQStage);    // [kD]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(Xs + kD);
+  float* hx = Xs + kD;                                               // [kScoreKeys] upper halves' sums
+  uint64_t* bars = reinterpret_cast<uint64_t*>(hx + kScoreKeys);
   uint64_t *k_bar = &bars[0], *q_bar = &bars[1], *s_bar = q_bar + kQStages, *c_bar = s_bar + 2, *q_free = c_bar + 2;
   constexpr int kBars = 1 + kQStages + 2 + 2 + kQStages;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kBars);
@@ -554,8 +559,8 @@ score_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
 
   if (tid == 0) {
     for (int i = 0; i < 1 + kQStages + 2; ++i) mbar_init(&bars[i], 1);
-    for (int i = 0; i < 2; ++i) mbar_init(&c_bar[i], kScoreKeys);
-    for (int i = 0; i < kQStages; ++i) mbar_init(&q_free[i], kScoreKeys);
+    for (int i = 0; i < 2; ++i) mbar_init(&c_bar[i], kKeyThreads);
+    for (int i = 0; i < kQStages; ++i) mbar_init(&q_free[i], kKeyThreads);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) tmem_alloc(tmem_slot, 512);
@@ -565,11 +570,12 @@ score_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;  // key tile kk, buffer buf: columns [kk * 256 + buf * 128, + 128)
   float h = 0.f;
-  const int j = j0 + tid;  // key threads: this thread's key
+  const int j = j0 + (tid & (kScoreKeys - 1));  // key threads: this thread's key
+  const int rhalf = tid >> 8;                   // key threads: which 64 rows of a Q block
 
-  if (warp == 9) {
+  if (warp == 17) {
     // =============================== copies (one lane) ===============================
-    if (tid == kScoreKeys + 32) {
+    if (tid == kKeyThreads + 32) {
       mbar_expect_tx(k_bar, 2 * kTileBytes);
       for (int kk = 0; kk < 2; ++kk) {
         tma_load_2d(Ks + kk * kTileBytes, &tmK, 0, unit * dm.cap + j0 + kk * kTile, k_bar);
@@ -585,9 +591,9 @@ score_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         bulk_load(qd + kTileBytes, sc.stats + ((size_t)unit * sc.Mpad + (size_t)rb * kTile) * 2, kStatBytes, &q_bar[st]);
       }
     }
-  } else if (warp == 8) {
+  } else if (warp == 16) {
     // =============================== products (one lane) ===============================
-    if (tid == kScoreKeys) {
+    if (tid == kKeyThreads) {
       constexpr uint32_t kIdesc = instr_desc(false);
       const uint32_t k_addr = smem_u32(Ks);
       mbar_wait_idle(k_bar, 0, status);
@@ -609,7 +615,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
   } else {
     // =============================== one key per thread ===============================
     const float scale2 = dm.scale * 1.4426950408889634f;
-    const int kk = warp >> 2;
+    const int kk = (warp >> 2) & 1;
     const uint32_t t_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16) + kk * 256;
     for (int rb = 0; rb < nblocks; ++rb) {
       const int buf = rb & 1, st = rb % kQStages;
@@ -621,7 +627,8 @@ score_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
       // row block can have columns beyond M
       const bool plain = (j0 + kScoreKeys - 1 < n - m + 1) && (rb * kTile + kTile <= M);
 #pragma unroll
-      for (int cc = 0; cc < 4; ++cc) {
+      for (int c2 = 0; c2 < 2; ++c2) {
+        const int cc = 2 * rhalf + c2;  // this thread's two groups of 32 rows
         float v[32];
         tmem_ld32(t_lane + buf * 128 + cc * 32, v);
         const float* stc = stt + cc * 32 * 2;
@@ -650,7 +657,10 @@ score_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     }
   }
 
-  // ---- c_j = w_j / (1 - w_j) * ||X - v_j||, w_j = h_j / M ----
+  // ---- the two halves of a key add up; then c_j = w_j / (1 - w_j) * ||X - v_j||, w_j = h_j / M ----
+  if (tid >= kScoreKeys && tid < kKeyThreads) hx[tid - kScoreKeys] = h;
+  __syncthreads();
+  if (tid < kScoreKeys) h += hx[tid];
   if (tid < kScoreKeys && j < n) {
     const __nv_bfloat16* vrow = V + ((size_t)unit * dm.cap + j) * kD;
     float acc = 0.f;
