@@ -40,7 +40,7 @@ constexpr int kThreads = 128;
 constexpr long long kWaitCycles = 2000000000LL;
 
 struct Scratch {
-  float* stats;  // [units][Mpad][2]: log2-domain softmax reference, 1 / sum of 2^(s - ref)
+  float* stats;  // [units][Mpad]: log2-domain softmax reference + log2(sum of 2^(s - ref)): alpha = 2^(s - stats)
   float* X;      // [units][kD]
   int Mpad;      // M rounded up to a multiple of kTile
 };
@@ -50,7 +50,7 @@ inline size_t carve(const Dims& dm, char* base, Scratch* out) {
   s.Mpad = (dm.R + kTile - 1) / kTile * kTile;
   size_t off = 0;
   s.stats = reinterpret_cast<float*>(base + off);
-  off = align_up(off + sizeof(float) * 2 * (size_t)dm.units * s.Mpad, 256);
+  off = align_up(off + sizeof(float) * (size_t)dm.units * s.Mpad, 256);
   s.X = reinterpret_cast<float*>(base + off);
   off = align_up(off + sizeof(float) * (size_t)dm.units * kD, 256);
   if (out) *out = s;
@@ -488,10 +488,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
           *reinterpret_cast<float4*>(orow + cc * 32 + i) = make_float4(v[i] * inv_l, v[i + 1] * inv_l, v[i + 2] * inv_l, v[i + 3] * inv_l);
       }
     }
-    if (R < M && half == 0) {
-      sc.stats[((size_t)unit * sc.Mpad + R) * 2] = m_ref;
-      sc.stats[((size_t)unit * sc.Mpad + R) * 2 + 1] = inv_l;
-    }
+    if (R < M && half == 0) sc.stats[(size_t)unit * sc.Mpad + R] = m_ref + __log2f(l);
   }
   tc_fence_before();
   __syncthreads();
@@ -518,7 +515,7 @@ xsum_kernel(Dims dm, const int* __restrict__ len, const float* __restrict__ o, S
 constexpr int kScoreKeys = 2 * kTile;            // keys per CTA: two key tiles share every Q block
 constexpr int kKeyThreads = 2 * kScoreKeys;       // two threads per key: each owns 64 of a block's 128 rows
 constexpr int kScoreThreads = kKeyThreads + 64;   // + a warp for the products + a warp for the copies
-constexpr int kStatBytes = kTile * 2 * 4;         // (reference, 1 / sum) of the 128 rows of a block
+constexpr int kStatBytes = kTile * 4;             // the softmax statistic of the 128 rows of a block
 constexpr int kQStage = kTileBytes + kStatBytes;
 constexpr int kQStages = 3;
 
@@ -588,7 +585,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         mbar_expect_tx(&q_bar[st], kQStage);
         tma_load_2d(qd, &tmQ, 0, unit * M + rb * kTile, &q_bar[st]);
         tma_load_2d(qd + kHalfBytes, &tmQ, 64, unit * M + rb * kTile, &q_bar[st]);
-        bulk_load(qd + kTileBytes, sc.stats + ((size_t)unit * sc.Mpad + (size_t)rb * kTile) * 2, kStatBytes, &q_bar[st]);
+        bulk_load(qd + kTileBytes, sc.stats + (size_t)unit * sc.Mpad + (size_t)rb * kTile, kStatBytes, &q_bar[st]);
       }
     }
   } else if (warp == 16) {
@@ -631,13 +628,16 @@ score_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         const int cc = 2 * rhalf + c2;  // this thread's two groups of 32 rows
         float v[32];
         tmem_ld32(t_lane + buf * 128 + cc * 32, v);
-        const float* stc = stt + cc * 32 * 2;
+        const float* stc = stt + cc * 32;
         if (plain) {
           float h4[4] = {0.f, 0.f, 0.f, 0.f};  // independent partial sums
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const float2 rs = *reinterpret_cast<const float2*>(stc + 2 * i);  // (reference, 1 / sum) of the row
-            h4[i & 3] = fmaf(fast_exp2(fmaf(v[i], scale2, -rs.x)), rs.y, h4[i & 3]);
+          for (int i = 0; i < 32; i += 4) {
+            const float4 rs = *reinterpret_cast<const float4*>(stc + i);  // statistics of four rows
+            h4[0] += fast_exp2(fmaf(v[i], scale2, -rs.x));
+            h4[1] += fast_exp2(fmaf(v[i + 1], scale2, -rs.y));
+            h4[2] += fast_exp2(fmaf(v[i + 2], scale2, -rs.z));
+            h4[3] += fast_exp2(fmaf(v[i + 3], scale2, -rs.w));
           }
           h += (h4[0] + h4[1]) + (h4[2] + h4[3]);
         } else {
@@ -646,7 +646,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             const int R = rb * kTile + cc * 32 + i;  // query row of this column
             // row R sees key j iff j <= n - m + (R % m)
             const bool vis = R < M && j < n - m + (R % m) + 1;
-            const float a = fast_exp2(fmaf(v[i], scale2, -stc[2 * i])) * stc[2 * i + 1];
+            const float a = fast_exp2(fmaf(v[i], scale2, -stc[i]));
             h += vis ? a : 0.f;
           }
         }
