@@ -129,7 +129,8 @@ def build_state(w, device, rank, pool):
     budget = lens0.clone() if w.ragged_min_len is not None else torch.full_like(lens0, w.budget)
     for layer in range(w.layers):
         c = P.EvictionCache(w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.capacity, w.n_new, w.torch_dtype,
-                            budget, w.base_mode, "fill", w.scale, max_evict=w.n_new, device=device)
+                            budget, w.base_mode, "fill", w.scale,
+                            max_evict=max(w.n_new, w.init_len + w.n_new - w.budget), device=device)
         K0, V0 = wl.initial_cache(w, device, layer)
         c.load(K0, V0, lens0)
         del K0, V0
