@@ -7,7 +7,7 @@
 #include <vector>
 
 #include "common.cuh"
-#include "decode_stream.cuh"
+#include "decode_tc.cuh"
 #include "generic_score.cuh"
 #include "prefill_tc.cuh"
 #include "select_compact.cuh"
@@ -200,10 +200,10 @@ static int decode_grid_limit() {
   int g = cached[dev].load(std::memory_order_acquire);
   if (g == 0) {
     int sms = 0, per_sm = 0;
-    const size_t smem = decode::smem_bytes();
-    if (cudaFuncSetAttribute(decode::decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+    const size_t smem = decode::tc_smem_bytes();
+    if (cudaFuncSetAttribute(decode::decode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode::decode_kernel, decode::kThreads, smem) != cudaSuccess)
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode::decode_tc_kernel, decode::kTcThreads, smem) != cudaSuccess)
       return 0;
     g = sms * per_sm;
     cached[dev].store(g > 0 ? g : -1, std::memory_order_release);
@@ -229,11 +229,11 @@ static int launch_decode_score(const Dims& dm, const void* q, const void* K, con
   const int grid_limit = decode_grid_limit();
   TensorMapEncodeFn encode = tensor_map_encoder();
   const bool carried = dm.base_mode == CAOTE_BASE_ACCUM || dm.base_mode == CAOTE_BASE_EXTERNAL;
-  if (grid_limit <= 0 || !encode || (carried && !aligned(base, 16))) return CAOTE_OK;
+  if (grid_limit <= 0 || !encode || (carried && !aligned(base, 16)) || !aligned(q, 16)) return CAOTE_OK;
   decode::Plan pl;
   decode::carve(dm, ws + kHeaderBytes, &pl, grid_limit);
   int* status = reinterpret_cast<int*>(ws);
-  CUtensorMap tmK, tmV;
+  CUtensorMap tmK, tmV, tmQ;
   const cuuint64_t gdim[2] = {(cuuint64_t)dm.D, (cuuint64_t)dm.units * (cuuint64_t)dm.cap};
   const cuuint64_t gstride[1] = {(cuuint64_t)dm.D * 2};
   const cuuint32_t box[2] = {64, (cuuint32_t)decode::kT};
@@ -247,14 +247,26 @@ static int launch_decode_score(const Dims& dm, const void* q, const void* K, con
       return CAOTE_ERR_CUDA;
     }
   }
+  {
+    // the query rows: boxes of 64 channels x 16 rows (a unit's heads, padded by its neighbours' or by zeros)
+    const cuuint64_t qdim[2] = {(cuuint64_t)dm.D, (cuuint64_t)dm.B * (cuuint64_t)dm.Hq};
+    const cuuint32_t qbox[2] = {64, 16};
+    CUresult r = encode(&tmQ, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(q), qdim, gstride, qbox, estride,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+      snprintf(g_cuda_error, sizeof(g_cuda_error), "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+      return CAOTE_ERR_CUDA;
+    }
+  }
   CAOTE_LAUNCH("decode_plan_kernel", st,
                decode::plan_kernel<<<1, 1024, 0, st>>>(dm.units, dm.Hkv, dm.cap, len, pl, status));
   const int tiles_per_unit = (dm.cap + decode::kT - 1) / decode::kT;
   const long long max_items = (long long)dm.units * ((tiles_per_unit + pl.tpi - 1) / pl.tpi);
   const int grid = (int)(max_items < grid_limit ? max_items : grid_limit);
   CAOTE_LAUNCH("decode_kernel", st,
-               decode::decode_kernel<<<grid, decode::kThreads, decode::smem_bytes(), st>>>(
-                   tmK, tmV, dm, (const __nv_bfloat16*)q, len, base, o, scores, pl, status));
+               decode::decode_tc_kernel<<<grid, decode::kTcThreads, decode::tc_smem_bytes(), st>>>(
+                   tmK, tmV, tmQ, dm, len, base, o, scores, pl, status));
   *used = true;
   return CAOTE_OK;
 }
