@@ -29,11 +29,14 @@ sys.path.insert(0, ROOT)
 
 from paper_2504_14051_b200 import workloads as wl  # noqa: E402
 
-# DRAM bytes (read + write) of one launch per unit of work, from ncu captures of reduced cases
-# (profiles/*_ncu.txt), scaled to the launch at hand by the units it processes; traffic grows in
-# proportion to them. A value is set to None when its kernel has changed since the capture.
+# DRAM bytes (read + write) of one launch per unit of work, from ncu captures (profiles/*.txt), scaled
+# to the launch at hand by the units it processes; traffic grows in proportion to them. The decode
+# figure is from the full-size c4 launch (a one-pass capture of the two DRAM counters): in the reduced
+# case part of the second pass over V is served by L2, at full size none of it is. A value is set to
+# None when its kernel has changed since the capture.
 NCU_TRAFFIC = {
-    "decode_kernel": {"bytes_per_token_head": 288304128 / 449880, "profile": "profiles/decode_kernel_c4_batch16_ncu.txt"},
+    "decode_tc_kernel": {"bytes_per_token_head": (1419558400 + 62669824) / 1834896,
+                         "profile": "profiles/decode_tc_kernel_c4_full_traffic.txt"},
     "prefill_attn_kernel": {"bytes_per_unit": (155871488 + 22343680) / 16, "profile": "profiles/prefill_kernels_c5p_batch2_ncu.txt"},
 }
 

@@ -264,7 +264,7 @@ static int launch_decode_score(const Dims& dm, const void* q, const void* K, con
   const int tiles_per_unit = (dm.cap + decode::kT - 1) / decode::kT;
   const long long max_items = (long long)dm.units * ((tiles_per_unit + pl.tpi - 1) / pl.tpi);
   const int grid = (int)(max_items < grid_limit ? max_items : grid_limit);
-  CAOTE_LAUNCH("decode_kernel", st,
+  CAOTE_LAUNCH("decode_tc_kernel", st,
                decode::decode_tc_kernel<<<grid, decode::kTcThreads, decode::tc_smem_bytes(), st>>>(
                    tmK, tmV, tmQ, dm, len, base, o, scores, pl, status));
   *used = true;

@@ -1,24 +1,26 @@
 // Single-query (decode) scoring path on the 5th-generation tensor cores (tcgen05 + TMEM) for bf16,
-// head_dim 128, group size <= 8. Same work list, records and flags as decode_stream.cuh (attention
-// items A(i), score items B(i) trailing by `lag`, one atomic ticket counter, the last arriver of a
-// unit merges its records); what differs is how a CTA works through its slots.
+// head_dim 128, group size <= 8. Work items, records and flags: see decode_common.cuh.
 //
 // Every product has the tile's 128 tokens on the M side, so a token owns one TMEM lane and one thread
 // from the logits to the score:
 //   S^T[token][head]    = K_tile (A, K-major) x Q^T (B: 16 rows = the unit's query heads, rest unused)
 //   O^T[channel][head]  = V_tile^T (A, MN-major view of the same staged bytes) x P^T (B: 16 rows =
 //                         bf16 hi parts of the 8 heads' numerators, then their lo parts)
-// One lane of an issuing warp queues the products, a producer warp fills the slot ring by TMA, and
-// the four token warps do the softmax numerators (lazy reference: O^T is rescaled only when a logit
-// tops the reference by more than 2^8), the logits' write-out, and in the score pass
-// ||X - v_j||^2 by plain subtraction over the token's own V row.
+// A CTA (one per SM) runs two pipelines side by side, each fed through its own ring of shared-memory
+// slots by its own producer warp (TMA):
+//   attention side  K and V tiles in turn. One lane of an issuing warp queues the products; four
+//                   attention warps turn S^T into softmax numerators (lazy reference: O^T is rescaled
+//                   only when a logit tops the reference by more than 2^8), write the logits out and
+//                   close the item (record, counter, merge by the last arriver).
+//   score side      V tiles with their logits and carried base scores. Four score warps compute
+//                   ||X - v_j||^2 by plain subtraction over the token's own V row, and the score.
 //
 // Waits are bounded by a clock limit; the first one that runs out records CAOTE_ERR_TIMEOUT and
-// raises the CTA's stop flag, after which every wait returns at once, the producer stops taking work
+// raises the CTA's stop flag, after which every wait returns at once, the producers stop taking work
 // and the CTA drains its copies and leaves. Indices stay in bounds whatever the buffers hold.
 #pragma once
 
-#include "decode_stream.cuh"
+#include "decode_common.cuh"
 #include "prefill_tc.cuh"
 
 namespace caote {
