@@ -35,9 +35,9 @@ from paper_2504_14051_b200 import workloads as wl  # noqa: E402
 # case part of the second pass over V is served by L2, at full size none of it is. A value is set to
 # None when its kernel has changed since the capture.
 NCU_TRAFFIC = {
-    "decode_tc_kernel": {"bytes_per_token_head": (1419558400 + 62669824) / 1834896,
+    "decode_tc_kernel": {"bytes_per_token_head": (1420590336 + 62974464) / 1834896,
                          "profile": "profiles/decode_tc_kernel_c4_full_traffic.txt"},
-    "prefill_attn_kernel": {"bytes_per_unit": (155871488 + 22343680) / 16, "profile": "profiles/prefill_kernels_c5p_batch2_ncu.txt"},
+    "prefill_attn_kernel": {"bytes_per_unit": (155834368 + 22759680) / 16, "profile": "profiles/prefill_kernels_c5p_batch2_ncu.txt"},
 }
 
 METRIC = "cached tokens scored+evicted/sec"
