@@ -97,6 +97,36 @@ def test_score_matches_oracle(shape, mode, dtype):
     assert torch.equal(scores2, scores) and torch.equal(o2.view(torch.int32), o.view(torch.int32))
 
 
+@pytest.mark.parametrize("mode", ["last_query", "accum"])
+def test_decode_items_of_several_tiles_with_late_large_logits(mode):
+    """Enough tiles that the decode kernel works in items of two tiles, with keys planted in the second
+    tile of an item that top everything before them by far more than 2^8: the running softmax reference
+    has to move and the output accumulated so far has to be rescaled. Sampled units against the oracle."""
+    B, Hq, Hkv, d, cap = 10, 32, 8, 128, 1280
+    G = Hq // Hkv
+    lens = [1280 - 37 * (i % 5) for i in range(B)]
+    q, K, V, lens_t = make_case(777, B, Hq, Hkv, d, cap, 1, torch.bfloat16, lens)
+    units = [(0, 0), (3, 5), (9, 7), (6, 2)]
+    for b, h in units:
+        K[b, h, 200] = (q[b, h * G, 0].float() * 3.0).to(K.dtype)       # tile 1: ~ +49 in the log2 domain
+        K[b, h, 450] = (q[b, h * G + 1, 0].float() * 1.0).to(K.dtype)   # tile 3: ~ +16
+        K[b, h, 700] = (q[b, h * G + 3, 0].float() * 2.0).to(K.dtype)   # tile 5: ~ +33
+    base = None
+    if mode == "accum":
+        g = torch.Generator(device="cpu").manual_seed(9)
+        base = (torch.rand((B, Hkv, cap), generator=g) * 2.0).to(DEV)
+    base_in = None if base is None else base.clone()
+    p, ws, o, scores = run_score(q, K, V, lens_t, 1, mode, base)
+    qs, Ks, Vs, ls, bs = sub_problem(q, K, V, lens_t, base_in, units, Hkv, G)
+    r = oracle.score(f32(qs), f32(Ks), f32(Vs), ls.cpu().numpy(), scale=d ** -0.5, n_new=1, base_mode=mode,
+                     base=None if bs is None else bs.double().cpu().numpy())
+    sg, og = f32(scores), f32(o)
+    for i, (b, h) in enumerate(units):
+        n = lens[b]
+        assert_close(sg[b, h, :n], r["scores"][i, 0, :n], f"unit ({b},{h}) scores")
+        assert_close(og[b, h * G:(h + 1) * G], r["o"][i], f"unit ({b},{h}) o")
+
+
 def test_c1_full_step_every_token():
     """Tiny fp32 configuration: scores of all 256 tokens, then evict 128 in one selection."""
     w = wl.WORKLOADS["c1"]
