@@ -197,6 +197,32 @@ CAOTE_API int caote_step(const caote_params_t* params, const void* q, const void
                int32_t* n_evict, int32_t compact_mode, void* workspace, size_t workspace_bytes,
                caote_stream_t stream);
 
+/* ---- FastCAOTE (Sec. 3.3) ------------------------------------------------------------------------
+ * The same score with the pre-eviction output replaced by the plain mean of the cached values:
+ *     c_j = w_j / (1 - w_j) * || (1/n) sum_i v_i - v_j ||_2 ,
+ * everything else (attention, o, base score per base_mode, normalisation, selection) as in caote_score.
+ * The mean does not depend on the current queries, so it is carried from step to step instead of being
+ * recomputed: vsum [B, Hkv, d] fp32 holds, per unit, the sum of its n valid V rows (new tokens
+ * included). On the single-query path this removes the second pass over V: K and V are read once. */
+
+/* vsum[u, :] = sum_{j < len} V[u, j, :] from scratch (one read of V); len 0 gives 0. */
+CAOTE_API int caote_vsum(const caote_params_t* params, const void* V, const int32_t* len, float* vsum,
+               caote_stream_t stream);
+
+/* caote_score with FastCAOTE scores. vsum: in, current for the cache as passed (16-byte aligned). */
+CAOTE_API int caote_score_fast(const caote_params_t* params, const void* q, const void* K, const void* V,
+                     const int32_t* len, float* base, const float* vsum, float* o, float* scores,
+                     void* workspace, size_t workspace_bytes, caote_stream_t stream);
+
+/* caote_step with FastCAOTE scores. vsum: in/out; the rows appended by this call are added before
+ * scoring and the rows it evicts are subtracted, so that it is current for the next call. Sums are kept
+ * in fp32: refresh with caote_vsum now and then over very long runs if the drift matters. */
+CAOTE_API int caote_step_fast(const caote_params_t* params, const void* q, const void* k_new, const void* v_new,
+                    void* K, void* V, float* base, int32_t* pos, int32_t* len, int32_t* n_seen,
+                    const int32_t* budget, float* vsum, float* o, float* scores, int32_t* evict_idx,
+                    int32_t max_evict, int32_t* n_evict, int32_t compact_mode, void* workspace,
+                    size_t workspace_bytes, caote_stream_t stream);
+
 /* Synchronise the stream, copy the status word to *status_out (host pointer) and reset it to CAOTE_OK.
  * The word holds the first device-side error since the last reset. */
 CAOTE_API int caote_read_status(void* workspace, caote_stream_t stream, int32_t* status_out);

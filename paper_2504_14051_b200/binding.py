@@ -86,6 +86,12 @@ def lib() -> ctypes.CDLL:
     L.caote_compact.argtypes = [pp, vp, vp, vp, vp, vp, vp, i32, vp, i32, vp, sz, vp]
     L.caote_step.restype = ctypes.c_int
     L.caote_step.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, i32, vp, sz, vp]
+    L.caote_vsum.restype = ctypes.c_int
+    L.caote_vsum.argtypes = [pp, vp, vp, vp, vp]
+    L.caote_score_fast.restype = ctypes.c_int
+    L.caote_score_fast.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    L.caote_step_fast.restype = ctypes.c_int
+    L.caote_step_fast.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, i32, vp, sz, vp]
     L.caote_read_status.restype = ctypes.c_int
     L.caote_read_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32)]
     L.caote_status_string.restype = ctypes.c_char_p
@@ -181,6 +187,28 @@ def caote_step(p, q, k_new, v_new, K, V, base, pos, lens, n_seen, budget, o, sco
                             _p(lens), _p(n_seen), _p(budget), _p(o), _p(scores), _p(evict_idx),
                             evict_idx.shape[-1], _p(n_evict), mode, _p(workspace), workspace.numel(),
                             _stream(stream)))
+
+
+def caote_vsum(p, V, lens, vsum, stream=None):
+    """vsum[u, :] = sum of the unit's valid V rows (FastCAOTE, Sec. 3.3)."""
+    _check("caote_vsum", lib().caote_vsum(ctypes.byref(p), _p(V), _p(lens), _p(vsum), _stream(stream)))
+
+
+def caote_score_fast(p, q, K, V, lens, base, vsum, o, scores, workspace, stream=None):
+    _check("caote_score_fast",
+           lib().caote_score_fast(ctypes.byref(p), _p(q), _p(K), _p(V), _p(lens), _p(base), _p(vsum), _p(o),
+                                  _p(scores), _p(workspace), workspace.numel(), _stream(stream)))
+
+
+def caote_step_fast(p, q, k_new, v_new, K, V, base, pos, lens, n_seen, budget, vsum, o, scores, evict_idx, n_evict,
+                    mode, workspace, stream=None):
+    if isinstance(mode, str):
+        mode = COMPACT_MODES[mode]
+    _check("caote_step_fast",
+           lib().caote_step_fast(ctypes.byref(p), _p(q), _p(k_new), _p(v_new), _p(K), _p(V), _p(base), _p(pos),
+                                 _p(lens), _p(n_seen), _p(budget), _p(vsum), _p(o), _p(scores), _p(evict_idx),
+                                 evict_idx.shape[-1], _p(n_evict), mode, _p(workspace), workspace.numel(),
+                                 _stream(stream)))
 
 
 def caote_read_status(workspace, stream=None) -> int:

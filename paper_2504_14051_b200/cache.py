@@ -15,7 +15,7 @@ from . import binding as C
 class EvictionCache:
     def __init__(self, batch, n_q_heads, n_kv_heads, head_dim, capacity, n_new, dtype, budget,
                  base_mode="last_query", compact_mode="fill", scale: Optional[float] = None,
-                 max_evict: Optional[int] = None, device="cuda"):
+                 max_evict: Optional[int] = None, device="cuda", method: str = "caote"):
         self.device = torch.device(device)
         scale = head_dim ** -0.5 if scale is None else scale
         self.params = C.make_params(batch, n_q_heads, n_kv_heads, head_dim, capacity, n_new, dtype, scale,
@@ -39,6 +39,10 @@ class EvictionCache:
         self.n_evict = torch.zeros((B,), dtype=torch.int32, device=dev)
         self.o = torch.zeros((B, Hq, m, d), dtype=torch.float32, device=dev)
         self.workspace = C.alloc_workspace(self.params, dev)
+        # FastCAOTE (Sec. 3.3) scores against the mean of the cached values: the per-unit sum of V rows is state
+        assert method in ("caote", "fast")
+        self.method = method
+        self.vsum = torch.zeros((B, Hkv, d), dtype=torch.float32, device=dev) if method == "fast" else None
 
     def load(self, K, V, lens, base=None, pos=None):
         """Install an existing cache state (copied into the owned buffers)."""
@@ -53,9 +57,16 @@ class EvictionCache:
         else:
             cap = self.K.shape[2]
             self.pos.copy_(torch.arange(cap, dtype=torch.int32, device=self.device).expand_as(self.pos))
+        if self.vsum is not None:
+            C.caote_vsum(self.params, self.V, self.lens, self.vsum)
 
     def step(self, q, k_new, v_new, stream=None):
         """One eviction step; returns the pre-eviction attention output o [B, Hq, m, d]."""
+        if self.vsum is not None:
+            C.caote_step_fast(self.params, q, k_new, v_new, self.K, self.V, self.base, self.pos, self.lens,
+                              self.n_seen, self.budget, self.vsum, self.o, self.scores, self.evict_idx, self.n_evict,
+                              self.compact_mode, self.workspace, stream)
+            return self.o
         C.caote_step(self.params, q, k_new, v_new, self.K, self.V, self.base, self.pos, self.lens, self.n_seen,
                      self.budget, self.o, self.scores, self.evict_idx, self.n_evict, self.compact_mode,
                      self.workspace, stream)

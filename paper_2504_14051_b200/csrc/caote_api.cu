@@ -145,7 +145,7 @@ static int allow_smem(KernelT kernel, size_t bytes) {
 
 template <typename T, int D>
 static int launch_generic_score(const Dims& dm, const void* q, const void* K, const void* V, const int* len,
-                                float* base, float* o, float* scores, char* ws, cudaStream_t st) {
+                                float* base, float* o, float* scores, char* ws, cudaStream_t st, const float* vsum) {
   generic::Scratch sc;
   generic::carve(dm, ws + kHeaderBytes, &sc);
   int* status = reinterpret_cast<int*>(ws);
@@ -168,7 +168,7 @@ static int launch_generic_score(const Dims& dm, const void* q, const void* K, co
     if (rc) return rc;
     dim3 grid((dm.cap + generic::kKT - 1) / generic::kKT, dm.units);
     CAOTE_LAUNCH("score_pass_kernel", st, generic::score_pass_kernel<T, D><<<grid, generic::kThreads, smem, st>>>(
-        dm, (const T*)q, (const T*)K, (const T*)V, len, base, sc, scores));
+        dm, (const T*)q, (const T*)K, (const T*)V, len, base, sc, scores, vsum));
   }
   return CAOTE_OK;
 }
@@ -201,9 +201,10 @@ static int decode_grid_limit() {
   if (g == 0) {
     int sms = 0, per_sm = 0;
     const size_t smem = decode::tc_smem_bytes();
-    if (cudaFuncSetAttribute(decode::decode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+    if (cudaFuncSetAttribute(decode::decode_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+        cudaFuncSetAttribute(decode::decode_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode::decode_tc_kernel, decode::kTcThreads, smem) != cudaSuccess)
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode::decode_tc_kernel<false>, decode::kTcThreads, smem) != cudaSuccess)
       return 0;
     g = sms * per_sm;
     cached[dev].store(g > 0 ? g : -1, std::memory_order_release);
@@ -224,7 +225,8 @@ static bool decode_shape_ok(const caote_params_t* p) {
 }
 
 static int launch_decode_score(const Dims& dm, const void* q, const void* K, const void* V, const int* len,
-                               float* base, float* o, float* scores, char* ws, cudaStream_t st, bool* used) {
+                               float* base, float* o, float* scores, char* ws, cudaStream_t st, bool* used,
+                               const float* vsum) {
   *used = false;
   const int grid_limit = decode_grid_limit();
   TensorMapEncodeFn encode = tensor_map_encoder();
@@ -264,9 +266,18 @@ static int launch_decode_score(const Dims& dm, const void* q, const void* K, con
   const int tiles_per_unit = (dm.cap + decode::kT - 1) / decode::kT;
   const long long max_items = (long long)dm.units * ((tiles_per_unit + pl.tpi - 1) / pl.tpi);
   const int grid = (int)(max_items < grid_limit ? max_items : grid_limit);
-  CAOTE_LAUNCH("decode_tc_kernel", st,
-               decode::decode_tc_kernel<<<grid, decode::kTcThreads, decode::tc_smem_bytes(), st>>>(
-                   tmK, tmV, tmQ, dm, len, base, o, scores, pl, status));
+  if (!vsum) {
+    CAOTE_LAUNCH("decode_tc_kernel", st,
+                 decode::decode_tc_kernel<false><<<grid, decode::kTcThreads, decode::tc_smem_bytes(), st>>>(
+                     tmK, tmV, tmQ, dm, len, base, o, scores, nullptr, pl, status));
+  } else {
+    // FastCAOTE: one pass over K and V, then scores from the stored logits and distances
+    CAOTE_LAUNCH("decode_tc_fast_kernel", st,
+                 decode::decode_tc_kernel<true><<<grid, decode::kTcThreads, decode::tc_smem_bytes(), st>>>(
+                     tmK, tmV, tmQ, dm, len, base, o, scores, vsum, pl, status));
+    dim3 fgrid(tiles_per_unit, dm.units);
+    CAOTE_LAUNCH("fast_finish_kernel", st, decode::fast_finish_kernel<<<fgrid, decode::kT, 0, st>>>(dm, len, base, scores, pl));
+  }
   *used = true;
   return CAOTE_OK;
 }
@@ -296,7 +307,7 @@ static int encode_rows_map(CUtensorMap* tm, const void* ptr, unsigned long long 
 }
 
 static int launch_prefill_score(const Dims& dm, const void* q, const void* K, const void* V, const int* len, float* o,
-                                float* scores, char* ws, cudaStream_t st, bool* used) {
+                                float* scores, char* ws, cudaStream_t st, bool* used, const float* vsum) {
   *used = false;
   TensorMapEncodeFn encode = tensor_map_encoder();
   if (!encode) return CAOTE_OK;
@@ -318,7 +329,11 @@ static int launch_prefill_score(const Dims& dm, const void* q, const void* K, co
                  prefill::attn_kernel<<<grid, prefill::kAttnThreads, prefill::attn_smem_bytes(), st>>>(tmQ, tmK64, tmV64, dm, len,
                                                                                                     sc, o, status));
   }
-  CAOTE_LAUNCH("prefill_xsum_kernel", st, prefill::xsum_kernel<<<dm.units, prefill::kD, 0, st>>>(dm, len, o, sc));
+  if (vsum) {
+    CAOTE_LAUNCH("fast_mean_kernel", st, fast::mean_kernel<<<dm.units, prefill::kD, 0, st>>>(dm.Hkv, dm.cap, prefill::kD, len, vsum, sc.X));
+  } else {
+    CAOTE_LAUNCH("prefill_xsum_kernel", st, prefill::xsum_kernel<<<dm.units, prefill::kD, 0, st>>>(dm, len, o, sc));
+  }
   {
     dim3 grid((dm.cap + prefill::kScoreKeys - 1) / prefill::kScoreKeys, dm.units);
     CAOTE_LAUNCH("prefill_score_kernel", st,
@@ -396,9 +411,10 @@ int caote_append(const caote_params_t* p, void* K, void* V, float* base, int32_t
   return CAOTE_OK;
 }
 
-int caote_score(const caote_params_t* p, const void* q, const void* K, const void* V, const int32_t* len,
-                float* base, float* o, float* scores, void* workspace, size_t workspace_bytes_,
-                caote_stream_t stream) {
+// caote_score (vsum == NULL) and caote_score_fast (vsum: the per-unit sums of the cached value rows).
+static int score_impl(const caote_params_t* p, const void* q, const void* K, const void* V, const int32_t* len,
+                      float* base, const float* vsum, float* o, float* scores, void* workspace, size_t workspace_bytes_,
+                      caote_stream_t stream) {
   if (!params_ok(p) || !q || !K || !V || !len || !o || !scores || !workspace) return CAOTE_ERR_INVALID_ARG;
   if (!params_supported(p)) return CAOTE_ERR_UNSUPPORTED;
   if ((p->base_mode == CAOTE_BASE_ACCUM || p->base_mode == CAOTE_BASE_EXTERNAL) && !base)
@@ -410,22 +426,51 @@ int caote_score(const caote_params_t* p, const void* q, const void* K, const voi
   const Dims dm = make_dims(p);
   cudaStream_t st = (cudaStream_t)stream;
   char* ws = (char*)workspace;
-  if (decode_shape_ok(p) && !(p->flags & 0)) {
+  if (decode_shape_ok(p)) {
     bool used = false;
-    rc = launch_decode_score(dm, q, K, V, len, base, o, scores, ws, st, &used);
+    rc = launch_decode_score(dm, q, K, V, len, base, o, scores, ws, st, &used, vsum);
     if (rc || used) return rc;
   }
   if (prefill_shape_ok(p)) {
     bool used = false;
-    rc = launch_prefill_score(dm, q, K, V, len, o, scores, ws, st, &used);
+    rc = launch_prefill_score(dm, q, K, V, len, o, scores, ws, st, &used, vsum);
     if (rc || used) return rc;
   }
   if (p->dtype == CAOTE_BF16) {
-    if (dm.D == 128) return launch_generic_score<__nv_bfloat16, 128>(dm, q, K, V, len, base, o, scores, ws, st);
-    return launch_generic_score<__nv_bfloat16, 64>(dm, q, K, V, len, base, o, scores, ws, st);
+    if (dm.D == 128) return launch_generic_score<__nv_bfloat16, 128>(dm, q, K, V, len, base, o, scores, ws, st, vsum);
+    return launch_generic_score<__nv_bfloat16, 64>(dm, q, K, V, len, base, o, scores, ws, st, vsum);
   }
-  if (dm.D == 128) return launch_generic_score<float, 128>(dm, q, K, V, len, base, o, scores, ws, st);
-  return launch_generic_score<float, 64>(dm, q, K, V, len, base, o, scores, ws, st);
+  if (dm.D == 128) return launch_generic_score<float, 128>(dm, q, K, V, len, base, o, scores, ws, st, vsum);
+  return launch_generic_score<float, 64>(dm, q, K, V, len, base, o, scores, ws, st, vsum);
+}
+
+int caote_score(const caote_params_t* p, const void* q, const void* K, const void* V, const int32_t* len,
+                float* base, float* o, float* scores, void* workspace, size_t workspace_bytes_,
+                caote_stream_t stream) {
+  return score_impl(p, q, K, V, len, base, nullptr, o, scores, workspace, workspace_bytes_, stream);
+}
+
+int caote_score_fast(const caote_params_t* p, const void* q, const void* K, const void* V, const int32_t* len,
+                     float* base, const float* vsum, float* o, float* scores, void* workspace,
+                     size_t workspace_bytes_, caote_stream_t stream) {
+  if (!vsum || !aligned(vsum, 16)) return CAOTE_ERR_INVALID_ARG;
+  return score_impl(p, q, K, V, len, base, vsum, o, scores, workspace, workspace_bytes_, stream);
+}
+
+int caote_vsum(const caote_params_t* p, const void* V, const int32_t* len, float* vsum, caote_stream_t stream) {
+  if (!params_ok(p) || !V || !len || !vsum) return CAOTE_ERR_INVALID_ARG;
+  if (!params_supported(p)) return CAOTE_ERR_UNSUPPORTED;
+  int rc = check_device();
+  if (rc) return rc;
+  const Dims dm = make_dims(p);
+  cudaStream_t st = (cudaStream_t)stream;
+  if (p->dtype == CAOTE_BF16) {
+    CAOTE_LAUNCH("fast_vsum_kernel", st, fast::vsum_kernel<__nv_bfloat16><<<dm.units, 256, 0, st>>>(
+        dm.Hkv, dm.cap, dm.D, (const __nv_bfloat16*)V, len, vsum));
+  } else {
+    CAOTE_LAUNCH("fast_vsum_kernel", st, fast::vsum_kernel<float><<<dm.units, 256, 0, st>>>(dm.Hkv, dm.cap, dm.D, (const float*)V, len, vsum));
+  }
+  return CAOTE_OK;
 }
 
 int caote_score_static(const caote_params_t* p, const void* q, const void* K, const void* V, const int32_t* len,
@@ -488,16 +533,30 @@ int caote_compact(const caote_params_t* p, void* K, void* V, float* base, int32_
   return CAOTE_OK;
 }
 
-int caote_step(const caote_params_t* p, const void* q, const void* k_new, const void* v_new, void* K, void* V,
-               float* base, int32_t* pos, int32_t* len, int32_t* n_seen, const int32_t* budget, float* o,
-               float* scores, int32_t* evict_idx, int32_t max_evict, int32_t* n_evict, int32_t compact_mode,
-               void* workspace, size_t workspace_bytes_, caote_stream_t stream) {
+// caote_step (vsum == NULL) and caote_step_fast (vsum kept current: += appended rows, -= evicted rows).
+static int step_impl(const caote_params_t* p, const void* q, const void* k_new, const void* v_new, void* K, void* V,
+                     float* base, int32_t* pos, int32_t* len, int32_t* n_seen, const int32_t* budget, float* vsum,
+                     float* o, float* scores, int32_t* evict_idx, int32_t max_evict, int32_t* n_evict,
+                     int32_t compact_mode, void* workspace, size_t workspace_bytes_, caote_stream_t stream) {
   int rc;
+  const bool bf16 = params_ok(p) && p->dtype == CAOTE_BF16;
   if (k_new || v_new) {
+    if (vsum) {
+      if (!params_ok(p) || !v_new || !len) return CAOTE_ERR_INVALID_ARG;
+      const Dims dm = make_dims(p);
+      cudaStream_t st = (cudaStream_t)stream;
+      if (bf16) {
+        CAOTE_LAUNCH("fast_vsum_add_kernel", st, fast::vsum_add_kernel<__nv_bfloat16><<<dm.units, dm.D, 0, st>>>(
+            dm.Hkv, dm.cap, dm.m, dm.D, (const __nv_bfloat16*)v_new, len, vsum));
+      } else {
+        CAOTE_LAUNCH("fast_vsum_add_kernel", st, fast::vsum_add_kernel<float><<<dm.units, dm.D, 0, st>>>(
+            dm.Hkv, dm.cap, dm.m, dm.D, (const float*)v_new, len, vsum));
+      }
+    }
     rc = caote_append(p, K, V, base, pos, len, n_seen, k_new, v_new, workspace, workspace_bytes_, stream);
     if (rc) return rc;
   }
-  rc = caote_score(p, q, K, V, len, base, o, scores, workspace, workspace_bytes_, stream);
+  rc = score_impl(p, q, K, V, len, base, vsum, o, scores, workspace, workspace_bytes_, stream);
   if (rc) return rc;
   if (compact_mode == CAOTE_COMPACT_FILL) {
     // selection, compaction and the length update in one launch (same results as the two calls below)
@@ -509,14 +568,42 @@ int caote_step(const caote_params_t* p, const void* q, const void* k_new, const 
     CAOTE_LAUNCH("select_compact_kernel", st,
                  sel::select_compact_kernel<<<dm.units, sel::kSelThreads, 0, st>>>(
                      dm.B, dm.Hkv, dm.cap, row_bytes, scores, (char*)K, (char*)V, base, pos, len, budget, evict_idx,
-                     max_evict, n_evict, hdr, hdr + 4));
+                     max_evict, n_evict, hdr, hdr + 4, vsum, bf16 ? 2 : 4));
     return CAOTE_OK;
   }
   rc = caote_select_evict(p, scores, len, budget, pos, evict_idx, max_evict, n_evict, workspace,
                           workspace_bytes_, stream);
   if (rc) return rc;
+  if (vsum) {
+    const Dims dm = make_dims(p);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (bf16) {
+      CAOTE_LAUNCH("fast_vsum_sub_kernel", st, fast::vsum_sub_kernel<__nv_bfloat16><<<dm.units, 128, 0, st>>>(
+          dm.Hkv, dm.cap, dm.D, (const __nv_bfloat16*)V, evict_idx, max_evict, n_evict, vsum));
+    } else {
+      CAOTE_LAUNCH("fast_vsum_sub_kernel", st, fast::vsum_sub_kernel<float><<<dm.units, 128, 0, st>>>(
+          dm.Hkv, dm.cap, dm.D, (const float*)V, evict_idx, max_evict, n_evict, vsum));
+    }
+  }
   return caote_compact(p, K, V, base, pos, len, evict_idx, max_evict, n_evict, compact_mode, workspace,
                        workspace_bytes_, stream);
+}
+
+int caote_step(const caote_params_t* p, const void* q, const void* k_new, const void* v_new, void* K, void* V,
+               float* base, int32_t* pos, int32_t* len, int32_t* n_seen, const int32_t* budget, float* o,
+               float* scores, int32_t* evict_idx, int32_t max_evict, int32_t* n_evict, int32_t compact_mode,
+               void* workspace, size_t workspace_bytes_, caote_stream_t stream) {
+  return step_impl(p, q, k_new, v_new, K, V, base, pos, len, n_seen, budget, nullptr, o, scores, evict_idx, max_evict,
+                   n_evict, compact_mode, workspace, workspace_bytes_, stream);
+}
+
+int caote_step_fast(const caote_params_t* p, const void* q, const void* k_new, const void* v_new, void* K, void* V,
+                    float* base, int32_t* pos, int32_t* len, int32_t* n_seen, const int32_t* budget, float* vsum,
+                    float* o, float* scores, int32_t* evict_idx, int32_t max_evict, int32_t* n_evict,
+                    int32_t compact_mode, void* workspace, size_t workspace_bytes_, caote_stream_t stream) {
+  if (!vsum || !aligned(vsum, 16)) return CAOTE_ERR_INVALID_ARG;
+  return step_impl(p, q, k_new, v_new, K, V, base, pos, len, n_seen, budget, vsum, o, scores, evict_idx, max_evict,
+                   n_evict, compact_mode, workspace, workspace_bytes_, stream);
 }
 
 int caote_read_status(void* workspace, caote_stream_t stream, int32_t* status_out) {

@@ -65,6 +65,7 @@ struct Plan {
   PartialRec* part;   // [max items]
   FinalRec* fin;      // [units]
   float* S;           // [units][capS / kT][G][kT] log2-domain logits, tile by tile
+  float* dist;        // [units][capS] ||mean(v) - v_j|| (FastCAOTE only)
   int tpi;            // tiles per item
   int capS;           // cap rounded up to a multiple of kT
 };
@@ -98,6 +99,7 @@ inline size_t carve(const Dims& dm, char* base, Plan* out, int grid) {
   pl.work = (int*)take(sizeof(int) * 4);
   pl.fin = (FinalRec*)take(sizeof(FinalRec) * (size_t)dm.units);
   pl.S = (float*)take(sizeof(float) * (size_t)dm.units * dm.G * pl.capS);
+  pl.dist = (float*)take(sizeof(float) * (size_t)dm.units * pl.capS);
   pl.part = (PartialRec*)take(sizeof(PartialRec) * max_items);
   if (out) *out = pl;
   return off;

@@ -15,6 +15,12 @@
 //   score side      V tiles with their logits and carried base scores. Four score warps compute
 //                   ||X - v_j||^2 by plain subtraction over the token's own V row, and the score.
 //
+// FastCAOTE (Sec. 3.3; template flag kFast): X is the plain mean of the cached values, known before
+// the pass (the caller keeps the per-unit sum of V rows), so V is read once: the score warps take
+// ||mean - v_j|| from the attention side's V tile while the softmax is under way and store it (4 bytes per
+// token); the score side and its ring stay idle, and fast_finish_kernel turns logits, final statistics
+// and distances into scores afterwards.
+//
 // Waits are bounded by a clock limit; the first one that runs out records CAOTE_ERR_TIMEOUT and
 // raises the CTA's stop flag, after which every wait returns at once, the producers stop taking work
 // and the CTA drains its copies and leaves. Indices stay in bounds whatever the buffers hold.
@@ -155,10 +161,12 @@ __device__ __forceinline__ Entry find_entry(int item, const Dims& dm, const Plan
   return e;
 }
 
+template <bool kFast>
 __global__ void __launch_bounds__(kTcThreads, 1)
 decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                  const __grid_constant__ CUtensorMap tmQ, Dims dm, const int* __restrict__ len,
-                 float* __restrict__ base, float* __restrict__ o, float* __restrict__ scores, Plan pl, int* status) {
+                 float* __restrict__ base, float* __restrict__ o, float* __restrict__ scores, const float* __restrict__ vsum,
+                 Plan pl, int* status) {
   extern __shared__ char smem_raw[];
   char* sm = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   char* tilesA = sm;                                                     // [kASlots][kTileBytes]
@@ -167,6 +175,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   char* pbuf = qbuf + kQBufs * kQBytes;                                  // [2][kPBytes]
   char* baseA = pbuf + 2 * kPBytes;                                      // [kASlots][kBaseRowBytes]
   char* sideB = baseA + kASlots * kBaseRowBytes;                         // [kBSlots][kBSideBytes]
+  float* xbuf = reinterpret_cast<float*>(sideB);                         // kFast: [kQBufs][kD + 4] sum of V rows, 1 / n
   char* finbuf = sideB + kBSlots * kBSideBytes;                          // [kFinBufs] FinalRec
   Desc* descA = reinterpret_cast<Desc*>(finbuf + kFinBufs * kFinalBytes);  // [kASlots]
   Desc* descB = descA + kASlots;                                         // [kBSlots]
@@ -197,7 +206,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   if (tid == 0) {
     for (int i = 0; i < kASlots; ++i) {
       mbar_init(&fullA[i], 1);
-      mbar_init(&emptyA[i], 5);
+      mbar_init(&emptyA[i], kFast ? 9 : 5);  // 4 attention warps + the issuing lane (+ 4 score warps)
     }
     for (int i = 0; i < kBSlots; ++i) {
       mbar_init(&fullB[i], 1);
@@ -257,7 +266,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
           d.type = kSlotKA;
           descA[s] = d;
           const bool first = (d.flags & kFlagFirst) != 0;
-          mbar_expect_tx(&fullA[s], kTileBytes + base_bytes + (first ? (uint32_t)kQBytes : 0u));
+          if (kFast && first) xbuf[(a_items % kQBufs) * (kD + 4) + kD] = 1.f / (float)e.n;
+          mbar_expect_tx(&fullA[s], kTileBytes + base_bytes + (first ? (uint32_t)kQBytes + (kFast ? kD * 4u : 0u) : 0u));
           tma_load_2d(tl, &tmK, 0, row, &fullA[s], pol_stream);
           tma_load_2d(tl + kHalfBytes, &tmK, 64, row, &fullA[s], pol_stream);
           if (use_base)
@@ -269,6 +279,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             const int qrow = (e.unit / dm.Hkv) * dm.Hq + (e.unit % dm.Hkv) * G;
             tma_load_2d(qb, &tmQ, 0, qrow, &fullA[s], pol_keep);
             tma_load_2d(qb + kQBytes / 2, &tmQ, 64, qrow, &fullA[s], pol_keep);
+            if (kFast) bulk_load(xbuf + (a_items % kQBufs) * (kD + 4), vsum + (size_t)e.unit * kD, kD * 4, &fullA[s]);
             ++a_items;
           }
           ctl[2] = ++issued;
@@ -309,7 +320,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     const uint64_t pol_stream = policy_evict_first();
     int issued = 0, b_items = 0;
     bool ok = true;
-    while (ok) {
+    while (ok && !kFast) {  // (FastCAOTE has no second pass over V: this ring stays empty)
       int w = 0;
       if (lane == 0) w = atomicAdd(&pl.work[1], 1);
       w = __shfl_sync(0xffffffffu, w, 0);
@@ -354,7 +365,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
       }
       ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
     }
-    if (lane == 0) {
+    if (lane == 0 && !kFast) {
       if (ok) {
         const int s = issued % kBSlots;
         if (mbar_wait(&emptyB[s], ((issued / kBSlots) & 1) ^ 1, &ctl[0])) {
@@ -676,6 +687,48 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   } else {
     // ================================ score warps (thread = token) ================================
     const int tok = tid - kTcTokenThreads;
+    if constexpr (kFast) {
+      // FastCAOTE: walk the attention ring; from every V tile take || mean(v) - v_j || of the token's row
+      int items = 0;
+      for (int i = 0;; ++i) {
+        const int s = i % kASlots;
+        const char* sl = tilesA + s * kTileBytes;
+        const bool got = warp_mbar_wait(&fullA[s], (i / kASlots) & 1, &ctl[0], lane);
+        if (token_any(2, !got)) {
+          if (tok == 0 && !ctl[0]) {
+            set_status(status, CAOTE_ERR_TIMEOUT);
+            ctl[0] = 1;
+          }
+          break;
+        }
+        const Desc d = descA[s];
+        if (d.type == kSlotStop) break;
+        if (d.type == kSlotKA) {
+          if (d.flags & kFlagFirst) ++items;
+        } else {
+          const float* xs = xbuf + ((items - 1) % kQBufs) * (kD + 4);
+          const float inv_n = xs[kD];
+          float n2a = 0.f, n2b = 0.f;
+#pragma unroll 2
+          for (int c = 0; c < 16; ++c) {
+            const uint4 raw = *reinterpret_cast<const uint4*>(sl + tile_off(tok, c));
+            const float4 x0 = *reinterpret_cast<const float4*>(xs + 8 * c);
+            const float4 x1 = *reinterpret_cast<const float4*>(xs + 8 * c + 4);
+            const float d0 = fmaf(x0.x, inv_n, -__uint_as_float(raw.x << 16)), d1 = fmaf(x0.y, inv_n, -__uint_as_float(raw.x & 0xffff0000u));
+            const float d2 = fmaf(x0.z, inv_n, -__uint_as_float(raw.y << 16)), d3 = fmaf(x0.w, inv_n, -__uint_as_float(raw.y & 0xffff0000u));
+            const float d4 = fmaf(x1.x, inv_n, -__uint_as_float(raw.z << 16)), d5 = fmaf(x1.y, inv_n, -__uint_as_float(raw.z & 0xffff0000u));
+            const float d6 = fmaf(x1.z, inv_n, -__uint_as_float(raw.w << 16)), d7 = fmaf(x1.w, inv_n, -__uint_as_float(raw.w & 0xffff0000u));
+            n2a = fmaf(d0, d0, n2a); n2b = fmaf(d1, d1, n2b);
+            n2a = fmaf(d2, d2, n2a); n2b = fmaf(d3, d3, n2b);
+            n2a = fmaf(d4, d4, n2a); n2b = fmaf(d5, d5, n2b);
+            n2a = fmaf(d6, d6, n2a); n2b = fmaf(d7, d7, n2b);
+          }
+          if (tok < d.n_valid) __stcg(pl.dist + (size_t)d.unit * pl.capS + (size_t)d.tile * kT + tok, sqrtf(n2a + n2b));
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&emptyA[s]);
+      }
+    } else
     for (;; ++seenB) {
       const int s = seenB % kBSlots;
       const char* sl = tilesB + s * kTileBytes;
@@ -746,6 +799,37 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   if (tid == kTcTokenThreads)
     for (int j = seenB; j < ctl[3]; ++j) mbar_wait(&fullB[j % kBSlots], (j / kBSlots) & 1, &dummy);
   if (warp == kTcIssueWarp) prefill::tmem_dealloc(tmem, kTmemCols);
+}
+
+// FastCAOTE, after decode_tc_kernel<true>: c_j = w_j / (1 - w_j) * || mean(v) - v_j || from the stored
+// logits, the unit's final softmax statistics and the stored distances. grid = (tiles, units), kT threads.
+__global__ void __launch_bounds__(kT)
+fast_finish_kernel(Dims dm, const int* __restrict__ len, float* __restrict__ base, float* __restrict__ scores, Plan pl) {
+  const int unit = blockIdx.y, tile = blockIdx.x, b = unit / dm.Hkv;
+  const int n = len[b], tok = tile * kT + threadIdx.x;
+  if (n <= 0 || n > dm.cap || tok >= n) return;
+  const int G = dm.G, mode = dm.base_mode;
+  const FinalRec* fr = pl.fin + unit;
+  float hj = 0.f;
+  if (mode != CAOTE_BASE_EXTERNAL) {
+    const float* Sg = pl.S + ((size_t)unit * (pl.capS / kT) + tile) * G * kT + threadIdx.x;
+    for (int g = 0; g < G; ++g) hj = fmaf(fast_exp2(__ldcg(Sg + g * kT) - fr->m[g]), fr->inv_l[g], hj);
+  }
+  const size_t slot = (size_t)unit * dm.cap + tok;
+  if (mode == CAOTE_BASE_ACCUM) {
+    hj += base[slot];
+    base[slot] = hj;
+  } else if (mode == CAOTE_BASE_EXTERNAL) {
+    hj = base[slot];
+  }
+  const float Htot = fr->H;
+  float ratio = 0.f;
+  if (Htot > 0.f) {
+    const float rest = Htot - hj;
+    ratio = (rest > 0.f) ? hj / rest : INFINITY;
+  }
+  const float dist = __ldcg(pl.dist + (size_t)unit * pl.capS + tok);
+  scores[slot] = (ratio == 0.f) ? 0.f : ((ratio == INFINITY) ? INFINITY : ratio * dist);
 }
 
 }  // namespace decode

@@ -310,7 +310,7 @@ template <typename T, int D>
 __global__ void __launch_bounds__(kThreads)
 score_pass_kernel(Dims dm, const T* __restrict__ q, const T* __restrict__ K, const T* __restrict__ V,
                   const int* __restrict__ len, float* __restrict__ base, Scratch sc,
-                  float* __restrict__ scores) {
+                  float* __restrict__ scores, const float* __restrict__ vsum) {
   constexpr int LD = D + 4;
   extern __shared__ __align__(16) float smem[];
   float* Qs = smem;              // kRT * LD
@@ -338,6 +338,7 @@ score_pass_kernel(Dims dm, const T* __restrict__ q, const T* __restrict__ K, con
     for (int ch = 0; ch < sc.chunks; ++ch) x += sc.osum[((size_t)unit * sc.chunks + ch) * D + tid];
     if (carried) x += sc.ytot[(size_t)unit * D + tid];
     Xs[tid] = (Htot > 0.f) ? x / Htot : 0.f;
+    if (vsum) Xs[tid] = vsum[(size_t)unit * D + tid] / (float)n;  // FastCAOTE (Sec. 3.3): the mean of the cached values
   }
   const int valid = min(kKT, n - j0);
   if (n_rows > 0) stage_rows<T, D, LD>(Ks, K + ((size_t)unit * dm.cap + j0) * D, kKT, valid);

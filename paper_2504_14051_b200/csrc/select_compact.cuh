@@ -5,6 +5,7 @@
 #pragma once
 
 #include "common.cuh"
+#include "fast.cuh"
 
 namespace caote {
 namespace sel {
@@ -197,11 +198,17 @@ __global__ void __launch_bounds__(kSelThreads)
 select_compact_kernel(int B, int Hkv, int cap, int row_bytes, const float* __restrict__ scores, char* __restrict__ K,
                       char* __restrict__ V, float* __restrict__ base, int* __restrict__ pos, int* __restrict__ len,
                       const int* __restrict__ budget, int* __restrict__ evict_idx, int max_evict,
-                      int* __restrict__ n_evict, int* status, int* ticket) {
+                      int* __restrict__ n_evict, int* status, int* ticket, float* __restrict__ vsum, int elt_bytes) {
   __shared__ int s_last;
   const int unit = blockIdx.x;
   const int k = select_unit(unit, Hkv, cap, scores, len, budget, pos, evict_idx, max_evict, n_evict, status);
   __syncthreads();  // evict_idx of this unit is written
+  if (vsum && k > 0) {  // FastCAOTE: the evicted rows leave the running sum of values before they are overwritten
+    const int* E = evict_idx + (size_t)unit * max_evict;
+    if (elt_bytes == 2) fast::vsum_sub_unit<__nv_bfloat16>(unit, k, cap, row_bytes / 2, (const __nv_bfloat16*)V, E, vsum);
+    else fast::vsum_sub_unit<float>(unit, k, cap, row_bytes / 4, (const float*)V, E, vsum);
+    __syncthreads();
+  }
   compact_fill_unit(unit, k, Hkv, cap, row_bytes, K, V, base, pos, len, evict_idx, max_evict);
   __syncthreads();
   if (threadIdx.x == 0) {

@@ -1,0 +1,121 @@
+"""FastCAOTE (Sec. 3.3) on the GPU against the oracle: scores with X = mean of the cached values, and the
+running per-unit sum of value rows that the library carries from step to step."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2504_14051_b200 as P
+from paper_2504_14051_b200 import workloads as wl
+
+from parity import assert_close, check_evicted, f32, sub_problem
+from test_gpu_parity import make_case
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+SHAPES = [
+    # B, Hq, Hkv, d, cap, m, lens, dtype      (path)
+    (2, 8, 2, 128, 300, 1, [257, 129], torch.bfloat16),        # single-query tensor-core path
+    (1, 7, 1, 128, 1100, 1, [1031], torch.bfloat16),
+    (3, 16, 2, 128, 200, 1, [200, 0, 65], torch.bfloat16),
+    (10, 32, 8, 128, 1280, 1, [1280 - 37 * (i % 5) for i in range(10)], torch.bfloat16),  # items of two tiles
+    (2, 16, 2, 128, 1200, 128, [1200, 777], torch.bfloat16),   # tensor-core prefill path
+    (2, 4, 2, 64, 80, 1, [63, 80], torch.float32),             # generic path
+    (1, 14, 2, 128, 400, 3, [333], torch.bfloat16),
+]
+
+
+def expected_fast(r, V, lens, units):
+    out = {}
+    Vf = f32(V)
+    for b, h in units:
+        n = int(lens[b])
+        out[(b, h)] = oracle.fast_scores(r["w"][b, h, :n], Vf[b, h, :n]) if n > 0 else np.zeros(0)
+    return out
+
+
+@pytest.mark.parametrize("mode", ["last_query", "chunk_sum", "accum", "external"])
+@pytest.mark.parametrize("shape", SHAPES)
+def test_fast_scores_match_oracle(shape, mode):
+    B, Hq, Hkv, d, cap, m, lens, dtype = shape
+    q, K, V, lens_t = make_case(4242 + SHAPES.index(shape), B, Hq, Hkv, d, cap, m, dtype, lens)
+    base = None
+    if mode in ("accum", "external"):
+        g = torch.Generator(device="cpu").manual_seed(5)
+        base = (torch.rand((B, Hkv, cap), generator=g) * 4.0).to(DEV)
+    base_in = None if base is None else base.clone()
+    p = P.make_params(B, Hq, Hkv, d, cap, m, dtype, d ** -0.5, mode)
+    ws = P.alloc_workspace(p, DEV)
+    vsum = torch.full((B, Hkv, d), float("nan"), dtype=torch.float32, device=DEV)
+    P.caote_vsum(p, V, lens_t, vsum)
+    for b, n in enumerate(lens):
+        ref = V[b, :, :n].double().sum(dim=1)
+        assert_close(vsum[b].double().cpu().numpy(), ref.cpu().numpy(), "vsum", rtol=1e-5, atol=1e-3)
+    o = torch.full(q.shape, float("nan"), dtype=torch.float32, device=DEV)
+    scores = torch.full((B, Hkv, cap), -7.0, dtype=torch.float32, device=DEV)
+    P.caote_score_fast(p, q, K, V, lens_t, base, vsum, o, scores, ws)
+    torch.cuda.synchronize()
+    assert P.caote_read_status(ws) == 0
+    r = oracle.score(f32(q), f32(K), f32(V), lens_t.cpu().numpy(), scale=d ** -0.5, n_new=m, base_mode=mode,
+                     base=None if base_in is None else base_in.double().cpu().numpy())
+    units = [(b, h) for b in range(B) for h in range(Hkv)]
+    exp = expected_fast(r, V, lens, units)
+    sg, og = f32(scores), f32(o)
+    for b, h in units:
+        n = lens[b]
+        if n == 0:
+            continue
+        assert_close(sg[b, h, :n], exp[(b, h)], f"{shape} {mode} fast scores ({b},{h})")
+        assert (sg[b, h, n:] == -7.0).all()
+    for b, n in enumerate(lens):
+        if n:
+            assert_close(og[b], r["o"][b], f"{shape} {mode} o[b={b}]")
+    if mode == "accum":
+        for b, n in enumerate(lens):
+            assert_close(f32(base)[b, :, :n], r["base"][b, :, :n], "accumulated base", rtol=1e-5, atol=1e-6)
+
+
+@pytest.mark.parametrize("name,kw,steps,compact", [
+    ("c4", dict(batch=3, budget=1500, init_len=1500, ragged_min_len=1100), 4, "fill"),
+    ("c4", dict(batch=2, budget=700, init_len=700, ragged_min_len=600), 3, "stable"),
+    ("c3", dict(budget=1024, init_len=1024, layers=1), 2, "fill"),
+])
+def test_fast_steps_keep_the_sum_current(name, kw, steps, compact):
+    """Several steps through caote_step_fast: before each step the state is copied out and the oracle scores
+    it; the running sum must equal the sum of the valid V rows after every step."""
+    w = wl.scaled(wl.WORKLOADS[name], **kw)
+    G, Hkv, m = w.group, w.n_kv_heads, w.n_new
+    lens0 = wl.initial_lengths(w, DEV)
+    budget = lens0.clone() if w.ragged_min_len is not None else torch.full_like(lens0, w.budget)
+    c = P.EvictionCache(w.batch, w.n_q_heads, Hkv, w.head_dim, w.capacity, m, w.torch_dtype, budget, w.base_mode, compact,
+                        w.scale, max_evict=m, device=DEV, method="fast")
+    K0, V0 = wl.initial_cache(w, DEV)
+    c.load(K0, V0, lens0)
+    units = [(b, h) for b in range(w.batch) for h in range(Hkv)][:6]
+    for t in range(steps):
+        q, kn, vn = wl.step_inputs(w, DEV, t)
+        K, V, lens = c.K.clone(), c.V.clone(), c.lens.clone()
+        base, pos, seen = c.base.clone(), c.pos.clone(), c.n_seen.clone()
+        for b in range(w.batch):
+            n = int(lens[b])
+            K[b, :, n:n + m], V[b, :, n:n + m] = kn[b], vn[b]
+            base[b, :, n:n + m] = 0.0
+            pos[b, :, n:n + m] = (seen[b] + torch.arange(m, device=DEV, dtype=torch.int32))[None, :]
+        lens = lens + m
+        c.step(q, kn, vn)
+        assert c.status() == 0
+        qs, Ks, Vs, ls, bs = sub_problem(q, K, V, lens, base if w.base_mode in ("accum", "external") else None, units, Hkv, G)
+        r = oracle.score(f32(qs), f32(Ks), f32(Vs), ls.cpu().numpy(), scale=w.scale, n_new=m, base_mode=w.base_mode,
+                         base=None if bs is None else bs.double().cpu().numpy())
+        sc, ev, posn = f32(c.scores), c.evict_idx.cpu().numpy(), pos.cpu().numpy()
+        for i, (b, h) in enumerate(units):
+            n = int(lens[b])
+            ref = oracle.fast_scores(r["w"][i, 0, :n], f32(Vs)[i, 0, :n])
+            assert_close(sc[b, h, :n], ref, f"{name} step {t} unit ({b},{h}) fast scores")
+            k = max(0, n - int(c.budget[b]))
+            check_evicted(ref, posn[b, h], n, k, ev[b, h, :k], f"{name} step {t} unit ({b},{h})")
+        for b in range(w.batch):
+            n = int(c.lens[b])
+            ref = c.V[b, :, :n].double().sum(dim=1).cpu().numpy()
+            assert_close(c.vsum[b].double().cpu().numpy(), ref, f"{name} step {t} vsum[b={b}]", rtol=1e-5, atol=2e-3)
