@@ -332,7 +332,7 @@ static int launch_prefill_score(const Dims& dm, const void* q, const void* K, co
   if (vsum) {
     CAOTE_LAUNCH("fast_mean_kernel", st, fast::mean_kernel<<<dm.units, prefill::kD, 0, st>>>(dm.Hkv, dm.cap, prefill::kD, len, vsum, sc.X));
   } else {
-    CAOTE_LAUNCH("prefill_xsum_kernel", st, prefill::xsum_kernel<<<dm.units, prefill::kD, 0, st>>>(dm, len, o, sc));
+    CAOTE_LAUNCH("prefill_xsum_kernel", st, prefill::xsum_kernel<<<dm.units, prefill::kXsumLanes * prefill::kD, 0, st>>>(dm, len, o, sc));
   }
   {
     dim3 grid((dm.cap + prefill::kScoreKeys - 1) / prefill::kScoreKeys, dm.units);
@@ -405,7 +405,7 @@ int caote_append(const caote_params_t* p, void* K, void* V, float* base, int32_t
   const Dims dm = make_dims(p);
   const int row_bytes = dm.D * (p->dtype == CAOTE_BF16 ? 2 : 4);
   cudaStream_t st = (cudaStream_t)stream;
-  CAOTE_LAUNCH("append_kernel", st, sel::append_kernel<<<dm.units, 256, 0, st>>>(dm.Hkv, dm.cap, dm.m, row_bytes, (char*)K, (char*)V, base, pos,
+  CAOTE_LAUNCH("append_kernel", st, sel::append_kernel<<<dim3(dm.units, (dm.m + 7) / 8), 256, 0, st>>>(dm.Hkv, dm.cap, dm.m, row_bytes, (char*)K, (char*)V, base, pos,
                                                len, n_seen, (const char*)k_new, (const char*)v_new,
                                                (int*)workspace, dm.B, (int*)workspace + 4));
   return CAOTE_OK;

@@ -496,20 +496,29 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
 }
 
 // X[unit] = mean of the unit's M rows of o. grid = units, 128 threads (one per channel).
-__global__ void __launch_bounds__(kD)
+constexpr int kXsumLanes = 8;  // row lanes per channel: 8 x 128 threads per unit
+__global__ void __launch_bounds__(kXsumLanes * kD)
 xsum_kernel(Dims dm, const int* __restrict__ len, const float* __restrict__ o, Scratch sc) {
-  const int unit = blockIdx.x, c = threadIdx.x;
+  __shared__ float part[kXsumLanes][kD];
+  const int unit = blockIdx.x, c = threadIdx.x % kD, lane = threadIdx.x / kD;
   const int n = len[unit / dm.Hkv];
   if (n == 0 || n < dm.m || n > dm.cap) return;
   const float* base = o + (size_t)unit * dm.R * kD + c;
   float acc[4] = {0.f, 0.f, 0.f, 0.f};
-  int r = 0;
-  for (; r + 4 <= dm.R; r += 4) {
+  int r = lane;
+  for (; r + 3 * kXsumLanes < dm.R; r += 4 * kXsumLanes) {
 #pragma unroll
-    for (int i = 0; i < 4; ++i) acc[i] += base[(size_t)(r + i) * kD];
+    for (int i = 0; i < 4; ++i) acc[i] += base[(size_t)(r + i * kXsumLanes) * kD];
   }
-  for (; r < dm.R; ++r) acc[0] += base[(size_t)r * kD];
-  sc.X[(size_t)unit * kD + c] = ((acc[0] + acc[1]) + (acc[2] + acc[3])) / (float)dm.R;
+  for (; r < dm.R; r += kXsumLanes) acc[0] += base[(size_t)r * kD];
+  part[lane][c] = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+  __syncthreads();
+  if (lane == 0) {
+    float s = 0.f;
+#pragma unroll
+    for (int l = 0; l < kXsumLanes; ++l) s += part[l][c];  // fixed order: reproducible
+    sc.X[(size_t)unit * kD + c] = s / (float)dm.R;
+  }
 }
 
 constexpr int kScoreKeys = 2 * kTile;            // keys per CTA: two key tiles share every Q block

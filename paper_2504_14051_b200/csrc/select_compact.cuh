@@ -282,7 +282,7 @@ __global__ void update_len_kernel(int B, int* __restrict__ len, const int* __res
   if (b < B) len[b] -= n_evict[b];
 }
 
-// Append m new rows per unit: one CTA per unit, one warp per row.
+// Append m new rows per unit: grid = (units, ceil(m / 8)), 8 warps per CTA, one warp per row.
 __global__ void __launch_bounds__(256)
 append_kernel(int Hkv, int cap, int m, int row_bytes, char* __restrict__ K, char* __restrict__ V,
               float* __restrict__ base, int* __restrict__ pos, int* __restrict__ len,
@@ -291,10 +291,10 @@ append_kernel(int Hkv, int cap, int m, int row_bytes, char* __restrict__ K, char
   const int unit = blockIdx.x, b = unit / Hkv;
   const int n = len[b];
   const bool fits = n >= 0 && n + m <= cap;
-  if (!fits && threadIdx.x == 0) set_status(status, CAOTE_ERR_OVERFLOW);
+  if (!fits && threadIdx.x == 0 && blockIdx.y == 0) set_status(status, CAOTE_ERR_OVERFLOW);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
   const int seen = n_seen ? n_seen[b] : n;
-  for (int i = warp; fits && i < m; i += nwarps) {
+  for (int i = blockIdx.y * nwarps + warp; fits && i < m; i += gridDim.y * nwarps) {
     const size_t dst = (size_t)unit * cap + n + i, src = (size_t)unit * m + i;
     warp_copy_row(K + dst * row_bytes, k_new + src * row_bytes, row_bytes, lane);
     warp_copy_row(V + dst * row_bytes, v_new + src * row_bytes, row_bytes, lane);
@@ -309,7 +309,7 @@ append_kernel(int Hkv, int cap, int m, int row_bytes, char* __restrict__ K, char
   __syncthreads();
   if (threadIdx.x == 0) {
     __threadfence();
-    s_last = (atomicAdd(ticket, 1) == (int)gridDim.x - 1);
+    s_last = (atomicAdd(ticket, 1) == (int)(gridDim.x * gridDim.y) - 1);
   }
   __syncthreads();
   if (s_last) {
