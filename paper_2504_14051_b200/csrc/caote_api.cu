@@ -324,10 +324,14 @@ static int launch_prefill_score(const Dims& dm, const void* q, const void* K, co
   if (!rc) rc = allow_smem(prefill::score_kernel, prefill::score_smem_bytes());
   if (rc) return rc;
   {
-    dim3 grid((dm.R + prefill::kTile - 1) / prefill::kTile, dm.units);
+    dim3 grid((dm.R + prefill::kTile - 1) / prefill::kTile, dm.units, sc.nsplit);
     CAOTE_LAUNCH("prefill_attn_kernel", st,
                  prefill::attn_kernel<<<grid, prefill::kAttnThreads, prefill::attn_smem_bytes(), st>>>(tmQ, tmK64, tmV64, dm, len,
                                                                                                     sc, o, status));
+  }
+  if (sc.nsplit > 1) {
+    dim3 grid((dm.R + 3) / 4, dm.units);
+    CAOTE_LAUNCH("prefill_attn_combine_kernel", st, prefill::attn_combine_kernel<<<grid, 4 * prefill::kD, 0, st>>>(dm, len, sc, o));
   }
   if (vsum) {
     CAOTE_LAUNCH("fast_mean_kernel", st, fast::mean_kernel<<<dm.units, prefill::kD, 0, st>>>(dm.Hkv, dm.cap, prefill::kD, len, vsum, sc.X));

@@ -43,7 +43,34 @@ struct Scratch {
   float* stats;  // [units][Mpad]: log2-domain softmax reference + log2(sum of 2^(s - ref)): alpha = 2^(s - stats)
   float* X;      // [units][kD]
   int Mpad;      // M rounded up to a multiple of kTile
+  int nsplit;    // key splits of the attention pass (1: none)
+  float* po;     // [units][nsplit][Mpad][kD] per-split outputs, normalised by their own sums (nsplit > 1)
+  float* pstat;  // [units][nsplit][Mpad] per-split statistics
 };
+
+// Few units and few query rows leave most SMs idle: the keys of a unit are then cut into up to 8 splits
+// that run as CTAs of their own; attn_combine_kernel merges them. A function of the shape only.
+inline int attn_splits(const Dims& dm) {
+  const long long ctas = (long long)((dm.R + kTile - 1) / kTile) * dm.units;
+  long long ns = 148 / (ctas > 0 ? ctas : 1);
+  const long long max_by_len = ((dm.cap + kTile - 1) / kTile) / 4;  // at least four tiles per split
+  if (ns > max_by_len) ns = max_by_len;
+  if (ns > 8) ns = 8;
+  return ns < 1 ? 1 : (int)ns;
+}
+// Split plan for a unit of n keys, the last m of them new (device and host agree on it): `ts` tiles per
+// split, `count` splits in use. The new block must lie inside the last split, so that every row sees at
+// least one key in every split it takes part in.
+__host__ __device__ inline void split_plan(int n, int m, int nsplit, int& ts, int& count) {
+  const int ntiles = (n + kTile - 1) / kTile;
+  for (int k = nsplit; k >= 1; --k) {
+    ts = (ntiles + k - 1) / k;
+    count = (ntiles + ts - 1) / ts;
+    if ((count - 1) * ts * kTile <= n - m) return;
+  }
+  ts = ntiles;
+  count = 1;
+}
 
 inline size_t carve(const Dims& dm, char* base, Scratch* out) {
   Scratch s;
@@ -53,6 +80,14 @@ inline size_t carve(const Dims& dm, char* base, Scratch* out) {
   off = align_up(off + sizeof(float) * (size_t)dm.units * s.Mpad, 256);
   s.X = reinterpret_cast<float*>(base + off);
   off = align_up(off + sizeof(float) * (size_t)dm.units * kD, 256);
+  s.nsplit = attn_splits(dm);
+  s.po = s.pstat = nullptr;
+  if (s.nsplit > 1) {
+    s.po = reinterpret_cast<float*>(base + off);
+    off = align_up(off + sizeof(float) * (size_t)dm.units * s.nsplit * s.Mpad * kD, 256);
+    s.pstat = reinterpret_cast<float*>(base + off);
+    off = align_up(off + sizeof(float) * (size_t)dm.units * s.nsplit * s.Mpad, 256);
+  }
   if (out) *out = s;
   return off;
 }
@@ -280,7 +315,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     if (tid == 0) set_status(status, CAOTE_ERR_BAD_LENGTH);
     return;
   }
-  const int ntiles = (n + kKeys - 1) / kKeys;
+  // this CTA's share of the unit's key tiles: [kt0, kt0 + ntiles)
+  int ts, nsp;
+  split_plan(n, m, sc.nsplit, ts, nsp);
+  const int split = blockIdx.z;
+  if (split >= nsp) return;
+  const int kt0 = split * ts;
+  const int ntiles = min(ts, (n + kKeys - 1) / kKeys - kt0);
 
   if (tid == 0) {
     for (int i = 0; i < kBars; ++i) mbar_init(&bars[i], 1);
@@ -302,7 +343,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
       tma_load_2d(Qs, &tmQ, 0, unit * M + row0, q_bar);
       tma_load_2d(Qs + kHalfBytes, &tmQ, 64, unit * M + row0, q_bar);
       for (int kt = 0; kt < ntiles; ++kt) {
-        const int st = kt % kKStages, row = unit * dm.cap + kt * kKeys;
+        const int st = kt % kKStages, row = unit * dm.cap + (kt0 + kt) * kKeys;
         if (kt >= kKStages) mbar_wait_idle(&k_free[st], ((kt / kKStages) - 1) & 1, status);  // S of tile kt - 3 is formed
         mbar_expect_tx(&k_bar[st], kKvTile);
         tma_load_2d(Ksm + st * kKvTile, &tmK64, 0, row, &k_bar[st]);
@@ -313,7 +354,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     // =============================== V loads (one lane) ===============================
     if (tid == kRowThreads + 64) {
       for (int kt = 0; kt < ntiles; ++kt) {
-        const int st = kt % kVStages, row = unit * dm.cap + kt * kKeys;
+        const int st = kt % kVStages, row = unit * dm.cap + (kt0 + kt) * kKeys;
         if (kt >= kVStages) mbar_wait_idle(&v_free[st], ((kt / kVStages) - 1) & 1, status);  // O += P V of tile kt - 2 is done
         mbar_expect_tx(&v_bar[st], kKvTile);
         tma_load_2d(Vsm + st * kKvTile, &tmV64, 0, row, &v_bar[st]);
@@ -387,12 +428,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     for (int kt = 0; kt < ntiles; ++kt) {
       mbar_wait(&s_bar[kt & 1], (kt >> 1) & 1, status);
       tc_fence_after();
-      const int j0 = kt * kKeys + half * 64;  // first key of this thread's half
+      const int j0 = (kt0 + kt) * kKeys + half * 64;  // first key of this thread's half
       const uint32_t t_s = t_lane + (kt & 1) * kKeys + half * 64;
       float sv[64];  // raw products; masked keys become -inf
       tmem_ld32(t_s, *reinterpret_cast<float(*)[32]>(&sv[0]));
       tmem_ld32(t_s + 32, *reinterpret_cast<float(*)[32]>(&sv[32]));
-      if (kt * kKeys + kKeys > n - m + 1) {  // only tiles that reach into the new block (or past the length) need the mask
+      if ((kt0 + kt) * kKeys + kKeys > n - m + 1) {  // only tiles that reach into the new block (or past the length) need the mask
 #pragma unroll
         for (int i = 0; i < 64; ++i) sv[i] = (j0 + i < nvis) ? sv[i] : -INFINITY;
       }
@@ -453,7 +494,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         tmem_st_wait();
         l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
       }
-      const int n_valid = min(kKeys, n - kt * kKeys);
+      const int n_valid = min(kKeys, n - (kt0 + kt) * kKeys);
       if (n_valid < kKeys) {
         // V rows behind the unit's length: clear them so that 0 * (stray NaN) cannot reach O
         mbar_wait(&v_bar[kt % kVStages], (kt / kVStages) & 1, status);
@@ -477,7 +518,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     asm volatile("bar.sync 1, %0;" ::"n"(kRowThreads) : "memory");
     l += xl[tid ^ kThreads];
     const float inv_l = 1.f / l;
-    float* orow = o + ((size_t)unit * M + R) * kD + half * 64;
+    // (with key splits: this split's output, normalised by its own sum, and its statistic go to scratch)
+    float* orow = (nsp > 1 ? sc.po + (((size_t)unit * sc.nsplit + split) * sc.Mpad + R) * kD
+                           : o + ((size_t)unit * M + R) * kD) + half * 64;
 #pragma unroll
     for (int cc = 0; cc < 2; ++cc) {
       float v[32];
@@ -488,7 +531,10 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
           *reinterpret_cast<float4*>(orow + cc * 32 + i) = make_float4(v[i] * inv_l, v[i + 1] * inv_l, v[i + 2] * inv_l, v[i + 3] * inv_l);
       }
     }
-    if (R < M && half == 0) sc.stats[(size_t)unit * sc.Mpad + R] = m_ref + __log2f(l);
+    if (R < M && half == 0) {
+      if (nsp > 1) sc.pstat[((size_t)unit * sc.nsplit + split) * sc.Mpad + R] = m_ref + __log2f(l);
+      else sc.stats[(size_t)unit * sc.Mpad + R] = m_ref + __log2f(l);
+    }
   }
   tc_fence_before();
   __syncthreads();
@@ -496,6 +542,31 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
 }
 
 // X[unit] = mean of the unit's M rows of o. grid = units, 128 threads (one per channel).
+// Merge the key splits of a unit: o = sum_s o_s 2^(stat_s - stat), stat = log2 sum_s 2^stat_s.
+// grid = (ceil(M / 4), units), 4 rows x 128 channels per CTA. Units that ran unsplit are left alone.
+__global__ void __launch_bounds__(4 * kD)
+attn_combine_kernel(Dims dm, const int* __restrict__ len, Scratch sc, float* __restrict__ o) {
+  const int unit = blockIdx.y, c = threadIdx.x % kD, R = blockIdx.x * 4 + threadIdx.x / kD;
+  const int n = len[unit / dm.Hkv];
+  if (n == 0 || n < dm.m || n > dm.cap || R >= dm.R) return;
+  int ts, nsp;
+  split_plan(n, dm.m, sc.nsplit, ts, nsp);
+  if (nsp <= 1) return;
+  float st[8], mx = -INFINITY;
+  for (int s = 0; s < nsp; ++s) {
+    st[s] = sc.pstat[((size_t)unit * sc.nsplit + s) * sc.Mpad + R];
+    mx = fmaxf(mx, st[s]);
+  }
+  float tot = 0.f, acc = 0.f;
+  for (int s = 0; s < nsp; ++s) {
+    const float w = exp2f(st[s] - mx);
+    tot += w;
+    acc = fmaf(sc.po[(((size_t)unit * sc.nsplit + s) * sc.Mpad + R) * kD + c], w, acc);
+  }
+  o[((size_t)unit * dm.R + R) * kD + c] = acc / tot;
+  if (c == 0) sc.stats[(size_t)unit * sc.Mpad + R] = mx + log2f(tot);
+}
+
 constexpr int kXsumLanes = 8;  // row lanes per channel: 8 x 128 threads per unit
 __global__ void __launch_bounds__(kXsumLanes * kD)
 xsum_kernel(Dims dm, const int* __restrict__ len, const float* __restrict__ o, Scratch sc) {
