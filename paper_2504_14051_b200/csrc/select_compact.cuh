@@ -81,38 +81,85 @@ __device__ __forceinline__ int select_unit(int unit, int Hkv, int cap, const flo
     return 1;
   }
 
-  if (tid == 0) { s_prefix = 0ull; s_remaining = k; }
+  // Radix select on the 64-bit keys, 8 bits per pass, most significant first. Up to kCached keys per
+  // thread stay in registers across the passes; a pass ends the search early when the whole bucket it
+  // lands in is needed (always the case once the remaining bits only tell equal scores apart and
+  // positions are unique).
+  constexpr int kCached = 8;
+  const bool cached = n <= kSelThreads * kCached;
+  unsigned long long kreg[kCached];
+#pragma unroll
+  for (int i = 0; i < kCached; ++i) {
+    const int j = tid + i * kSelThreads;
+    kreg[i] = (cached && j < n) ? make_key(sc[j], ps ? ps[j] : j) : ~0ull;
+  }
+  __shared__ int s_done;
+  if (tid == 0) { s_prefix = 0ull; s_remaining = k; s_done = 0; }
+  unsigned long long kth = ~0ull;
   for (int pass = 0; pass < 8; ++pass) {
     const int shift = 56 - 8 * pass;
     if (tid < 256) hist[tid] = 0u;
     __syncthreads();
     const unsigned long long prefix = s_prefix;
     const unsigned long long mask = (pass == 0) ? 0ull : (~0ull << (shift + 8));
-    for (int j = tid; j < n; j += kSelThreads) {
-      const unsigned long long key = make_key(sc[j], ps ? ps[j] : j);
-      if ((key & mask) == prefix) atomicAdd(&hist[(unsigned int)(key >> shift) & 255u], 1u);
-    }
-    __syncthreads();
-    if (tid == 0) {
-      int rem = s_remaining;
-      int dgt = 0;
-      for (; dgt < 256; ++dgt) {
-        const int c = (int)hist[dgt];
-        if (rem <= c) break;
-        rem -= c;
+    if (cached) {
+#pragma unroll
+      for (int i = 0; i < kCached; ++i) {
+        const int j = tid + i * kSelThreads;
+        if (j < n && (kreg[i] & mask) == prefix) atomicAdd(&hist[(unsigned int)(kreg[i] >> shift) & 255u], 1u);
       }
-      if (dgt > 255) dgt = 255;
-      s_remaining = rem;
-      s_prefix = prefix | ((unsigned long long)dgt << shift);
+    } else {
+      for (int j = tid; j < n; j += kSelThreads) {
+        const unsigned long long key = make_key(sc[j], ps ? ps[j] : j);
+        if ((key & mask) == prefix) atomicAdd(&hist[(unsigned int)(key >> shift) & 255u], 1u);
+      }
     }
     __syncthreads();
+    if (warp == 0) {
+      // the first digit whose cumulative count reaches the number still wanted: 8 bins per lane
+      unsigned int c[8], sum = 0u;
+#pragma unroll
+      for (int q = 0; q < 8; ++q) { c[q] = hist[8 * lane + q]; sum += c[q]; }
+      unsigned int incl = sum;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const unsigned int t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+      }
+      const unsigned int rem = (unsigned int)s_remaining;
+      const unsigned int reach = __ballot_sync(0xffffffffu, rem <= incl);
+      const int f = reach ? __ffs((int)reach) - 1 : 31;
+      if (lane == f) {
+        unsigned int r = rem - (incl - sum);
+        int q = 0;
+        for (; q < 7; ++q) {
+          if (r <= c[q]) break;
+          r -= c[q];
+        }
+        s_remaining = (int)r;
+        s_prefix = prefix | ((unsigned long long)(8 * lane + q) << shift);
+        s_done = (r == c[q]) ? 1 : 0;
+      }
+    }
+    __syncthreads();
+    if (s_done || pass == 7) {
+      kth = s_prefix | (shift ? ((1ull << shift) - 1ull) : 0ull);  // the largest key that is taken
+      break;
+    }
   }
-  const unsigned long long kth = s_prefix;  // the k-th smallest key
   if (tid == 0) s_running = 0;
   __syncthreads();
-  for (int j0 = 0; j0 < n; j0 += kSelThreads) {
+  for (int j0 = 0, i = 0; j0 < n; j0 += kSelThreads, ++i) {
     const int j = j0 + tid;
-    const int flag = (j < n) && (make_key(sc[j], ps ? ps[j] : j) <= kth);
+    unsigned long long key = ~0ull;
+    if (cached) {
+#pragma unroll
+      for (int q = 0; q < kCached; ++q)
+        if (q == i) key = kreg[q];
+    } else if (j < n) {
+      key = make_key(sc[j], ps ? ps[j] : j);
+    }
+    const int flag = (j < n) && (key <= kth);
     const unsigned int ballot = __ballot_sync(0xffffffffu, flag);
     const int in_warp = __popc(ballot & ((1u << lane) - 1u));
     if (lane == 0) s_warp_tot[warp] = __popc(ballot);
