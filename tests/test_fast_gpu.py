@@ -119,3 +119,38 @@ def test_fast_steps_keep_the_sum_current(name, kw, steps, compact):
             n = int(c.lens[b])
             ref = c.V[b, :, :n].double().sum(dim=1).cpu().numpy()
             assert_close(c.vsum[b].double().cpu().numpy(), ref, f"{name} step {t} vsum[b={b}]", rtol=1e-5, atol=2e-3)
+
+
+def test_fast_scores_rank_like_caote_scores():
+    """Sec. 3.3 reports a Spearman correlation >= 0.8 between FastCAOTE and CAOTE scores on real models.
+    Here: the same check on synthetic decode caches (keys partly aligned with the queries, so that the
+    weights are far from uniform), on the GPU's scores, with the oracle's correlation beside it."""
+    from scipy.stats import spearmanr
+
+    B, Hq, Hkv, d, cap = 4, 16, 4, 128, 1536
+    lens = [1536, 1400, 1290, 1025]
+    q, K, V, lens_t = make_case(99, B, Hq, Hkv, d, cap, 1, torch.bfloat16, lens)
+    G = Hq // Hkv
+    for b in range(B):            # every 16th key leans towards one of the unit's queries
+        for h in range(Hkv):
+            K[b, h, ::16] = (K[b, h, ::16].float() + 0.6 * q[b, h * G, 0].float()).to(K.dtype)
+    p = P.make_params(B, Hq, Hkv, d, cap, 1, torch.bfloat16, d ** -0.5, "last_query")
+    ws = P.alloc_workspace(p, DEV)
+    o = torch.zeros(q.shape, dtype=torch.float32, device=DEV)
+    caote = torch.zeros((B, Hkv, cap), dtype=torch.float32, device=DEV)
+    fast = torch.zeros_like(caote)
+    vsum = torch.zeros((B, Hkv, d), dtype=torch.float32, device=DEV)
+    P.caote_score(p, q, K, V, lens_t, None, o, caote, ws)
+    P.caote_vsum(p, V, lens_t, vsum)
+    P.caote_score_fast(p, q, K, V, lens_t, None, vsum, o, fast, ws)
+    torch.cuda.synchronize()
+    assert P.caote_read_status(ws) == 0
+    r = oracle.score(f32(q), f32(K), f32(V), lens_t.cpu().numpy(), scale=d ** -0.5, n_new=1, base_mode="last_query")
+    cg, fg, Vf = f32(caote), f32(fast), f32(V)
+    for b in range(B):
+        n = lens[b]
+        for h in range(Hkv):
+            rho_gpu = spearmanr(cg[b, h, :n], fg[b, h, :n]).statistic
+            rho_ref = spearmanr(r["scores"][b, h, :n], oracle.fast_scores(r["w"][b, h, :n], Vf[b, h, :n])).statistic
+            assert rho_gpu >= 0.8, f"unit ({b},{h}): Spearman {rho_gpu}"
+            assert abs(rho_gpu - rho_ref) < 5e-3, f"unit ({b},{h}): GPU {rho_gpu} vs oracle {rho_ref}"
