@@ -38,6 +38,8 @@ NCU_TRAFFIC = {
     # per launch at the workload's own size: (read + write) of profiles/decode_tc_kernel_c4_full_traffic.txt
     "decode_tc_kernel": {"per_launch": {"c4": 1421127168 + 63072512, "c5d": 780569856 + 34433792},
                          "profile": "profiles/decode_tc_kernel_c4_full_traffic.txt"},
+    "decode_tc_fast_kernel": {"per_launch": {"c4": 956221696 + 57498880},
+                              "profile": "profiles/decode_tc_kernel_c4_full_traffic.txt"},
     "prefill_attn_kernel": {"bytes_per_unit": (155385088 + 17509632) / 16, "profile": "profiles/prefill_kernels_c5p_batch2_ncu.txt"},
 }
 
@@ -239,7 +241,7 @@ def run_ours(args, w0, rank, world, device):
     if w.n_new == 1:
         # measured only at the named workloads' full sizes: smaller cases get part of their second pass from L2
         full_size = w.batch == wl.WORKLOADS[w0.name].batch
-        decode_traffic = NCU_TRAFFIC.get(top, {}).get("per_launch", {}).get(w0.name) if full_size else None  # (no entry for the fast kernel)
+        decode_traffic = NCU_TRAFFIC.get(top, {}).get("per_launch", {}).get(w0.name) if full_size else None
         bytes_per_launch = algo["per_step"] / launches_per_step_top
         achieved = bytes_per_launch / (per_launch_ms * 1e-3) / 1e9
         roofline = {"bound": "hbm", "kernel": top, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
