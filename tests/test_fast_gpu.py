@@ -154,3 +154,41 @@ def test_fast_scores_rank_like_caote_scores():
             rho_ref = spearmanr(r["scores"][b, h, :n], oracle.fast_scores(r["w"][b, h, :n], Vf[b, h, :n])).statistic
             assert rho_gpu >= 0.8, f"unit ({b},{h}): Spearman {rho_gpu}"
             assert abs(rho_gpu - rho_ref) < 5e-3, f"unit ({b},{h}): GPU {rho_gpu} vs oracle {rho_ref}"
+
+
+@pytest.mark.parametrize("name,units", [("c4", [(0, 0), (17, 3), (63, 1)]), ("c5d", [(7, 7)])])
+def test_fast_full_size_step_on_sampled_units(name, units):
+    """One FastCAOTE step at the size and launch configuration the benchmark times; the oracle follows a sample."""
+    w = wl.WORKLOADS[name]
+    G, Hkv, m = w.group, w.n_kv_heads, w.n_new
+    lens0 = wl.initial_lengths(w, DEV)
+    budget = lens0.clone() if w.ragged_min_len is not None else torch.full_like(lens0, w.budget)
+    c = P.EvictionCache(w.batch, w.n_q_heads, Hkv, w.head_dim, w.capacity, m, w.torch_dtype, budget, w.base_mode, "fill",
+                        w.scale, max_evict=m, device=DEV, method="fast")
+    K0, V0 = wl.initial_cache(w, DEV)
+    c.load(K0, V0, lens0)
+    del K0, V0
+    q, kn, vn = wl.step_inputs(w, DEV, 0)
+    lens = c.lens.clone() + m
+    sub = {}
+    for b, h in units:  # the unit's state with the new token appended the way the step will
+        n = int(lens[b])
+        Ku, Vu = c.K[b, h, :n].clone(), c.V[b, h, :n].clone()
+        Ku[n - m:], Vu[n - m:] = kn[b, h], vn[b, h]
+        sub[(b, h)] = (Ku, Vu, c.base[b, h, :n].clone(), c.pos[b, h, :n].clone(), int(c.n_seen[b]))
+    c.step(q, kn, vn)
+    assert c.status() == 0
+    sc, ev = f32(c.scores), c.evict_idx.cpu().numpy()
+    for b, h in units:
+        Ku, Vu, bu, pu, seen = sub[(b, h)]
+        n = Ku.shape[0]
+        bu[n - m:] = 0.0
+        pu[n - m:] = seen + torch.arange(m, device=DEV, dtype=torch.int32)
+        r = oracle.score(f32(q[b:b + 1, h * G:(h + 1) * G]), f32(Ku)[None, None], f32(Vu)[None, None], np.array([n], dtype=np.int32),
+                         scale=w.scale, n_new=m, base_mode=w.base_mode,
+                         base=bu.double().cpu().numpy()[None, None] if w.base_mode in ("accum", "external") else None)
+        ref = oracle.fast_scores(r["w"][0, 0, :n], f32(Vu))
+        assert_close(sc[b, h, :n], ref, f"{name} unit ({b},{h}) fast scores")
+        assert_close(f32(c.o)[b, h * G:(h + 1) * G], r["o"][0], f"{name} unit ({b},{h}) o")
+        k = max(0, n - int(c.budget[b]))
+        check_evicted(ref, pu.cpu().numpy(), n, k, ev[b, h, :k], f"{name} unit ({b},{h})")
