@@ -123,6 +123,13 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const float (&v)[16]) 
   asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
 
+// Two floats -> packed bf16x2 (x0 in the low half), round to nearest even.
+__device__ __forceinline__ uint32_t pack_bf16x2(float x0, float x1) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(x1), "f"(x0));
+  return r;
+}
+
 // Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 16; A K-major or MN-major, B K-major.
 __host__ __device__ constexpr uint32_t idesc_n16(bool a_mn_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn_major ? 1u : 0u) << 15) | ((16u >> 3) << 17) | ((128u >> 4) << 24);
@@ -544,17 +551,24 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         // P^T rows g (hi part) and 8 + g (lo part), column = token; row 7 carries the base score
         char* pb = pbuf + sb * kPBytes + (tok >> 6) * 2048 + (tok & 7) * 2;
         const int chunk = (tok & 63) >> 3;
+        float pv[8];
 #pragma unroll
         for (int g = 0; g < 8; ++g) {
           const bool base_row = use_base && g == 7;
-          if (g < G || base_row) {
-            float p = base_row ? bval : fast_exp2(sv[g] - ref[g]);
-            if (!base_row) lpart[g] += p;
-            const __nv_bfloat16 hi = __float2bfloat16_rn(p);
-            const __nv_bfloat16 lo = __float2bfloat16_rn(p - __bfloat162float(hi));
-            char* at = pb + g * 128 + ((chunk ^ g) << 4);
-            *reinterpret_cast<__nv_bfloat16*>(at) = hi;
-            *reinterpret_cast<__nv_bfloat16*>(at + 1024) = lo;
+          pv[g] = base_row ? bval : (g < G ? fast_exp2(sv[g] - ref[g]) : 0.f);
+          if (g < G) lpart[g] += pv[g];
+        }
+#pragma unroll
+        for (int g = 0; g < 8; g += 2) {  // two heads per conversion; a row no head owns gets the zeros it holds anyway
+          if (g < G || (use_base && g == 6)) {
+            const uint32_t hi2 = pack_bf16x2(pv[g], pv[g + 1]);
+            const uint32_t lo2 = pack_bf16x2(pv[g] - __uint_as_float(hi2 << 16), pv[g + 1] - __uint_as_float(hi2 & 0xffff0000u));
+            char* at0 = pb + g * 128 + ((chunk ^ g) << 4);
+            char* at1 = pb + (g + 1) * 128 + ((chunk ^ (g + 1)) << 4);
+            *reinterpret_cast<unsigned short*>(at0) = (unsigned short)(hi2 & 0xffffu);
+            *reinterpret_cast<unsigned short*>(at1) = (unsigned short)(hi2 >> 16);
+            *reinterpret_cast<unsigned short*>(at0 + 1024) = (unsigned short)(lo2 & 0xffffu);
+            *reinterpret_cast<unsigned short*>(at1 + 1024) = (unsigned short)(lo2 >> 16);
           }
         }
         if (d.n_valid < kT) {
