@@ -84,6 +84,15 @@ def test_host_side_argument_checks_return_before_any_launch():
     assert lib.caote_compact(bp, fake, fake, None, None, fake, fake, 4, fake, 7, ws, need, None) == C.ERR_INVALID_ARG
     assert lib.caote_append(bp, fake, fake, None, None, None, None, fake, fake, ws, need, None) == C.ERR_INVALID_ARG
     assert lib.caote_read_status(None, None, None) == C.ERR_INVALID_ARG
+    # FastCAOTE entry points: the running sum of value rows is mandatory and 16-byte aligned
+    assert lib.caote_vsum(bp, fake, fake, None, None) == C.ERR_INVALID_ARG
+    assert lib.caote_vsum(None, fake, fake, fake, None) == C.ERR_INVALID_ARG
+    assert lib.caote_score_fast(bp, fake, fake, fake, fake, fake, None, fake, fake, ws, need, None) == C.ERR_INVALID_ARG
+    assert lib.caote_score_fast(bp, fake, fake, fake, fake, fake, ctypes.c_void_p(4100), fake, fake, ws, need,
+                                None) == C.ERR_INVALID_ARG
+    assert lib.caote_score_fast(bp, fake, fake, fake, fake, fake, fake, fake, fake, ws, need - 1, None) == C.ERR_INVALID_ARG
+    assert lib.caote_step_fast(bp, fake, fake, fake, fake, fake, fake, fake, fake, fake, fake, None, fake, fake, fake, 1,
+                               fake, 0, ws, need, None) == C.ERR_INVALID_ARG
     assert C.caote_launch_count() == before
 
 
