@@ -200,9 +200,10 @@ static int decode_grid_limit() {
   int g = cached[dev].load(std::memory_order_acquire);
   if (g == 0) {
     int sms = 0, per_sm = 0;
-    const size_t smem = decode::tc_smem_bytes();
+    const size_t smem = decode::tc_smem_bytes(false);
+    const size_t smem_fast = decode::tc_smem_bytes(true);
     if (cudaFuncSetAttribute(decode::decode_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
-        cudaFuncSetAttribute(decode::decode_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+        cudaFuncSetAttribute(decode::decode_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_fast) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode::decode_tc_kernel<false>, decode::kTcThreads, smem) != cudaSuccess)
       return 0;
@@ -268,12 +269,12 @@ static int launch_decode_score(const Dims& dm, const void* q, const void* K, con
   const int grid = (int)(max_items < grid_limit ? max_items : grid_limit);
   if (!vsum) {
     CAOTE_LAUNCH("decode_tc_kernel", st,
-                 decode::decode_tc_kernel<false><<<grid, decode::kTcThreads, decode::tc_smem_bytes(), st>>>(
+                 decode::decode_tc_kernel<false><<<grid, decode::kTcThreads, decode::tc_smem_bytes(false), st>>>(
                      tmK, tmV, tmQ, dm, len, base, o, scores, nullptr, pl, status));
   } else {
     // FastCAOTE: one pass over K and V, then scores from the stored logits and distances
     CAOTE_LAUNCH("decode_tc_fast_kernel", st,
-                 decode::decode_tc_kernel<true><<<grid, decode::kTcThreads, decode::tc_smem_bytes(), st>>>(
+                 decode::decode_tc_kernel<true><<<grid, decode::kTcThreads, decode::tc_smem_bytes(true), st>>>(
                      tmK, tmV, tmQ, dm, len, base, o, scores, vsum, pl, status));
     dim3 fgrid(tiles_per_unit, dm.units);
     CAOTE_LAUNCH("fast_finish_kernel", st, decode::fast_finish_kernel<<<fgrid, decode::kT, 0, st>>>(dm, len, base, scores, pl));

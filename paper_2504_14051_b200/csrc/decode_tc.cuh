@@ -46,10 +46,15 @@ constexpr uint32_t kTmemCols = 64;                 // S^T x 2 (16 columns each),
 constexpr int kBaseRowBytes = kT * 4;              // the carried base scores of one tile
 constexpr int kBSideBytes = 8 * kT * 4;            // score slot: logits of up to 7 heads (rows 0..6), base scores (row 7)
 
-inline size_t tc_smem_bytes() {
-  return 1024 + (size_t)(kASlots + kBSlots) * kTileBytes + kQBufs * kQBytes + 2 * kPBytes + kASlots * kBaseRowBytes +
-         kBSlots * kBSideBytes + kFinBufs * kFinalBytes + sizeof(Desc) * (kASlots + kBSlots) +
-         sizeof(float) * (2 * 4 * 8 + 4 * 8 + 4 + 8) + 8 * (2 * (kASlots + kBSlots) + 8) + 64;
+constexpr int kASlotsFast = 6;                     // FastCAOTE: no score ring, a deeper attention ring instead
+constexpr int kQBufsFast = 4;
+constexpr int kXBufBytes = kQBufsFast * (kD + 4) * 4;  // FastCAOTE: per query buffer the sum of V rows and 1 / n
+
+inline size_t tc_smem_bytes(bool fast) {
+  const size_t a = fast ? kASlotsFast : kASlots;
+  return 1024 + a * kTileBytes + (fast ? 0 : (size_t)kBSlots * kTileBytes) + (fast ? kQBufsFast : kQBufs) * kQBytes + 2 * kPBytes + a * kBaseRowBytes +
+         (fast ? (size_t)kXBufBytes : (size_t)kBSlots * kBSideBytes + kFinBufs * kFinalBytes) + sizeof(Desc) * (kASlotsFast + kBSlots) +
+         sizeof(float) * (2 * 4 * 8 + 4 * 8 + 4 + 8) + 8 * (2 * (kASlotsFast + kBSlots) + 8) + 64;
 }
 
 __device__ __forceinline__ void wait_or_stop(uint64_t* bar, uint32_t parity, volatile int* stop, int* status) {
@@ -174,25 +179,29 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                  const __grid_constant__ CUtensorMap tmQ, Dims dm, const int* __restrict__ len,
                  float* __restrict__ base, float* __restrict__ o, float* __restrict__ scores, const float* __restrict__ vsum,
                  Plan pl, int* status) {
+  // FastCAOTE has no score ring: its shared memory goes to a deeper attention ring
+  constexpr int kA = kFast ? kASlotsFast : kASlots;
+  constexpr int kQ = kFast ? kQBufsFast : kQBufs;  // a buffer is reused only after every reader of its item has moved on:
+                                                   // that takes one more buffer with the deeper ring
   extern __shared__ char smem_raw[];
   char* sm = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  char* tilesA = sm;                                                     // [kASlots][kTileBytes]
-  char* tilesB = tilesA + kASlots * kTileBytes;                          // [kBSlots][kTileBytes]
-  char* qbuf = tilesB + kBSlots * kTileBytes;                            // [kQBufs][kQBytes]
-  char* pbuf = qbuf + kQBufs * kQBytes;                                  // [2][kPBytes]
-  char* baseA = pbuf + 2 * kPBytes;                                      // [kASlots][kBaseRowBytes]
-  char* sideB = baseA + kASlots * kBaseRowBytes;                         // [kBSlots][kBSideBytes]
-  float* xbuf = reinterpret_cast<float*>(sideB);                         // kFast: [kQBufs][kD + 4] sum of V rows, 1 / n
-  char* finbuf = sideB + kBSlots * kBSideBytes;                          // [kFinBufs] FinalRec
-  Desc* descA = reinterpret_cast<Desc*>(finbuf + kFinBufs * kFinalBytes);  // [kASlots]
-  Desc* descB = descA + kASlots;                                         // [kBSlots]
+  char* tilesA = sm;                                                     // [kA][kTileBytes]
+  char* tilesB = tilesA + kA * kTileBytes;                               // [kBSlots][kTileBytes] (none with kFast)
+  char* qbuf = tilesB + (kFast ? 0 : kBSlots * kTileBytes);                            // [kQ][kQBytes]
+  char* pbuf = qbuf + kQ * kQBytes;                                  // [2][kPBytes]
+  char* baseA = pbuf + 2 * kPBytes;                                      // [kA][kBaseRowBytes]
+  char* sideB = baseA + kA * kBaseRowBytes;                         // [kBSlots][kBSideBytes]
+  float* xbuf = reinterpret_cast<float*>(sideB);                         // kFast: [kQ][kD + 4] sum of V rows, 1 / n
+  char* finbuf = sideB + (kFast ? kXBufBytes : kBSlots * kBSideBytes);                          // [kFinBufs] FinalRec
+  Desc* descA = reinterpret_cast<Desc*>(finbuf + (kFast ? 0 : kFinBufs * kFinalBytes));  // [kA]
+  Desc* descB = descA + kA;                                         // [kBSlots]
   float* red = reinterpret_cast<float*>(descB + kBSlots);                // [2][4][8] warp maxima
   float* wl = red + 2 * 4 * 8;                                           // [4][8] warp sums
   float* whb = wl + 4 * 8;                                               // [4]
   float* wxx = whb + 4;                                                  // [8]
-  uint64_t* fullA = reinterpret_cast<uint64_t*>(wxx + 8);                // [kASlots]
-  uint64_t* emptyA = fullA + kASlots;                                    // [kASlots] 4 attention warps + the issuing lane
-  uint64_t* fullB = emptyA + kASlots;                                    // [kBSlots]
+  uint64_t* fullA = reinterpret_cast<uint64_t*>(wxx + 8);                // [kA]
+  uint64_t* emptyA = fullA + kA;                                    // [kA] 4 attention warps + the issuing lane
+  uint64_t* fullB = emptyA + kA;                                    // [kBSlots]
   uint64_t* emptyB = fullB + kBSlots;                                    // [kBSlots] 4 score warps
   uint64_t* s_bar = emptyB + kBSlots;                                    // [2] S^T formed
   uint64_t* p_bar = s_bar + 2;                                           // [2] P^T written
@@ -211,7 +220,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   const int tiles_per_unit = pl.capS / kT;
 
   if (tid == 0) {
-    for (int i = 0; i < kASlots; ++i) {
+    for (int i = 0; i < kA; ++i) {
       mbar_init(&fullA[i], 1);
       mbar_init(&emptyA[i], kFast ? 9 : 5);  // 4 attention warps + the issuing lane (+ 4 score warps)
     }
@@ -231,7 +240,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     ctl[3] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (tid < (kASlots + kBSlots) * (int)(sizeof(Desc) / sizeof(int))) reinterpret_cast<int*>(descA)[tid] = 0;
+  if (tid < (kA + kBSlots) * (int)(sizeof(Desc) / sizeof(int))) reinterpret_cast<int*>(descA)[tid] = 0;
   // rows of P^T that no head writes stay zero for the whole kernel
   for (int i = tid; i < 2 * kPBytes / 16; i += kTcThreads) reinterpret_cast<uint4*>(pbuf)[i] = make_uint4(0u, 0u, 0u, 0u);
   fence_async_smem();
@@ -267,31 +276,31 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
           d.nitems = e.nitems;
           const int row = e.unit * dm.cap + t * kT;
           const uint32_t base_bytes = use_base ? (uint32_t)min(kT, dm.cap - t * kT) * 4u : 0u;
-          int s = issued % kASlots;
-          if (!(ok = mbar_wait(&emptyA[s], ((issued / kASlots) & 1) ^ 1, &ctl[0]))) break;
+          int s = issued % kA;
+          if (!(ok = mbar_wait(&emptyA[s], ((issued / kA) & 1) ^ 1, &ctl[0]))) break;
           char* tl = tilesA + s * kTileBytes;
           d.type = kSlotKA;
           descA[s] = d;
           const bool first = (d.flags & kFlagFirst) != 0;
-          if (kFast && first) xbuf[(a_items % kQBufs) * (kD + 4) + kD] = 1.f / (float)e.n;
+          if (kFast && first) xbuf[(a_items % kQ) * (kD + 4) + kD] = 1.f / (float)e.n;
           mbar_expect_tx(&fullA[s], kTileBytes + base_bytes + (first ? (uint32_t)kQBytes + (kFast ? kD * 4u : 0u) : 0u));
           tma_load_2d(tl, &tmK, 0, row, &fullA[s], pol_stream);
           tma_load_2d(tl + kHalfBytes, &tmK, 64, row, &fullA[s], pol_stream);
           if (use_base)
-            bulk_load(baseA + (a_tiles % kASlots) * kBaseRowBytes, base + (size_t)e.unit * dm.cap + t * kT, base_bytes, &fullA[s]);
+            bulk_load(baseA + (a_tiles % kA) * kBaseRowBytes, base + (size_t)e.unit * dm.cap + t * kT, base_bytes, &fullA[s]);
           ++a_tiles;
           if (first) {
             // the unit's query rows (16 rows from its first head on; only the first G are used)
-            char* qb = qbuf + (a_items % kQBufs) * kQBytes;
+            char* qb = qbuf + (a_items % kQ) * kQBytes;
             const int qrow = (e.unit / dm.Hkv) * dm.Hq + (e.unit % dm.Hkv) * G;
             tma_load_2d(qb, &tmQ, 0, qrow, &fullA[s], pol_keep);
             tma_load_2d(qb + kQBytes / 2, &tmQ, 64, qrow, &fullA[s], pol_keep);
-            if (kFast) bulk_load(xbuf + (a_items % kQBufs) * (kD + 4), vsum + (size_t)e.unit * kD, kD * 4, &fullA[s]);
+            if (kFast) bulk_load(xbuf + (a_items % kQ) * (kD + 4), vsum + (size_t)e.unit * kD, kD * 4, &fullA[s]);
             ++a_items;
           }
           ctl[2] = ++issued;
-          s = issued % kASlots;
-          if (!(ok = mbar_wait(&emptyA[s], ((issued / kASlots) & 1) ^ 1, &ctl[0]))) break;
+          s = issued % kA;
+          if (!(ok = mbar_wait(&emptyA[s], ((issued / kA) & 1) ^ 1, &ctl[0]))) break;
           tl = tilesA + s * kTileBytes;
           d.type = kSlotVA;
           descA[s] = d;
@@ -305,8 +314,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     }
     if (lane == 0) {
       if (ok) {
-        const int s = issued % kASlots;
-        if (mbar_wait(&emptyA[s], ((issued / kASlots) & 1) ^ 1, &ctl[0])) {
+        const int s = issued % kA;
+        if (mbar_wait(&emptyA[s], ((issued / kA) & 1) ^ 1, &ctl[0])) {
           descA[s].type = kSlotStop;
           mbar_arrive(&fullA[s]);
           ctl[2] = ++issued;
@@ -399,7 +408,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
       auto issue_qk = [&](int s, const Desc& d) {
         if (d.flags & kFlagFirst) ++q_items;
         const uint32_t ka = smem_u32(tilesA + s * kTileBytes);
-        const uint32_t qa = smem_u32(qbuf + ((q_items - 1) % kQBufs) * kQBytes);
+        const uint32_t qa = smem_u32(qbuf + ((q_items - 1) % kQ) * kQBytes);
         prefill::tc_fence_after();
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks)
@@ -410,8 +419,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
       };
       for (int i = 0;; ++i) {
         if (i <= qk_queued) continue;  // a K slot whose product went out early; it may be refilled by now
-        const int s = i % kASlots;
-        wait_or_stop_idle(&fullA[s], (i / kASlots) & 1, &ctl[0], status);
+        const int s = i % kA;
+        wait_or_stop_idle(&fullA[s], (i / kA) & 1, &ctl[0], status);
         if (ctl[0]) break;
         const Desc d = descA[s];
         if (d.type == kSlotStop) break;
@@ -421,8 +430,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         } else {
           // queue the next tile's S^T first, if its K tile has landed: it then overlaps this tile's softmax
           {
-            const int j = i + 1, s2 = j % kASlots;
-            if (mbar_try_wait(&fullA[s2], (j / kASlots) & 1)) {
+            const int j = i + 1, s2 = j % kA;
+            if (mbar_try_wait(&fullA[s2], (j / kA) & 1)) {
               const Desc d2 = descA[s2];
               if (d2.type == kSlotKA) {
                 issue_qk(s2, d2);
@@ -460,8 +469,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     int a_cnt = 0, red_par = 0;
 
     for (;; ++seenA) {
-      const int s = seenA % kASlots;
-      const bool got = warp_mbar_wait(&fullA[s], (seenA / kASlots) & 1, &ctl[0], lane);
+      const int s = seenA % kA;
+      const bool got = warp_mbar_wait(&fullA[s], (seenA / kA) & 1, &ctl[0], lane);
       if (token_any(1, !got)) {
         if (tid == 0 && !ctl[0]) {
           set_status(status, CAOTE_ERR_TIMEOUT);
@@ -504,7 +513,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         }
         float bval = 0.f;
         if (use_base) {
-          bval = valid ? reinterpret_cast<const float*>(baseA + (a_cnt % kASlots) * kBaseRowBytes)[tok] : 0.f;
+          bval = valid ? reinterpret_cast<const float*>(baseA + (a_cnt % kA) * kBaseRowBytes)[tok] : 0.f;
           hbpart += bval;
         }
         if (token_any(1, over)) {
@@ -574,8 +583,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         if (d.n_valid < kT) {
           // rows behind the unit's length hold whatever the cache has there: clear them in the V tile
           // (next slot) so that a zero weight times a stray NaN cannot reach the accumulators
-          const int s2 = (seenA + 1) % kASlots;
-          wait_or_stop(&fullA[s2], ((seenA + 1) / kASlots) & 1, &ctl[0], status);
+          const int s2 = (seenA + 1) % kA;
+          wait_or_stop(&fullA[s2], ((seenA + 1) / kA) & 1, &ctl[0], status);
           if (!valid) {
             char* vt = tilesA + s2 * kTileBytes;
 #pragma unroll
@@ -705,9 +714,9 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
       // FastCAOTE: walk the attention ring; from every V tile take || mean(v) - v_j || of the token's row
       int items = 0;
       for (int i = 0;; ++i) {
-        const int s = i % kASlots;
+        const int s = i % kA;
         const char* sl = tilesA + s * kTileBytes;
-        const bool got = warp_mbar_wait(&fullA[s], (i / kASlots) & 1, &ctl[0], lane);
+        const bool got = warp_mbar_wait(&fullA[s], (i / kA) & 1, &ctl[0], lane);
         if (token_any(2, !got)) {
           if (tok == 0 && !ctl[0]) {
             set_status(status, CAOTE_ERR_TIMEOUT);
@@ -720,7 +729,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
         if (d.type == kSlotKA) {
           if (d.flags & kFlagFirst) ++items;
         } else {
-          const float* xs = xbuf + ((items - 1) % kQBufs) * (kD + 4);
+          const float* xs = xbuf + ((items - 1) % kQ) * (kD + 4);
           const float inv_n = xs[kD];
           float n2a = 0.f, n2b = 0.f;
 #pragma unroll 2
@@ -809,7 +818,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   prefill::tc_fence_after();
   const int dummy = 0;
   if (tid == 0)
-    for (int j = seenA; j < ctl[2]; ++j) mbar_wait(&fullA[j % kASlots], (j / kASlots) & 1, &dummy);
+    for (int j = seenA; j < ctl[2]; ++j) mbar_wait(&fullA[j % kA], (j / kA) & 1, &dummy);
   if (tid == kTcTokenThreads)
     for (int j = seenB; j < ctl[3]; ++j) mbar_wait(&fullB[j % kBSlots], (j / kBSlots) & 1, &dummy);
   if (warp == kTcIssueWarp) prefill::tmem_dealloc(tmem, kTmemCols);
