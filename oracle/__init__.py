@@ -9,7 +9,8 @@ Pins (see the CPU tests): attention against torch's fp64 scaled-dot-product atte
 leave-one-out recomputation (Theorem 3.2) and against the weight-renormalisation identity
 (Theorem 3.1); closed forms for q = 0 and n = 2; invariances; the H2O mass theorem (Appendix D.1);
 selection against a tuple sort; compaction against multiset preservation. The FastCAOTE and joint
-multi-token helpers are pinned by their reductions to the single-token score and by brute force.
+multi-token helpers are pinned by their reductions to the single-token score and by brute force; the
+post-eviction output against torch attention over the retained set and against the correction formula.
 """
 from __future__ import annotations
 
@@ -138,6 +139,38 @@ def joint_score(w, V, evicted) -> float:
     n, d = V.shape
     return float(_load().caote_oracle_joint_score(_ptr(w, ctypes.c_double), _ptr(V, ctypes.c_float),
                                                   n, d, _ptr(E, ctypes.c_int32), len(E)))
+
+
+def post_evict_output(q, K, V, lens, evict, *, scale: float, n_new: int = 1) -> np.ndarray:
+    """Attention output over the retained tokens (Sec. 2: the budgeted cache attends over what it kept).
+
+    Written from the definition, row by row: query i of the block sees slots j <= n - m + i; the evicted
+    slots ``evict[b][h]`` are taken out; softmax over what is left, in double. A row left with nothing to
+    see gets zeros. q [B,Hq,m,d], K/V [B,Hkv,cap,d]; returns [B,Hq,m,d] float64.
+    """
+    q, K, V = _f32(q).astype(np.float64), _f32(K).astype(np.float64), _f32(V).astype(np.float64)
+    B, Hq, m, d = q.shape
+    Hkv = K.shape[1]
+    G = Hq // Hkv
+    assert m == n_new
+    out = np.zeros((B, Hq, m, d), dtype=np.float64)
+    for b in range(B):
+        n = int(lens[b])
+        if n == 0:
+            continue
+        for h in range(Hkv):
+            gone = np.zeros(n, dtype=bool)
+            gone[np.asarray(evict[b][h], dtype=np.int64)] = True
+            for g in range(G):
+                for i in range(m):
+                    keep = ~gone
+                    keep[n - m + i + 1:] = False
+                    if not keep.any():
+                        continue
+                    s = scale * (K[b, h, :n][keep] @ q[b, h * G + g, i])
+                    w = np.exp(s - s.max())
+                    out[b, h * G + g, i] = (w / w.sum()) @ V[b, h, :n][keep]
+    return out
 
 
 def select_evict(scores, lens, budget, pos=None) -> Tuple[list, np.ndarray]:

@@ -297,6 +297,45 @@ def test_fast_and_joint_scores():
 
 
 # ---------------------------------------------------------------- the paper's printed numbers
+def test_post_evict_output_is_attention_over_the_retained_tokens():
+    """Pins: (1) torch fp64 scaled-dot-product attention on the retained keys with the causal-in-block mask;
+    (2) the correction formula of Sec. 3.1, o' = (o - sum alpha_e v_e) / (1 - sum alpha_e), built from the
+    pre-eviction output and weights that oracle.score returns for one head and one query; (3) evicting
+    nothing gives the pre-eviction output back."""
+    rng = np.random.default_rng(31)
+    B, Hq, Hkv, d, cap, m = 2, 4, 2, 16, 40, 3
+    lens = np.array([37, 12], dtype=np.int32)
+    q = rng.standard_normal((B, Hq, m, d)).astype(np.float32)
+    K = rng.standard_normal((B, Hkv, cap, d)).astype(np.float32)
+    V = rng.standard_normal((B, Hkv, cap, d)).astype(np.float32)
+    scale = d ** -0.5
+    evict = [[np.array([0, 5, 35, 36]), np.array([7])], [np.array([10, 11]), np.array([], dtype=np.int64)]]
+    got = oracle.post_evict_output(q, K, V, lens, evict, scale=scale, n_new=m)
+    G = Hq // Hkv
+    for b in range(B):
+        n = int(lens[b])
+        for h in range(Hkv):
+            keep = np.setdiff1d(np.arange(n), evict[b][h])
+            kt = torch.from_numpy(K[b, h, keep]).double()[None, None]
+            vt = torch.from_numpy(V[b, h, keep]).double()[None, None]
+            mask = torch.from_numpy(keep[None, :] <= (n - m + np.arange(m))[:, None])  # [m, kept]
+            for g in range(G):
+                qt = torch.from_numpy(q[b, h * G + g]).double()[None, None]
+                ref = torch.nn.functional.scaled_dot_product_attention(qt, kt, vt, attn_mask=mask[None, None], scale=scale)
+                np.testing.assert_allclose(got[b, h * G + g], ref[0, 0].numpy(), rtol=1e-12, atol=1e-13)
+    none = [[np.array([], dtype=np.int64)] * Hkv for _ in range(B)]
+    r = oracle.score(q, K, V, lens, scale=scale, n_new=m, base_mode="chunk_sum")
+    np.testing.assert_allclose(oracle.post_evict_output(q, K, V, lens, none, scale=scale, n_new=m), r["o"], rtol=1e-12, atol=1e-13)
+    # one head, one query: w of oracle.score is that query's attention row
+    q1, n1 = q[:1, :1, :1], np.array([37], dtype=np.int32)
+    r1 = oracle.score(q1, K[:1, :1], V[:1, :1], n1, scale=scale, n_new=1, base_mode="last_query")
+    E = np.array([3, 8, 20])
+    a = r1["w"][0, 0, E]
+    want = (r1["o"][0, 0, 0] - a @ V[0, 0, E].astype(np.float64)) / (1.0 - a.sum())
+    got1 = oracle.post_evict_output(q1, K[:1, :1], V[:1, :1], n1, [[E]], scale=scale, n_new=1)
+    np.testing.assert_allclose(got1[0, 0, 0], want, rtol=1e-11, atol=1e-13)
+
+
 def test_flop_model_matches_printed_ratios():
     """Appendix C: the FLOP formulas with Llama-3.1-8B dimensions reproduce the printed ratio tables."""
     path = os.path.join(os.path.dirname(__file__), "golden", "appendix_c_flop_ratios.txt")
