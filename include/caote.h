@@ -223,6 +223,21 @@ CAOTE_API int caote_step_fast(const caote_params_t* params, const void* q, const
                     int32_t max_evict, int32_t* n_evict, int32_t compact_mode, void* workspace,
                     size_t workspace_bytes, caote_stream_t stream);
 
+/* Post-eviction attention output (Sec. 2: the budgeted cache attends over the retained tokens only;
+ * Sec. 3.1, proof of Theorem 3.2): for every query row r of this call,
+ *     o_post_r = (o_r - sum_{e in E_r} alpha_{r,e} v_e) / (1 - sum_{e in E_r} alpha_{r,e}),
+ * E_r = the evicted slots row r can see, alpha = the row's pre-eviction softmax weights; i.e. the softmax
+ * attention over the retained tokens. A row whose visible tokens are all evicted gets 0.
+ * Call it after caote_select_evict and BEFORE caote_compact (evict_idx refers to the slots as scored):
+ *   q, K, V, len as passed to caote_score; evict_idx, max_evict, n_evict as written by caote_select_evict;
+ *   o  in:  the pre-eviction output caote_score wrote, [B, Hq, m, d] fp32;
+ *   o_post out, same shape (may alias o).
+ * Needs no workspace. It recomputes the rows' softmax normalisers with one pass over K on the CUDA cores:
+ * a correction step for callers that want it, not part of the timed path. */
+CAOTE_API int caote_post_evict_output(const caote_params_t* params, const void* q, const void* K, const void* V,
+                            const int32_t* len, const int32_t* evict_idx, int32_t max_evict,
+                            const int32_t* n_evict, const float* o, float* o_post, caote_stream_t stream);
+
 /* Synchronise the stream, copy the status word to *status_out (host pointer) and reset it to CAOTE_OK.
  * The word holds the first device-side error since the last reset. */
 CAOTE_API int caote_read_status(void* workspace, caote_stream_t stream, int32_t* status_out);

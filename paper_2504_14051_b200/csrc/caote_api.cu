@@ -9,6 +9,7 @@
 #include "common.cuh"
 #include "decode_tc.cuh"
 #include "generic_score.cuh"
+#include "post_evict.cuh"
 #include "prefill_tc.cuh"
 #include "select_compact.cuh"
 
@@ -387,6 +388,19 @@ static int static_scratch_address(char** out) {
   return CAOTE_OK;
 }
 
+template <typename T, int D>
+static int launch_post_evict(const Dims& dm, const void* q, const void* K, const void* V, const int* len,
+                             const int* evict_idx, int max_evict, const int* n_evict, const float* o, float* o_post,
+                             cudaStream_t st) {
+  const size_t smem = post::smem_bytes<D>();
+  int rc = allow_smem(post::post_evict_kernel<T, D>, smem);
+  if (rc) return rc;
+  dim3 grid((dm.R + post::kRows - 1) / post::kRows, dm.units);
+  CAOTE_LAUNCH("post_evict_kernel", st, post::post_evict_kernel<T, D><<<grid, 32 * post::kRows, smem, st>>>(
+      dm, (const T*)q, (const T*)K, (const T*)V, len, evict_idx, max_evict, n_evict, o, o_post));
+  return CAOTE_OK;
+}
+
 }  // namespace caote
 
 using namespace caote;
@@ -609,6 +623,25 @@ int caote_step_fast(const caote_params_t* p, const void* q, const void* k_new, c
   if (!vsum || !aligned(vsum, 16)) return CAOTE_ERR_INVALID_ARG;
   return step_impl(p, q, k_new, v_new, K, V, base, pos, len, n_seen, budget, vsum, o, scores, evict_idx, max_evict,
                    n_evict, compact_mode, workspace, workspace_bytes_, stream);
+}
+
+int caote_post_evict_output(const caote_params_t* p, const void* q, const void* K, const void* V, const int32_t* len,
+                            const int32_t* evict_idx, int32_t max_evict, const int32_t* n_evict, const float* o,
+                            float* o_post, caote_stream_t stream) {
+  if (!params_ok(p) || !q || !K || !V || !len || !evict_idx || !n_evict || !o || !o_post || max_evict < 1)
+    return CAOTE_ERR_INVALID_ARG;
+  if (!params_supported(p)) return CAOTE_ERR_UNSUPPORTED;
+  if (!aligned(q, 16) || !aligned(K, 16) || !aligned(V, 16)) return CAOTE_ERR_INVALID_ARG;
+  int rc = check_device();
+  if (rc) return rc;
+  const Dims dm = make_dims(p);
+  cudaStream_t st = (cudaStream_t)stream;
+  if (p->dtype == CAOTE_BF16) {
+    if (dm.D == 128) return launch_post_evict<__nv_bfloat16, 128>(dm, q, K, V, len, evict_idx, max_evict, n_evict, o, o_post, st);
+    return launch_post_evict<__nv_bfloat16, 64>(dm, q, K, V, len, evict_idx, max_evict, n_evict, o, o_post, st);
+  }
+  if (dm.D == 128) return launch_post_evict<float, 128>(dm, q, K, V, len, evict_idx, max_evict, n_evict, o, o_post, st);
+  return launch_post_evict<float, 64>(dm, q, K, V, len, evict_idx, max_evict, n_evict, o, o_post, st);
 }
 
 int caote_read_status(void* workspace, caote_stream_t stream, int32_t* status_out) {
