@@ -721,13 +721,17 @@ score_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
           }
           h += (h4[0] + h4[1]) + (h4[2] + h4[3]);
         } else {
+          // row R sees key j iff j <= n - m + (R % m), i.e. iff (R % m) >= j - (n - m); R % m is carried
+          // along instead of being divided out for every pair
+          const int need = j - (n - m);
+          const int R0 = rb * kTile + cc * 32;
+          int rm = R0 % m;
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
-            const int R = rb * kTile + cc * 32 + i;  // query row of this column
-            // row R sees key j iff j <= n - m + (R % m)
-            const bool vis = R < M && j < n - m + (R % m) + 1;
+            const bool vis = (R0 + i < M) && (rm >= need);
             const float a = fast_exp2(fmaf(v[i], scale2, -stc[i]));
             h += vis ? a : 0.f;
+            if (++rm == m) rm = 0;
           }
         }
       }
