@@ -40,7 +40,7 @@ NCU_TRAFFIC = {
                          "profile": "profiles/decode_tc_kernel_c4_full_traffic.txt"},
     "decode_tc_fast_kernel": {"per_launch": {"c4": 956084992 + 56993536},
                               "profile": "profiles/decode_tc_kernel_c4_full_traffic.txt"},
-    "prefill_attn_kernel": {"bytes_per_unit": (155385088 + 17509632) / 16, "profile": "profiles/prefill_kernels_c5p_batch2_ncu.txt"},
+    "prefill_attn_kernel": {"bytes_per_unit": (156274688 + 23372288) / 16, "profile": "profiles/prefill_kernels_c5p_batch2_ncu.txt"},
 }
 
 METRIC = "cached tokens scored+evicted/sec"
