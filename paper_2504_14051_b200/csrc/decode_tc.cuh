@@ -645,7 +645,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
             float mfin[8], lfin[8], acc[8];
 #pragma unroll
             for (int g = 0; g < 8; ++g) { mfin[g] = -INFINITY; lfin[g] = 0.f; acc[g] = 0.f; }
-#pragma unroll 2
+#pragma unroll 4
             for (int c = 0; c < d.nitems; ++c) {
               const float4 m0 = __ldcg(reinterpret_cast<const float4*>(p0[c].m));
               const float4 m1 = __ldcg(reinterpret_cast<const float4*>(p0[c].m + 4));
@@ -655,7 +655,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
               mfin[6] = fmaxf(mfin[6], m1.z); mfin[7] = fmaxf(mfin[7], m1.w);
             }
             float hbsum = 0.f;
-#pragma unroll 2
+#pragma unroll 4
             for (int c = 0; c < d.nitems; ++c) {
               const float4 m0 = __ldcg(reinterpret_cast<const float4*>(p0[c].m));
               const float4 m1 = __ldcg(reinterpret_cast<const float4*>(p0[c].m + 4));
