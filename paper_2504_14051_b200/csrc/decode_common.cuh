@@ -59,6 +59,7 @@ struct Desc {         // what a slot holds
 
 struct Plan {
   int* item_prefix;   // [units + 1] exclusive prefix of items per unit
+  int4* item_info;    // [items] (unit, first item of the unit, items of the unit, tokens of the unit)
   int* counter;       // [units] A items of the unit whose records are written
   int* ready;         // [units] 1 once FinalRec is written
   int* work;          // [2] next attention item, next score item
@@ -94,6 +95,7 @@ inline size_t carve(const Dims& dm, char* base, Plan* out, int grid) {
   pl.capS = tiles_per_unit * kT;
   const size_t max_items = (size_t)dm.units * tiles_per_unit;  // sized for tpi = 1
   pl.item_prefix = (int*)take(sizeof(int) * ((size_t)dm.units + 1));
+  pl.item_info = (int4*)take(sizeof(int4) * max_items);
   pl.counter = (int*)take(sizeof(int) * (size_t)dm.units);
   pl.ready = (int*)take(sizeof(int) * (size_t)dm.units);
   pl.work = (int*)take(sizeof(int) * 4);
@@ -133,7 +135,13 @@ plan_kernel(int units, int Hkv, int cap, const int* __restrict__ len, Plan pl, i
     __syncthreads();
     int before = carry;
     for (int w = 0; w < warp; ++w) before += warp_tot[w];
-    if (u < units) pl.item_prefix[u + 1] = before + incl;
+    if (u < units) {
+      pl.item_prefix[u + 1] = before + incl;
+      // what a CTA needs to know about an item it takes, in one load
+      const int first = before + incl - ni;
+      const int4 info = make_int4(u, first, ni, len[u / Hkv]);
+      for (int k = 0; k < ni; ++k) pl.item_info[first + k] = info;
+    }
     __syncthreads();
     if (tid == 1023) carry = before + incl;
     __syncthreads();

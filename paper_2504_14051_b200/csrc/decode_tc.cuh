@@ -149,25 +149,15 @@ struct Entry {  // a work item a producer is feeding into its ring
   int item, unit, item0, nitems, n, t_begin, t_end;
 };
 
-// The item -> unit lookup (32-ary search over the item prefix, one probe per lane) and the item's tile
-// range; warp-collective, every lane gets the same entry.
+// An item's unit and tile range from the plan's item table; every lane gets the same entry.
 __device__ __forceinline__ Entry find_entry(int item, const Dims& dm, const Plan& pl, const int* __restrict__ len, int lane) {
-  int lo = 0, hi = dm.units;
-  while (hi - lo > 1) {
-    const int step = (hi - lo + 31) / 32;
-    const int probe = lo + lane * step;
-    const int val = (probe < hi) ? __ldg(pl.item_prefix + probe) : 0x7fffffff;
-    const unsigned mask = __ballot_sync(0xffffffffu, val <= item);
-    const int k = 31 - __clz((int)mask);
-    lo = lo + k * step;
-    hi = min(hi, lo + step);
-  }
+  const int4 info = __ldcg(pl.item_info + item);
   Entry e;
   e.item = item;
-  e.unit = lo;
-  e.item0 = pl.item_prefix[lo];
-  e.nitems = pl.item_prefix[lo + 1] - e.item0;
-  e.n = len[lo / dm.Hkv];
+  e.unit = info.x;
+  e.item0 = info.y;
+  e.nitems = info.z;
+  e.n = info.w;
   e.t_begin = (item - e.item0) * pl.tpi;
   e.t_end = min(e.t_begin + pl.tpi, (e.n + kT - 1) / kT);
   return e;
