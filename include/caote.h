@@ -223,6 +223,19 @@ CAOTE_API int caote_step_fast(const caote_params_t* params, const void* q, const
                     int32_t max_evict, int32_t* n_evict, int32_t compact_mode, void* workspace,
                     size_t workspace_bytes, caote_stream_t stream);
 
+/* caote_score with the other way of extending the single-head, single-query score to a group of query
+ * heads and to a block of queries: instead of adding the rows' attention weights and applying the general
+ * form once per unit, add up the exact single-query errors (Sec. 3.1 score, Theorem 3.2, row by row) of
+ * the rows that define the base score,
+ *     scores[u, j] = sum_r alpha_{r,j} / (1 - alpha_{r,j}) * || o_r - v_j ||_2 ,
+ * r over the last row of every group head (LAST_QUERY) or over all rows (CHUNK_SUM); other base modes
+ * return CAOTE_ERR_UNSUPPORTED. With one head and one query it equals caote_score. Arguments as in
+ * caote_score (no base). Runs on the any-shape fp32 CUDA-core kernels (two dot products of length d per
+ * (row, token) pair): a correctness path for comparing the two aggregations, not tuned. */
+CAOTE_API int caote_score_sum_errors(const caote_params_t* params, const void* q, const void* K, const void* V,
+                           const int32_t* len, float* o, float* scores, void* workspace,
+                           size_t workspace_bytes, caote_stream_t stream);
+
 /* Post-eviction attention output (Sec. 2: the budgeted cache attends over the retained tokens only;
  * Sec. 3.1, proof of Theorem 3.2): for every query row r of this call,
  *     o_post_r = (o_r - sum_{e in E_r} alpha_{r,e} v_e) / (1 - sum_{e in E_r} alpha_{r,e}),

@@ -92,6 +92,8 @@ def lib() -> ctypes.CDLL:
     L.caote_score_fast.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     L.caote_step_fast.restype = ctypes.c_int
     L.caote_step_fast.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp, i32, vp, sz, vp]
+    L.caote_score_sum_errors.restype = ctypes.c_int
+    L.caote_score_sum_errors.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     L.caote_post_evict_output.restype = ctypes.c_int
     L.caote_post_evict_output.argtypes = [pp, vp, vp, vp, vp, vp, i32, vp, vp, vp, vp]
     L.caote_read_status.restype = ctypes.c_int
@@ -211,6 +213,13 @@ def caote_step_fast(p, q, k_new, v_new, K, V, base, pos, lens, n_seen, budget, v
                                  _p(lens), _p(n_seen), _p(budget), _p(vsum), _p(o), _p(scores), _p(evict_idx),
                                  evict_idx.shape[-1], _p(n_evict), mode, _p(workspace), workspace.numel(),
                                  _stream(stream)))
+
+
+def caote_score_sum_errors(p, q, K, V, lens, o, scores, workspace, stream=None):
+    """Scores as the sum over the counted query rows of the exact single-query eviction errors."""
+    _check("caote_score_sum_errors",
+           lib().caote_score_sum_errors(ctypes.byref(p), _p(q), _p(K), _p(V), _p(lens), _p(o), _p(scores),
+                                        _p(workspace), workspace.numel(), _stream(stream)))
 
 
 def caote_post_evict_output(p, q, K, V, lens, evict_idx, n_evict, o, o_post, stream=None):

@@ -146,7 +146,8 @@ static int allow_smem(KernelT kernel, size_t bytes) {
 
 template <typename T, int D>
 static int launch_generic_score(const Dims& dm, const void* q, const void* K, const void* V, const int* len,
-                                float* base, float* o, float* scores, char* ws, cudaStream_t st, const float* vsum) {
+                                float* base, float* o, float* scores, char* ws, cudaStream_t st, const float* vsum,
+                                bool sum_errors = false) {
   generic::Scratch sc;
   generic::carve(dm, ws + kHeaderBytes, &sc);
   int* status = reinterpret_cast<int*>(ws);
@@ -162,6 +163,15 @@ static int launch_generic_score(const Dims& dm, const void* q, const void* K, co
   {
     dim3 grid(sc.chunks, dm.units);
     CAOTE_LAUNCH("attn_combine_kernel", st, generic::attn_combine_kernel<T, D><<<grid, D, 0, st>>>(dm, len, sc, o));
+  }
+  if (sum_errors) {
+    const size_t smem = generic::sum_errors_smem(D);
+    int rc = allow_smem(generic::sum_errors_kernel<T, D>, smem);
+    if (rc) return rc;
+    dim3 grid((dm.cap + generic::kKT - 1) / generic::kKT, dm.units);
+    CAOTE_LAUNCH("sum_errors_kernel", st, generic::sum_errors_kernel<T, D><<<grid, generic::kThreads, smem, st>>>(
+        dm, (const T*)q, (const T*)K, (const T*)V, len, o, sc, scores));
+    return CAOTE_OK;
   }
   {
     const size_t smem = generic::score_smem(D);
@@ -467,6 +477,26 @@ int caote_score(const caote_params_t* p, const void* q, const void* K, const voi
                 float* base, float* o, float* scores, void* workspace, size_t workspace_bytes_,
                 caote_stream_t stream) {
   return score_impl(p, q, K, V, len, base, nullptr, o, scores, workspace, workspace_bytes_, stream);
+}
+
+int caote_score_sum_errors(const caote_params_t* p, const void* q, const void* K, const void* V, const int32_t* len,
+                           float* o, float* scores, void* workspace, size_t workspace_bytes_, caote_stream_t stream) {
+  if (!params_ok(p) || !q || !K || !V || !len || !o || !scores || !workspace) return CAOTE_ERR_INVALID_ARG;
+  if (!params_supported(p)) return CAOTE_ERR_UNSUPPORTED;
+  if (p->base_mode != CAOTE_BASE_LAST_QUERY && p->base_mode != CAOTE_BASE_CHUNK_SUM) return CAOTE_ERR_UNSUPPORTED;
+  if (workspace_bytes_ < workspace_bytes(p) || !aligned(workspace, 256)) return CAOTE_ERR_INVALID_ARG;
+  if (!aligned(q, 16) || !aligned(K, 16) || !aligned(V, 16) || !aligned(o, 16)) return CAOTE_ERR_INVALID_ARG;
+  int rc = check_device();
+  if (rc) return rc;
+  const Dims dm = make_dims(p);
+  cudaStream_t st = (cudaStream_t)stream;
+  char* ws = (char*)workspace;
+  if (p->dtype == CAOTE_BF16) {
+    if (dm.D == 128) return launch_generic_score<__nv_bfloat16, 128>(dm, q, K, V, len, nullptr, o, scores, ws, st, nullptr, true);
+    return launch_generic_score<__nv_bfloat16, 64>(dm, q, K, V, len, nullptr, o, scores, ws, st, nullptr, true);
+  }
+  if (dm.D == 128) return launch_generic_score<float, 128>(dm, q, K, V, len, nullptr, o, scores, ws, st, nullptr, true);
+  return launch_generic_score<float, 64>(dm, q, K, V, len, nullptr, o, scores, ws, st, nullptr, true);
 }
 
 int caote_score_fast(const caote_params_t* p, const void* q, const void* K, const void* V, const int32_t* len,

@@ -438,6 +438,103 @@ inline size_t partial_smem(int D) {
   const int LD = D + 4;
   return sizeof(float) * (size_t)(kRT * LD + 2 * kKT * LD + kRT * kKT + kKT + kThreads);
 }
+// Sum-of-errors aggregation: instead of adding the rows' weights and applying the general form once,
+// add up the exact single-query errors (Theorem 3.2, row by row) of the rows that define the base score:
+//     c_j = sum_r alpha_{r,j} / (1 - alpha_{r,j}) * || o_r - v_j ||_2 .
+// Needs o and the row statistics of attn_partial / attn_combine. grid = (key tiles, units), kThreads;
+// thread (r = tid / 16, c0 = tid % 16) owns row slot r and keys c0 + 16 i of the tile.
+template <typename T, int D>
+__global__ void __launch_bounds__(kThreads)
+sum_errors_kernel(Dims dm, const T* __restrict__ q, const T* __restrict__ K, const T* __restrict__ V,
+                  const int* __restrict__ len, const float* __restrict__ o, Scratch sc, float* __restrict__ scores) {
+  constexpr int LD = D + 4;
+  extern __shared__ __align__(16) float smem[];
+  float* Qs = smem;              // kRT * LD
+  float* Os = Qs + kRT * LD;     // kRT * LD
+  float* Ks = Os + kRT * LD;     // kKT * LD
+  float* Vs = Ks + kKT * LD;     // kKT * LD
+  float* Hred = Vs + kKT * LD;   // kRT * kKT
+  float* st = Hred + kRT * kKT;  // kRT * 2
+
+  const int unit = blockIdx.y;
+  const int b = unit / dm.Hkv, h = unit % dm.Hkv;
+  const int n = len[b];
+  const int j0 = blockIdx.x * kKT;
+  if (n == 0 || n < dm.m || n > dm.cap || j0 >= n) return;
+  const int tid = threadIdx.x, r = tid >> 4, c0 = tid & 15;
+  const int mode = dm.base_mode;
+  const int n_rows = (mode == CAOTE_BASE_LAST_QUERY) ? dm.G : dm.R;
+  const int valid = min(kKT, n - j0);
+  stage_rows<T, D, LD>(Ks, K + ((size_t)unit * dm.cap + j0) * D, kKT, valid);
+  stage_rows<T, D, LD>(Vs, V + ((size_t)unit * dm.cap + j0) * D, kKT, valid);
+
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  for (int t0 = 0; t0 < n_rows; t0 += kRT) {
+    __syncthreads();
+    for (int idx = tid; idx < kRT * (D / 4); idx += kThreads) {
+      const int rr = idx / (D / 4), c4 = idx % (D / 4);
+      const int t = t0 + rr;
+      float4 qv = make_float4(0.f, 0.f, 0.f, 0.f), ov = qv;
+      if (t < n_rows) {
+        const int row = (mode == CAOTE_BASE_LAST_QUERY) ? t * dm.m + dm.m - 1 : t;
+        qv = load4(q + q_offset(dm, b, h, row) + c4 * 4);
+        ov = *reinterpret_cast<const float4*>(o + q_offset(dm, b, h, row) + c4 * 4);
+      }
+      *reinterpret_cast<float4*>(Qs + rr * LD + c4 * 4) = qv;
+      *reinterpret_cast<float4*>(Os + rr * LD + c4 * 4) = ov;
+    }
+    if (tid < kRT) {
+      const int t = t0 + tid;
+      float mx = 0.f, il = 0.f;
+      if (t < n_rows) {
+        const int row = (mode == CAOTE_BASE_LAST_QUERY) ? t * dm.m + dm.m - 1 : t;
+        mx = sc.stats[((size_t)unit * sc.Rpad + row) * 2];
+        il = sc.stats[((size_t)unit * sc.Rpad + row) * 2 + 1];
+      }
+      st[tid * 2] = mx;
+      st[tid * 2 + 1] = il;
+    }
+    __syncthreads();
+    const int t = t0 + r;
+    if (t < n_rows) {
+      const int row = (mode == CAOTE_BASE_LAST_QUERY) ? t * dm.m + dm.m - 1 : t;
+      const int n_vis = n - dm.m + (row % dm.m) + 1;
+      const float mx = st[r * 2], l = 1.f / st[r * 2 + 1];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int jj = c0 + 16 * i, j = j0 + jj;
+        if (j < n_vis) {
+          const float e = expf(logit<D>(Qs + r * LD, Ks + jj * LD, dm.scale) - mx);
+          const float rest = l - e;  // the other tokens' share of the row's softmax sum
+          float d2 = 0.f;
+#pragma unroll 8
+          for (int c = 0; c < D; c += 4) {
+            const float4 ov = *reinterpret_cast<const float4*>(Os + r * LD + c);
+            const float4 vv = *reinterpret_cast<const float4*>(Vs + jj * LD + c);
+            const float a0 = ov.x - vv.x, a1 = ov.y - vv.y, a2 = ov.z - vv.z, a3 = ov.w - vv.w;
+            d2 = fmaf(a0, a0, d2); d2 = fmaf(a1, a1, d2); d2 = fmaf(a2, a2, d2); d2 = fmaf(a3, a3, d2);
+          }
+          acc[i] += (rest > 0.f) ? e / rest * sqrtf(d2) : INFINITY;
+        }
+      }
+    }
+  }
+  __syncthreads();
+#pragma unroll
+  for (int i = 0; i < 4; ++i) Hred[r * kKT + c0 + 16 * i] = acc[i];
+  __syncthreads();
+  if (tid < kKT && j0 + tid < n) {
+    float cj = 0.f;
+    for (int rr = 0; rr < kRT; ++rr) cj += Hred[rr * kKT + tid];
+    scores[(size_t)unit * dm.cap + j0 + tid] = cj;
+  }
+}
+
+inline size_t sum_errors_smem(int D) {
+  const int LD = D + 4;
+  return sizeof(float) * (size_t)(2 * kRT * LD + 2 * kKT * LD + kRT * kKT + kRT * 2);
+}
+
 inline size_t score_smem(int D) {
   const int LD = D + 4;
   return sizeof(float) * (size_t)(kRT * LD + kKT * LD + kRT * kKT + D + kRT * 2 + kKT);

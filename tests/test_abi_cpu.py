@@ -93,6 +93,9 @@ def test_host_side_argument_checks_return_before_any_launch():
     assert lib.caote_score_fast(bp, fake, fake, fake, fake, fake, fake, fake, fake, ws, need - 1, None) == C.ERR_INVALID_ARG
     assert lib.caote_step_fast(bp, fake, fake, fake, fake, fake, fake, fake, fake, fake, fake, None, fake, fake, fake, 1,
                                fake, 0, ws, need, None) == C.ERR_INVALID_ARG
+    # sum-of-errors aggregation: defined for LAST_QUERY and CHUNK_SUM only (p is ACCUM)
+    assert lib.caote_score_sum_errors(bp, fake, fake, fake, fake, fake, fake, ws, need, None) == C.ERR_UNSUPPORTED
+    assert lib.caote_score_sum_errors(bp, None, fake, fake, fake, fake, fake, ws, need, None) == C.ERR_INVALID_ARG
     # post-eviction output: every pointer is mandatory, max_evict >= 1
     assert lib.caote_post_evict_output(bp, fake, fake, fake, fake, None, 4, fake, fake, fake, None) == C.ERR_INVALID_ARG
     assert lib.caote_post_evict_output(bp, fake, fake, fake, fake, fake, 0, fake, fake, fake, None) == C.ERR_INVALID_ARG
