@@ -36,9 +36,9 @@ from paper_2504_14051_b200 import workloads as wl  # noqa: E402
 # None when its kernel has changed since the capture.
 NCU_TRAFFIC = {
     # per launch at the workload's own size: (read + write) of profiles/decode_tc_kernel_c4_full_traffic.txt
-    "decode_tc_kernel": {"per_launch": {"c4": 1421538816 + 62786304, "c5d": 781206528 + 34503168},
+    "decode_tc_kernel": {"per_launch": {"c4": 1420990976 + 62851584, "c5d": 780532736 + 34983680},
                          "profile": "profiles/decode_tc_kernel_c4_full_traffic.txt"},
-    "decode_tc_fast_kernel": {"per_launch": {"c4": 956084992 + 56993536},
+    "decode_tc_fast_kernel": {"per_launch": {"c4": 956031488 + 56979456},
                               "profile": "profiles/decode_tc_kernel_c4_full_traffic.txt"},
     "prefill_attn_kernel": {"bytes_per_unit": (156274688 + 23372288) / 16, "profile": "profiles/prefill_kernels_c5p_batch2_ncu.txt"},
 }
