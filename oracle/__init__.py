@@ -9,8 +9,9 @@ Pins (see the CPU tests): attention against torch's fp64 scaled-dot-product atte
 leave-one-out recomputation (Theorem 3.2) and against the weight-renormalisation identity
 (Theorem 3.1); closed forms for q = 0 and n = 2; invariances; the H2O mass theorem (Appendix D.1);
 selection against a tuple sort; compaction against multiset preservation. The FastCAOTE and joint
-multi-token helpers are pinned by their reductions to the single-token score and by brute force; the
-post-eviction output against torch attention over the retained set and against the correction formula.
+multi-token helpers are pinned by their reductions to the single-token score and by brute force (the
+greedy sequence by recomputing the output from scratch after every pick, by the joint score of the set it
+chose and by exhaustive search over pairs); the post-eviction output against torch attention over the retained set and against the correction formula.
 """
 from __future__ import annotations
 
@@ -67,6 +68,8 @@ def _load():
         lib.caote_oracle_fast_scores.argtypes = [dp, fp, ctypes.c_int, ctypes.c_int, dp]
         lib.caote_oracle_joint_score.restype = ctypes.c_double
         lib.caote_oracle_joint_score.argtypes = [dp, fp, ctypes.c_int, ctypes.c_int, ip, ctypes.c_int]
+        lib.caote_oracle_greedy_evict.restype = ctypes.c_int
+        lib.caote_oracle_greedy_evict.argtypes = [dp, fp, ip, ctypes.c_int, ctypes.c_int, ctypes.c_int, ip, dp, dp]
         _lib = lib
     return _lib
 
@@ -139,6 +142,30 @@ def joint_score(w, V, evicted) -> float:
     n, d = V.shape
     return float(_load().caote_oracle_joint_score(_ptr(w, ctypes.c_double), _ptr(V, ctypes.c_float),
                                                   n, d, _ptr(E, ctypes.c_int32), len(E)))
+
+
+def greedy_evict(w, V, k: int, pos=None):
+    """Greedy multi-token eviction of one unit (Appendix B chained): k times evict the token whose removal
+    changes the current output least, renormalise the weights of the rest and update the output.
+
+    w [n] normalised weights, V [n,d], pos [n] tie-break keys or None (slot index). Returns
+    (order [k] slots in eviction order, step_score [k] each pick's score at its step,
+    cum_err [k] distance between the original output and the output after each eviction).
+    """
+    w = np.ascontiguousarray(np.asarray(w, dtype=np.float64))
+    V = _f32(V)
+    n, d = V.shape
+    order = np.zeros(k, dtype=np.int32)
+    step = np.zeros(k, dtype=np.float64)
+    cum = np.zeros(k, dtype=np.float64)
+    pos_a = None if pos is None else np.ascontiguousarray(np.asarray(pos, dtype=np.int32))
+    rc = _load().caote_oracle_greedy_evict(_ptr(w, ctypes.c_double), _ptr(V, ctypes.c_float),
+                                           _ptr(pos_a, ctypes.c_int32), n, d, int(k),
+                                           _ptr(order, ctypes.c_int32), _ptr(step, ctypes.c_double),
+                                           _ptr(cum, ctypes.c_double))
+    if rc != 0:
+        raise ValueError("caote_oracle_greedy_evict: bad argument (need 0 <= k < n)")
+    return order, step, cum
 
 
 def post_evict_output(q, K, V, lens, evict, *, scale: float, n_new: int = 1) -> np.ndarray:

@@ -252,3 +252,65 @@ double caote_oracle_joint_score(const double* w, const float* V, int n, int d, c
   free(acc);
   return sqrt(nrm) / (1.0 - gone);
 }
+
+/* Greedy multi-token eviction (Appendix B, the two-token derivation chained k times): evict one token,
+ * renormalise what is left, evict the next one from the updated state.
+ *   repeat k times over the tokens still present:
+ *     c_j = w_j / (1 - w_j) * || X - v_j ||_2 on the CURRENT weights and output (Sec. 3.1 score; 1 - w_j
+ *           as the sum of the other present weights);
+ *     e   = the present token with the smallest (c_j, pos_j) (pos == NULL: the slot index);
+ *     X  <- (X - w_e v_e) / (1 - w_e),  w_i <- w_i / (1 - w_e) for the others   (Appendix B, alpha' and X').
+ * One unit. w in: normalised weights of the n tokens (sum 1). Outputs: order[t] = slot evicted at step t,
+ * step_score[t] = its score at that step (the output error of that single step), cum_err[t] = the distance
+ * between the ORIGINAL output and the output after t + 1 evictions (which the closed-form joint score of
+ * Appendix B gives for the evicted set). Any output may be NULL. k < n required. Returns 0, or -1. */
+int caote_oracle_greedy_evict(const double* w_in, const float* V, const int32_t* pos, int n, int d, int k,
+                              int32_t* order, double* step_score, double* cum_err) {
+  if (n < 1 || d < 1 || k < 0 || k >= n) return -1;
+  double* w = (double*)malloc(sizeof(double) * (size_t)n);
+  char* present = (char*)malloc((size_t)n);
+  double* X = (double*)calloc((size_t)d, sizeof(double));
+  double* X0 = (double*)malloc(sizeof(double) * (size_t)d);
+  for (int j = 0; j < n; ++j) {
+    w[j] = w_in[j];
+    present[j] = 1;
+    for (int c = 0; c < d; ++c) X[c] += w[j] * (double)V[(size_t)j * d + c];
+  }
+  memcpy(X0, X, sizeof(double) * (size_t)d);
+  for (int t = 0; t < k; ++t) {
+    int best = -1;
+    double best_c = 0.0;
+    for (int j = 0; j < n; ++j) {
+      if (!present[j]) continue;
+      double rest = 0.0;
+      for (int i = 0; i < n; ++i)
+        if (present[i] && i != j) rest += w[i];
+      const double c = (rest == 0.0) ? INFINITY : w[j] / rest * l2_distance(X, V + (size_t)j * d, d);
+      const int pj = pos ? pos[j] : j;
+      if (best < 0 || c < best_c || (c == best_c && pj < (pos ? pos[best] : best))) {
+        best = j;
+        best_c = c;
+      }
+    }
+    const double we = w[best];
+    double rest = 0.0;
+    for (int i = 0; i < n; ++i)
+      if (present[i] && i != best) rest += w[i];
+    present[best] = 0;
+    for (int c = 0; c < d; ++c) X[c] = (X[c] - we * (double)V[(size_t)best * d + c]) / rest;
+    for (int i = 0; i < n; ++i)
+      if (present[i]) w[i] /= rest;
+    if (order) order[t] = best;
+    if (step_score) step_score[t] = best_c;
+    if (cum_err) {
+      double acc = 0.0;
+      for (int c = 0; c < d; ++c) acc += (X0[c] - X[c]) * (X0[c] - X[c]);
+      cum_err[t] = sqrt(acc);
+    }
+  }
+  free(w);
+  free(present);
+  free(X);
+  free(X0);
+  return 0;
+}
