@@ -151,10 +151,12 @@ CAOTE_API int caote_score(const caote_params_t* params, const void* q, const voi
  * image; every GPU that loads the library holds it from load until the process exits. The caller
  * passes only inputs and outputs, with the meaning, layout and alignment they have in caote_score.
  *   status_out  device pointer to one int32, or NULL. Receives the status word of this call (CAOTE_OK
- *               or the first device-side error); stream-ordered like the other outputs.
+ *               or the first device-side error); stream-ordered like the other outputs. Left untouched
+ *               when the call itself returns an error code.
  * Limits and rules:
  *   - A shape with caote_workspace_bytes(params) > CAOTE_STATIC_SCRATCH_BYTES is rejected with
- *     CAOTE_ERR_TOO_LARGE before anything is enqueued.
+ *     CAOTE_ERR_TOO_LARGE, and every argument caote_score would refuse is refused with the same code,
+ *     before anything is enqueued or the array is touched.
  *   - The call itself allocates and frees nothing: no cudaMalloc / cudaFree, no allocating library
  *     routine. It enqueues a 256-byte memset of the scratch header, the kernels of caote_score and a
  *     4-byte device-to-device copy.

@@ -417,6 +417,29 @@ using namespace caote;
 
 extern "C" {
 
+// Host-side checks of caote_append / caote_score arguments; nothing is enqueued before they pass.
+static int append_args_check(const caote_params_t* p, const void* K, const void* V, const int32_t* len, const void* k_new,
+                             const void* v_new, const void* workspace, size_t workspace_bytes_) {
+  if (!params_ok(p) || !K || !V || !len || !k_new || !v_new || !workspace) return CAOTE_ERR_INVALID_ARG;
+  if (!params_supported(p)) return CAOTE_ERR_UNSUPPORTED;
+  if (workspace_bytes_ < kHeaderBytes || !aligned(workspace, 256)) return CAOTE_ERR_INVALID_ARG;
+  if (!aligned(K, 16) || !aligned(V, 16) || !aligned(k_new, 16) || !aligned(v_new, 16)) return CAOTE_ERR_INVALID_ARG;
+  return CAOTE_OK;
+}
+static int score_args_check(const caote_params_t* p, const void* q, const void* K, const void* V, const int32_t* len,
+                            const float* base, const float* o, const float* scores) {
+  if (!params_ok(p) || !q || !K || !V || !len || !o || !scores) return CAOTE_ERR_INVALID_ARG;
+  if (!params_supported(p)) return CAOTE_ERR_UNSUPPORTED;
+  if ((p->base_mode == CAOTE_BASE_ACCUM || p->base_mode == CAOTE_BASE_EXTERNAL) && !base)
+    return CAOTE_ERR_INVALID_ARG;
+  if (!aligned(q, 16) || !aligned(K, 16) || !aligned(V, 16) || !aligned(o, 16)) return CAOTE_ERR_INVALID_ARG;
+  return CAOTE_OK;
+}
+static int score_workspace_check(const caote_params_t* p, const void* workspace, size_t workspace_bytes_) {
+  if (!workspace || workspace_bytes_ < workspace_bytes(p) || !aligned(workspace, 256)) return CAOTE_ERR_INVALID_ARG;
+  return CAOTE_OK;
+}
+
 size_t caote_workspace_bytes(const caote_params_t* params) {
   if (!params_ok(params) || !params_supported(params)) return 0;
   return workspace_bytes(params);
@@ -425,11 +448,9 @@ size_t caote_workspace_bytes(const caote_params_t* params) {
 int caote_append(const caote_params_t* p, void* K, void* V, float* base, int32_t* pos, int32_t* len,
                  int32_t* n_seen, const void* k_new, const void* v_new, void* workspace,
                  size_t workspace_bytes_, caote_stream_t stream) {
-  if (!params_ok(p) || !K || !V || !len || !k_new || !v_new || !workspace) return CAOTE_ERR_INVALID_ARG;
-  if (!params_supported(p)) return CAOTE_ERR_UNSUPPORTED;
-  if (workspace_bytes_ < kHeaderBytes || !aligned(workspace, 256)) return CAOTE_ERR_INVALID_ARG;
-  if (!aligned(K, 16) || !aligned(V, 16) || !aligned(k_new, 16) || !aligned(v_new, 16)) return CAOTE_ERR_INVALID_ARG;
-  int rc = check_device();
+  int rc = append_args_check(p, K, V, len, k_new, v_new, workspace, workspace_bytes_);
+  if (rc) return rc;
+  rc = check_device();
   if (rc) return rc;
   const Dims dm = make_dims(p);
   const int row_bytes = dm.D * (p->dtype == CAOTE_BF16 ? 2 : 4);
@@ -444,13 +465,9 @@ int caote_append(const caote_params_t* p, void* K, void* V, float* base, int32_t
 static int score_impl(const caote_params_t* p, const void* q, const void* K, const void* V, const int32_t* len,
                       float* base, const float* vsum, float* o, float* scores, void* workspace, size_t workspace_bytes_,
                       caote_stream_t stream) {
-  if (!params_ok(p) || !q || !K || !V || !len || !o || !scores || !workspace) return CAOTE_ERR_INVALID_ARG;
-  if (!params_supported(p)) return CAOTE_ERR_UNSUPPORTED;
-  if ((p->base_mode == CAOTE_BASE_ACCUM || p->base_mode == CAOTE_BASE_EXTERNAL) && !base)
-    return CAOTE_ERR_INVALID_ARG;
-  if (workspace_bytes_ < workspace_bytes(p) || !aligned(workspace, 256)) return CAOTE_ERR_INVALID_ARG;
-  if (!aligned(q, 16) || !aligned(K, 16) || !aligned(V, 16) || !aligned(o, 16)) return CAOTE_ERR_INVALID_ARG;
-  int rc = check_device();
+  int rc = score_args_check(p, q, K, V, len, base, o, scores);
+  if (!rc) rc = score_workspace_check(p, workspace, workspace_bytes_);
+  if (!rc) rc = check_device();
   if (rc) return rc;
   const Dims dm = make_dims(p);
   cudaStream_t st = (cudaStream_t)stream;
@@ -524,10 +541,11 @@ int caote_vsum(const caote_params_t* p, const void* V, const int32_t* len, float
 
 int caote_score_static(const caote_params_t* p, const void* q, const void* K, const void* V, const int32_t* len,
                        float* base, float* o, float* scores, int32_t* status_out, caote_stream_t stream) {
-  if (!params_ok(p)) return CAOTE_ERR_INVALID_ARG;
-  if (!params_supported(p)) return CAOTE_ERR_UNSUPPORTED;
+  // everything caote_score would refuse is refused here, before anything touches the stream or the array
+  int rc = score_args_check(p, q, K, V, len, base, o, scores);
+  if (rc) return rc;
   if (workspace_bytes(p) > kStaticScratchBytes) return CAOTE_ERR_TOO_LARGE;
-  int rc = check_device();
+  rc = check_device();
   if (rc) return rc;
   char* scratch = nullptr;
   rc = static_scratch_address(&scratch);  // first call on this device: looks the address up
@@ -587,11 +605,17 @@ static int step_impl(const caote_params_t* p, const void* q, const void* k_new, 
                      float* base, int32_t* pos, int32_t* len, int32_t* n_seen, const int32_t* budget, float* vsum,
                      float* o, float* scores, int32_t* evict_idx, int32_t max_evict, int32_t* n_evict,
                      int32_t compact_mode, void* workspace, size_t workspace_bytes_, caote_stream_t stream) {
-  int rc;
-  const bool bf16 = params_ok(p) && p->dtype == CAOTE_BF16;
+  // every host-visible check of the calls below runs before the first launch
+  int rc = score_args_check(p, q, K, V, len, base, o, scores);
+  if (!rc) rc = score_workspace_check(p, workspace, workspace_bytes_);
+  if (!rc && (k_new || v_new)) rc = append_args_check(p, K, V, len, k_new, v_new, workspace, workspace_bytes_);
+  if (!rc && (!budget || !evict_idx || !n_evict || max_evict < 1)) rc = CAOTE_ERR_INVALID_ARG;
+  if (!rc && compact_mode != CAOTE_COMPACT_FILL && compact_mode != CAOTE_COMPACT_STABLE) rc = CAOTE_ERR_INVALID_ARG;
+  if (!rc) rc = check_device();
+  if (rc) return rc;
+  const bool bf16 = p->dtype == CAOTE_BF16;
   if (k_new || v_new) {
     if (vsum) {
-      if (!params_ok(p) || !v_new || !len) return CAOTE_ERR_INVALID_ARG;
       const Dims dm = make_dims(p);
       cudaStream_t st = (cudaStream_t)stream;
       if (bf16) {

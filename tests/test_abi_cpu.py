@@ -100,6 +100,27 @@ def test_host_side_argument_checks_return_before_any_launch():
     assert lib.caote_post_evict_output(bp, fake, fake, fake, fake, None, 4, fake, fake, fake, None) == C.ERR_INVALID_ARG
     assert lib.caote_post_evict_output(bp, fake, fake, fake, fake, fake, 0, fake, fake, fake, None) == C.ERR_INVALID_ARG
     assert lib.caote_post_evict_output(bp, fake, fake, fake, fake, fake, 4, fake, fake, None, None) == C.ERR_INVALID_ARG
+    # the whole-step entry points validate append, score and selection arguments before their first launch
+    # (the FastCAOTE step would otherwise have added the new rows to the running sum already)
+    okp = C.make_params(1, 4, 2, 64, 32, 1, torch.float32, 0.125, "last_query")
+    okb, okneed = ctypes.byref(okp), C.caote_workspace_bytes(okp)
+    for bad_K in (None, ctypes.c_void_p(4100)):
+        assert lib.caote_step_fast(okb, fake, fake, fake, bad_K, fake, None, fake, fake, fake, fake, fake, fake, fake, fake,
+                                   1, fake, 0, ws, okneed, None) == C.ERR_INVALID_ARG
+        assert lib.caote_step(okb, fake, fake, fake, bad_K, fake, None, fake, fake, fake, fake, fake, fake, fake, 1, fake,
+                              0, ws, okneed, None) == C.ERR_INVALID_ARG
+    assert lib.caote_step_fast(okb, fake, fake, fake, fake, fake, None, fake, fake, fake, fake, fake, fake, fake, fake, 1,
+                               fake, 0, ws, okneed - 1, None) == C.ERR_INVALID_ARG          # workspace too small
+    assert lib.caote_step_fast(okb, fake, fake, fake, fake, fake, None, fake, fake, fake, None, fake, fake, fake, fake, 1,
+                               fake, 0, ws, okneed, None) == C.ERR_INVALID_ARG              # no budget
+    assert lib.caote_step_fast(ctypes.byref(p96), fake, fake, fake, fake, fake, None, fake, fake, fake, fake, fake, fake,
+                               fake, fake, 1, fake, 0, ws, 1 << 20, None) == C.ERR_UNSUPPORTED
+    # the no-allocation variant refuses what caote_score refuses, before it touches its built-in array
+    assert lib.caote_score_static(okb, None, fake, fake, fake, None, fake, fake, None, None) == C.ERR_INVALID_ARG
+    assert lib.caote_score_static(okb, fake, ctypes.c_void_p(4100), fake, fake, None, fake, fake, None, None) == C.ERR_INVALID_ARG
+    assert lib.caote_score_static(bp, fake, fake, fake, fake, None, fake, fake, None, None) == C.ERR_INVALID_ARG  # accum, no base
+    big = C.make_params(64, 28, 4, 128, 8196, 1, torch.bfloat16, 0.1, "accum")
+    assert lib.caote_score_static(ctypes.byref(big), fake, fake, fake, fake, fake, fake, fake, None, None) == C.ERR_TOO_LARGE
     assert C.caote_launch_count() == before
 
 
