@@ -276,6 +276,19 @@ typedef struct {
 CAOTE_API int caote_trace_enable(int on);
 CAOTE_API int caote_trace_collect(caote_trace_entry_t* out, int32_t max_entries, int32_t* n_out);
 
+/* Process-wide settings, for tests and tuning runs. (The paper has no counterpart.)
+ *   CAOTE_OPT_WAIT_CYCLES     clock cycles after which a device-side wait of the single-query cluster kernel
+ *                             gives up (default 2e9, about a second). The kernel then records
+ *                             CAOTE_ERR_TIMEOUT in the status word and still returns; its outputs are
+ *                             undefined, the caches and the workspace stay usable. value >= 1.
+ *   CAOTE_OPT_DECODE_CLUSTER  CTAs per thread-block cluster on the single-query path: 0 = chosen from the
+ *                             shape (default), 1..16 = forced (shapes it cannot serve take the next path),
+ *                             -1 = do not use the cluster kernel.
+ * Takes effect for launches made after the call. Returns CAOTE_ERR_INVALID_ARG for an unknown option or a
+ * value out of range. */
+typedef enum { CAOTE_OPT_WAIT_CYCLES = 1, CAOTE_OPT_DECODE_CLUSTER = 2 } caote_option_t;
+CAOTE_API int caote_set_option(int32_t option, int64_t value);
+
 /* Number of kernels this library has launched from this process since it was loaded. */
 CAOTE_API int64_t caote_launch_count(void);
 

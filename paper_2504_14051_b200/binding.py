@@ -108,6 +108,8 @@ def lib() -> ctypes.CDLL:
     L.caote_trace_collect.argtypes = [ctypes.POINTER(TraceEntry), i32, ctypes.POINTER(ctypes.c_int32)]
     L.caote_launch_count.restype = ctypes.c_int64
     L.caote_launch_count.argtypes = []
+    L.caote_set_option.restype = ctypes.c_int
+    L.caote_set_option.argtypes = [ctypes.c_int32, ctypes.c_int64]
     _lib = L
     return L
 
@@ -249,6 +251,13 @@ def caote_trace_collect(max_entries: int = 32) -> dict:
     n = ctypes.c_int32(0)
     _check("caote_trace_collect", lib().caote_trace_collect(buf, max_entries, ctypes.byref(n)))
     return {buf[i].name.decode(): (int(buf[i].launches), float(buf[i].total_ms)) for i in range(n.value)}
+
+
+OPT_WAIT_CYCLES, OPT_DECODE_CLUSTER = 1, 2
+
+
+def caote_set_option(option: int, value: int) -> None:
+    _check("caote_set_option", lib().caote_set_option(int(option), int(value)))
 
 
 def caote_launch_count() -> int:

@@ -7,6 +7,7 @@
 #include <vector>
 
 #include "common.cuh"
+#include "decode_cluster.cuh"
 #include "decode_tc.cuh"
 #include "generic_score.cuh"
 #include "post_evict.cuh"
@@ -16,6 +17,8 @@
 namespace caote {
 
 static std::atomic<long long> g_launches{0};
+static std::atomic<long long> g_wait_cycles{2000000000LL};  // CAOTE_OPT_WAIT_CYCLES
+static std::atomic<int> g_decode_cluster{0};                // CAOTE_OPT_DECODE_CLUSTER: 0 auto, -1 off, else the size
 static thread_local char g_cuda_error[256] = "";
 
 static int cuda_fail(cudaError_t e, const char* what) {
@@ -234,6 +237,123 @@ static bool decode_shape_ok(const caote_params_t* p) {
   return p->dtype == CAOTE_BF16 && p->head_dim == 128 && p->n_new == 1 && G <= 8 &&
          !(carried && (G > 7 || p->capacity % 4 != 0)) &&
          (long long)p->batch * p->n_kv_heads * p->capacity < (1LL << 31);
+}
+
+// ---- single-query path on thread-block clusters ---------------------------------------------------------
+// Clusters of `c` CTAs of the cluster kernel that can be resident on the current device at once; 0 if none.
+static int cluster_capacity(int c) {
+  static std::atomic<int> cached[64][dcl::kMaxC + 1];
+  int dev = 0;
+  if (c < 1 || c > dcl::kMaxC || cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+  int n = cached[dev][c].load(std::memory_order_acquire);
+  if (n == 0) {
+    const size_t smem = dcl::smem_bytes();
+    n = -1;
+    if (cudaFuncSetAttribute(dcl::decode_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) == cudaSuccess &&
+        cudaFuncSetAttribute(dcl::decode_cluster_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3((unsigned)c * 64u);
+      cfg.blockDim = dim3(dcl::kThreads);
+      cfg.dynamicSmemBytes = smem;
+      cudaLaunchAttribute at[1];
+      at[0].id = cudaLaunchAttributeClusterDimension;
+      at[0].val.clusterDim.x = (unsigned)c;
+      at[0].val.clusterDim.y = 1;
+      at[0].val.clusterDim.z = 1;
+      cfg.attrs = at;
+      cfg.numAttrs = 1;
+      int got = 0;
+      if (cudaOccupancyMaxActiveClusters(&got, dcl::decode_cluster_kernel, &cfg) == cudaSuccess && got > 0) n = got;
+    }
+    (void)cudaGetLastError();
+    cached[dev][c].store(n, std::memory_order_release);
+  }
+  return n > 0 ? n : 0;
+}
+
+// Cluster size for these dimensions: every CTA must be able to keep its share of a full unit (kMaxT
+// tiles), and among the sizes that can, the one with the smallest estimate of rounds x (tiles per CTA +
+// a fixed cost per unit for the merge) wins. 0: no size fits (the unit is too long, or no cluster can run).
+static int choose_cluster(const Dims& dm, int* clusters_out) {
+  const int cap_tiles = (dm.cap + decode::kT - 1) / decode::kT;
+  const int forced = g_decode_cluster.load(std::memory_order_relaxed);
+  if (forced < 0) return 0;
+  int best = 0, best_n = 0;
+  double best_cost = 0.0;
+  for (int c = 1; c <= dcl::kMaxC; ++c) {
+    if (forced > 0 && c != forced) continue;
+    if ((cap_tiles + c - 1) / c > dcl::kMaxT) continue;
+    const int n = cluster_capacity(c);
+    if (n <= 0) continue;
+    const long long rounds = ((long long)dm.units + n - 1) / n;
+    const double cost = (double)rounds * ((double)cap_tiles / c + 2.0 + 0.05 * c);
+    if (best == 0 || cost < best_cost) {
+      best = c;
+      best_n = n;
+      best_cost = cost;
+    }
+  }
+  *clusters_out = best_n;
+  return best;
+}
+
+static int encode_decode_maps(const Dims& dm, const void* q, const void* K, const void* V, unsigned q_rows,
+                              CUtensorMap* tmK, CUtensorMap* tmV, CUtensorMap* tmQ, TensorMapEncodeFn encode) {
+  const cuuint64_t gdim[2] = {(cuuint64_t)dm.D, (cuuint64_t)dm.units * (cuuint64_t)dm.cap};
+  const cuuint64_t gstride[1] = {(cuuint64_t)dm.D * 2};
+  const cuuint32_t box[2] = {64, (cuuint32_t)decode::kT};
+  const cuuint32_t estride[2] = {1, 1};
+  for (int i = 0; i < 3; ++i) {
+    // K, V: boxes of 64 channels x 128 tokens; q: 64 channels x q_rows rows (a unit's heads, padded by its
+    // neighbours' or by zeros)
+    const cuuint64_t qdim[2] = {(cuuint64_t)dm.D, (cuuint64_t)dm.B * (cuuint64_t)dm.Hq};
+    const cuuint32_t qbox[2] = {64, q_rows};
+    CUresult r = encode(i == 0 ? tmK : (i == 1 ? tmV : tmQ), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+                        const_cast<void*>(i == 0 ? K : (i == 1 ? V : q)), i < 2 ? gdim : qdim, gstride, i < 2 ? box : qbox,
+                        estride, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+      snprintf(g_cuda_error, sizeof(g_cuda_error), "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+      return CAOTE_ERR_CUDA;
+    }
+  }
+  return CAOTE_OK;
+}
+
+static int launch_decode_cluster(const Dims& dm, const void* q, const void* K, const void* V, const int* len,
+                                 float* base, float* o, float* scores, char* ws, cudaStream_t st, bool* used) {
+  *used = false;
+  TensorMapEncodeFn encode = tensor_map_encoder();
+  const bool carried = dm.base_mode == CAOTE_BASE_ACCUM || dm.base_mode == CAOTE_BASE_EXTERNAL;
+  if (!encode || (carried && !aligned(base, 16)) || !aligned(q, 16)) return CAOTE_OK;
+  int clusters = 0;
+  const int c = choose_cluster(dm, &clusters);
+  if (c == 0) return CAOTE_OK;
+  CUtensorMap tmK, tmV, tmQ;
+  int rc = encode_decode_maps(dm, q, K, V, 8, &tmK, &tmV, &tmQ, encode);
+  if (rc) return rc;
+  if (clusters > dm.units) clusters = dm.units;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(clusters * c));
+  cfg.blockDim = dim3(dcl::kThreads);
+  cfg.dynamicSmemBytes = dcl::smem_bytes();
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = (unsigned)c;
+  at[0].val.clusterDim.y = 1;
+  at[0].val.clusterDim.z = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  int* status = reinterpret_cast<int*>(ws);
+  const long long wait_cycles = g_wait_cycles.load(std::memory_order_relaxed);
+  CAOTE_LAUNCH("decode_cluster_kernel", st, {
+    cudaError_t e = cudaLaunchKernelEx(&cfg, dcl::decode_cluster_kernel, tmK, tmV, tmQ, dm, len, base, o, scores, status,
+                                       wait_cycles);
+    if (e != cudaSuccess) return cuda_fail(e, "decode_cluster_kernel");
+  });
+  *used = true;
+  return CAOTE_OK;
 }
 
 static int launch_decode_score(const Dims& dm, const void* q, const void* K, const void* V, const int* len,
@@ -474,6 +594,10 @@ static int score_impl(const caote_params_t* p, const void* q, const void* K, con
   char* ws = (char*)workspace;
   if (decode_shape_ok(p)) {
     bool used = false;
+    if (!vsum) {
+      rc = launch_decode_cluster(dm, q, K, V, len, base, o, scores, ws, st, &used);
+      if (rc || used) return rc;
+    }
     rc = launch_decode_score(dm, q, K, V, len, base, o, scores, ws, st, &used, vsum);
     if (rc || used) return rc;
   }
@@ -760,6 +884,21 @@ int caote_trace_collect(caote_trace_entry_t* out, int32_t max_entries, int32_t* 
   }
   *n_out = n;
   return rc;
+}
+
+int caote_set_option(int32_t option, int64_t value) {
+  switch (option) {
+    case CAOTE_OPT_WAIT_CYCLES:
+      if (value < 1) return CAOTE_ERR_INVALID_ARG;
+      g_wait_cycles.store((long long)value, std::memory_order_relaxed);
+      return CAOTE_OK;
+    case CAOTE_OPT_DECODE_CLUSTER:
+      if (value < -1 || value > dcl::kMaxC) return CAOTE_ERR_INVALID_ARG;
+      g_decode_cluster.store((int)value, std::memory_order_relaxed);
+      return CAOTE_OK;
+    default:
+      return CAOTE_ERR_INVALID_ARG;
+  }
 }
 
 int64_t caote_launch_count(void) { return (int64_t)g_launches.load(std::memory_order_relaxed); }
