@@ -240,8 +240,30 @@ static bool decode_shape_ok(const caote_params_t* p) {
 }
 
 // ---- single-query path on thread-block clusters ---------------------------------------------------------
+typedef void (*ClusterKernel)(const CUtensorMap, const CUtensorMap, const CUtensorMap, Dims, const int*, float*, float*,
+                              float*, int*, long long);
+template <int kMode>
+static ClusterKernel cluster_kernel_for_g(int g) {
+  switch (g) {
+    case 1: return dcl::decode_cluster_kernel<1, kMode>;
+    case 2: return dcl::decode_cluster_kernel<2, kMode>;
+    case 3: return dcl::decode_cluster_kernel<3, kMode>;
+    case 4: return dcl::decode_cluster_kernel<4, kMode>;
+    case 5: return dcl::decode_cluster_kernel<5, kMode>;
+    case 6: return dcl::decode_cluster_kernel<6, kMode>;
+    case 7: return dcl::decode_cluster_kernel<7, kMode>;
+    default: return dcl::decode_cluster_kernel<8, kMode>;
+  }
+}
+// The instantiation for a group size and a base mode (LAST_QUERY and CHUNK_SUM coincide for one query).
+static ClusterKernel cluster_kernel(int g, int base_mode) {
+  if (base_mode == CAOTE_BASE_ACCUM) return cluster_kernel_for_g<CAOTE_BASE_ACCUM>(g > 7 ? 7 : g);
+  if (base_mode == CAOTE_BASE_EXTERNAL) return cluster_kernel_for_g<CAOTE_BASE_EXTERNAL>(g > 7 ? 7 : g);
+  return cluster_kernel_for_g<CAOTE_BASE_LAST_QUERY>(g);
+}
+
 // Clusters of `c` CTAs of the cluster kernel that can be resident on the current device at once; 0 if none.
-static int cluster_capacity(int c) {
+static int cluster_capacity(int c, ClusterKernel kernel) {
   static std::atomic<int> cached[64][dcl::kMaxC + 1];
   int dev = 0;
   if (c < 1 || c > dcl::kMaxC || cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
@@ -249,8 +271,8 @@ static int cluster_capacity(int c) {
   if (n == 0) {
     const size_t smem = dcl::smem_bytes();
     n = -1;
-    if (cudaFuncSetAttribute(dcl::decode_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) == cudaSuccess &&
-        cudaFuncSetAttribute(dcl::decode_cluster_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) == cudaSuccess &&
+        cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
       cudaLaunchConfig_t cfg = {};
       cfg.gridDim = dim3((unsigned)c * 64u);
       cfg.blockDim = dim3(dcl::kThreads);
@@ -263,7 +285,7 @@ static int cluster_capacity(int c) {
       cfg.attrs = at;
       cfg.numAttrs = 1;
       int got = 0;
-      if (cudaOccupancyMaxActiveClusters(&got, dcl::decode_cluster_kernel, &cfg) == cudaSuccess && got > 0) n = got;
+      if (cudaOccupancyMaxActiveClusters(&got, kernel, &cfg) == cudaSuccess && got > 0) n = got;
     }
     (void)cudaGetLastError();
     cached[dev][c].store(n, std::memory_order_release);
@@ -274,7 +296,7 @@ static int cluster_capacity(int c) {
 // Cluster size for these dimensions: every CTA must be able to keep its share of a full unit (kMaxT
 // tiles), and among the sizes that can, the one with the smallest estimate of rounds x (tiles per CTA +
 // a fixed cost per unit for the merge) wins. 0: no size fits (the unit is too long, or no cluster can run).
-static int choose_cluster(const Dims& dm, int* clusters_out) {
+static int choose_cluster(const Dims& dm, ClusterKernel kernel, int* clusters_out) {
   const int cap_tiles = (dm.cap + decode::kT - 1) / decode::kT;
   const int forced = g_decode_cluster.load(std::memory_order_relaxed);
   if (forced < 0) return 0;
@@ -283,7 +305,7 @@ static int choose_cluster(const Dims& dm, int* clusters_out) {
   for (int c = 1; c <= dcl::kMaxC; ++c) {
     if (forced > 0 && c != forced) continue;
     if ((cap_tiles + c - 1) / c > dcl::kMaxT) continue;
-    const int n = cluster_capacity(c);
+    const int n = cluster_capacity(c, kernel);
     if (n <= 0) continue;
     const long long rounds = ((long long)dm.units + n - 1) / n;
     const double cost = (double)rounds * ((double)cap_tiles / c + 2.0 + 0.05 * c);
@@ -326,8 +348,24 @@ static int launch_decode_cluster(const Dims& dm, const void* q, const void* K, c
   TensorMapEncodeFn encode = tensor_map_encoder();
   const bool carried = dm.base_mode == CAOTE_BASE_ACCUM || dm.base_mode == CAOTE_BASE_EXTERNAL;
   if (!encode || (carried && !aligned(base, 16)) || !aligned(q, 16)) return CAOTE_OK;
+  const ClusterKernel kernel = cluster_kernel(dm.G, dm.base_mode);
+  // (the attributes below are per function: every instantiation gets them the first time it is used)
+  static std::mutex attr_mu;
+  static std::vector<std::pair<int, ClusterKernel>> attr_done;
+  {
+    int dev = 0;
+    CAOTE_CUDA(cudaGetDevice(&dev));
+    std::lock_guard<std::mutex> lk(attr_mu);
+    bool done = false;
+    for (auto& e : attr_done) done |= (e.first == dev && e.second == kernel);
+    if (!done) {
+      CAOTE_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dcl::smem_bytes()));
+      CAOTE_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+      attr_done.push_back({dev, kernel});
+    }
+  }
   int clusters = 0;
-  const int c = choose_cluster(dm, &clusters);
+  const int c = choose_cluster(dm, kernel, &clusters);
   if (c == 0) return CAOTE_OK;
   CUtensorMap tmK, tmV, tmQ;
   int rc = encode_decode_maps(dm, q, K, V, 8, &tmK, &tmV, &tmQ, encode);
@@ -348,7 +386,7 @@ static int launch_decode_cluster(const Dims& dm, const void* q, const void* K, c
   int* status = reinterpret_cast<int*>(ws);
   const long long wait_cycles = g_wait_cycles.load(std::memory_order_relaxed);
   CAOTE_LAUNCH("decode_cluster_kernel", st, {
-    cudaError_t e = cudaLaunchKernelEx(&cfg, dcl::decode_cluster_kernel, tmK, tmV, tmQ, dm, len, base, o, scores, status,
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, tmK, tmV, tmQ, dm, len, base, o, scores, status,
                                        wait_cycles);
     if (e != cudaSuccess) return cuda_fail(e, "decode_cluster_kernel");
   });

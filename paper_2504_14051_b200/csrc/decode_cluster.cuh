@@ -258,6 +258,9 @@ struct Sched {
   }
 };
 
+// kG: query heads per KV head; kMode: the base mode. Compile-time so that the per-head loops carry no
+// predicates and the paths of the other modes are not in the instruction stream.
+template <int kG, int kMode>
 __global__ void __launch_bounds__(kThreads, 1)
 decode_cluster_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                       const __grid_constant__ CUtensorMap tmQ, Dims dm, const int* __restrict__ len,
@@ -297,9 +300,9 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
   float* xword = reinterpret_cast<float*>(tmem_slot + 1);              // where the peers' "done reading" words land
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int G = dm.G, mode = dm.base_mode;
-  const bool use_base = (mode == CAOTE_BASE_ACCUM || mode == CAOTE_BASE_EXTERNAL);
-  const bool counted = (mode != CAOTE_BASE_EXTERNAL);
+  constexpr int G = kG, mode = kMode;
+  constexpr bool use_base = (mode == CAOTE_BASE_ACCUM || mode == CAOTE_BASE_EXTERNAL);
+  constexpr bool counted = (mode != CAOTE_BASE_EXTERNAL);
   const float scale2 = dm.scale * 1.4426950408889634f;
 
   Sched sch;
