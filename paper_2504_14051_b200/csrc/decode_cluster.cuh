@@ -25,10 +25,11 @@
 // other tokens' numerators) and every other token's complement is 1 - alpha with alpha <= 1/2; the
 // carried base scores are treated the same way. The heads' complements, all non-negative, are added.
 //
-// Warp roles (512 threads): warps 0..3 softmax group, warps 4..7 and 8..11 two keeper groups that take
-// the CTA's tiles in turn (thread = token = TMEM lane in all three); one lane each of warps 12..15 issues
-// the K copies, the V copies, the S^T products and the O^T products. Three token warps per scheduler: a
-// single warp cannot hide the latency of its own instruction stream.
+// Warp roles (512 threads): warps 0..3 softmax group, then kNB = 2 keeper groups of four warps that take the
+// CTA's tiles in turn (thread = token = TMEM lane in all of them); one lane each of the last four warps
+// issues the K copies, the V copies, the S^T products and the O^T products. Several token warps per
+// scheduler: a single warp cannot hide the latency of its own instruction stream. (Three keeper groups at
+// 96 registers per thread were slower: 246 us against 218 us on the batched 8k-token decode workload.)
 //
 // Flow control between units. Buffers that peers write (records, X) are reused every unit. A record of
 // unit u + 1 is pushed only after this CTA has seen round 2 of unit u complete, and round 2 includes a
@@ -76,9 +77,10 @@ constexpr int kStash = 7;                 // value tiles a CTA keeps in TMEM
 constexpr int kMaxT = 9;                  // tiles of one unit per CTA: the stash + 2 held in the V ring
 constexpr int kMaxC = 16;                 // largest cluster
 constexpr int kGroup = 128;               // threads of a token group
-constexpr int kThreads = 3 * kGroup + 128;  // softmax group, two keeper groups, four single-lane warps
-constexpr int kWarpK = 12, kWarpV = 13, kWarpQK = 14, kWarpPV = 15;
-constexpr int kMaxKeep = (kMaxT + 1) / 2;   // tiles of one unit per keeper group
+constexpr int kNB = 2;                    // keeper groups
+constexpr int kThreads = (1 + kNB) * kGroup + 128;  // softmax group, keeper groups, four single-lane warps
+constexpr int kWarpK = 4 * (1 + kNB), kWarpV = kWarpK + 1, kWarpQK = kWarpK + 2, kWarpPV = kWarpK + 3;
+constexpr int kMaxKeep = (kMaxT + kNB - 1) / kNB;   // tiles of one unit per keeper group
 constexpr int kQBufBytes = 2048;          // 8 query rows x 128 channels as two 64-channel boxes
 constexpr int kPBytes = 4096;             // 16 rows x 128 tokens as two 64-token boxes
 constexpr int kStatFloats = 36;           // per CTA: ref[8] lrest[8] pmax[8] smax[8] brest bmax pad pad
@@ -101,8 +103,8 @@ struct Fin {        // per unit, every CTA computes its own copy
 
 inline size_t smem_bytes() {
   return 1024 + (size_t)(kKS + kVS) * kTileBytes + 2 * kQBufBytes + kPBytes + kVS * (kT * 4) +
-         kMaxC * kStatFloats * 4 + kXoFloats * 4 + 2 * kD * 4 + 2 * sizeof(Fin) + 2 * kMaxC * 8 * 4 /* fac */ +
-         2 * 32 * 4 /* red */ + 4 * 28 * 4 /* gred */ + kStatFloats * 4 /* mystat */ + kLenTab * 4 + 40 * 8 /* barriers */ + 64;
+         kMaxC * kStatFloats * 4 + kXoFloats * 4 + 2 * kD * 4 + kNB * sizeof(Fin) + kNB * kMaxC * 8 * 4 /* fac */ +
+         2 * 32 * 4 /* red */ + 4 * 28 * 4 /* gred */ + kStatFloats * 4 /* mystat */ + kLenTab * 4 + 64 * 8 /* barriers, control words */ + 64;
 }
 
 // ---- cluster PTX ------------------------------------------------------------------------------------
@@ -276,9 +278,9 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
   float* xstats = baseV + kVS * kT;                                    // [C][kStatFloats]    written by the peers
   float* xo = xstats + kMaxC * kStatFloats;                            // [C][slice][8]       written by the peers
   float* xnX = xo + kXoFloats;                                         // [2][kD]  -X         written by the owners
-  Fin* fins = reinterpret_cast<Fin*>(xnX + 2 * kD);                    // [2] one copy per keeper group
-  float* facs = reinterpret_cast<float*>(fins + 2);                    // [2][C][8] 2^(ref_c - m) / l per record and head
-  float* red = facs + 2 * kMaxC * 8;                                       // [2][4][8] warp maxima of the softmax group
+  Fin* fins = reinterpret_cast<Fin*>(xnX + 2 * kD);                    // [kNB] one copy per keeper group
+  float* facs = reinterpret_cast<float*>(fins + kNB);                  // [kNB][C][8] 2^(ref_c - m) / l per record and head
+  float* red = facs + kNB * kMaxC * 8;                                       // [2][4][8] warp maxima of the softmax group
   float* gred = red + 2 * 32;                                          // [4 warps][28] closing sums of the softmax group
   float* mystat = gred + 4 * 28;                                       // [kStatFloats] this CTA's record
   int* slen = reinterpret_cast<int*>(mystat + kStatFloats);            // [kLenTab]
@@ -320,7 +322,7 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
   const int slice = (kD + C - 1) / C;                                   // channels per owner
   const int my_ch0 = min(rank * slice, kD), my_nch = min(slice, kD - my_ch0);
   const uint32_t r1_bytes = (uint32_t)(C * (kStatFloats * 4 + 8 * my_nch * 4));
-  const uint32_t r2_bytes = (uint32_t)(kD * 4 + 2 * C * 4);
+  const uint32_t r2_bytes = (uint32_t)(kD * 4 + kNB * C * 4);
 
   if (tid == 0) {
     for (int i = 0; i < kKS; ++i) { mbar_init(&kfull[i], 1); mbar_init(&kempty[i], 1); }
@@ -711,9 +713,9 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
     }
   } else {
     // ================================ keeper groups (thread = token of the tile) ================================
-    // Group bg takes the CTA's tiles j with (j & 1) == bg: it keeps their logits and value rows during the
+    // Group bg takes the CTA's tiles j with j % kNB == bg: it keeps their logits and value rows during the
     // attention pass and scores them after the merge. Both groups finish the softmax statistics for
-    // themselves (no hand-over between them); the owner's channels are split between them by parity.
+    // themselves (no hand-over between them); the owner's channels are dealt to them in turn.
     const int bg = (warp >> 2) - 1, gw = warp & 3;
     const int tok = tid & (kGroup - 1);
     const uint32_t lane_base = (uint32_t)(32 * gw) << 16;
@@ -731,8 +733,8 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
 
       // ===================== attention pass: keep logits and value rows =====================
 #pragma unroll 1
-      for (int jj = 0; 2 * jj + bg < w.T; ++jj) {
-        const int j = 2 * jj + bg, tj = ti + j;
+      for (int jj = 0; kNB * jj + bg < w.T; ++jj) {
+        const int j = kNB * jj + bg, tj = ti + j;
         const int t = w.t0 + j;
         const int n_valid = min(kT, w.n - t * kT);
         const int vs = tj % kVS, sb = tj % kSB;
@@ -748,12 +750,13 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
         for (int hd = 0; hd < 8; ++hd) sv[hd] = (valid && hd < G) ? sv[hd] * scale2 : -INFINITY;
         wait_bounded(&vfull[vs], (tj / kVS) & 1, &ctl[0], status, wait_cycles, false);
         const float bval = (use_base && valid) ? baseV[vs * kT + tok] : 0.f;
-        switch (jj) {  // (static indices keep the arrays in registers; jj is uniform over the group)
-#define CAOTE_KEEP(q) case q: { _Pragma("unroll") for (int hd = 0; hd < 8; ++hd) keep[q][hd] = sv[hd]; keepb[q] = bval; } break;
-          CAOTE_KEEP(0) CAOTE_KEEP(1) CAOTE_KEEP(2) CAOTE_KEEP(3)
-          default: { _Pragma("unroll") for (int hd = 0; hd < 8; ++hd) keep[kMaxKeep - 1][hd] = sv[hd]; keepb[kMaxKeep - 1] = bval; } break;
-#undef CAOTE_KEEP
-        }
+#pragma unroll
+        for (int q = 0; q < kMaxKeep; ++q)  // (static indices keep the arrays in registers)
+          if (q == jj) {
+#pragma unroll
+            for (int hd = 0; hd < 8; ++hd) keep[q][hd] = sv[hd];
+            keepb[q] = bval;
+          }
         if (j < kStash) {
           const char* vt = tilesV + vs * kTileBytes;
 #pragma unroll
@@ -830,9 +833,9 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
         const float inv_H = (fin->Htot > 0.f) ? 1.f / fin->Htot : 0.f;
         float* xdst = xnX + (mu & 1) * kD;
         const int r = tok & 7;
-        const int nq = (my_nch - bg + 1) / 2;  // channels of this group's parity
+        const int nq = (my_nch - bg + kNB - 1) / kNB;  // channels dealt to this group
         for (int q0 = 0; q0 < nq; q0 += kGroup / 8) {
-          const int cl = 2 * (q0 + (tok >> 3)) + bg;
+          const int cl = kNB * (q0 + (tok >> 3)) + bg;
           const bool act = cl < my_nch;
           float v0 = 0.f, v1 = 0.f;
           if (act) {
@@ -857,7 +860,7 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
         }
       }
       group_sync(1 + bg);  // every thread of this group is done with the records: tell the peers
-      if (tok < C) push_f32(map_to_rank(smem_u32(xword + 2 * rank + bg), tok), 0.f, map_to_rank(smem_u32(r2), tok));
+      if (tok < C) push_f32(map_to_rank(smem_u32(xword + kNB * rank + bg), tok), 0.f, map_to_rank(smem_u32(r2), tok));
       wait_bounded(r2, mu & 1, &ctl[0], status, wait_cycles, false);
       if (bg == 0 && tok == 0) {
         // the next unit's merge: what the peers will push into this CTA
@@ -869,23 +872,24 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
       {
         const float Htot = fin->Htot, hbsum = fin->hbsum, fbmax = fin->bmax, fbrest = fin->brest;
         const float* nX = xnX + (mu & 1) * kD;
-        const int mine = (w.T + 1 - bg) / 2;                             // tiles this group kept
-        const int first_held = (kStash + 1 - bg) / 2;                    // smallest jj with 2 jj + bg >= kStash
+        const int mine = (w.T + kNB - 1 - bg) / kNB;                     // tiles this group kept
+        const int first_held = (kStash + kNB - 1 - bg) / kNB;            // smallest jj with kNB jj + bg >= kStash
         const int nheld = max(mine - first_held, 0);
 #pragma unroll 1
         for (int jx = 0; jx < mine; ++jx) {
           const int jj = (jx < nheld) ? first_held + jx : jx - nheld;
-          const int j = 2 * jj + bg;
+          const int j = kNB * jj + bg;
           const int t = w.t0 + j;
           const int n_valid = min(kT, w.n - t * kT);
           const bool valid = tok < n_valid;
-          float sl[8], bold;
-          switch (jj) {
-#define CAOTE_TAKE(q) case q: { _Pragma("unroll") for (int hd = 0; hd < 8; ++hd) sl[hd] = keep[q][hd]; bold = keepb[q]; } break;
-            CAOTE_TAKE(0) CAOTE_TAKE(1) CAOTE_TAKE(2) CAOTE_TAKE(3)
-            default: { _Pragma("unroll") for (int hd = 0; hd < 8; ++hd) sl[hd] = keep[kMaxKeep - 1][hd]; bold = keepb[kMaxKeep - 1]; } break;
-#undef CAOTE_TAKE
-          }
+          float sl[8], bold = 0.f;
+#pragma unroll
+          for (int q = 0; q < kMaxKeep; ++q)
+            if (q == jj) {
+#pragma unroll
+              for (int hd = 0; hd < 8; ++hd) sl[hd] = keep[q][hd];
+              bold = keepb[q];
+            }
           float asum = 0.f, comp = 0.f;
           if (counted) {
 #pragma unroll
