@@ -28,11 +28,11 @@ constexpr int kThreads = 256;
 constexpr int kCombineRows = 32; // rows per combine CTA
 
 struct Scratch {
-  float* part_ml;  // [units][splits][Rpad][2]
+  float* part_ml;  // [units][splits][Rpad][2]   (max logit, sum of exp(s - max) over all keys but the first one at the max)
   float* part_o;   // [units][splits][Rpad][D]
   float* part_y;   // [units][splits][D]
   float* part_hb;  // [units][splits]
-  float* stats;    // [units][Rpad][2]   (max, 1/sum)
+  float* stats;    // [units][Rpad][4]   (max, 1/sum, (sum without the row's top key) / sum, unused)
   float* osum;     // [units][chunks][D]
   float* ytot;     // [units][D]
   float* hbtot;    // [units]
@@ -70,7 +70,7 @@ inline size_t carve(const Dims& dm, char* base, Scratch* out) {
   s.part_o = take(us * s.Rpad * dm.D);
   s.part_y = take(us * dm.D);
   s.part_hb = take(us);
-  s.stats = take((size_t)dm.units * s.Rpad * 2);
+  s.stats = take((size_t)dm.units * s.Rpad * 4);
   s.osum = take((size_t)dm.units * s.chunks * dm.D);
   s.ytot = take((size_t)dm.units * dm.D);
   s.hbtot = take((size_t)dm.units);
@@ -157,7 +157,9 @@ attn_partial_kernel(Dims dm, const T* __restrict__ q, const T* __restrict__ K, c
   const T* Ku = K + (size_t)unit * dm.cap * D;
   const T* Vu = V + (size_t)unit * dm.cap * D;
 
-  float m_run = -INFINITY, l_run = 0.f;
+  // l_rest: sum of exp(s - m_run) over the keys so far EXCEPT the first key that sits at the maximum (whose
+  // term is exactly 1): the row's 1 - alpha of its top key is then l_rest / (l_rest + 1), a sum of the others
+  float m_run = -INFINITY, l_rest = 0.f;
   float o_acc[OC];
 #pragma unroll
   for (int i = 0; i < OC; ++i) o_acc[i] = 0.f;
@@ -182,22 +184,24 @@ attn_partial_kernel(Dims dm, const T* __restrict__ q, const T* __restrict__ K, c
 #pragma unroll
     for (int o = 8; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
     const float m_new = fmaxf(m_run, mx);
-    float corr = 1.f, lsum = 0.f;
-    if (m_new == -INFINITY) {
+    const bool new_top = mx > m_run;  // this tile holds a key above everything before it
+    // (no branch here: the two rows of a warp vote together below)
+    const float corr = (m_run == -INFINITY) ? 0.f : expf(m_run - m_new);
+    float lsum = 0.f;
+    bool found = false;  // the first key of the tile at the new maximum (smallest key index) is left out of the sum
 #pragma unroll
-      for (int i = 0; i < 4; ++i) Ps[r * kKT + c0 + 16 * i] = 0.f;
-    } else {
-      corr = (m_run == -INFINITY) ? 0.f : expf(m_run - m_new);
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const float p = (s[i] == -INFINITY) ? 0.f : expf(s[i] - m_new);
-        Ps[r * kKT + c0 + 16 * i] = p;
-        lsum += p;
-      }
+    for (int i = 0; i < 4; ++i) {
+      const float p = (s[i] == -INFINITY) ? 0.f : expf(s[i] - m_new);
+      Ps[r * kKT + c0 + 16 * i] = p;
+      const unsigned at_top = (__ballot_sync(0xffffffffu, new_top && s[i] == m_new) >> (threadIdx.x & 16)) & 0xffffu;
+      const bool skip = !found && at_top != 0u && (int)(__ffs(at_top) - 1) == c0;
+      found |= at_top != 0u;
+      lsum += skip ? 0.f : p;
     }
 #pragma unroll
     for (int o = 8; o > 0; o >>= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, o);
-    l_run = l_run * corr + lsum;
+    // the old top key (term 1 before) joins the others when a new top appears
+    l_rest = l_rest * corr + ((new_top && m_run != -INFINITY) ? corr : 0.f) + lsum;
     m_run = m_new;
 #pragma unroll
     for (int i = 0; i < OC; ++i) o_acc[i] *= corr;
@@ -229,7 +233,7 @@ attn_partial_kernel(Dims dm, const T* __restrict__ q, const T* __restrict__ K, c
   if (row_ok) {
     if (c0 == 0) {
       sc.part_ml[(us * sc.Rpad + r_glob) * 2 + 0] = m_run;
-      sc.part_ml[(us * sc.Rpad + r_glob) * 2 + 1] = l_run;
+      sc.part_ml[(us * sc.Rpad + r_glob) * 2 + 1] = l_rest;
     }
     float* po = sc.part_o + (us * sc.Rpad + r_glob) * D;
     *reinterpret_cast<float4*>(po + c0 * 4) = make_float4(o_acc[0], o_acc[1], o_acc[2], o_acc[3]);
@@ -275,22 +279,26 @@ attn_combine_kernel(Dims dm, const int* __restrict__ len, Scratch sc, float* __r
     float mx = -INFINITY;
     for (int s = 0; s < sc.splits; ++s)
       mx = fmaxf(mx, sc.part_ml[(((size_t)unit * sc.splits + s) * sc.Rpad + r) * 2]);
-    float l = 0.f, acc = 0.f;
+    float l_rest = 0.f, acc = 0.f;
+    bool top_seen = false;  // the first split at the overall maximum keeps its top key apart; the others' join the rest
     for (int s = 0; s < sc.splits; ++s) {
       const size_t idx = ((size_t)unit * sc.splits + s) * sc.Rpad + r;
       const float ms = sc.part_ml[idx * 2];
       if (ms == -INFINITY) continue;
       const float f = expf(ms - mx);
-      l = fmaf(sc.part_ml[idx * 2 + 1], f, l);
+      l_rest = fmaf(sc.part_ml[idx * 2 + 1], f, l_rest);
+      if (ms == mx && !top_seen) top_seen = true;
+      else l_rest += f;
       acc = fmaf(sc.part_o[idx * D + c], f, acc);
     }
-    const float inv_l = 1.f / l;
+    const float inv_l = 1.f / (l_rest + 1.f);
     const float val = acc * inv_l;
     o[q_offset(dm, b, h, r) + c] = val;
     if (row_counted(dm, r)) osum += val;
     if (c == 0) {
-      sc.stats[((size_t)unit * sc.Rpad + r) * 2 + 0] = mx;
-      sc.stats[((size_t)unit * sc.Rpad + r) * 2 + 1] = inv_l;
+      sc.stats[((size_t)unit * sc.Rpad + r) * 4 + 0] = mx;
+      sc.stats[((size_t)unit * sc.Rpad + r) * 4 + 1] = inv_l;
+      sc.stats[((size_t)unit * sc.Rpad + r) * 4 + 2] = l_rest * inv_l;
     }
   }
   sc.osum[((size_t)unit * sc.chunks + chunk) * D + c] = osum;
@@ -315,10 +323,11 @@ score_pass_kernel(Dims dm, const T* __restrict__ q, const T* __restrict__ K, con
   extern __shared__ __align__(16) float smem[];
   float* Qs = smem;              // kRT * LD
   float* Ks = Qs + kRT * LD;     // kKT * LD
-  float* Hred = Ks + kKT * LD;   // kRT * kKT
-  float* Xs = Hred + kRT * kKT;  // D
-  float* st = Xs + D;            // kRT * 2
-  float* wq = st + kRT * 2;      // kKT: w_j / (1 - w_j)
+  float* Hred = Ks + kKT * LD;   // kRT * kKT  sums of the rows' weights of a key
+  float* Cred = Hred + kRT * kKT;  // kRT * kKT  sums of the rows' complements 1 - alpha of a key
+  float* Xs = Cred + kRT * kKT;  // D
+  float* st = Xs + D;            // kRT * 4
+  float* wq = st + kRT * 4;      // kKT: w_j / (1 - w_j)
 
   const int unit = blockIdx.y;
   const int b = unit / dm.Hkv, h = unit % dm.Hkv;
@@ -343,7 +352,9 @@ score_pass_kernel(Dims dm, const T* __restrict__ q, const T* __restrict__ K, con
   const int valid = min(kKT, n - j0);
   if (n_rows > 0) stage_rows<T, D, LD>(Ks, K + ((size_t)unit * dm.cap + j0) * D, kKT, valid);
 
-  float hacc[4] = {0.f, 0.f, 0.f, 0.f};
+  // hacc: sum over the counted rows of alpha_{r,j}; cacc: sum of 1 - alpha_{r,j}, where the row's top key takes
+  // (sum of the others) / sum from the attention pass and everybody else 1 - alpha <= 1/2: no cancellation
+  float hacc[4] = {0.f, 0.f, 0.f, 0.f}, cacc[4] = {0.f, 0.f, 0.f, 0.f};
   for (int t0 = 0; t0 < n_rows; t0 += kRT) {
     __syncthreads();
     // counted row number t -> row of the unit
@@ -359,48 +370,66 @@ score_pass_kernel(Dims dm, const T* __restrict__ q, const T* __restrict__ K, con
     }
     if (tid < kRT) {
       const int t = t0 + tid;
-      float mx = 0.f, il = 0.f;
+      float mx = 0.f, il = 0.f, cr = 0.f;
       if (t < n_rows) {
         const int row = (mode == CAOTE_BASE_LAST_QUERY) ? t * dm.m + dm.m - 1 : t;
-        mx = sc.stats[((size_t)unit * sc.Rpad + row) * 2];
-        il = sc.stats[((size_t)unit * sc.Rpad + row) * 2 + 1];
+        mx = sc.stats[((size_t)unit * sc.Rpad + row) * 4];
+        il = sc.stats[((size_t)unit * sc.Rpad + row) * 4 + 1];
+        cr = sc.stats[((size_t)unit * sc.Rpad + row) * 4 + 2];
       }
-      st[tid * 2] = mx;
-      st[tid * 2 + 1] = il;
+      st[tid * 4] = mx;
+      st[tid * 4 + 1] = il;
+      st[tid * 4 + 2] = cr;
     }
     __syncthreads();
     const int t = t0 + r;
     if (t < n_rows) {
       const int row = (mode == CAOTE_BASE_LAST_QUERY) ? t * dm.m + dm.m - 1 : t;
       const int n_vis = n - dm.m + (row % dm.m) + 1;
-      const float mx = st[r * 2], il = st[r * 2 + 1];
+      const float mx = st[r * 4], il = st[r * 4 + 1], cr = st[r * 4 + 2];
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         const int j = j0 + c0 + 16 * i;
-        if (j < n_vis) hacc[i] += expf(logit<D>(Qs + r * LD, Ks + (c0 + 16 * i) * LD, dm.scale) - mx) * il;
+        if (j < n_vis) {
+          const float sl = logit<D>(Qs + r * LD, Ks + (c0 + 16 * i) * LD, dm.scale);
+          const float a = expf(sl - mx) * il;
+          hacc[i] += a;
+          cacc[i] += (sl == mx) ? cr : 1.f - a;
+        } else {
+          cacc[i] += 1.f;  // a row that cannot see the key gives all its weight to the others
+        }
       }
     }
   }
   __syncthreads();
 #pragma unroll
-  for (int i = 0; i < 4; ++i) Hred[r * kKT + c0 + 16 * i] = hacc[i];
+  for (int i = 0; i < 4; ++i) {
+    Hred[r * kKT + c0 + 16 * i] = hacc[i];
+    Cred[r * kKT + c0 + 16 * i] = cacc[i];
+  }
   __syncthreads();
   if (tid < kKT) {
     const int j = j0 + tid;
     float ratio = 0.f;
     if (j < n) {
-      float hj = 0.f;
-      for (int rr = 0; rr < kRT; ++rr) hj += Hred[rr * kKT + tid];
-      if (mode == CAOTE_BASE_ACCUM) {
-        hj += base[(size_t)unit * dm.cap + j];
-        base[(size_t)unit * dm.cap + j] = hj;
-      } else if (mode == CAOTE_BASE_EXTERNAL) {
-        hj = base[(size_t)unit * dm.cap + j];
+      float hj = 0.f, rest = 0.f;  // rest = (1 - w_j) * Htot as a sum of non-negative parts
+      for (int rr = 0; rr < kRT; ++rr) {
+        hj += Hred[rr * kKT + tid];
+        rest += Cred[rr * kKT + tid];
       }
-      if (Htot > 0.f) {
-        const float rest = Htot - hj;  // (1 - w_j) * Htot
-        ratio = (rest > 0.f) ? hj / rest : INFINITY;
+      if (carried) {
+        // (the carried scores' own complement is a plain difference: a single carried score that holds almost
+        // all of their sum is outside what this any-shape path resolves)
+        const float bj = base[(size_t)unit * dm.cap + j];
+        rest += hb - bj;
+        if (mode == CAOTE_BASE_ACCUM) {
+          hj += bj;
+          base[(size_t)unit * dm.cap + j] = hj;
+        } else {
+          hj = bj;
+        }
       }
+      if (Htot > 0.f && hj > 0.f) ratio = (rest > 0.f) ? hj / rest : INFINITY;
     }
     wq[tid] = ratio;
   }
@@ -485,27 +514,30 @@ sum_errors_kernel(Dims dm, const T* __restrict__ q, const T* __restrict__ K, con
     }
     if (tid < kRT) {
       const int t = t0 + tid;
-      float mx = 0.f, il = 0.f;
+      float mx = 0.f, il = 0.f, cr = 0.f;
       if (t < n_rows) {
         const int row = (mode == CAOTE_BASE_LAST_QUERY) ? t * dm.m + dm.m - 1 : t;
-        mx = sc.stats[((size_t)unit * sc.Rpad + row) * 2];
-        il = sc.stats[((size_t)unit * sc.Rpad + row) * 2 + 1];
+        mx = sc.stats[((size_t)unit * sc.Rpad + row) * 4];
+        il = sc.stats[((size_t)unit * sc.Rpad + row) * 4 + 1];
+        cr = sc.stats[((size_t)unit * sc.Rpad + row) * 4 + 2];
       }
-      st[tid * 2] = mx;
-      st[tid * 2 + 1] = il;
+      st[tid * 4] = mx;
+      st[tid * 4 + 1] = il;
+      st[tid * 4 + 2] = cr;
     }
     __syncthreads();
     const int t = t0 + r;
     if (t < n_rows) {
       const int row = (mode == CAOTE_BASE_LAST_QUERY) ? t * dm.m + dm.m - 1 : t;
       const int n_vis = n - dm.m + (row % dm.m) + 1;
-      const float mx = st[r * 2], l = 1.f / st[r * 2 + 1];
+      const float mx = st[r * 4], il = st[r * 4 + 1], cr = st[r * 4 + 2];
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         const int jj = c0 + 16 * i, j = j0 + jj;
         if (j < n_vis) {
-          const float e = expf(logit<D>(Qs + r * LD, Ks + jj * LD, dm.scale) - mx);
-          const float rest = l - e;  // the other tokens' share of the row's softmax sum
+          const float sl = logit<D>(Qs + r * LD, Ks + jj * LD, dm.scale);
+          const float e = expf(sl - mx) * il;              // alpha
+          const float rest = (sl == mx) ? cr : 1.f - e;    // 1 - alpha: the others' share, without cancellation
           float d2 = 0.f;
 #pragma unroll 8
           for (int c = 0; c < D; c += 4) {
@@ -532,12 +564,12 @@ sum_errors_kernel(Dims dm, const T* __restrict__ q, const T* __restrict__ K, con
 
 inline size_t sum_errors_smem(int D) {
   const int LD = D + 4;
-  return sizeof(float) * (size_t)(2 * kRT * LD + 2 * kKT * LD + kRT * kKT + kRT * 2);
+  return sizeof(float) * (size_t)(2 * kRT * LD + 2 * kKT * LD + kRT * kKT + kRT * 4);
 }
 
 inline size_t score_smem(int D) {
   const int LD = D + 4;
-  return sizeof(float) * (size_t)(kRT * LD + kKT * LD + kRT * kKT + D + kRT * 2 + kKT);
+  return sizeof(float) * (size_t)(kRT * LD + kKT * LD + 2 * kRT * kKT + D + kRT * 4 + kKT);
 }
 
 }  // namespace generic

@@ -263,3 +263,88 @@ def test_append_and_status_word():
     P.caote_select_evict(p, scores, lens, torch.tensor([1, 17], dtype=torch.int32, device=DEV), None, ev, ne, ws)
     assert P.caote_read_status(ws) == P.binding.ERR_OVERFLOW
     assert ne.tolist() == [0, 1]
+
+
+def dominant_case(seed, B, Hq, Hkv, d, cap, m, dtype, lens, eps, slot):
+    """Every query row of every head is (nearly) the same vector q0 and one key per unit is c * q0, with c chosen
+    so that this key takes all but about `eps` of every row's weight: 1 - w_j ~ eps must then not be formed by
+    cancellation."""
+    g = torch.Generator(device="cpu").manual_seed(seed)
+    q0 = torch.randn((B, Hkv, 1, 1, d), generator=g)
+    q = (q0 + 0.02 * torch.randn((B, Hkv, Hq // Hkv, m, d), generator=g)).reshape(B, Hq, m, d)
+    K = torch.randn((B, Hkv, cap, d), generator=g)
+    V = torch.randn((B, Hkv, cap, d), generator=g)
+    for b in range(B):
+        for h in range(Hkv):
+            v0 = q0[b, h, 0, 0]
+            others = torch.exp((K[b, h, :lens[b]] @ v0) * d ** -0.5).sum()  # the other keys' numerators for q0
+            logit = float(torch.log(others / eps))
+            K[b, h, slot] = v0 * (logit / (d ** -0.5 * float(v0 @ v0)))
+    return (q.to(dtype).to(DEV), K.to(dtype).to(DEV), V.to(dtype).to(DEV),
+            torch.tensor(lens, dtype=torch.int32, device=DEV))
+
+
+@pytest.mark.parametrize("eps", [1e-1, 1e-2, 1e-3, 1e-4])
+@pytest.mark.parametrize("shape", [
+    # B, Hq, Hkv, d, cap, m, lens, mode, dtype            path
+    (2, 8, 2, 128, 1600, 1, [1531, 700], "last_query", torch.bfloat16),   # single query, G 4
+    (1, 7, 1, 128, 9000, 1, [8193], "accum", torch.bfloat16),             # single query, G 7, carried base scores
+    (2, 8, 1, 128, 300, 1, [257, 300], "last_query", torch.bfloat16),     # single query, G 8, few tiles
+    (1, 8, 2, 128, 700, 128, [640], "chunk_sum", torch.bfloat16),         # block of queries, tensor-core path
+    (1, 4, 2, 64, 200, 3, [150], "chunk_sum", torch.float32),             # any-shape path
+    (1, 4, 2, 64, 200, 1, [190], "last_query", torch.float32),            # any-shape path, one query
+])
+def test_token_holding_almost_all_the_weight(shape, eps):
+    """One token of every unit holds all but ~eps of the weight (Sec. 3.2 normalisation; the oracle forms 1 - w_j
+    as the sum of the other weights). Down to eps = 1e-3 its score and everybody else's stay within the stated
+    tolerance. At 1e-4 the planted token's own score is bounded by something else: X - v_j is then a difference
+    of two fp32 vectors that agree to four digits, which leaves the distance about three digits; it is held
+    to 2e-2 there, everybody else to the stated tolerance."""
+    B, Hq, Hkv, d, cap, m, lens, mode, dtype = shape
+    slot = 77
+    q, K, V, lens_t = dominant_case(int(-np.log10(eps)) * 31 + Hq, B, Hq, Hkv, d, cap, m, dtype, lens, eps, slot)
+    base = None
+    if mode == "accum":
+        g = torch.Generator(device="cpu").manual_seed(3)
+        base = (torch.rand((B, Hkv, cap), generator=g) * 1e-9).to(DEV)
+    base_in = None if base is None else base.clone()
+    p, ws, o, scores = run_score(q, K, V, lens_t, m, mode, base)
+    r = oracle_for(q, K, V, lens_t, scale=d ** -0.5, n_new=m, base_mode=mode, base=base_in)
+    for b in range(B):
+        comp = 1.0 - r["w"][b, :, slot]
+        assert (comp < 6 * eps).all() and (comp > eps / 6).all(), f"construction: 1 - w = {comp}, wanted ~{eps}"
+    if eps >= 1e-3:
+        check_scores_and_o(r, scores, o, lens_t, f"{shape} eps {eps}")
+    else:
+        sg = f32(scores).astype(np.float64)
+        for b, n in enumerate(lens):
+            rest = np.ones(n, dtype=bool)
+            rest[slot] = False
+            assert_close(sg[b, :, :n][:, rest], r["scores"][b, :, :n][:, rest], f"{shape} eps {eps} others")
+            assert_close(sg[b, :, slot], r["scores"][b, :, slot], f"{shape} eps {eps} planted token", rtol=2e-2)
+            assert_close(f32(o)[b], r["o"][b], "o")
+
+
+@pytest.mark.parametrize("mode,m,dtype,d", [("last_query", 1, torch.bfloat16, 128), ("accum", 1, torch.bfloat16, 128),
+                                            ("chunk_sum", 64, torch.bfloat16, 128), ("chunk_sum", 2, torch.float32, 64)])
+def test_equal_values_and_dominant_base_score(mode, m, dtype, d):
+    """All value rows equal: X equals every v_j up to the rounding of the accumulated output, so every score is
+    (within the absolute tolerance) zero. And a carried base score that holds almost all of the normaliser
+    (accumulated mode, single-query path) keeps an accurate complement."""
+    B, Hq, Hkv, cap, n = 1, 8, 2, 1500, 1409
+    q, K, V, lens_t = make_case(91, B, Hq, Hkv, d, cap, m, dtype, [n])
+    Veq = V[:, :, :1].expand_as(V).contiguous()
+    base = torch.rand((B, Hkv, cap), device=DEV) if mode == "accum" else None
+    base_in = None if base is None else base.clone()
+    _, _, o, scores = run_score(q, K, Veq, lens_t, m, mode, base)
+    r = oracle_for(q, K, Veq, lens_t, scale=d ** -0.5, n_new=m, base_mode=mode, base=base_in)
+    assert np.abs(r["scores"][0, :, :n]).max() < 1e-12
+    check_scores_and_o(r, scores, o, lens_t, "equal values")
+    if mode == "accum":
+        base = torch.rand((B, Hkv, cap), device=DEV) * 1e-2
+        base[:, :, 500] = 3e5
+        base_in = base.clone()
+        _, _, o, scores = run_score(q, K, V, lens_t, m, mode, base)
+        r = oracle_for(q, K, V, lens_t, scale=d ** -0.5, n_new=m, base_mode=mode, base=base_in)
+        assert (1.0 - r["w"][0, :, 500] < 1e-3).all()
+        check_scores_and_o(r, scores, o, lens_t, "dominant carried base score")
