@@ -29,19 +29,24 @@ sys.path.insert(0, ROOT)
 
 from paper_2504_14051_b200 import workloads as wl  # noqa: E402
 
-# DRAM bytes (read + write) of one launch per unit of work, from ncu captures (profiles/*.txt), scaled
-# to the launch at hand by the units it processes; traffic grows in proportion to them. The decode
-# figure is from the full-size c4 launch (a one-pass capture of the two DRAM counters): in the reduced
-# case part of the second pass over V is served by L2, at full size none of it is. A value is set to
-# None when its kernel has changed since the capture.
-NCU_TRAFFIC = {
-    # per launch at the workload's own size: (read + write) of profiles/decode_tc_kernel_c4_full_traffic.txt
-    "decode_tc_kernel": {"per_launch": {"c4": 1420990976 + 62851584, "c5d": 780532736 + 34983680},
-                         "profile": "profiles/decode_tc_kernel_c4_full_traffic.txt"},
-    "decode_tc_fast_kernel": {"per_launch": {"c4": 956031488 + 56979456},
-                              "profile": "profiles/decode_tc_kernel_c4_full_traffic.txt"},
-    "prefill_attn_kernel": {"bytes_per_unit": (156274688 + 23372288) / 16, "profile": "profiles/prefill_kernels_c5p_batch2_ncu.txt"},
-}
+# DRAM bytes (read + write) of one launch, taken by ncu: the summaries under profiles/ carry one line per
+# (kernel, workload) of the form
+#     traffic_bytes_per_launch: <kernel> <workload> <bytes>
+# and this table is read from them, so that a figure can only be reported together with the capture it
+# comes from. A summary whose kernel has changed since the capture is deleted or re-taken, never edited here.
+def load_ncu_traffic():
+    table = {}
+    pdir = os.path.join(ROOT, "profiles")
+    if os.path.isdir(pdir):
+        for fn in sorted(os.listdir(pdir)):
+            if not fn.endswith((".txt", ".md")):
+                continue
+            for ln in open(os.path.join(pdir, fn)):
+                if ln.startswith("traffic_bytes_per_launch:"):
+                    _, kernel, workload, nbytes = ln.split()
+                    table[(kernel, workload)] = (int(float(nbytes)), "profiles/" + fn)
+    return table
+
 
 METRIC = "cached tokens scored+evicted/sec"
 UNIT = "token-heads/s"
@@ -179,7 +184,9 @@ def aggregate_over_ranks(ms: float, units_this_rank: float, world: int, device):
     return float(t_all.item()), float(th_all.item())
 
 
-def run_ours(args, w0, rank, world, device):
+def run_ours(args, w0, rank, world, device, light=False):
+    """Times `args.steps` steps of workload w0 on this rank. light=True (the secondary records): device-resident
+    timing, per-kernel times and roofline only."""
     import paper_2504_14051_b200 as P
 
     pool = min(args.pool, args.steps + args.warmup)
@@ -238,17 +245,18 @@ def run_ours(args, w0, rank, world, device):
     launches_per_step_top = trace[top][0] / trace_steps
     peaks = load_peaks()
     algo = algorithmic_bytes(w, th_per_step, units)
+    traffic_table = load_ncu_traffic()
+    full_size = w.batch == wl.WORKLOADS[w0.name].batch and args.method == "caote"
+    traffic_entry = traffic_table.get((top, w0.name)) if full_size else None  # captured at the named full sizes only
     if w.n_new == 1:
-        # measured only at the named workloads' full sizes: smaller cases get part of their second pass from L2
-        full_size = w.batch == wl.WORKLOADS[w0.name].batch
-        decode_traffic = NCU_TRAFFIC.get(top, {}).get("per_launch", {}).get(w0.name) if full_size else None
+        decode_traffic = traffic_entry[0] if traffic_entry else None
         bytes_per_launch = algo["per_step"] / launches_per_step_top
         achieved = bytes_per_launch / (per_launch_ms * 1e-3) / 1e9
         roofline = {"bound": "hbm", "kernel": top, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "frac": achieved / peaks["hbm_gbs"], "frac_of_nominal_8000": achieved / 8000.0,
                     "peak_source": peaks["source"] + " copy bandwidth",
                     "traffic": decode_traffic,
-                    "traffic_source": NCU_TRAFFIC[top]["profile"] if decode_traffic else None,
+                    "traffic_source": traffic_entry[1] if traffic_entry else None,
                     "algorithmic_bytes_per_launch": bytes_per_launch,
                     "algorithmic_bytes_per_token_head": algo["per_token_head"],
                     "step_frac": (algo["per_step"] / (ms_per_step * 1e-3) / 1e9) / peaks["hbm_gbs"]}
@@ -258,10 +266,20 @@ def run_ours(args, w0, rank, world, device):
         roofline = {"bound": "tensor", "kernel": top, "achieved": achieved, "peak": peaks["bf16_tflops_sustained"],
                     "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops_sustained"],
                     "peak_source": peaks["source"] + " cuBLAS bf16 sustained",
-                    "traffic": (NCU_TRAFFIC[top]["bytes_per_unit"] * units if NCU_TRAFFIC.get(top) else None),
-                    "traffic_source": NCU_TRAFFIC[top]["profile"] if NCU_TRAFFIC.get(top) else None,
+                    "traffic": traffic_entry[0] if traffic_entry else None,
+                    "traffic_source": traffic_entry[1] if traffic_entry else None,
                     "useful_flops_per_launch": fl_per_launch,
+                    "note": "achieved counts the attention's own 4 M n d per unit (QK^T and PV); the kernels execute "
+                            "8 M n d (PV in two bf16 parts, K Q^T again in the score pass)",
+                    "step_useful_tflops": flops_per_step / (ms_per_step * 1e-3) / 1e12,
+                    "step_executed_tflops": 2.0 * flops_per_step / (ms_per_step * 1e-3) / 1e12,
                     "step_frac": (flops_per_step / (ms_per_step * 1e-3) / 1e12) / peaks["bf16_tflops_sustained"]}
+
+    if light:
+        return {"workload": w0.name, "steps": steps, "warmup": warmup, "ms_per_step": ms_per_step, "value": value,
+                "unit": UNIT, "dtype": w.dtype, "n_new": w.n_new, "layers": w.layers,
+                "token_heads_per_step": th_per_step, "kernels": kernels, "roofline": roofline,
+                "clocks": clk.summary()}, w
 
     # -------- end to end: per-step inputs from pinned host memory, results read back every step
     host_in = [[tuple(x.cpu().pin_memory() for x in inp[t]) for t in range(pool)] for inp in inputs]
@@ -396,6 +414,11 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--method", default="caote", choices=["caote", "fast"],
                     help="caote: the CAOTE score (the headline); fast: FastCAOTE (Sec. 3.3), X = mean of the cached values")
+    ap.add_argument("--dry-run", action="store_true",
+                    help="exercise the launcher and the cross-rank aggregation on CPU (gloo) with made-up per-rank "
+                         "figures; no CUDA work, not a measurement")
+    ap.add_argument("--no-secondary", action="store_true",
+                    help="skip the short chunked-prefill runs that the default line carries beside the headline")
     ap.add_argument("--batch", type=int, default=None,
                     help="override the workload's batch (smaller cases for profiler captures; not a bench line)")
     args = ap.parse_args()
@@ -406,9 +429,37 @@ def main():
         # chunked prefill is timed in its steady state: the cache already holds `budget` tokens, so every
         # timed step scores budget + m tokens per unit and evicts m (the regime of all but the first chunks)
         w = wl.scaled(w, init_len=w.budget)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
+        # asked for N replicas but started as a plain process: become the launcher (one rank per GPU)
+        if not args.dry_run and torch.cuda.device_count() < args.gpus:
+            print(f"bench.py: --gpus {args.gpus} but {torch.cuda.device_count()} CUDA device(s) visible", file=sys.stderr)
+            return 2
+        import socket
+
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            port = sk.getsockname()[1]
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+               "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+        os.execv(sys.executable, cmd)
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "ours" and world != args.gpus:
+        print(f"bench.py: --gpus {args.gpus} does not match WORLD_SIZE {world}", file=sys.stderr)
+        return 2
+    if args.dry_run:
+        # every rank reports (10 + 5 rank) ms for (1000 + rank) units; the line shows what the aggregation made of it
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        if world > 1:
+            torch.distributed.init_process_group("gloo")
+        ms, units = aggregate_over_ranks(10.0 + 5.0 * rank, 1000.0 + rank, world, torch.device("cpu"))
+        if rank == 0:
+            print(json.dumps({"dry_run": True, "n_gpus": world, "ms_per_step": ms, "units": units,
+                              "value": units / (ms * 1e-3), "scaling": "weak"}), flush=True)
+        if world > 1:
+            torch.distributed.destroy_process_group()
+        return 0
 
     if args.impl == "reference":
         if rank != 0:
@@ -431,6 +482,20 @@ def main():
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         torch.distributed.init_process_group("nccl", device_id=device)
     out, wr = run_ours(args, w, rank, world, device)
+    if world == 1 and w.name == "c4" and args.batch is None and args.method == "caote" and not args.no_secondary:
+        # the metric's other half (% of tensor peak on chunked prefill): short steady-state runs of the two
+        # prefill workloads, device-resident timing only; the headline keys above are not touched
+        import copy
+
+        out["secondary"] = {}
+        for name, nsteps in (("c5p", 8), ("c3", 16)):
+            torch.cuda.empty_cache()
+            a2 = copy.copy(args)
+            a2.steps, a2.warmup, a2.pool = nsteps, 3, 4
+            w2 = wl.WORKLOADS[name]
+            w2 = wl.scaled(w2, init_len=w2.budget)
+            rec, _ = run_ours(a2, w2, rank, world, device, light=True)
+            out["secondary"][name] = rec
     if rank == 0:
         if not args.no_cpu_baseline:
             out["cpu_baseline"] = cpu_baseline(w)

@@ -182,6 +182,25 @@ CAOTE_API int caote_select_evict(const caote_params_t* params, const float* scor
                        int32_t max_evict, int32_t* n_evict, void* workspace,
                        size_t workspace_bytes, caote_stream_t stream);
 
+/* Greedy multi-token eviction (Appendix B, "Extending CAOTE to multi-token eviction": evicting token 1 and then
+ * token 2 from the renormalised state, chained): instead of taking the k lowest scores of one scoring pass,
+ * evict one token at a time and let every eviction change the scores of the rest. Per unit, with
+ * non-negative weights h_j (any base score: accumulated H2O scores after caote_score, or scores of the
+ * caller's own), w_j = h_j / sum_i h_i and X = sum_j w_j v_j, repeat k = max(0, len - budget) times:
+ *     e = arg min_j  w_j / (1 - w_j) * || X - v_j ||_2   over the tokens still present (ties: smaller pos),
+ *     X <- (X - w_e v_e) / (1 - w_e),   w_i <- w_i / (1 - w_e)   (the paper's alpha' and X').
+ * After t evictions the distance between the original and the current X is the paper's closed-form joint
+ * score of the evicted set. With k = 1 the result is that of caote_select_evict on the CAOTE scores.
+ *   V [B, Hkv, cap, d] I/O dtype, in;  h [B, Hkv, cap] fp32, in (negative values count as 0);
+ *   evict_idx[u, 0..k) out: the evicted slots in ascending order (what caote_compact takes);
+ *   order[u, 0..k) out, nullable: the same slots in the order they were evicted;  n_evict[b] = k out.
+ * capacity <= 24576 (the unit's weights and distances stay in shared memory), else CAOTE_ERR_UNSUPPORTED.
+ * Cost: one sweep over the unit's value rows per eviction (from L2 after the first). */
+CAOTE_API int caote_select_evict_greedy(const caote_params_t* params, const void* V, const float* h,
+                              const int32_t* len, const int32_t* budget, const int32_t* pos,
+                              int32_t* evict_idx, int32_t* order, int32_t max_evict, int32_t* n_evict,
+                              void* workspace, size_t workspace_bytes, caote_stream_t stream);
+
 /* Remove the evicted slots from K, V, base, pos in place and set len[b] -= n_evict[b], so that the
  * cache is back within budget before the next block arrives (Sec. 2, budgeted block-wise flow).
  * mode is a caote_compact_mode_t. base, pos nullable. evict_idx rows must be ascending and unique

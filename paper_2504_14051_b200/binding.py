@@ -106,6 +106,8 @@ def lib() -> ctypes.CDLL:
     L.caote_trace_enable.argtypes = [ctypes.c_int]
     L.caote_trace_collect.restype = ctypes.c_int
     L.caote_trace_collect.argtypes = [ctypes.POINTER(TraceEntry), i32, ctypes.POINTER(ctypes.c_int32)]
+    L.caote_select_evict_greedy.restype = ctypes.c_int
+    L.caote_select_evict_greedy.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, i32, vp, vp, sz, vp]
     L.caote_launch_count.restype = ctypes.c_int64
     L.caote_launch_count.argtypes = []
     L.caote_set_option.restype = ctypes.c_int
@@ -173,6 +175,12 @@ def caote_select_evict(p, scores, lens, budget, pos, evict_idx, n_evict, workspa
            lib().caote_select_evict(ctypes.byref(p), _p(scores), _p(lens), _p(budget), _p(pos), _p(evict_idx),
                                     evict_idx.shape[-1], _p(n_evict), _p(workspace), workspace.numel(),
                                     _stream(stream)))
+
+
+def caote_select_evict_greedy(p, V, h, lens, budget, pos, evict_idx, order, n_evict, workspace, stream=None):
+    _check("caote_select_evict_greedy", lib().caote_select_evict_greedy(
+        ctypes.byref(p), _p(V), _p(h), _p(lens), _p(budget), _p(pos), _p(evict_idx), _p(order), evict_idx.shape[-1],
+        _p(n_evict), _p(workspace), workspace.numel() * workspace.element_size(), _stream(stream)))
 
 
 def caote_compact(p, K, V, base, pos, lens, evict_idx, n_evict, mode, workspace, stream=None):

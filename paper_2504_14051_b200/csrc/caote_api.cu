@@ -10,6 +10,7 @@
 #include "decode_cluster.cuh"
 #include "decode_tc.cuh"
 #include "generic_score.cuh"
+#include "greedy.cuh"
 #include "post_evict.cuh"
 #include "prefill_tc.cuh"
 #include "select_compact.cuh"
@@ -569,6 +570,17 @@ static int launch_post_evict(const Dims& dm, const void* q, const void* K, const
   return CAOTE_OK;
 }
 
+template <typename T, int D>
+static int launch_greedy(const Dims& dm, const void* V, const float* h, const int* len, const int* budget, const int* pos,
+                         int* evict_idx, int* order, int max_evict, int* n_evict, int* status, cudaStream_t st) {
+  const size_t smem = greedy::smem_bytes(dm.cap, D);
+  int rc = allow_smem(greedy::greedy_kernel<T, D>, smem);
+  if (rc) return rc;
+  CAOTE_LAUNCH("greedy_select_kernel", st, greedy::greedy_kernel<T, D><<<dm.units, greedy::kThreads, smem, st>>>(
+      dm.Hkv, dm.cap, (const T*)V, h, len, budget, pos, evict_idx, order, max_evict, n_evict, status));
+  return CAOTE_OK;
+}
+
 }  // namespace caote
 
 using namespace caote;
@@ -734,6 +746,27 @@ int caote_select_evict(const caote_params_t* p, const float* scores, const int32
   CAOTE_LAUNCH("select_kernel", st, sel::select_kernel<<<dm.units, sel::kSelThreads, 0, st>>>(
       dm.Hkv, dm.cap, scores, len, budget, pos, evict_idx, max_evict, n_evict, (int*)workspace));
   return CAOTE_OK;
+}
+
+int caote_select_evict_greedy(const caote_params_t* p, const void* V, const float* h, const int32_t* len,
+                              const int32_t* budget, const int32_t* pos, int32_t* evict_idx, int32_t* order,
+                              int32_t max_evict, int32_t* n_evict, void* workspace, size_t workspace_bytes_,
+                              caote_stream_t stream) {
+  if (!params_ok(p) || !V || !h || !len || !budget || !evict_idx || !n_evict || !workspace || max_evict < 1)
+    return CAOTE_ERR_INVALID_ARG;
+  if (!params_supported(p) || p->capacity > greedy::kMaxTokens) return CAOTE_ERR_UNSUPPORTED;
+  if (workspace_bytes_ < kHeaderBytes || !aligned(workspace, 256) || !aligned(V, 16)) return CAOTE_ERR_INVALID_ARG;
+  int rc = check_device();
+  if (rc) return rc;
+  const Dims dm = make_dims(p);
+  cudaStream_t st = (cudaStream_t)stream;
+  int* status = (int*)workspace;
+  if (p->dtype == CAOTE_BF16) {
+    if (dm.D == 128) return launch_greedy<__nv_bfloat16, 128>(dm, V, h, len, budget, pos, evict_idx, order, max_evict, n_evict, status, st);
+    return launch_greedy<__nv_bfloat16, 64>(dm, V, h, len, budget, pos, evict_idx, order, max_evict, n_evict, status, st);
+  }
+  if (dm.D == 128) return launch_greedy<float, 128>(dm, V, h, len, budget, pos, evict_idx, order, max_evict, n_evict, status, st);
+  return launch_greedy<float, 64>(dm, V, h, len, budget, pos, evict_idx, order, max_evict, n_evict, status, st);
 }
 
 int caote_compact(const caote_params_t* p, void* K, void* V, float* base, int32_t* pos, int32_t* len,

@@ -56,3 +56,26 @@ def test_single_rank_needs_no_process_group():
     import bench
 
     assert bench.aggregate_over_ranks(3.5, 7.0, 1, torch.device("cpu")) == (3.5, 7.0)
+
+
+@pytest.mark.timeout(300)
+def test_bench_gpus_flag_launches_that_many_ranks():
+    """`bench.py --gpus 2` started as a plain process must become two ranks by itself (never print an N = 1 line
+    for an N = 2 request). --dry-run keeps it on CPU: launcher, rendezvous and the two reductions are real, the
+    per-rank figures are made up (rank r: 10 + 5 r ms, 1000 + r units)."""
+    import json
+    import subprocess
+
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_PORT")}
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--dry-run"], env=env,
+                         capture_output=True, text=True, timeout=280)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [ln for ln in res.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1, res.stdout
+    out = json.loads(lines[0])
+    assert out["n_gpus"] == 2 and out["ms_per_step"] == 15.0 and out["units"] == 2001.0
+    # a world size that does not match the request is an error, not a silently smaller run
+    env2 = dict(env, WORLD_SIZE="1", RANK="0", LOCAL_RANK="0")
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--dry-run"], env=env2,
+                         capture_output=True, text=True, timeout=120)
+    assert res.returncode != 0 and "does not match" in res.stderr
