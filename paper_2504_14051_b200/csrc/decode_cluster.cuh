@@ -693,7 +693,7 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
       // the peers' copies of the previous unit's records must have been read before they are overwritten
       if (mu >= 1) wait_bounded(r2, (mu - 1) & 1, &ctl[0], status, wait_cycles, false);
       group_sync(0);
-      {
+      if (!ctl[0]) {  // (a CTA that has given up pushes nothing more: its peers may be on their way out)
         // statistics to every peer (one 16-byte piece per thread and peer)
         const uint32_t st_local = smem_u32(xstats + rank * kStatFloats), bar_local = smem_u32(r1);
         for (int p = tok; p < 9 * C; p += kGroup) {
@@ -853,17 +853,19 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
 #pragma unroll
           for (int off = 4; off > 0; off >>= 1) xs += __shfl_xor_sync(0xffffffffu, xs, off);
           const float nxv = -(xs * inv_H);
-          if (act) {
+          if (act && !ctl[0]) {
             for (int peer = r; peer < C; peer += 8)
               push_f32(map_to_rank(smem_u32(xdst + my_ch0 + cl), peer), nxv, map_to_rank(smem_u32(r2), peer));
           }
         }
       }
       group_sync(1 + bg);  // every thread of this group is done with the records: tell the peers
-      if (tok < C) push_f32(map_to_rank(smem_u32(xword + kNB * rank + bg), tok), 0.f, map_to_rank(smem_u32(r2), tok));
+      if (tok < C && !ctl[0]) push_f32(map_to_rank(smem_u32(xword + kNB * rank + bg), tok), 0.f, map_to_rank(smem_u32(r2), tok));
       wait_bounded(r2, mu & 1, &ctl[0], status, wait_cycles, false);
-      if (bg == 0 && tok == 0) {
-        // the next unit's merge: what the peers will push into this CTA
+      if (bg == 0 && tok == 0 && !ctl[0]) {
+        // the next unit's merge: what the peers will push into this CTA. (Not after a wait of this CTA has run
+        // out: the phase may then still be open, and a second arrival on an open phase whose arrival count is
+        // already used up is not defined.)
         mbar_expect_tx(r1, r1_bytes);
         mbar_expect_tx(r2, r2_bytes);
       }

@@ -348,3 +348,30 @@ def test_equal_values_and_dominant_base_score(mode, m, dtype, d):
         r = oracle_for(q, K, V, lens_t, scale=d ** -0.5, n_new=m, base_mode=mode, base=base_in)
         assert (1.0 - r["w"][0, :, 500] < 1e-3).all()
         check_scores_and_o(r, scores, o, lens_t, "dominant carried base score")
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_library_stays_usable():
+    """The single-query kernel bounds every device-side wait by a clock limit. With the limit set far below the
+    latency of a memory copy the waits for the first tiles run out: the call must still return, record
+    CAOTE_ERR_TIMEOUT in the status word, and leave the library, the workspace and the caches usable - the same
+    call with the default limit then gives the oracle's result."""
+    B, Hq, Hkv, d, cap = 6, 8, 2, 128, 1100
+    lens = [1031, 900, 1100, 513, 1024, 257]
+    q, K, V, lens_t = make_case(4242, B, Hq, Hkv, d, cap, 1, torch.bfloat16, lens)
+    p = P.make_params(B, Hq, Hkv, d, cap, 1, torch.bfloat16, d ** -0.5, "last_query")
+    ws = P.alloc_workspace(p, DEV)
+    o = torch.zeros(q.shape, dtype=torch.float32, device=DEV)
+    scores = torch.zeros((B, Hkv, cap), dtype=torch.float32, device=DEV)
+    P.caote_set_option(P.binding.OPT_WAIT_CYCLES, 200)
+    try:
+        P.caote_score(p, q, K, V, lens_t, None, o, scores, ws)
+        torch.cuda.synchronize()  # the call came back
+        assert P.caote_read_status(ws) == P.binding.ERR_TIMEOUT
+    finally:
+        P.caote_set_option(P.binding.OPT_WAIT_CYCLES, 2_000_000_000)
+    assert P.caote_read_status(ws) == 0  # reading resets the word
+    P.caote_score(p, q, K, V, lens_t, None, o, scores, ws)
+    torch.cuda.synchronize()
+    assert P.caote_read_status(ws) == 0
+    r = oracle_for(q, K, V, lens_t, scale=d ** -0.5, n_new=1, base_mode="last_query")
+    check_scores_and_o(r, scores, o, lens_t, "after a timed-out call")
