@@ -33,9 +33,13 @@ def make_cache(w, compact="fill"):
     return c
 
 
-def lockstep(w, steps, units=None, compact="fill"):
-    """Run `steps` steps; check every step against the oracle on `units` (default: all)."""
+def lockstep(w, steps, units=None, compact="fill", random_base=False):
+    """Run `steps` steps; check every step against the oracle on `units` (default: all). random_base: the carried
+    base scores start from seeded positive values instead of zero (a cache that has been running for a while)."""
     c = make_cache(w, compact)
+    if random_base:
+        g = torch.Generator(device="cpu").manual_seed(w.seed + 1)
+        c.base.copy_((torch.rand(c.base.shape, generator=g) * 3.0).to(DEV))
     G, Hkv, m = w.group, w.n_kv_heads, w.n_new
     if units is None:
         units = [(b, h) for b in range(w.batch) for h in range(Hkv)]
@@ -81,13 +85,13 @@ def lockstep(w, steps, units=None, compact="fill"):
 
 
 def test_c2_decode_with_sinks_lockstep():
-    w = wl.scaled(wl.WORKLOADS["c2"], steps=6)
-    lockstep(w, 6)
+    w = wl.scaled(wl.WORKLOADS["c2"], steps=64)
+    lockstep(w, 64)
 
 
 def test_c3_chunked_prefill_reduced_lockstep():
     w = wl.scaled(wl.WORKLOADS["c3"], budget=1024, init_len=1024, layers=1)
-    lockstep(w, 2)
+    lockstep(w, 6)
 
 
 def test_c3_chunked_prefill_fills_before_it_evicts():
@@ -97,14 +101,14 @@ def test_c3_chunked_prefill_fills_before_it_evicts():
 
 def test_c4_ragged_accumulated_reduced_lockstep():
     w = wl.scaled(wl.WORKLOADS["c4"], batch=3, budget=1500, init_len=1500, ragged_min_len=1100)
-    lockstep(w, 4)
+    lockstep(w, 32)
 
 
 def test_c5_prefill_then_decode_reduced_lockstep():
     wp = wl.scaled(wl.WORKLOADS["c5p"], batch=1, budget=1536, init_len=1536)
     lockstep(wp, 1, units=[(0, 0), (0, 7)])
     wd = wl.scaled(wl.WORKLOADS["c5d"], batch=2, budget=1536, init_len=1536)
-    lockstep(wd, 3)
+    lockstep(wd, 16)
 
 
 @pytest.mark.parametrize("name,units", [
@@ -119,3 +123,9 @@ def test_full_size_step_on_sampled_units(name, units):
     if w.n_new > 1:
         w = wl.scaled(w, init_len=w.budget, layers=1)
     lockstep(w, 1, units=units)
+
+
+def test_full_size_c4_steps_with_carried_base_scores():
+    """Two full-size steps of the accumulated-score workload starting from non-zero carried base scores (row 7 of
+    the P operand and the base tiles staged beside the value tiles are in play from the first launch on)."""
+    lockstep(wl.WORKLOADS["c4"], 2, units=[(5, 2), (40, 0), (63, 3)], random_base=True)

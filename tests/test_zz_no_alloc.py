@@ -5,10 +5,11 @@ already owns the whole GPU, a plug-in that is handed tensors but no allocator, a
 an allocation could stall the device. They cannot supply the workspace that caote_score wants, so
 caote_score_static takes none and works on a fixed array inside the library instead.
 
-Checked here, through the C ABI: the same inputs give the same outputs as caote_score, on two calls
-in a row (the array is shared and keeps the previous call's contents, so the second call runs on a
-dirty array), for a shape served by the single-query kernel and one served by the generic kernels;
-and a shape whose scratch would not fit the array is refused before anything runs.
+Checked here, through the C ABI: the same inputs give the same outputs as caote_score and as the CPU
+oracle, on two calls in a row (the array is shared and keeps the previous call's contents, so the
+second call runs on a dirty array), for shapes served by the single-query kernel, by the tensor-core
+kernels for a block of queries and by the any-shape kernels; the amount of device memory in use does not
+move across a call; and a shape whose scratch would not fit the array is refused before anything runs.
 
 This file sorts last on purpose, so a run that stops at the first failure has already run the rest.
 """
@@ -20,7 +21,7 @@ import torch
 import paper_2504_14051_b200 as P
 from paper_2504_14051_b200 import binding as C
 
-from parity import ATOL, RTOL, assert_close, f32
+from parity import ATOL, RTOL, assert_close, check_scores_and_o, f32, oracle_for
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
@@ -38,7 +39,8 @@ def _inputs(seed, B, Hq, Hkv, d, cap, m, lens):
 @pytest.mark.parametrize("shape,mode", [
     ((3, 14, 2, 128, 1500, 1, [1500, 1031, 77]), "accum"),       # single-query kernel, carried base score
     ((2, 8, 2, 128, 700, 1, [700, 513]), "last_query"),          # single-query kernel
-    ((1, 8, 2, 128, 400, 64, [390]), "chunk_sum"),               # generic kernels (a block of 64 queries)
+    ((1, 8, 2, 128, 400, 64, [390]), "chunk_sum"),               # tensor-core kernels for a block of 64 queries
+    ((1, 4, 2, 64, 300, 3, [290]), "chunk_sum"),                 # any-shape kernels (head_dim 64, 3 queries)
 ])
 def test_static_scratch_matches_workspace_call_twice(shape, mode):
     B, Hq, Hkv, d, cap, m, lens = shape
@@ -57,13 +59,19 @@ def test_static_scratch_matches_workspace_call_twice(shape, mode):
     P.caote_score(p, q, K, V, lens_t, base_ref if mode == "accum" else None, o_ref, sc_ref, ws)
     assert P.caote_read_status(ws) == 0
 
+    r = oracle_for(q, K, V, lens_t, scale=d ** -0.5, n_new=m, base_mode=mode, base=base0 if mode == "accum" else None)
     for call in range(2):
         o, sc = outputs()
         base = base0.clone()
         status = torch.full((1,), 99, dtype=torch.int32, device=DEV)
+        torch.cuda.synchronize()
+        free_before, in_use_before = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated()
         P.caote_score_static(p, q, K, V, lens_t, base if mode == "accum" else None, o, sc, status)
         torch.cuda.synchronize()
+        # nothing was allocated or freed on the device by the call (neither through torch nor behind its back)
+        assert torch.cuda.memory_allocated() == in_use_before and torch.cuda.mem_get_info()[0] == free_before
         assert status.item() == 0, f"call {call}: device status {status.item()}"
+        check_scores_and_o(r, sc, o, lens_t, f"{shape} {mode} call {call} against the oracle")
         what = f"{shape} {mode} call {call}"
         assert_close(f32(sc), f32(sc_ref), what + " scores", rtol=RTOL, atol=ATOL)
         assert_close(f32(o)[[b for b, n in enumerate(lens) if n > 0]],
