@@ -782,13 +782,16 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
         const int hd = 2 * gw + (lane >> 4), rl = lane & 15;
         const bool have = rl < C;
         const float* st = xstats + rl * kStatFloats;
-        const float rc = have ? st[hd] : -INFINITY;
+        // with carried base scores the eighth half-warp has no head (G <= 7): it merges the base scores instead,
+        // (sum of the others, largest) with the score itself as the key, through the same steps
+        const bool is_base = use_base && hd == 7;
+        const float rc = have ? (is_base ? 0.f : st[hd]) : -INFINITY;
         float m_fin = rc;
 #pragma unroll
         for (int off = 8; off > 0; off >>= 1) m_fin = fmaxf(m_fin, __shfl_xor_sync(0xffffffffu, m_fin, off));
         const float f = (rc == -INFINITY) ? 0.f : fast_exp2(rc - m_fin);
-        const float lr = have ? st[8 + hd] * f : 0.f, pm = have ? st[16 + hd] * f : 0.f;
-        const float sx = have ? st[24 + hd] : -INFINITY;
+        const float lr = have ? (is_base ? st[32] : st[8 + hd] * f) : 0.f, pm = have ? (is_base ? st[33] : st[16 + hd] * f) : 0.f;
+        const float sx = have ? (is_base ? st[33] : st[24 + hd]) : -INFINITY;
         float smx = sx;
 #pragma unroll
         for (int off = 8; off > 0; off >>= 1) smx = fmaxf(smx, __shfl_xor_sync(0xffffffffu, smx, off));
@@ -805,27 +808,19 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
           fin->inv_l[hd] = inv_l;
           fin->smax[hd] = smx;
           fin->crest[hd] = lsum * inv_l;
-        }
-        if (have) fac[rl * 8 + hd] = (use_base && hd == 7) ? 1.f : f * inv_l;
-        if (gw == 0) {
-          // carried base scores: the largest one apart from the sum of the others (both half-warps do it)
-          const float bm = have ? st[33] : 0.f, br = have ? st[32] : 0.f;
-          float bmx = bm;
-#pragma unroll
-          for (int off = 8; off > 0; off >>= 1) bmx = fmaxf(bmx, __shfl_xor_sync(0xffffffffu, bmx, off));
-          const uint32_t bb = (__ballot_sync(0xffffffffu, have && bm == bmx) >> (lane & 16)) & 0xffffu;
-          const int bstar = __ffs(bb) - 1;
-          float brs = br + ((rl != bstar) ? bm : 0.f);
-#pragma unroll
-          for (int off = 8; off > 0; off >>= 1) brs += __shfl_xor_sync(0xffffffffu, brs, off);
-          if (lane == 0) {
-            const float hbsum = use_base ? brs + bmx : 0.f;
-            fin->hbsum = hbsum;
-            fin->bmax = bmx;
-            fin->brest = brs;
-            fin->Htot = (counted ? (float)G : 0.f) + hbsum;
+          if (is_base) {
+            fin->hbsum = l;
+            fin->bmax = smx;
+            fin->brest = lsum;
+            fin->Htot = (counted ? (float)G : 0.f) + l;
+          } else if (!use_base && hd == 0) {
+            fin->hbsum = 0.f;
+            fin->bmax = 0.f;
+            fin->brest = 0.f;
+            fin->Htot = (float)G;
           }
         }
+        if (have) fac[rl * 8 + hd] = is_base ? 1.f : f * inv_l;
       }
       group_sync(1 + bg);
       {
