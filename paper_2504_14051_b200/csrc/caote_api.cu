@@ -519,7 +519,28 @@ static int launch_prefill_score(const Dims& dm, const void* q, const void* K, co
   return CAOTE_OK;
 }
 
+// The split heuristics of the prefill and any-shape paths look at the SM count: keep it current for this device
+// (cached per device; left at its default when there is no device, e.g. when only sizes are asked for).
+static void refresh_sm_count() {
+  static std::atomic<int> cached[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+    (void)cudaGetLastError();
+    return;
+  }
+  int n = cached[dev].load(std::memory_order_acquire);
+  if (n == 0) {
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) {
+      (void)cudaGetLastError();
+      return;
+    }
+    cached[dev].store(n, std::memory_order_release);
+  }
+  g_sm_count = n;
+}
+
 static size_t workspace_bytes(const caote_params_t* p) {
+  refresh_sm_count();
   const Dims dm = make_dims(p);
   size_t need = generic::carve(dm, nullptr, nullptr);
   if (decode_shape_ok(p)) {

@@ -23,6 +23,10 @@ struct Dims {
 
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// SMs of the current device, as far as the host-side split heuristics are concerned. The entry points refresh
+// it from the device attribute before they size or carve a workspace; without a device it stays at 148.
+inline int g_sm_count = 148;
+
 // Record the first device-side error in the status word (never overwrites an earlier one).
 __device__ inline void set_status(int* status, int code) { atomicCAS(status, 0, code); }
 

@@ -46,7 +46,7 @@ inline int round_up(int x, int a) { return (x + a - 1) / a * a; }
 inline int choose_splits(const Dims& dm) {
   const int row_tiles = (dm.R + kRT - 1) / kRT;
   const long ctas = (long)dm.units * row_tiles;
-  int s = (int)((148L * 4 + ctas - 1) / ctas);
+  int s = (int)(((long)g_sm_count * 4 + ctas - 1) / ctas);
   const int max_by_cap = (dm.cap + 2 * kKT - 1) / (2 * kKT);
   if (s > max_by_cap) s = max_by_cap;
   if (s > 32) s = 32;

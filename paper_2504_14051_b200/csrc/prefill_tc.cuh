@@ -52,7 +52,7 @@ struct Scratch {
 // that run as CTAs of their own; attn_combine_kernel merges them. A function of the shape only.
 inline int attn_splits(const Dims& dm) {
   const long long ctas = (long long)((dm.R + kTile - 1) / kTile) * dm.units;
-  long long ns = 148 / (ctas > 0 ? ctas : 1);
+  long long ns = g_sm_count / (ctas > 0 ? ctas : 1);
   const long long max_by_len = ((dm.cap + kTile - 1) / kTile) / 4;  // at least four tiles per split
   if (ns > max_by_len) ns = max_by_len;
   if (ns > 8) ns = 8;
@@ -255,8 +255,8 @@ __device__ __forceinline__ uint64_t desc_mn_major(uint32_t tile_addr, int ks) {
 
 
 // ---- attention pass ---------------------------------------------------------------------------------
-// Keys are walked in tiles of 64 so that three K/V stages, two P buffers (bf16 hi and lo parts each) and
-// the Q block fit in shared memory together; the tensor pipe then always has the next S = Q K^T queued
+// Keys are walked in tiles of 128: three K stages, two V stages and the Q block in shared memory, two S buffers,
+// O and one P buffer (bf16 hi and lo parts) in TMEM; the tensor pipe then always has the next S = Q K^T queued
 // while the threads are busy with the softmax of the current tile:
 //   tensor pipe:  QK(t+1)  PV(t)  QK(t+2)  PV(t+1) ...
 //   threads:      softmax(t) ............ softmax(t+1) ...
@@ -272,7 +272,7 @@ inline size_t attn_smem_bytes() {
   return 1024 + kTileBytes + (size_t)(kKStages + kVStages) * kKvTile + 2 * kRowThreads * sizeof(float) + 256;
 }
 
-// K-major / MN-major descriptors of k-step ks of a 64-key tile (boxes of 64 rows: kKvHalf apart).
+// K-major / MN-major descriptors of k-step ks of a key tile (boxes of kKeys rows x 64 channels: kKvHalf apart).
 __device__ __forceinline__ uint64_t desc_k_major64(uint32_t tile_addr, int ks) {
   return smem_desc(tile_addr + (ks >> 2) * kKvHalf + (ks & 3) * 32, 16, 1024);
 }
@@ -541,7 +541,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
   if (warp == 0) tmem_dealloc(tmem, 512);
 }
 
-// X[unit] = mean of the unit's M rows of o. grid = units, 128 threads (one per channel).
 // Merge the key splits of a unit: o = sum_s o_s 2^(stat_s - stat), stat = log2 sum_s 2^stat_s.
 // grid = (ceil(M / 4), units), 4 rows x 128 channels per CTA. Units that ran unsplit are left alone.
 __global__ void __launch_bounds__(4 * kD)
@@ -567,6 +566,7 @@ attn_combine_kernel(Dims dm, const int* __restrict__ len, Scratch sc, float* __r
   if (c == 0) sc.stats[(size_t)unit * sc.Mpad + R] = mx + log2f(tot);
 }
 
+// X[unit] = mean of the unit's M rows of o. grid = units, kXsumLanes x 128 threads (row lanes x channels).
 constexpr int kXsumLanes = 8;  // row lanes per channel: 8 x 128 threads per unit
 __global__ void __launch_bounds__(kXsumLanes * kD)
 xsum_kernel(Dims dm, const int* __restrict__ len, const float* __restrict__ o, Scratch sc) {
