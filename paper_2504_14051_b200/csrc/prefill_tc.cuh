@@ -28,6 +28,7 @@
 #include <cuda.h>
 
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace caote {
 namespace prefill {
@@ -92,23 +93,17 @@ inline size_t carve(const Dims& dm, char* base, Scratch* out) {
   return off;
 }
 
-// ---- PTX wrappers ---------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-  return ok != 0;
-}
+// ---- PTX wrappers (ptx.cuh), the waits built on them, and the tcgen05 wrappers ----------------------------
+using ptx::smem_u32;
+using ptx::mbar_init;
+using ptx::mbar_expect_tx;
+using ptx::mbar_arrive;
+using ptx::mbar_try_wait;
+using ptx::tma_load_2d;
+using ptx::bulk_load;
+using ptx::fence_async_smem;
+using ptx::fast_exp2;
+using ptx::tile_off;
 // Bounded wait. On expiry the error is recorded and the caller carries on (see the file comment).
 __device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, int* status) {
   if (mbar_try_wait(bar, parity)) return;
@@ -133,12 +128,6 @@ __device__ __forceinline__ void mbar_wait_idle(uint64_t* bar, uint32_t parity, i
     }
   }
 }
-__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -228,19 +217,10 @@ __device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-__device__ __forceinline__ float fast_exp2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
 __device__ __forceinline__ uint32_t pack_bf16(float x0, float x1) {
   uint32_t r;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(x1), "f"(x0));
   return r;
-}
-// Byte offset of 16-byte chunk `chunk16` (0..15 along 128 bf16) of row `row` in a staged tile.
-__device__ __forceinline__ uint32_t tile_off(int row, int chunk16) {
-  return (uint32_t)((chunk16 >> 3) * kHalfBytes + row * 128 + (((chunk16 & 7) ^ (row & 7)) << 4));
 }
 // Descriptors of k-step ks (16 of the 128 contraction elements) of a staged tile.
 //   K-major: contraction along the 128-byte rows: 32 bytes per step inside a box, second box after 4.
@@ -281,9 +261,6 @@ __device__ __forceinline__ uint64_t desc_mn_major64(uint32_t tile_addr, int ks) 
 }
 __host__ __device__ constexpr uint32_t instr_desc_n(bool b_mn_major, uint32_t n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((n >> 3) << 17) | ((128u >> 4) << 24);
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
 // o and row statistics of 128 query rows of one unit. grid = (row blocks, units), 352 threads:
@@ -601,11 +578,6 @@ constexpr int kQStages = 3;
 
 inline size_t score_smem_bytes() {
   return 1024 + 2 * kTileBytes + kQStages * (size_t)kQStage + (kD + kScoreKeys) * sizeof(float) + 256;
-}
-__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
-  asm volatile(
-      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-      ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 
 // CAOTE scores of 256 keys of one unit. grid = (key tile pairs, units), 576 threads: warps 0..15 are the
