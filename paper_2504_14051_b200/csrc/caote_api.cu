@@ -4,6 +4,7 @@
 #include <cstdio>
 #include <cstring>
 #include <mutex>
+#include <utility>
 #include <vector>
 
 #include "common.cuh"
@@ -91,6 +92,23 @@ struct TraceScope {
     }                                      \
     if (rc__ != CAOTE_OK) return rc__;     \
   } while (0)
+
+// Launch with the programmatic-serialization attribute: the kernel may be scheduled while its predecessor in the
+// stream is still running and waits for it in its first statement (ptx::pdl_wait). Only for kernels that do so.
+template <typename... KArgs, typename... Args>
+static void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  (void)cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);  // (errors are picked up by after_launch)
+}
 
 static bool params_ok(const caote_params_t* p) {
   if (!p) return false;
@@ -377,13 +395,15 @@ static int launch_decode_cluster(const Dims& dm, const void* q, const void* K, c
   cfg.blockDim = dim3(dcl::kThreads);
   cfg.dynamicSmemBytes = dcl::smem_bytes();
   cfg.stream = st;
-  cudaLaunchAttribute at[1];
+  cudaLaunchAttribute at[2];
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = (unsigned)c;
   at[0].val.clusterDim.y = 1;
   at[0].val.clusterDim.z = 1;
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // (the kernel starts with ptx::pdl_wait)
+  at[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   int* status = reinterpret_cast<int*>(ws);
   const long long wait_cycles = g_wait_cycles.load(std::memory_order_relaxed);
   CAOTE_LAUNCH("decode_cluster_kernel", st, {
@@ -433,21 +453,21 @@ static int launch_decode_score(const Dims& dm, const void* q, const void* K, con
     }
   }
   CAOTE_LAUNCH("decode_plan_kernel", st,
-               decode::plan_kernel<<<1, 1024, 0, st>>>(dm.units, dm.Hkv, dm.cap, len, pl, status));
+               launch_pdl(decode::plan_kernel, dim3(1), dim3(1024), 0, st, dm.units, dm.Hkv, dm.cap, len, pl, status));
   const int tiles_per_unit = (dm.cap + decode::kT - 1) / decode::kT;
   const long long max_items = (long long)dm.units * ((tiles_per_unit + pl.tpi - 1) / pl.tpi);
   const int grid = (int)(max_items < grid_limit ? max_items : grid_limit);
   if (!vsum) {
     CAOTE_LAUNCH("decode_tc_kernel", st,
-                 decode::decode_tc_kernel<false><<<grid, decode::kTcThreads, decode::tc_smem_bytes(false), st>>>(
+                 launch_pdl(decode::decode_tc_kernel<false>, dim3(grid), dim3(decode::kTcThreads), decode::tc_smem_bytes(false), st, 
                      tmK, tmV, tmQ, dm, len, base, o, scores, nullptr, pl, status));
   } else {
     // FastCAOTE: one pass over K and V, then scores from the stored logits and distances
     CAOTE_LAUNCH("decode_tc_fast_kernel", st,
-                 decode::decode_tc_kernel<true><<<grid, decode::kTcThreads, decode::tc_smem_bytes(true), st>>>(
+                 launch_pdl(decode::decode_tc_kernel<true>, dim3(grid), dim3(decode::kTcThreads), decode::tc_smem_bytes(true), st, 
                      tmK, tmV, tmQ, dm, len, base, o, scores, vsum, pl, status));
     dim3 fgrid(tiles_per_unit, dm.units);
-    CAOTE_LAUNCH("fast_finish_kernel", st, decode::fast_finish_kernel<<<fgrid, decode::kT, 0, st>>>(dm, len, base, scores, pl));
+    CAOTE_LAUNCH("fast_finish_kernel", st, launch_pdl(decode::fast_finish_kernel, dim3(fgrid), dim3(decode::kT), 0, st, dm, len, base, scores, pl));
   }
   *used = true;
   return CAOTE_OK;
@@ -497,22 +517,22 @@ static int launch_prefill_score(const Dims& dm, const void* q, const void* K, co
   {
     dim3 grid((dm.R + prefill::kTile - 1) / prefill::kTile, dm.units, sc.nsplit);
     CAOTE_LAUNCH("prefill_attn_kernel", st,
-                 prefill::attn_kernel<<<grid, prefill::kAttnThreads, prefill::attn_smem_bytes(), st>>>(tmQ, tmK64, tmV64, dm, len,
+                 launch_pdl(prefill::attn_kernel, dim3(grid), dim3(prefill::kAttnThreads), prefill::attn_smem_bytes(), st, tmQ, tmK64, tmV64, dm, len,
                                                                                                     sc, o, status));
   }
   if (sc.nsplit > 1) {
     dim3 grid((dm.R + 3) / 4, dm.units);
-    CAOTE_LAUNCH("prefill_attn_combine_kernel", st, prefill::attn_combine_kernel<<<grid, 4 * prefill::kD, 0, st>>>(dm, len, sc, o));
+    CAOTE_LAUNCH("prefill_attn_combine_kernel", st, launch_pdl(prefill::attn_combine_kernel, dim3(grid), dim3(4 * prefill::kD), 0, st, dm, len, sc, o));
   }
   if (vsum) {
     CAOTE_LAUNCH("fast_mean_kernel", st, fast::mean_kernel<<<dm.units, prefill::kD, 0, st>>>(dm.Hkv, dm.cap, prefill::kD, len, vsum, sc.X));
   } else {
-    CAOTE_LAUNCH("prefill_xsum_kernel", st, prefill::xsum_kernel<<<dm.units, prefill::kXsumLanes * prefill::kD, 0, st>>>(dm, len, o, sc));
+    CAOTE_LAUNCH("prefill_xsum_kernel", st, launch_pdl(prefill::xsum_kernel, dim3(dm.units), dim3(prefill::kXsumLanes * prefill::kD), 0, st, dm, len, o, sc));
   }
   {
     dim3 grid((dm.cap + prefill::kScoreKeys - 1) / prefill::kScoreKeys, dm.units);
     CAOTE_LAUNCH("prefill_score_kernel", st,
-                 prefill::score_kernel<<<grid, prefill::kScoreThreads, prefill::score_smem_bytes(), st>>>(
+                 launch_pdl(prefill::score_kernel, dim3(grid), dim3(prefill::kScoreThreads), prefill::score_smem_bytes(), st, 
                      tmQ, tmK, dm, (const __nv_bfloat16*)V, len, sc, scores, status));
   }
   *used = true;
@@ -646,7 +666,7 @@ int caote_append(const caote_params_t* p, void* K, void* V, float* base, int32_t
   const Dims dm = make_dims(p);
   const int row_bytes = dm.D * (p->dtype == CAOTE_BF16 ? 2 : 4);
   cudaStream_t st = (cudaStream_t)stream;
-  CAOTE_LAUNCH("append_kernel", st, sel::append_kernel<<<dim3(dm.units, (dm.m + 7) / 8), 256, 0, st>>>(dm.Hkv, dm.cap, dm.m, row_bytes, (char*)K, (char*)V, base, pos,
+  CAOTE_LAUNCH("append_kernel", st, launch_pdl(sel::append_kernel, dim3(dim3(dm.units, (dm.m + 7) / 8)), dim3(256), 0, st, dm.Hkv, dm.cap, dm.m, row_bytes, (char*)K, (char*)V, base, pos,
                                                len, n_seen, (const char*)k_new, (const char*)v_new,
                                                (int*)workspace, dm.B, (int*)workspace + 4));
   return CAOTE_OK;
@@ -764,7 +784,7 @@ int caote_select_evict(const caote_params_t* p, const float* scores, const int32
   if (rc) return rc;
   const Dims dm = make_dims(p);
   cudaStream_t st = (cudaStream_t)stream;
-  CAOTE_LAUNCH("select_kernel", st, sel::select_kernel<<<dm.units, sel::kSelThreads, 0, st>>>(
+  CAOTE_LAUNCH("select_kernel", st, launch_pdl(sel::select_kernel, dim3(dm.units), dim3(sel::kSelThreads), 0, st, 
       dm.Hkv, dm.cap, scores, len, budget, pos, evict_idx, max_evict, n_evict, (int*)workspace));
   return CAOTE_OK;
 }
@@ -805,14 +825,14 @@ int caote_compact(const caote_params_t* p, void* K, void* V, float* base, int32_
   const int row_bytes = dm.D * (p->dtype == CAOTE_BF16 ? 2 : 4);
   cudaStream_t st = (cudaStream_t)stream;
   if (mode == CAOTE_COMPACT_FILL) {
-    CAOTE_LAUNCH("compact_fill_kernel", st, sel::compact_fill_kernel<<<dm.units, 256, 0, st>>>(dm.Hkv, dm.cap, row_bytes, (char*)K, (char*)V, base, pos,
+    CAOTE_LAUNCH("compact_fill_kernel", st, launch_pdl(sel::compact_fill_kernel, dim3(dm.units), dim3(256), 0, st, dm.Hkv, dm.cap, row_bytes, (char*)K, (char*)V, base, pos,
                                                        len, evict_idx, max_evict, n_evict));
   } else {
     dim3 grid(dm.units, 3);
     CAOTE_LAUNCH("compact_stable_kernel", st, sel::compact_stable_kernel<<<grid, 256, (size_t)sel::kStableTile * row_bytes, st>>>(
         dm.Hkv, dm.cap, row_bytes, (char*)K, (char*)V, base, pos, len, evict_idx, max_evict, n_evict));
   }
-  CAOTE_LAUNCH("update_len_kernel", st, sel::update_len_kernel<<<(dm.B + 127) / 128, 128, 0, st>>>(dm.B, len, n_evict));
+  CAOTE_LAUNCH("update_len_kernel", st, launch_pdl(sel::update_len_kernel, dim3((dm.B + 127) / 128), dim3(128), 0, st, dm.B, len, n_evict));
   return CAOTE_OK;
 }
 
@@ -855,7 +875,7 @@ static int step_impl(const caote_params_t* p, const void* q, const void* k_new, 
     cudaStream_t st = (cudaStream_t)stream;
     int* hdr = reinterpret_cast<int*>(workspace);
     CAOTE_LAUNCH("select_compact_kernel", st,
-                 sel::select_compact_kernel<<<dm.units, sel::kSelThreads, 0, st>>>(
+                 launch_pdl(sel::select_compact_kernel, dim3(dm.units), dim3(sel::kSelThreads), 0, st, 
                      dm.B, dm.Hkv, dm.cap, row_bytes, scores, (char*)K, (char*)V, base, pos, len, budget, evict_idx,
                      max_evict, n_evict, hdr, hdr + 4, vsum, bf16 ? 2 : 4));
     return CAOTE_OK;

@@ -268,6 +268,8 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
                       const __grid_constant__ CUtensorMap tmQ, Dims dm, const int* __restrict__ len,
                       float* __restrict__ base, float* __restrict__ o, float* __restrict__ scores, int* status,
                       long long wait_cycles) {
+  ptx::pdl_wait();
+  ptx::pdl_trigger();
   extern __shared__ char smem_raw[];
   char* sm = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   char* tilesK = sm;                                                   // [kKS][kTileBytes]

@@ -111,6 +111,8 @@ inline size_t carve(const Dims& dm, char* base, Plan* out, int grid) {
 // ---- plan: items per unit, their prefix sum, and cleared counters / flags (one CTA) -------------
 __global__ void __launch_bounds__(1024)
 plan_kernel(int units, int Hkv, int cap, const int* __restrict__ len, Plan pl, int* status) {
+  ptx::pdl_wait();
+  ptx::pdl_trigger();
   __shared__ int warp_tot[32];
   __shared__ int carry;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;

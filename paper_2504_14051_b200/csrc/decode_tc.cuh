@@ -169,6 +169,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                  const __grid_constant__ CUtensorMap tmQ, Dims dm, const int* __restrict__ len,
                  float* __restrict__ base, float* __restrict__ o, float* __restrict__ scores, const float* __restrict__ vsum,
                  Plan pl, int* status) {
+  ptx::pdl_wait();
+  ptx::pdl_trigger();
   // FastCAOTE has no score ring: its shared memory goes to a deeper attention ring
   constexpr int kA = kFast ? kASlotsFast : kASlots;
   constexpr int kQ = kFast ? kQBufsFast : kQBufs;  // a buffer is reused only after every reader of its item has moved on:
@@ -818,6 +820,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
 // logits, the unit's final softmax statistics and the stored distances. grid = (tiles, units), kT threads.
 __global__ void __launch_bounds__(kT)
 fast_finish_kernel(Dims dm, const int* __restrict__ len, float* __restrict__ base, float* __restrict__ scores, Plan pl) {
+  ptx::pdl_wait();
+  ptx::pdl_trigger();
   const int unit = blockIdx.y, tile = blockIdx.x, b = unit / dm.Hkv;
   const int n = len[b], tok = tile * kT + threadIdx.x;
   if (n <= 0 || n > dm.cap || tok >= n) return;

@@ -271,6 +271,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK64,
             const __grid_constant__ CUtensorMap tmV64, Dims dm, const int* __restrict__ len, Scratch sc,
             float* __restrict__ o, int* status) {
+  ptx::pdl_wait();
+  ptx::pdl_trigger();
   extern __shared__ char smem_raw[];
   char* sm = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   char* Qs = sm;
@@ -522,6 +524,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
 // grid = (ceil(M / 4), units), 4 rows x 128 channels per CTA. Units that ran unsplit are left alone.
 __global__ void __launch_bounds__(4 * kD)
 attn_combine_kernel(Dims dm, const int* __restrict__ len, Scratch sc, float* __restrict__ o) {
+  ptx::pdl_wait();
+  ptx::pdl_trigger();
   const int unit = blockIdx.y, c = threadIdx.x % kD, R = blockIdx.x * 4 + threadIdx.x / kD;
   const int n = len[unit / dm.Hkv];
   if (n == 0 || n < dm.m || n > dm.cap || R >= dm.R) return;
@@ -547,6 +551,8 @@ attn_combine_kernel(Dims dm, const int* __restrict__ len, Scratch sc, float* __r
 constexpr int kXsumLanes = 8;  // row lanes per channel: 8 x 128 threads per unit
 __global__ void __launch_bounds__(kXsumLanes * kD)
 xsum_kernel(Dims dm, const int* __restrict__ len, const float* __restrict__ o, Scratch sc) {
+  ptx::pdl_wait();
+  ptx::pdl_trigger();
   __shared__ float part[kXsumLanes][kD];
   const int unit = blockIdx.x, c = threadIdx.x % kD, lane = threadIdx.x / kD;
   const int n = len[unit / dm.Hkv];
@@ -588,6 +594,8 @@ __global__ void __launch_bounds__(kScoreThreads, 1)
 score_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, Dims dm,
              const __nv_bfloat16* __restrict__ V, const int* __restrict__ len, Scratch sc,
              float* __restrict__ scores, int* status) {
+  ptx::pdl_wait();
+  ptx::pdl_trigger();
   extern __shared__ char smem_raw[];
   char* sm = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   char* Ks = sm;                                                     // [2] key tiles

@@ -69,6 +69,15 @@ __device__ __forceinline__ uint64_t policy_evict_last() {
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
+// ---- programmatic dependent launch ------------------------------------------------------------------------
+// A kernel launched with the programmatic-serialization attribute may be scheduled while the kernel before it in
+// the stream is still running. pdl_wait() blocks until that kernel has completed and its writes are visible: it
+// is the first statement of every kernel launched that way, before any global access. pdl_trigger() lets the NEXT
+// kernel of the stream be scheduled once every CTA of this one has got this far (it then sits in its own
+// pdl_wait()): launch latency and prologue overlap the tail of this kernel. Both are no-ops in a plain launch.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- math -----------------------------------------------------------------------------------------------
 // 2^x, hardware approximation (2 ulp); 2^-inf = 0.
 __device__ __forceinline__ float fast_exp2(float x) {

@@ -5,6 +5,7 @@
 #pragma once
 
 #include "common.cuh"
+#include "ptx.cuh"
 #include "fast.cuh"
 
 namespace caote {
@@ -183,6 +184,8 @@ __global__ void __launch_bounds__(kSelThreads)
 select_kernel(int Hkv, int cap, const float* __restrict__ scores, const int* __restrict__ len,
               const int* __restrict__ budget, const int* __restrict__ pos, int* __restrict__ evict_idx,
               int max_evict, int* __restrict__ n_evict, int* status) {
+  ptx::pdl_wait();
+  ptx::pdl_trigger();
   select_unit(blockIdx.x, Hkv, cap, scores, len, budget, pos, evict_idx, max_evict, n_evict, status);
 }
 
@@ -235,6 +238,8 @@ __global__ void __launch_bounds__(256)
 compact_fill_kernel(int Hkv, int cap, int row_bytes, char* __restrict__ K, char* __restrict__ V,
                     float* __restrict__ base, int* __restrict__ pos, const int* __restrict__ len,
                     const int* __restrict__ evict_idx, int max_evict, const int* __restrict__ n_evict) {
+  ptx::pdl_wait();
+  ptx::pdl_trigger();
   compact_fill_unit(blockIdx.x, n_evict[blockIdx.x / Hkv], Hkv, cap, row_bytes, K, V, base, pos, len, evict_idx, max_evict);
 }
 
@@ -246,6 +251,8 @@ select_compact_kernel(int B, int Hkv, int cap, int row_bytes, const float* __res
                       char* __restrict__ V, float* __restrict__ base, int* __restrict__ pos, int* __restrict__ len,
                       const int* __restrict__ budget, int* __restrict__ evict_idx, int max_evict,
                       int* __restrict__ n_evict, int* status, int* ticket, float* __restrict__ vsum, int elt_bytes) {
+  ptx::pdl_wait();
+  ptx::pdl_trigger();
   __shared__ int s_last;
   const int unit = blockIdx.x;
   const int k = select_unit(unit, Hkv, cap, scores, len, budget, pos, evict_idx, max_evict, n_evict, status);
@@ -279,6 +286,8 @@ __global__ void __launch_bounds__(256)
 compact_stable_kernel(int Hkv, int cap, int row_bytes, char* __restrict__ K, char* __restrict__ V,
                       float* __restrict__ base, int* __restrict__ pos, const int* __restrict__ len,
                       const int* __restrict__ evict_idx, int max_evict, const int* __restrict__ n_evict) {
+  ptx::pdl_wait();
+  ptx::pdl_trigger();
   extern __shared__ __align__(16) char tile[];  // kStableTile * max(row_bytes, 8)
   const int unit = blockIdx.x, b = unit / Hkv, which = blockIdx.y;
   const int k = n_evict[b];
@@ -325,6 +334,8 @@ compact_stable_kernel(int Hkv, int cap, int row_bytes, char* __restrict__ K, cha
 
 // len[b] -= n_evict[b], after every unit of the sequence has been compacted.
 __global__ void update_len_kernel(int B, int* __restrict__ len, const int* __restrict__ n_evict) {
+  ptx::pdl_wait();
+  ptx::pdl_trigger();
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b < B) len[b] -= n_evict[b];
 }
@@ -335,6 +346,8 @@ append_kernel(int Hkv, int cap, int m, int row_bytes, char* __restrict__ K, char
               float* __restrict__ base, int* __restrict__ pos, int* __restrict__ len,
               int* __restrict__ n_seen, const char* __restrict__ k_new,
               const char* __restrict__ v_new, int* status, int B, int* ticket) {
+  ptx::pdl_wait();
+  ptx::pdl_trigger();
   const int unit = blockIdx.x, b = unit / Hkv;
   const int n = len[b];
   const bool fits = n >= 0 && n + m <= cap;
