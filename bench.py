@@ -412,7 +412,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--pool", type=int, default=64, help="distinct per-step input sets kept on the device")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--method", default="caote", choices=["caote", "fast"],
+    ap.add_argument("--method", default="caote", choices=["caote", "fast", "sum_errors", "post_evict"],
                     help="caote: the CAOTE score (the headline); fast: FastCAOTE (Sec. 3.3), X = mean of the cached values")
     ap.add_argument("--dry-run", action="store_true",
                     help="exercise the launcher and the cross-rank aggregation on CPU (gloo) with made-up per-rank "

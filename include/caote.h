@@ -266,11 +266,25 @@ CAOTE_API int caote_score_sum_errors(const caote_params_t* params, const void* q
  *   q, K, V, len as passed to caote_score; evict_idx, max_evict, n_evict as written by caote_select_evict;
  *   o  in:  the pre-eviction output caote_score wrote, [B, Hq, m, d] fp32;
  *   o_post out, same shape (may alias o).
- * Needs no workspace. It recomputes the rows' softmax normalisers with one pass over K on the CUDA cores:
- * a correction step for callers that want it, not part of the timed path. */
+ * Needs no workspace. It recomputes the rows' softmax normalisers with one pass over K on the CUDA cores;
+ * caote_post_evict_output_ws below avoids that pass where it can. */
 CAOTE_API int caote_post_evict_output(const caote_params_t* params, const void* q, const void* K, const void* V,
                             const int32_t* len, const int32_t* evict_idx, int32_t max_evict,
                             const int32_t* n_evict, const float* o, float* o_post, caote_stream_t stream);
+
+/* The same result from the softmax statistics that scoring already produced (Sec. 3.1: the weights
+ * alpha_{r,e} of the evicted tokens are all the correction needs): `workspace` is the one the caote_score /
+ * caote_step... call that scored these slots ran on, with the same params, and nothing else has run on it
+ * since except caote_select_evict[_greedy]. The tensor-core kernels (single-query decode on thread-block
+ * clusters; chunked prefill) leave every row's log-sum-exp there and say so in the workspace header; this
+ * call then reads q, o and only the evicted K / V rows, which makes it a small fraction of a scoring call.
+ * After any other scoring path the header says "none" and the call does what caote_post_evict_output does.
+ * Arguments as above; workspace (device, 256-byte aligned) of at least caote_workspace_bytes(params),
+ * read only. Errors as above, and CAOTE_ERR_INVALID_ARG for a missing, short or misaligned workspace. */
+CAOTE_API int caote_post_evict_output_ws(const caote_params_t* params, const void* q, const void* K, const void* V,
+                               const int32_t* len, const int32_t* evict_idx, int32_t max_evict,
+                               const int32_t* n_evict, const float* o, float* o_post, const void* workspace,
+                               size_t workspace_bytes, caote_stream_t stream);
 
 /* Synchronise the stream, copy the status word to *status_out (host pointer) and reset it to CAOTE_OK.
  * The word holds the first device-side error since the last reset. */

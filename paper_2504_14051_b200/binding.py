@@ -96,6 +96,8 @@ def lib() -> ctypes.CDLL:
     L.caote_score_sum_errors.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     L.caote_post_evict_output.restype = ctypes.c_int
     L.caote_post_evict_output.argtypes = [pp, vp, vp, vp, vp, vp, i32, vp, vp, vp, vp]
+    L.caote_post_evict_output_ws.restype = ctypes.c_int
+    L.caote_post_evict_output_ws.argtypes = [pp, vp, vp, vp, vp, vp, i32, vp, vp, vp, vp, sz, vp]
     L.caote_read_status.restype = ctypes.c_int
     L.caote_read_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32)]
     L.caote_status_string.restype = ctypes.c_char_p
@@ -237,6 +239,14 @@ def caote_post_evict_output(p, q, K, V, lens, evict_idx, n_evict, o, o_post, str
     _check("caote_post_evict_output",
            lib().caote_post_evict_output(ctypes.byref(p), _p(q), _p(K), _p(V), _p(lens), _p(evict_idx),
                                          evict_idx.shape[-1], _p(n_evict), _p(o), _p(o_post), _stream(stream)))
+
+
+def caote_post_evict_output_ws(p, q, K, V, lens, evict_idx, n_evict, o, o_post, workspace, stream=None):
+    """The same from the softmax statistics the scoring call left in `workspace`, where it left any."""
+    _check("caote_post_evict_output_ws",
+           lib().caote_post_evict_output_ws(ctypes.byref(p), _p(q), _p(K), _p(V), _p(lens), _p(evict_idx),
+                                            evict_idx.shape[-1], _p(n_evict), _p(o), _p(o_post), _p(workspace),
+                                            workspace.numel(), _stream(stream)))
 
 
 def caote_read_status(workspace, stream=None) -> int:

@@ -1,7 +1,11 @@
 """A budgeted KV cache driven through the C ABI: the call a user of the library makes per step.
 
 Holds the caller-owned device buffers (K, V, base, pos, len, scores, ...) and forwards each step to
-``caote_step`` (append the new tokens, score, select, compact). No arithmetic happens here.
+``caote_step`` (append the new tokens, score, select, compact), or, for the variants that have no fused entry
+point, to the same calls one after the other. No arithmetic happens here.
+
+method: "caote" (Sec. 3.2 score), "fast" (FastCAOTE, Sec. 3.3), "sum_errors" (the per-row errors added up),
+"post_evict" (the "caote" step that also returns the attention output over the retained tokens, Sec. 3.1).
 """
 from __future__ import annotations
 
@@ -40,9 +44,10 @@ class EvictionCache:
         self.o = torch.zeros((B, Hq, m, d), dtype=torch.float32, device=dev)
         self.workspace = C.alloc_workspace(self.params, dev)
         # FastCAOTE (Sec. 3.3) scores against the mean of the cached values: the per-unit sum of V rows is state
-        assert method in ("caote", "fast")
+        assert method in ("caote", "fast", "sum_errors", "post_evict")
         self.method = method
         self.vsum = torch.zeros((B, Hkv, d), dtype=torch.float32, device=dev) if method == "fast" else None
+        self.o_post = torch.zeros_like(self.o) if method == "post_evict" else None
 
     def load(self, K, V, lens, base=None, pos=None):
         """Install an existing cache state (copied into the owned buffers)."""
@@ -61,7 +66,23 @@ class EvictionCache:
             C.caote_vsum(self.params, self.V, self.lens, self.vsum)
 
     def step(self, q, k_new, v_new, stream=None):
-        """One eviction step; returns the pre-eviction attention output o [B, Hq, m, d]."""
+        """One eviction step; returns the pre-eviction attention output o [B, Hq, m, d] (method "post_evict":
+        the output over the retained tokens)."""
+        if self.method in ("sum_errors", "post_evict"):
+            p, ws = self.params, self.workspace
+            C.caote_append(p, self.K, self.V, self.base, self.pos, self.lens, self.n_seen, k_new, v_new, ws, stream)
+            if self.method == "sum_errors":
+                C.caote_score_sum_errors(p, q, self.K, self.V, self.lens, self.o, self.scores, ws, stream)
+            else:
+                C.caote_score(p, q, self.K, self.V, self.lens, self.base, self.o, self.scores, ws, stream)
+            C.caote_select_evict(p, self.scores, self.lens, self.budget, self.pos, self.evict_idx, self.n_evict, ws,
+                                 stream)
+            if self.method == "post_evict":
+                C.caote_post_evict_output_ws(p, q, self.K, self.V, self.lens, self.evict_idx, self.n_evict, self.o,
+                                             self.o_post, ws, stream)
+            C.caote_compact(p, self.K, self.V, self.base, self.pos, self.lens, self.evict_idx, self.n_evict,
+                            self.compact_mode, ws, stream)
+            return self.o_post if self.method == "post_evict" else self.o
         if self.vsum is not None:
             C.caote_step_fast(self.params, q, k_new, v_new, self.K, self.V, self.base, self.pos, self.lens,
                               self.n_seen, self.budget, self.vsum, self.o, self.scores, self.evict_idx, self.n_evict,

@@ -601,13 +601,15 @@ static int static_scratch_address(char** out) {
 template <typename T, int D>
 static int launch_post_evict(const Dims& dm, const void* q, const void* K, const void* V, const int* len,
                              const int* evict_idx, int max_evict, const int* n_evict, const float* o, float* o_post,
-                             cudaStream_t st) {
+                             const char* ws, cudaStream_t st) {
   const size_t smem = post::smem_bytes<D>();
   int rc = allow_smem(post::post_evict_kernel<T, D>, smem);
   if (rc) return rc;
   dim3 grid((dm.R + post::kRows - 1) / post::kRows, dm.units);
   CAOTE_LAUNCH("post_evict_kernel", st, post::post_evict_kernel<T, D><<<grid, 32 * post::kRows, smem, st>>>(
-      dm, (const T*)q, (const T*)K, (const T*)V, len, evict_idx, max_evict, n_evict, o, o_post));
+      dm, (const T*)q, (const T*)K, (const T*)V, len, evict_idx, max_evict, n_evict, o, o_post,
+      ws ? reinterpret_cast<const int*>(ws) + kStatTagIndex : nullptr,
+      ws ? reinterpret_cast<const float*>(ws + kHeaderBytes) : nullptr, (dm.R + prefill::kTile - 1) / prefill::kTile * prefill::kTile));
   return CAOTE_OK;
 }
 
@@ -915,9 +917,9 @@ int caote_step_fast(const caote_params_t* p, const void* q, const void* k_new, c
                    n_evict, compact_mode, workspace, workspace_bytes_, stream);
 }
 
-int caote_post_evict_output(const caote_params_t* p, const void* q, const void* K, const void* V, const int32_t* len,
-                            const int32_t* evict_idx, int32_t max_evict, const int32_t* n_evict, const float* o,
-                            float* o_post, caote_stream_t stream) {
+static int post_evict_impl(const caote_params_t* p, const void* q, const void* K, const void* V, const int32_t* len,
+                           const int32_t* evict_idx, int32_t max_evict, const int32_t* n_evict, const float* o,
+                           float* o_post, const char* ws, caote_stream_t stream) {
   if (!params_ok(p) || !q || !K || !V || !len || !evict_idx || !n_evict || !o || !o_post || max_evict < 1)
     return CAOTE_ERR_INVALID_ARG;
   if (!params_supported(p)) return CAOTE_ERR_UNSUPPORTED;
@@ -927,11 +929,27 @@ int caote_post_evict_output(const caote_params_t* p, const void* q, const void* 
   const Dims dm = make_dims(p);
   cudaStream_t st = (cudaStream_t)stream;
   if (p->dtype == CAOTE_BF16) {
-    if (dm.D == 128) return launch_post_evict<__nv_bfloat16, 128>(dm, q, K, V, len, evict_idx, max_evict, n_evict, o, o_post, st);
-    return launch_post_evict<__nv_bfloat16, 64>(dm, q, K, V, len, evict_idx, max_evict, n_evict, o, o_post, st);
+    if (dm.D == 128) return launch_post_evict<__nv_bfloat16, 128>(dm, q, K, V, len, evict_idx, max_evict, n_evict, o, o_post, ws, st);
+    return launch_post_evict<__nv_bfloat16, 64>(dm, q, K, V, len, evict_idx, max_evict, n_evict, o, o_post, ws, st);
   }
-  if (dm.D == 128) return launch_post_evict<float, 128>(dm, q, K, V, len, evict_idx, max_evict, n_evict, o, o_post, st);
-  return launch_post_evict<float, 64>(dm, q, K, V, len, evict_idx, max_evict, n_evict, o, o_post, st);
+  if (dm.D == 128) return launch_post_evict<float, 128>(dm, q, K, V, len, evict_idx, max_evict, n_evict, o, o_post, ws, st);
+  return launch_post_evict<float, 64>(dm, q, K, V, len, evict_idx, max_evict, n_evict, o, o_post, ws, st);
+}
+
+int caote_post_evict_output(const caote_params_t* p, const void* q, const void* K, const void* V, const int32_t* len,
+                            const int32_t* evict_idx, int32_t max_evict, const int32_t* n_evict, const float* o,
+                            float* o_post, caote_stream_t stream) {
+  return post_evict_impl(p, q, K, V, len, evict_idx, max_evict, n_evict, o, o_post, nullptr, stream);
+}
+
+int caote_post_evict_output_ws(const caote_params_t* p, const void* q, const void* K, const void* V, const int32_t* len,
+                               const int32_t* evict_idx, int32_t max_evict, const int32_t* n_evict, const float* o,
+                               float* o_post, const void* workspace, size_t workspace_bytes_, caote_stream_t stream) {
+  if (!params_ok(p)) return CAOTE_ERR_INVALID_ARG;
+  if (!params_supported(p)) return CAOTE_ERR_UNSUPPORTED;
+  const int rc = score_workspace_check(p, workspace, workspace_bytes_);
+  if (rc) return rc;
+  return post_evict_impl(p, q, K, V, len, evict_idx, max_evict, n_evict, o, o_post, (const char*)workspace, stream);
 }
 
 int caote_read_status(void* workspace, caote_stream_t stream, int32_t* status_out) {

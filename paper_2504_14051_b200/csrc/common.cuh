@@ -13,6 +13,12 @@ namespace caote {
 // [0, 256)            header: int32 status word at offset 0
 // [256, ...)          per-call scratch, carved by the entry point that uses it
 constexpr size_t kHeaderBytes = 256;
+// Word kStatTagIndex of the workspace header says which softmax statistics the last scoring call left at
+// workspace + kHeaderBytes for the post-eviction output to reuse (reference + log2(sum) of the log2-domain
+// logits): per query head of a unit ([units][8], single-query cluster kernel), per query row of a unit
+// ([units][padded rows], tensor-core prefill kernels), or none.
+constexpr int kStatTagIndex = 8;
+constexpr int kStatNone = 0, kStatPerHead = 1, kStatPerRow = 2;
 
 struct Dims {
   int B, Hq, Hkv, G, D, cap, m, R;  // R = G * m query rows per unit

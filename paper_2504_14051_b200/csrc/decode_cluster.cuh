@@ -338,6 +338,7 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
     ctl[0] = 0;
     ctl[1] = 0;
     ctl[2] = 0;
+    if (blockIdx.x == 0) status[kStatTagIndex] = kStatPerHead;  // which statistics this call leaves behind
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     // the first unit's merge: what the peers will push into this CTA
     mbar_expect_tx(r1, r1_bytes);
@@ -806,7 +807,10 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
         const float l = lsum + pmf;
         const float inv_l = (hd < G && l > 0.f) ? __fdividef(1.f, l) : 0.f;
         if (rl == 0) {
-          fin->m[hd] = (hd < G) ? m_fin + __log2f(l) : 0.f;
+          const float mstat = (hd < G) ? m_fin + __log2f(l) : 0.f;
+          fin->m[hd] = mstat;
+          if (bg == 0 && rank == 0 && hd < G)  // left for the post-eviction output: alpha_j = 2^(s_j - mstat)
+            reinterpret_cast<float*>(reinterpret_cast<char*>(status) + kHeaderBytes)[(size_t)w.unit * 8 + hd] = mstat;
           fin->inv_l[hd] = inv_l;
           fin->smax[hd] = smx;
           fin->crest[hd] = lsum * inv_l;

@@ -116,7 +116,7 @@ plan_kernel(int units, int Hkv, int cap, const int* __restrict__ len, Plan pl, i
   __shared__ int warp_tot[32];
   __shared__ int carry;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (tid == 0) { carry = 0; pl.item_prefix[0] = 0; pl.work[0] = 0; pl.work[1] = 0; }
+  if (tid == 0) { carry = 0; pl.item_prefix[0] = 0; pl.work[0] = 0; pl.work[1] = 0; status[kStatTagIndex] = kStatNone; }
   __syncthreads();
   for (int u0 = 0; u0 < units; u0 += 1024) {
     const int u = u0 + tid;

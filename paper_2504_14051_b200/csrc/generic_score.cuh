@@ -132,6 +132,7 @@ attn_partial_kernel(Dims dm, const T* __restrict__ q, const T* __restrict__ K, c
   const int unit = blockIdx.z, split = blockIdx.y, rt = blockIdx.x;
   const int b = unit / dm.Hkv, h = unit % dm.Hkv;
   const int n = len[b];
+  if (threadIdx.x == 0 && unit == 0 && split == 0 && rt == 0) status[kStatTagIndex] = kStatNone;
   if (n == 0) return;
   if (n < dm.m || n > dm.cap) {
     if (threadIdx.x == 0) set_status(status, CAOTE_ERR_BAD_LENGTH);

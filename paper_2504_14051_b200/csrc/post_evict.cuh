@@ -2,9 +2,12 @@
 // output of each query row becomes once the evicted tokens are gone and the remaining attention weights
 // are renormalised,
 //     o'_r = (o_r - sum_{e in E} alpha_{r,e} v_e) / (1 - sum_{e in E} alpha_{r,e}),
-// E = the evicted slots the row can see. The weights alpha_{r,e} need the row's softmax normaliser, which
-// this kernel recomputes with one pass over K (fp32 on the CUDA cores, any dtype, head_dim 64 or 128); it
-// is a correction step outside the timed path and is not tuned.
+// E = the evicted slots the row can see. The weights alpha_{r,e} need the row's softmax normaliser. Where the
+// scoring call that ran just before on the same workspace has left the rows' statistics there (the cluster
+// decode kernel: one per query head; the tensor-core prefill kernels: one per row; both as reference +
+// log2(sum) of the log2-domain logits), they are used and the kernel touches only q, the evicted K / V rows
+// and o; the kind of statistics present is a tag in the workspace header. Otherwise the normaliser is
+// recomputed with one pass over K (fp32 on the CUDA cores, any dtype, head_dim 64 or 128).
 // grid = (ceil(R / kRows), units), 256 threads: one warp per query row.
 #pragma once
 
@@ -23,7 +26,8 @@ template <typename T, int D>
 __global__ void __launch_bounds__(32 * kRows)
 post_evict_kernel(Dims dm, const T* __restrict__ q, const T* __restrict__ K, const T* __restrict__ V,
                   const int* __restrict__ len, const int* __restrict__ evict_idx, int max_evict,
-                  const int* __restrict__ n_evict, const float* __restrict__ o, float* __restrict__ o_post) {
+                  const int* __restrict__ n_evict, const float* __restrict__ o, float* __restrict__ o_post,
+                  const int* __restrict__ stat_tag, const float* __restrict__ stats, int prefill_stride) {
   constexpr int LD = D + 4, CPL = D / 32;  // channels per lane
   extern __shared__ __align__(16) float smem[];
   float* Ks = smem;             // [kKeys][LD]
@@ -41,9 +45,15 @@ post_evict_kernel(Dims dm, const T* __restrict__ q, const T* __restrict__ K, con
   const T* Ku = K + (size_t)unit * dm.cap * D;
   const T* Vu = V + (size_t)unit * dm.cap * D;
 
+  // statistics left by the scoring call? (1: per query head, 2: per row; anything else: none)
+  const int tag = stat_tag ? *stat_tag : 0;
+  const bool have_stat = (tag == kStatPerHead && m == 1) || tag == kStatPerRow;
+  float stat2 = 0.f;  // alpha = 2^(log2(e) * scale * <q, k> - stat2)
+  if (have_stat && row_ok)
+    stat2 = (tag == kStatPerHead) ? stats[(size_t)unit * 8 + g] : stats[(size_t)unit * prefill_stride + r];
   // pass over the keys: running maximum and sum of exp of this row's logits, two keys per lane and tile
   float mx = -INFINITY, l = 0.f;
-  for (int kt = 0; kt < n; kt += kKeys) {
+  for (int kt = 0; kt < (have_stat ? 0 : n); kt += kKeys) {
     __syncthreads();
     for (int idx = tid; idx < kKeys * (D / 4); idx += blockDim.x) {
       const int rr = idx / (D / 4), c4 = idx % (D / 4);
@@ -90,7 +100,7 @@ post_evict_kernel(Dims dm, const T* __restrict__ q, const T* __restrict__ K, con
       vv[c] = to_float(Vu[(size_t)j * D + lane * CPL + c]);
     }
     const float s = warp_sum(part) * dm.scale;
-    const float a = __expf(s - M) / Z;
+    const float a = have_stat ? exp2f(s * 1.4426950408889634f - stat2) : __expf(s - M) / Z;
     A += a;
 #pragma unroll
     for (int c = 0; c < CPL; ++c) Y[c] = fmaf(a, vv[c], Y[c]);

@@ -289,6 +289,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
   const int unit = blockIdx.y, row0 = blockIdx.x * kTile;
   const int b = unit / dm.Hkv;
   const int n = len[b], M = dm.R, m = dm.m;
+  if (tid == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) status[kStatTagIndex] = kStatPerRow;
   if (n == 0) return;
   if (n < m || n > dm.cap) {
     if (tid == 0) set_status(status, CAOTE_ERR_BAD_LENGTH);

@@ -100,6 +100,12 @@ def test_host_side_argument_checks_return_before_any_launch():
     assert lib.caote_post_evict_output(bp, fake, fake, fake, fake, None, 4, fake, fake, fake, None) == C.ERR_INVALID_ARG
     assert lib.caote_post_evict_output(bp, fake, fake, fake, fake, fake, 0, fake, fake, fake, None) == C.ERR_INVALID_ARG
     assert lib.caote_post_evict_output(bp, fake, fake, fake, fake, fake, 4, fake, fake, None, None) == C.ERR_INVALID_ARG
+    # ... and the variant that reuses the scoring call's statistics also wants that call's workspace
+    assert lib.caote_post_evict_output_ws(bp, fake, fake, fake, fake, fake, 4, fake, fake, fake, None, need, None) == C.ERR_INVALID_ARG
+    assert lib.caote_post_evict_output_ws(bp, fake, fake, fake, fake, fake, 4, fake, fake, fake, ws, need - 1, None) == C.ERR_INVALID_ARG
+    assert lib.caote_post_evict_output_ws(bp, fake, fake, fake, fake, fake, 4, fake, fake, fake, ctypes.c_void_p(4100), need,
+                                          None) == C.ERR_INVALID_ARG
+    assert lib.caote_post_evict_output_ws(bp, fake, fake, fake, fake, None, 4, fake, fake, fake, ws, need, None) == C.ERR_INVALID_ARG
     # the whole-step entry points validate append, score and selection arguments before their first launch
     # (the FastCAOTE step would otherwise have added the new rows to the running sum already)
     okp = C.make_params(1, 4, 2, 64, 32, 1, torch.float32, 0.125, "last_query")

@@ -20,7 +20,11 @@ CASES = [
     (2, 4, 2, 64, 80, 1, [63, 80], [40, 80], torch.float32),             # one sequence evicts nothing
     (1, 8, 2, 128, 520, 128, [515], [387], torch.bfloat16),              # block of 128 queries, evict 128
     (2, 6, 2, 64, 96, 5, [90, 17], [60, 3], torch.float32),              # most of a short sequence goes
+    (3, 32, 8, 128, 4224, 1, [4129, 515, 2000], [4096, 512, 2000], torch.bfloat16),  # several tiles per unit
+    (1, 12, 2, 128, 700, 33, [640], [500], torch.bfloat16),              # ragged block, 6 heads per group
 ]
+# cases whose scoring call runs on the tensor-core kernels and so leaves the rows' statistics in the workspace
+LEAVES_STATS = {0, 1, 3, 5, 6}
 
 
 @pytest.mark.parametrize("case", CASES)
@@ -56,3 +60,50 @@ def test_post_evict_output_matches_oracle(case):
     P.caote_post_evict_output(p, q, K, V, lens_t, evict_idx, n_evict, o2, o2)
     torch.cuda.synchronize()
     assert torch.equal(o2, o_post)
+    # from the statistics the scoring call left in the workspace
+    o3 = torch.full_like(o, float("nan"))
+    K3 = K
+    if CASES.index(case) in LEAVES_STATS:
+        # the statistics stand in for the pass over K: only the evicted rows of K may be read, so every other row
+        # can hold anything (a pass over K would turn the result into NaN)
+        K3 = torch.full_like(K, float("nan"))
+        for b in range(B):
+            for h in range(Hkv):
+                idx = torch.as_tensor(np.asarray(evict[b][h], dtype=np.int64), device=DEV)
+                K3[b, h, idx] = K[b, h, idx]
+    P.caote_post_evict_output_ws(p, q, K3, V, lens_t, evict_idx, n_evict, o, o3, ws)
+    torch.cuda.synchronize()
+    assert P.caote_read_status(ws) == 0
+    got3 = f32(o3)
+    for b in range(B):
+        assert_close(got3[b], ref[b], f"{case} o_post from the workspace statistics [b={b}]")
+
+
+def test_statistics_of_another_scoring_path_are_not_used():
+    """A tensor-core scoring call followed, on the same workspace, by one on the any-shape path: the second call
+    marks the workspace as holding no statistics and the post-eviction output falls back to its pass over K."""
+    B, Hq, Hkv, d, cap, dtype = 1, 8, 2, 128, 300, torch.bfloat16
+    lens, budget = [257], [250]
+    q, K, V, lens_t = make_case(77, B, Hq, Hkv, d, cap, 1, dtype, lens)
+    p1 = P.make_params(B, Hq, Hkv, d, cap, 1, dtype, d ** -0.5, "last_query")
+    ws = P.alloc_workspace(p1, DEV)
+    o = torch.zeros(q.shape, dtype=torch.float32, device=DEV)
+    scores = torch.zeros((B, Hkv, cap), dtype=torch.float32, device=DEV)
+    P.caote_score(p1, q, K, V, lens_t, None, o, scores, ws)          # cluster kernel: leaves statistics
+    P.caote_set_option(P.OPT_DECODE_CLUSTER, -1)
+    try:
+        scale = 0.5 * d ** -0.5                                       # other logits: the old statistics would be wrong
+        p2 = P.make_params(B, Hq, Hkv, d, cap, 1, dtype, scale, "last_query")
+        P.caote_score(p2, q, K, V, lens_t, None, o, scores, ws)      # streaming kernel: leaves none
+    finally:
+        P.caote_set_option(P.OPT_DECODE_CLUSTER, 0)
+    evict_idx = torch.zeros((B, Hkv, 7), dtype=torch.int32, device=DEV)
+    n_evict = torch.zeros((B,), dtype=torch.int32, device=DEV)
+    P.caote_select_evict(p2, scores, lens_t, torch.tensor(budget, dtype=torch.int32, device=DEV), None, evict_idx, n_evict, ws)
+    o_post = torch.full_like(o, float("nan"))
+    P.caote_post_evict_output_ws(p2, q, K, V, lens_t, evict_idx, n_evict, o, o_post, ws)
+    torch.cuda.synchronize()
+    assert P.caote_read_status(ws) == 0
+    ev = evict_idx.cpu().numpy()
+    ref = oracle.post_evict_output(f32(q), f32(K), f32(V), lens, [[ev[0, h] for h in range(Hkv)]], scale=scale, n_new=1)
+    assert_close(f32(o_post)[0], ref[0], "fallback to the pass over K")
