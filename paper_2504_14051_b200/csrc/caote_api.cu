@@ -533,7 +533,7 @@ static int launch_prefill_score(const Dims& dm, const void* q, const void* K, co
     dim3 grid((dm.cap + prefill::kScoreKeys - 1) / prefill::kScoreKeys, dm.units);
     CAOTE_LAUNCH("prefill_score_kernel", st,
                  launch_pdl(prefill::score_kernel, dim3(grid), dim3(prefill::kScoreThreads), prefill::score_smem_bytes(), st, 
-                     tmQ, tmK, dm, (const __nv_bfloat16*)V, len, sc, scores, status));
+                     tmQ, tmK, tmV64, dm, len, sc, scores, status));
   }
   *used = true;
   return CAOTE_OK;

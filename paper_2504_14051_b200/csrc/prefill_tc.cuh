@@ -182,6 +182,51 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
 #pragma unroll
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
+// The same load without the wait, and the wait as a statement that the 32 registers pass through: whatever reads
+// them afterwards depends on the wait, so the compiler cannot move such a read in front of it. Between the two
+// the thread may do anything that does not touch r.
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32_wait(uint32_t (&r)[32]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+      : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),
+        "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]), "+r"(r[16]),
+        "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]),
+        "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+      :: "memory");
+}
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16_wait(uint32_t (&r)[16]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+      : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),
+        "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
+      :: "memory");
+}
+// Sixteen floats from shared memory, issued where the statement stands (the compiler may not sink it towards the
+// first use: the point is to have the loads in flight while other work is done).
+__device__ __forceinline__ void lds16_issue(const float* p, float4 (&s)[4]) {
+  const uint32_t a = smem_u32(p);
+#pragma unroll
+  for (int k = 0; k < 4; ++k)
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                 : "=f"(s[k].x), "=f"(s[k].y), "=f"(s[k].z), "=f"(s[k].w) : "r"(a + 16 * k));
+}
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
@@ -580,11 +625,70 @@ constexpr int kScoreKeys = 2 * kTile;            // keys per CTA: two key tiles 
 constexpr int kKeyThreads = 2 * kScoreKeys;       // two threads per key: each owns 64 of a block's 128 rows
 constexpr int kScoreThreads = kKeyThreads + 64;   // + a warp for the products + a warp for the copies
 constexpr int kStatBytes = kTile * 4;             // the softmax statistic of the 128 rows of a block
-constexpr int kQStage = kTileBytes + kStatBytes;
-constexpr int kQStages = 3;
+constexpr int kQStages = 4;                       // Q blocks: a stage is free again once its products are done
+constexpr int kSStages = 8;                       // their rows' statistics: free once the key threads have used them
 
 inline size_t score_smem_bytes() {
-  return 1024 + 2 * kTileBytes + kQStages * (size_t)kQStage + (kD + kScoreKeys) * sizeof(float) + 256;
+  return 1024 + (2 + kQStages) * (size_t)kTileBytes + kSStages * (size_t)kStatBytes + (kD + kScoreKeys) * sizeof(float) + 256;
+}
+
+// 2^x for two arguments at once on the FMA pipe instead of the special-function unit: x = i + f with i the nearest
+// integer (taken from the low bits of x + 1.5 * 2^23), 2^f on [-1/2, 1/2] by a polynomial of degree 4 that is exact at
+// f = 0 (relative error below 3e-6), and i added to the exponent field. Arguments below -126 give about 2^-126.
+// The score pass is bound by the special-function unit's 16 results per clock and SM (one exponential per
+// (row, key) pair); it hands a quarter of them to this routine.
+__device__ __forceinline__ float2 poly_exp2x2(float2 x) {
+  constexpr float kMagic = 12582912.f;
+  x.x = fmaxf(x.x, -126.f);
+  x.y = fmaxf(x.y, -126.f);
+  const float2 t = __fadd2_rn(x, make_float2(kMagic, kMagic));
+  const float2 r = __fadd2_rn(t, make_float2(-kMagic, -kMagic));
+  const float2 f = __ffma2_rn(r, make_float2(-1.f, -1.f), x);
+  float2 p = __ffma2_rn(make_float2(0.009589649736881256f, 0.009589649736881256f), f,
+                        make_float2(0.05590599775314331f, 0.05590599775314331f));
+  p = __ffma2_rn(p, f, make_float2(0.24023915827274323f, 0.24023915827274323f));
+  p = __ffma2_rn(p, f, make_float2(0.6931241154670715f, 0.6931241154670715f));
+  p = __ffma2_rn(p, f, make_float2(1.f, 1.f));
+  return make_float2(__int_as_float(__float_as_int(p.x) + (__float_as_int(t.x) << 23)),
+                     __int_as_float(__float_as_int(p.y) + (__float_as_int(t.y) << 23)));
+}
+
+// Adds to a key's running sum the attention weights 2^(s * scale2 - statistic) of 16 rows (v: the logits of the
+// key against these rows, st: the rows' statistics). plain: no row is masked. Of every eight exponentials six go to
+// the special-function unit and two to the polynomial.
+__device__ __forceinline__ void score_piece16(const uint32_t (&v)[16], const float4 (&st)[4], float scale2, bool plain,
+                                              int R0, int M, int m, int need, float2 (&hacc)[2], float& hmasked) {
+  if (plain) {
+#pragma unroll
+    for (int i = 0; i < 16; i += 8) {
+      const float4 ra = st[i / 4], rb = st[i / 4 + 1];
+      const float a0 = fast_exp2(fmaf(__uint_as_float(v[i]), scale2, -ra.x));
+      const float a1 = fast_exp2(fmaf(__uint_as_float(v[i + 1]), scale2, -ra.y));
+      const float a2 = fast_exp2(fmaf(__uint_as_float(v[i + 2]), scale2, -ra.z));
+      const float a3 = fast_exp2(fmaf(__uint_as_float(v[i + 3]), scale2, -ra.w));
+      const float a4 = fast_exp2(fmaf(__uint_as_float(v[i + 4]), scale2, -rb.x));
+      const float a5 = fast_exp2(fmaf(__uint_as_float(v[i + 5]), scale2, -rb.y));
+      const float2 a67 = poly_exp2x2(make_float2(fmaf(__uint_as_float(v[i + 6]), scale2, -rb.z),
+                                                 fmaf(__uint_as_float(v[i + 7]), scale2, -rb.w)));
+      hacc[0] = __fadd2_rn(hacc[0], make_float2(a0, a1));
+      hacc[1] = __fadd2_rn(hacc[1], make_float2(a2, a3));
+      hacc[0] = __fadd2_rn(hacc[0], make_float2(a4, a5));
+      hacc[1] = __fadd2_rn(hacc[1], a67);
+    }
+  } else {
+    // row R sees key j iff j <= n - m + (R % m), i.e. iff (R % m) >= need; R % m is carried along instead of
+    // being divided out for every pair
+    const float stf[16] = {st[0].x, st[0].y, st[0].z, st[0].w, st[1].x, st[1].y, st[1].z, st[1].w,
+                           st[2].x, st[2].y, st[2].z, st[2].w, st[3].x, st[3].y, st[3].z, st[3].w};
+    int rm = R0 % m;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const bool vis = (R0 + i < M) && (rm >= need);
+      const float a = fast_exp2(fmaf(__uint_as_float(v[i]), scale2, -stf[i]));
+      hmasked += vis ? a : 0.f;
+      if (++rm == m) rm = 0;
+    }
+  }
 }
 
 // CAOTE scores of 256 keys of one unit. grid = (key tile pairs, units), 576 threads: warps 0..15 are the
@@ -592,20 +696,23 @@ inline size_t score_smem_bytes() {
 // lower eight take rows 0..63 of every Q block, the upper eight rows 64..127), one lane of warp 16 issues
 // the products, one lane of warp 17 the copies.
 __global__ void __launch_bounds__(kScoreThreads, 1)
-score_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, Dims dm,
-             const __nv_bfloat16* __restrict__ V, const int* __restrict__ len, Scratch sc,
+score_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+             const __grid_constant__ CUtensorMap tmV, Dims dm, const int* __restrict__ len, Scratch sc,
              float* __restrict__ scores, int* status) {
   ptx::pdl_wait();
   ptx::pdl_trigger();
   extern __shared__ char smem_raw[];
   char* sm = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   char* Ks = sm;                                                     // [2] key tiles
-  char* Qst = Ks + 2 * kTileBytes;                                   // [kQStages][Q block, row statistics]
-  float* Xs = reinterpret_cast<float*>(Qst + kQStages * kQStage);    // [kD]
+  char* Qst = Ks + 2 * kTileBytes;                                   // [kQStages] Q blocks
+  float* Sst = reinterpret_cast<float*>(Qst + kQStages * kTileBytes);  // [kSStages][kTile] row statistics
+  float* Xs = Sst + kSStages * kTile;                                // [kD]
   float* hx = Xs + kD;                                               // [kScoreKeys] upper halves' sums
   uint64_t* bars = reinterpret_cast<uint64_t*>(hx + kScoreKeys);
-  uint64_t *k_bar = &bars[0], *q_bar = &bars[1], *s_bar = q_bar + kQStages, *c_bar = s_bar + 2, *q_free = c_bar + 2;
-  constexpr int kBars = 1 + kQStages + 2 + 2 + kQStages;
+  uint64_t *k_bar = &bars[0], *v_bar = &bars[1], *q_bar = &bars[2], *q_done = q_bar + kQStages, *st_bar = q_done + kQStages,
+           *s_bar = st_bar + kSStages, *c_bar = s_bar + 2, *st_free = c_bar + 2;
+  constexpr int kBars1 = 2 + 2 * kQStages + kSStages + 2;  // single arrivals (a copy's bytes, a commit)
+  constexpr int kBars = kBars1 + 2 + kSStages;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kBars);
 
   const int tid = threadIdx.x, warp = tid >> 5;
@@ -616,9 +723,9 @@ score_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
   const int nblocks = (M + kTile - 1) / kTile;
 
   if (tid == 0) {
-    for (int i = 0; i < 1 + kQStages + 2; ++i) mbar_init(&bars[i], 1);
-    for (int i = 0; i < 2; ++i) mbar_init(&c_bar[i], kKeyThreads);
-    for (int i = 0; i < kQStages; ++i) mbar_init(&q_free[i], kKeyThreads);
+    for (int i = 0; i < kBars1; ++i) mbar_init(&bars[i], 1);
+    for (int i = 0; i < 2; ++i) mbar_init(&c_bar[i], kKeyThreads / 32);  // one arrival per key warp
+    for (int i = 0; i < kSStages; ++i) mbar_init(&st_free[i], kKeyThreads / 32);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) tmem_alloc(tmem_slot, 512);
@@ -640,13 +747,23 @@ score_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         tma_load_2d(Ks + kk * kTileBytes + kHalfBytes, &tmK, 64, unit * dm.cap + j0 + kk * kTile, k_bar);
       }
       for (int rb = 0; rb < nblocks; ++rb) {
-        const int st = rb % kQStages;
-        if (rb >= kQStages) mbar_wait_idle(&q_free[st], ((rb / kQStages) - 1) & 1, status);  // block rb - 3 is reduced
-        char* qd = Qst + st * kQStage;
-        mbar_expect_tx(&q_bar[st], kQStage);
+        const int st = rb % kQStages, ss = rb % kSStages;
+        if (rb >= kQStages) mbar_wait_idle(&q_done[st], ((rb / kQStages) - 1) & 1, status);  // the products of block rb - 4 are done
+        char* qd = Qst + st * kTileBytes;
+        mbar_expect_tx(&q_bar[st], kTileBytes);
         tma_load_2d(qd, &tmQ, 0, unit * M + rb * kTile, &q_bar[st]);
         tma_load_2d(qd + kHalfBytes, &tmQ, 64, unit * M + rb * kTile, &q_bar[st]);
-        bulk_load(qd + kTileBytes, sc.stats + (size_t)unit * sc.Mpad + (size_t)rb * kTile, kStatBytes, &q_bar[st]);
+        if (rb >= kSStages) mbar_wait_idle(&st_free[ss], ((rb / kSStages) - 1) & 1, status);  // block rb - 8 is summed
+        mbar_expect_tx(&st_bar[ss], kStatBytes);
+        bulk_load(Sst + ss * kTile, sc.stats + (size_t)unit * sc.Mpad + (size_t)rb * kTile, kStatBytes, &st_bar[ss]);
+      }
+      // the value rows of the CTA's keys, for the distances at the end: into the first two Q stages once the last
+      // product has read its Q block (a commit covers every product before it)
+      mbar_wait_idle(&q_done[(nblocks - 1) % kQStages], ((nblocks - 1) / kQStages) & 1, status);
+      mbar_expect_tx(v_bar, 2 * kTileBytes);
+      for (int kk = 0; kk < 2; ++kk) {
+        tma_load_2d(Qst + kk * kTileBytes, &tmV, 0, unit * dm.cap + j0 + kk * kTile, v_bar);
+        tma_load_2d(Qst + kk * kTileBytes + kHalfBytes, &tmV, 64, unit * dm.cap + j0 + kk * kTile, v_bar);
       }
     }
   } else if (warp == 16) {
@@ -660,7 +777,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         mbar_wait_idle(&q_bar[st], (rb / kQStages) & 1, status);
         if (rb >= 2) mbar_wait_idle(&c_bar[buf], ((rb - 2) >> 1) & 1, status);  // its S buffers have been read
         tc_fence_after();
-        const uint32_t q_addr = smem_u32(Qst + st * kQStage);
+        const uint32_t q_addr = smem_u32(Qst + st * kTileBytes);
 #pragma unroll
         for (int kk = 0; kk < 2; ++kk) {
 #pragma unroll
@@ -668,75 +785,92 @@ score_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             umma(tmem + kk * 256 + buf * 128, desc_k_major(k_addr + kk * kTileBytes, ks), desc_k_major(q_addr, ks), kIdesc, ks > 0);
         }
         umma_commit(&s_bar[buf]);
+        umma_commit(&q_done[st]);
       }
+      // (no arrival may still be on its way to this CTA's barriers when the CTA ends)
+      if (nblocks > 0) mbar_wait_idle(&q_done[(nblocks - 1) % kQStages], ((nblocks - 1) / kQStages) & 1, status);
     }
   } else {
     // =============================== one key per thread ===============================
+    // A thread's 64 rows of a Q block go through registers in four pieces of 16. Two register sets take turns: while
+    // one piece is summed, the next piece's logits (TMEM) and statistics (shared memory) are already on their way, so
+    // neither latency is waited for. The S buffer is handed back to the products as soon as its last piece is in
+    // registers, not when it has been summed.
     const float scale2 = dm.scale * 1.4426950408889634f;
     const int kk = (warp >> 2) & 1;
-    const uint32_t t_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16) + kk * 256;
+    const uint32_t t_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16) + kk * 256 + rhalf * 64;
+    const int lane = tid & 31;
+    const int need = j - (n - m);  // row R sees key j iff (R % m) >= need
+    uint32_t va[16], vb[16];
+    float4 sa[4], sb[4];
+    float2 hacc[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+    mbar_wait(&s_bar[0], 0, status);
+    mbar_wait(&st_bar[0], 0, status);
+    tc_fence_after();
+    tmem_ld16_issue(t_lane, va);
+    lds16_issue(Sst + rhalf * 64, sa);
     for (int rb = 0; rb < nblocks; ++rb) {
-      const int buf = rb & 1, st = rb % kQStages;
-      mbar_wait(&q_bar[st], (rb / kQStages) & 1, status);  // the row statistics have landed
-      mbar_wait(&s_bar[buf], (rb >> 1) & 1, status);
-      tc_fence_after();
-      const float* stt = reinterpret_cast<const float*>(Qst + st * kQStage + kTileBytes);
+      const int buf = rb & 1, ss = rb % kSStages;
       // only the keys of the new block itself are masked (causal inside the block), and only the last
       // row block can have columns beyond M
       const bool plain = (j0 + kScoreKeys - 1 < n - m + 1) && (rb * kTile + kTile <= M);
-#pragma unroll
-      for (int c2 = 0; c2 < 2; ++c2) {
-        const int cc = 2 * rhalf + c2;  // this thread's two groups of 32 rows
-        float v[32];
-        tmem_ld32(t_lane + buf * 128 + cc * 32, v);
-        const float* stc = stt + cc * 32;
-        if (plain) {
-          float h4[4] = {0.f, 0.f, 0.f, 0.f};  // independent partial sums
-#pragma unroll
-          for (int i = 0; i < 32; i += 4) {
-            const float4 rs = *reinterpret_cast<const float4*>(stc + i);  // statistics of four rows
-            h4[0] += fast_exp2(fmaf(v[i], scale2, -rs.x));
-            h4[1] += fast_exp2(fmaf(v[i + 1], scale2, -rs.y));
-            h4[2] += fast_exp2(fmaf(v[i + 2], scale2, -rs.z));
-            h4[3] += fast_exp2(fmaf(v[i + 3], scale2, -rs.w));
-          }
-          h += (h4[0] + h4[1]) + (h4[2] + h4[3]);
-        } else {
-          // row R sees key j iff j <= n - m + (R % m), i.e. iff (R % m) >= j - (n - m); R % m is carried
-          // along instead of being divided out for every pair
-          const int need = j - (n - m);
-          const int R0 = rb * kTile + cc * 32;
-          int rm = R0 % m;
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const bool vis = (R0 + i < M) && (rm >= need);
-            const float a = fast_exp2(fmaf(v[i], scale2, -stc[i]));
-            h += vis ? a : 0.f;
-            if (++rm == m) rm = 0;
-          }
-        }
-      }
+      const int R0 = rb * kTile + rhalf * 64;
+      const uint32_t t_s = t_lane + buf * 128;
+      const float* stc = Sst + ss * kTile + rhalf * 64;
+      // piece 0 (in va / sa); piece 1 on its way
+      tmem_ld16_wait(va);
+      tmem_ld16_issue(t_s + 16, vb);
+      lds16_issue(stc + 16, sb);
+      score_piece16(va, sa, scale2, plain, R0, M, m, need, hacc, h);
+      // piece 1; piece 2 on its way
+      tmem_ld16_wait(vb);
+      tmem_ld16_issue(t_s + 32, va);
+      lds16_issue(stc + 32, sa);
+      score_piece16(vb, sb, scale2, plain, R0 + 16, M, m, need, hacc, h);
+      // piece 2; piece 3 on its way
+      tmem_ld16_wait(va);
+      tmem_ld16_issue(t_s + 48, vb);
+      lds16_issue(stc + 48, sb);
+      score_piece16(va, sa, scale2, plain, R0 + 32, M, m, need, hacc, h);
+      // piece 3; the S buffer is free, the next block's piece 0 on its way
+      tmem_ld16_wait(vb);
       tc_fence_before();
-      mbar_arrive(&c_bar[buf]);
-      mbar_arrive(&q_free[st]);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&c_bar[buf]);  // this warp holds its part of the S buffer in registers
+      if (rb + 1 < nblocks) {
+        const int ss1 = (rb + 1) % kSStages;
+        mbar_wait(&s_bar[buf ^ 1], ((rb + 1) >> 1) & 1, status);
+        mbar_wait(&st_bar[ss1], ((rb + 1) / kSStages) & 1, status);  // the next block's row statistics have landed
+        tc_fence_after();
+        tmem_ld16_issue(t_lane + (buf ^ 1) * 128, va);
+        lds16_issue(Sst + ss1 * kTile + rhalf * 64, sa);
+      }
+      score_piece16(vb, sb, scale2, plain, R0 + 48, M, m, need, hacc, h);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&st_free[ss]);  // ... and is done with the block's statistics
     }
+    h += (hacc[0].x + hacc[0].y) + (hacc[1].x + hacc[1].y);
   }
 
   // ---- the two halves of a key add up; then c_j = w_j / (1 - w_j) * ||X - v_j||, w_j = h_j / M ----
   if (tid >= kScoreKeys && tid < kKeyThreads) hx[tid - kScoreKeys] = h;
   __syncthreads();
   if (tid < kScoreKeys) h += hx[tid];
+  if (tid < kScoreKeys) mbar_wait(v_bar, 0, status);
   if (tid < kScoreKeys && j < n) {
-    const __nv_bfloat16* vrow = V + ((size_t)unit * dm.cap + j) * kD;
+    // the key's value row: 16 chunks of 8 channels in the staged tile (two boxes of 64 channels, 128-byte swizzle)
+    const char* vt = Qst + (tid >> 7) * kTileBytes;
     float acc = 0.f;
 #pragma unroll
-    for (int c = 0; c < kD; c += 8) {
-      float f[8];
-      load8(vrow + c, f);
+    for (int c = 0; c < 16; ++c) {
+      const uint4 raw = *reinterpret_cast<const uint4*>(vt + tile_off(tid & (kTile - 1), c));
+      const uint32_t w4[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        const float d0 = Xs[c + e] - f[e];
+      for (int e = 0; e < 4; ++e) {
+        const float d0 = Xs[8 * c + 2 * e] - __uint_as_float(w4[e] << 16);
+        const float d1 = Xs[8 * c + 2 * e + 1] - __uint_as_float(w4[e] & 0xffff0000u);
         acc = fmaf(d0, d0, acc);
+        acc = fmaf(d1, d1, acc);
       }
     }
     const float Htot = (float)M;
