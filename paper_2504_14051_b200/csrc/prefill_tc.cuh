@@ -281,8 +281,8 @@ __device__ __forceinline__ uint64_t desc_mn_major(uint32_t tile_addr, int ks) {
 
 // ---- attention pass ---------------------------------------------------------------------------------
 // Keys are walked in tiles of 128: three K stages, two V stages and the Q block in shared memory, two S buffers,
-// O and one P buffer (bf16 hi and lo parts) in TMEM; the tensor pipe then always has the next S = Q K^T queued
-// while the threads are busy with the softmax of the current tile:
+// and O in TMEM, P (bf16 hi and lo parts) written over the S it came from; the tensor pipe then always has the next
+// S = Q K^T queued while the threads are busy with the softmax of the current tile:
 //   tensor pipe:  QK(t+1)  PV(t)  QK(t+2)  PV(t+1) ...
 //   threads:      softmax(t) ............ softmax(t+1) ...
 constexpr int kKeys = 128;                   // keys per tile of the attention pass
@@ -358,7 +358,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  // columns: S0 [0,128), S1 [128,256), O [256,384), P hi [384,448), P lo [448,512) (two bf16 per column)
+  // columns: S0 [0,128), S1 [128,256), O [256,384). P of a tile takes the place of its S once the row threads have
+  // read that: hi part in the buffer's columns [0,64), lo part in [64,128) (two bf16 per column), so P is double-
+  // buffered like S and the softmax of a tile does not wait for the previous tile's O += P V
   const uint32_t tmem = *tmem_slot;
 
   if (warp == 9) {
@@ -420,7 +422,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         mbar_wait_idle(&v_bar[kt % kVStages], (kt / kVStages) & 1, status);
         tc_fence_after();
         const uint64_t vd = vdesc0 + (uint64_t)(((kt % kVStages) * kKvTile) >> 4);
-        const uint32_t p_tmem = tmem + 384;
+        const uint32_t p_tmem = tmem + (kt & 1) * kKeys;
         if (kt == 0) {
           umma_ts(tmem + 256, p_tmem, vd, kIdescO, false);
         } else {
@@ -447,7 +449,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     const float scale2 = dm.scale * 1.4426950408889634f;
     const uint32_t t_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16);
     const uint32_t t_o = t_lane + 256 + half * 64;
-    const uint32_t t_p = t_lane + 384 + half * 32;  // this half's 64 keys = 32 packed columns (hi); lo at + 64
     float m_ref = -INFINITY, l = 0.f;
 
     for (int kt = 0; kt < ntiles; ++kt) {
@@ -512,8 +513,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
           lo[c] = __byte_perm(__float_as_uint(r0) + 0x8000u, __float_as_uint(r1) + 0x8000u, 0x7632);  // rounded
           ls[c & 3] += p0 + p1;
         }
-        // the one P buffer is still being read by the product of the previous tile until o_bar says so
-        if (kt >= 1) mbar_wait(&o_bar[(kt - 1) & 1], ((kt - 1) >> 1) & 1, status);
+        // P goes where S was: both halves of the row have read their S columns (the barrier above), and the
+        // product that read the buffer's previous P was issued before the product that formed this S
+        const uint32_t t_p = t_lane + (kt & 1) * kKeys + half * 32;  // this half's 64 keys = 32 packed columns
         tmem_st32u(t_p, hi);
         tmem_st32u(t_p + 64, lo);
         tmem_st_wait();
