@@ -807,10 +807,7 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
         const float l = lsum + pmf;
         const float inv_l = (hd < G && l > 0.f) ? __fdividef(1.f, l) : 0.f;
         if (rl == 0) {
-          const float mstat = (hd < G) ? m_fin + __log2f(l) : 0.f;
-          fin->m[hd] = mstat;
-          if (bg == 0 && rank == 0 && hd < G)  // left for the post-eviction output: alpha_j = 2^(s_j - mstat)
-            reinterpret_cast<float*>(reinterpret_cast<char*>(status) + kHeaderBytes)[(size_t)w.unit * 8 + hd] = mstat;
+          fin->m[hd] = (hd < G) ? m_fin + __log2f(l) : 0.f;
           fin->inv_l[hd] = inv_l;
           fin->smax[hd] = smx;
           fin->crest[hd] = lsum * inv_l;
@@ -967,6 +964,9 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
           }
         }
       }
+      // the heads' log-sum-exp, left for the post-eviction output (alpha_j = 2^(s_j - m)); off the merge's path
+      if (bg == 0 && rank == 0 && tok < G)
+        reinterpret_cast<float*>(reinterpret_cast<char*>(status) + kHeaderBytes)[(size_t)w.unit * 8 + tok] = fin->m[tok];
       ti += w.T;
       ++mu;
     }
