@@ -317,9 +317,16 @@ CAOTE_API int caote_trace_collect(caote_trace_entry_t* out, int32_t max_entries,
  *   CAOTE_OPT_DECODE_CLUSTER  CTAs per thread-block cluster on the single-query path: 0 = chosen from the
  *                             shape (default), 1..16 = forced (shapes it cannot serve take the next path),
  *                             -1 = do not use the cluster kernel.
+ *   CAOTE_OPT_SIDE_BY_SIDE    1 (default): on the single-query path, when the clusters leave enough SMs idle and
+ *                             the units do not divide evenly among them, the last sequences of the batch are
+ *                             scored by the streaming kernel on a second stream of the library's own, beside the
+ *                             cluster kernel; the caller's stream waits for both. 0 = never. 2..65 = always,
+ *                             with the last value - 1 sequences on the streaming kernel (tests, tuning). (The second stream
+ *                             and two events are created on first use, one set per device; caote_score_static
+ *                             never uses them.)
  * Takes effect for launches made after the call. Returns CAOTE_ERR_INVALID_ARG for an unknown option or a
  * value out of range. */
-typedef enum { CAOTE_OPT_WAIT_CYCLES = 1, CAOTE_OPT_DECODE_CLUSTER = 2 } caote_option_t;
+typedef enum { CAOTE_OPT_WAIT_CYCLES = 1, CAOTE_OPT_DECODE_CLUSTER = 2, CAOTE_OPT_SIDE_BY_SIDE = 3 } caote_option_t;
 CAOTE_API int caote_set_option(int32_t option, int64_t value);
 
 /* Number of kernels this library has launched from this process since it was loaded. */

@@ -271,7 +271,7 @@ def caote_trace_collect(max_entries: int = 32) -> dict:
     return {buf[i].name.decode(): (int(buf[i].launches), float(buf[i].total_ms)) for i in range(n.value)}
 
 
-OPT_WAIT_CYCLES, OPT_DECODE_CLUSTER = 1, 2
+OPT_WAIT_CYCLES, OPT_DECODE_CLUSTER, OPT_SIDE_BY_SIDE = 1, 2, 3
 
 
 def caote_set_option(option: int, value: int) -> None:

@@ -20,6 +20,7 @@ namespace caote {
 
 static std::atomic<long long> g_launches{0};
 static std::atomic<long long> g_wait_cycles{2000000000LL};  // CAOTE_OPT_WAIT_CYCLES
+static std::atomic<int> g_side_by_side{1};                  // CAOTE_OPT_SIDE_BY_SIDE: 0 off, 1 when it pays
 static std::atomic<int> g_decode_cluster{0};                // CAOTE_OPT_DECODE_CLUSTER: 0 auto, -1 off, else the size
 static thread_local char g_cuda_error[256] = "";
 
@@ -416,16 +417,21 @@ static int launch_decode_cluster(const Dims& dm, const void* q, const void* K, c
 }
 
 static int launch_decode_score(const Dims& dm, const void* q, const void* K, const void* V, const int* len,
-                               float* base, float* o, float* scores, char* ws, cudaStream_t st, bool* used,
-                               const float* vsum) {
+                               float* base, float* o, float* scores, int* status, char* scratch, float* rowstat,
+                               int stat_tag, int grid_cap, cudaStream_t st, bool* used, const float* vsum) {
+  // status: the workspace header; scratch: where the plan and the records go; rowstat: [units][8] for the heads'
+  // log-sum-exp (or null); stat_tag: what the header's statistics tag becomes (< 0: left alone);
+  // grid_cap > 0: at most that many CTAs (when the kernel shares the GPU with the cluster kernel)
   *used = false;
-  const int grid_limit = decode_grid_limit();
+  int grid_limit = decode_grid_limit();
+  if (grid_cap > 0 && grid_limit > grid_cap) grid_limit = grid_cap;
   TensorMapEncodeFn encode = tensor_map_encoder();
   const bool carried = dm.base_mode == CAOTE_BASE_ACCUM || dm.base_mode == CAOTE_BASE_EXTERNAL;
   if (grid_limit <= 0 || !encode || (carried && !aligned(base, 16)) || !aligned(q, 16)) return CAOTE_OK;
   decode::Plan pl;
-  decode::carve(dm, ws + kHeaderBytes, &pl, grid_limit);
-  int* status = reinterpret_cast<int*>(ws);
+  decode::carve(dm, scratch, &pl, grid_limit);
+  pl.rowstat = rowstat;
+  pl.stat_tag = stat_tag;
   CUtensorMap tmK, tmV, tmQ;
   const cuuint64_t gdim[2] = {(cuuint64_t)dm.D, (cuuint64_t)dm.units * (cuuint64_t)dm.cap};
   const cuuint64_t gstride[1] = {(cuuint64_t)dm.D * 2};
@@ -470,6 +476,98 @@ static int launch_decode_score(const Dims& dm, const void* q, const void* K, con
     CAOTE_LAUNCH("fast_finish_kernel", st, launch_pdl(decode::fast_finish_kernel, dim3(fgrid), dim3(decode::kT), 0, st, dm, len, base, scores, pl));
   }
   *used = true;
+  return CAOTE_OK;
+}
+
+
+// The heads' log-sum-exp of every unit ([units][8] floats) sits right behind the workspace header on the single-
+// query paths; the streaming kernel's plan and records follow it.
+static size_t rowstat_bytes(const Dims& dm) { return align_up(sizeof(float) * 8 * (size_t)dm.units, 256); }
+
+// The same problem restricted to `count` sequences (the caller offsets the pointers).
+static Dims sub_dims(const Dims& dm, int count) {
+  Dims d = dm;
+  d.B = count;
+  d.units = count * dm.Hkv;
+  return d;
+}
+
+// SMs the cluster kernel occupies on these dimensions.
+static int side_clusters_sms(const Dims& d, int base_mode) {
+  int n = 0;
+  const int c = choose_cluster(d, cluster_kernel(d.G, base_mode), &n);
+  if (n > d.units) n = d.units;
+  return c * n;
+}
+
+// ---- two kernels side by side --------------------------------------------------------------------------------
+// A cluster of C CTAs takes one unit at a time, the GPU holds n such clusters, and n C is often well below the SM
+// count (a cluster lives inside one GPC) while units / n is rarely whole: the last round runs a few clusters and
+// the SMs outside the clusters idle throughout. When that costs enough, the last `tail` sequences of the batch go
+// to the streaming kernel instead, on a second stream and on as many CTAs as there are SMs outside the clusters, at
+// the same time as the cluster kernel works on the others. Returns the number of tail sequences (0: one kernel).
+// The estimates only rank the options; rates in bytes per second per SM and per cluster round are measured ones.
+static int plan_side_by_side(const Dims& dm, int base_mode) {
+  const int mode = g_side_by_side.load(std::memory_order_relaxed);
+  if (mode == 0 || dm.B < 2) return 0;
+  if (mode >= 2) {  // forced: the last mode - 1 sequences, if the cluster kernel can take the others
+    const int tail = mode - 1 < dm.B ? mode - 1 : dm.B - 1;
+    return side_clusters_sms(sub_dims(dm, dm.B - tail), base_mode) > 0 ? tail : 0;
+  }
+  const double unit_bytes = (double)dm.cap * dm.D * 4.0;  // K and V rows, bf16
+  // measured: the cluster kernel moves about 33 GB/s of K and V per SM it occupies (3.7 TB/s on 112 SMs, 4.5 on 135);
+  // the streaming kernel beside it about 15 GB/s per SM (8 units of 16 385 tokens on 36 SMs in 118 us), after some
+  // 15 us for its plan launch and pipeline fill
+  const double cluster_rate_per_sm = 33e9, stream_rate_per_sm = 15e9, stream_fixed = 15e-6;
+  auto cluster_time = [&](int seqs, int* idle) {
+    const Dims d = sub_dims(dm, seqs);
+    int n = 0;
+    const int c = choose_cluster(d, cluster_kernel(dm.G, base_mode), &n);
+    if (c == 0 || n == 0) return -1.0;
+    if (n > d.units) n = d.units;
+    *idle = g_sm_count - n * c;
+    const long long rounds = ((long long)d.units + n - 1) / n;
+    return (double)rounds * (unit_bytes * n / (cluster_rate_per_sm * n * c));
+  };
+  int idle = 0;
+  const double alone = cluster_time(dm.B, &idle);
+  if (alone <= 0.0) return 0;
+  int best = 0;
+  // Worth it only for an estimated 10 % or more: the join delays whatever follows, and the cluster kernel itself
+  // slows down a little next to a second kernel (256 ragged units of about 7 k tokens with 13 SMs outside the
+  // clusters: 204 us with 16 units moved away against 209 us with all of them, no gain left after the join).
+  double best_t = alone * 0.90;
+  for (int tail = 1; tail < dm.B && tail <= 16; ++tail) {
+    const double tc = cluster_time(dm.B - tail, &idle);
+    if (tc <= 0.0 || idle < 8) continue;
+    const double ts = stream_fixed + (double)tail * dm.Hkv * unit_bytes / (idle * stream_rate_per_sm);
+    const double t = tc > ts ? tc : ts;
+    if (t < best_t) {
+      best_t = t;
+      best = tail;
+    }
+  }
+  return best;
+}
+
+// The second stream and the two events of the fork and the join, one set per device, made on first use.
+struct SideStream {
+  cudaStream_t stream = nullptr;
+  cudaEvent_t fork = nullptr, join = nullptr;
+};
+static std::mutex g_side_mu;
+static int side_stream(SideStream* out) {
+  static SideStream per_dev[64];
+  int dev = 0;
+  CAOTE_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return CAOTE_ERR_UNSUPPORTED;
+  SideStream& ss = per_dev[dev];
+  if (!ss.stream) {
+    CAOTE_CUDA(cudaStreamCreateWithFlags(&ss.stream, cudaStreamNonBlocking));
+    CAOTE_CUDA(cudaEventCreateWithFlags(&ss.fork, cudaEventDisableTiming));
+    CAOTE_CUDA(cudaEventCreateWithFlags(&ss.join, cudaEventDisableTiming));
+  }
+  *out = ss;
   return CAOTE_OK;
 }
 
@@ -564,7 +662,7 @@ static size_t workspace_bytes(const caote_params_t* p) {
   const Dims dm = make_dims(p);
   size_t need = generic::carve(dm, nullptr, nullptr);
   if (decode_shape_ok(p)) {
-    const size_t need2 = decode::carve(dm, nullptr, nullptr, 0);
+    const size_t need2 = rowstat_bytes(dm) + decode::carve(dm, nullptr, nullptr, 0);
     if (need2 > need) need = need2;
   }
   if (prefill_shape_ok(p)) {
@@ -677,7 +775,7 @@ int caote_append(const caote_params_t* p, void* K, void* V, float* base, int32_t
 // caote_score (vsum == NULL) and caote_score_fast (vsum: the per-unit sums of the cached value rows).
 static int score_impl(const caote_params_t* p, const void* q, const void* K, const void* V, const int32_t* len,
                       float* base, const float* vsum, float* o, float* scores, void* workspace, size_t workspace_bytes_,
-                      caote_stream_t stream) {
+                      caote_stream_t stream, bool allow_side_stream = true) {
   int rc = score_args_check(p, q, K, V, len, base, o, scores);
   if (!rc) rc = score_workspace_check(p, workspace, workspace_bytes_);
   if (!rc) rc = check_device();
@@ -687,11 +785,46 @@ static int score_impl(const caote_params_t* p, const void* q, const void* K, con
   char* ws = (char*)workspace;
   if (decode_shape_ok(p)) {
     bool used = false;
+    int* status = reinterpret_cast<int*>(ws);
+    float* rowstat = reinterpret_cast<float*>(ws + kHeaderBytes);
+    char* scratch = ws + kHeaderBytes + rowstat_bytes(dm);
     if (!vsum) {
+      const bool carried = dm.base_mode == CAOTE_BASE_ACCUM || dm.base_mode == CAOTE_BASE_EXTERNAL;
+      const int tail = (allow_side_stream && decode_grid_limit() > 0 && tensor_map_encoder() && aligned(q, 16) &&
+                        (!carried || aligned(base, 16))) ? plan_side_by_side(dm, dm.base_mode) : 0;
+      if (tail > 0) {
+        // the first B - tail sequences on the cluster kernel, the last `tail` on the streaming kernel beside it
+        const int head = dm.B - tail;
+        const Dims dh = sub_dims(dm, head), dt = sub_dims(dm, tail);
+        SideStream ss;
+        std::lock_guard<std::mutex> lk(g_side_mu);
+        TraceScope region("decode_side_by_side", st);  // (tracing: the time from the fork to the join)
+        rc = side_stream(&ss);
+        if (rc) return rc;
+        CAOTE_CUDA(cudaEventRecord(ss.fork, st));
+        CAOTE_CUDA(cudaStreamWaitEvent(ss.stream, ss.fork, 0));
+        rc = launch_decode_cluster(dh, q, K, V, len, base, o, scores, ws, st, &used);
+        if (rc) return rc;
+        if (used) {
+          const size_t uo = (size_t)head * dm.Hkv, qo = (size_t)head * dm.Hq * dm.D;
+          bool used_t = false;
+          rc = launch_decode_score(dt, (const __nv_bfloat16*)q + qo, (const __nv_bfloat16*)K + uo * dm.cap * dm.D,
+                                   (const __nv_bfloat16*)V + uo * dm.cap * dm.D, len + head, base ? base + uo * dm.cap : nullptr,
+                                   o + qo, scores + uo * dm.cap, status, scratch, rowstat + uo * 8, -1,
+                                   g_sm_count - side_clusters_sms(dh, dm.base_mode), ss.stream, &used_t, nullptr);
+          if (!rc && !used_t) rc = CAOTE_ERR_CUDA;  // (its preconditions were checked above)
+          const cudaError_t e1 = cudaEventRecord(ss.join, ss.stream);
+          const cudaError_t e2 = cudaStreamWaitEvent(st, ss.join, 0);
+          if (rc) return rc;
+          if (e1 != cudaSuccess) return cuda_fail(e1, "cudaEventRecord");
+          if (e2 != cudaSuccess) return cuda_fail(e2, "cudaStreamWaitEvent");
+          return CAOTE_OK;
+        }
+      }
       rc = launch_decode_cluster(dm, q, K, V, len, base, o, scores, ws, st, &used);
       if (rc || used) return rc;
     }
-    rc = launch_decode_score(dm, q, K, V, len, base, o, scores, ws, st, &used, vsum);
+    rc = launch_decode_score(dm, q, K, V, len, base, o, scores, status, scratch, rowstat, kStatPerHead, 0, st, &used, vsum);
     if (rc || used) return rc;
   }
   if (prefill_shape_ok(p)) {
@@ -770,7 +903,8 @@ int caote_score_static(const caote_params_t* p, const void* q, const void* K, co
   cudaStream_t st = (cudaStream_t)stream;
   // the array keeps whatever the previous call left: the status word has to start at zero
   CAOTE_CUDA(cudaMemsetAsync(scratch, 0, kHeaderBytes, st));
-  rc = caote_score(p, q, K, V, len, base, o, scores, scratch, kStaticScratchBytes, stream);
+  // (no second stream here: making one allocates)
+  rc = score_impl(p, q, K, V, len, base, nullptr, o, scores, scratch, kStaticScratchBytes, stream, false);
   if (rc) return rc;
   if (status_out) CAOTE_CUDA(cudaMemcpyAsync(status_out, scratch, sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
   return CAOTE_OK;
@@ -1021,6 +1155,10 @@ int caote_set_option(int32_t option, int64_t value) {
     case CAOTE_OPT_WAIT_CYCLES:
       if (value < 1) return CAOTE_ERR_INVALID_ARG;
       g_wait_cycles.store((long long)value, std::memory_order_relaxed);
+      return CAOTE_OK;
+    case CAOTE_OPT_SIDE_BY_SIDE:
+      if (value < 0 || value > 1 + 64) return CAOTE_ERR_INVALID_ARG;
+      g_side_by_side.store((int)value, std::memory_order_relaxed);
       return CAOTE_OK;
     case CAOTE_OPT_DECODE_CLUSTER:
       if (value < -1 || value > dcl::kMaxC) return CAOTE_ERR_INVALID_ARG;

@@ -70,6 +70,8 @@ struct Plan {
   float* dist;        // [units][capS] ||mean(v) - v_j|| (FastCAOTE only)
   int tpi;            // tiles per item
   int capS;           // cap rounded up to a multiple of kT
+  float* rowstat;     // [units][8] the heads' log-sum-exp (log2 domain), left for the post-eviction output; may be null
+  int stat_tag;       // what the plan kernel writes into the workspace header's statistics tag; < 0: leaves it alone
 };
 
 inline int tiles_per_item(const Dims& dm, int grid) {
@@ -104,6 +106,8 @@ inline size_t carve(const Dims& dm, char* base, Plan* out, int grid) {
   pl.S = (float*)take(sizeof(float) * (size_t)dm.units * dm.G * pl.capS);
   pl.dist = (float*)take(sizeof(float) * (size_t)dm.units * pl.capS);
   pl.part = (PartialRec*)take(sizeof(PartialRec) * max_items);
+  pl.rowstat = nullptr;
+  pl.stat_tag = kStatNone;
   if (out) *out = pl;
   return off;
 }
@@ -116,7 +120,10 @@ plan_kernel(int units, int Hkv, int cap, const int* __restrict__ len, Plan pl, i
   __shared__ int warp_tot[32];
   __shared__ int carry;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (tid == 0) { carry = 0; pl.item_prefix[0] = 0; pl.work[0] = 0; pl.work[1] = 0; status[kStatTagIndex] = kStatNone; }
+  if (tid == 0) {
+    carry = 0; pl.item_prefix[0] = 0; pl.work[0] = 0; pl.work[1] = 0;
+    if (pl.stat_tag >= 0) status[kStatTagIndex] = pl.stat_tag;
+  }
   __syncthreads();
   for (int u0 = 0; u0 < units; u0 += 1024) {
     const int u = u0 + tid;

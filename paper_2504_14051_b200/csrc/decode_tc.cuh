@@ -678,7 +678,11 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 const float on = acc[g] * inv_l;
                 o[((size_t)b * dm.Hq + h * G + g) * kD + tok] = on;
                 if (softmax_counted) xsum += on;
-                if (tid == 0) { fr->m[g] = mfin[g]; fr->inv_l[g] = inv_l; }
+                if (tid == 0) {
+                  fr->m[g] = mfin[g];
+                  fr->inv_l[g] = inv_l;
+                  if (pl.rowstat) pl.rowstat[(size_t)d.unit * 8 + g] = mfin[g] + log2f(lfin[g]);
+                }
               }
             }
             const float xv = (Htot > 0.f) ? xsum / Htot : 0.f;
