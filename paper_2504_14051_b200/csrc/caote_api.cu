@@ -4,6 +4,7 @@
 #include <cstdio>
 #include <cstring>
 #include <mutex>
+#include <type_traits>
 #include <utility>
 #include <vector>
 
@@ -703,11 +704,27 @@ static int launch_post_evict(const Dims& dm, const void* q, const void* K, const
   const size_t smem = post::smem_bytes<D>();
   int rc = allow_smem(post::post_evict_kernel<T, D>, smem);
   if (rc) return rc;
+  const int* tag = ws ? reinterpret_cast<const int*>(ws) + kStatTagIndex : nullptr;
+  const float* stats = ws ? reinterpret_cast<const float*>(ws + kHeaderBytes) : nullptr;
+  const int stat_stride = (dm.R + prefill::kTile - 1) / prefill::kTile * prefill::kTile;
+  // Blocks of queries in bf16 / d 128 may have per-row statistics in the workspace (only the device knows which path
+  // scored them): the kernel for that case goes first and returns at once if they are not there; the general
+  // kernel after it returns at once if they are.
+  int rows_kernel = 0;
+  if constexpr (std::is_same<T, __nv_bfloat16>::value && D == 128) {
+    if (ws && dm.m > 1 && aligned(o, 16) && aligned(o_post, 16)) {
+      rc = allow_smem(post::post_evict_rows_kernel, post::rows_smem_bytes());
+      if (rc) return rc;
+      dim3 rgrid((dm.R + post::kBlockRows - 1) / post::kBlockRows, dm.units);
+      CAOTE_LAUNCH("post_evict_rows_kernel", st, post::post_evict_rows_kernel<<<rgrid, 256, post::rows_smem_bytes(), st>>>(
+          dm, (const T*)q, (const T*)K, (const T*)V, len, evict_idx, max_evict, n_evict, o, o_post, tag, stats, stat_stride));
+      rows_kernel = 1;
+    }
+  }
   dim3 grid((dm.R + post::kRows - 1) / post::kRows, dm.units);
   CAOTE_LAUNCH("post_evict_kernel", st, post::post_evict_kernel<T, D><<<grid, 32 * post::kRows, smem, st>>>(
-      dm, (const T*)q, (const T*)K, (const T*)V, len, evict_idx, max_evict, n_evict, o, o_post,
-      ws ? reinterpret_cast<const int*>(ws) + kStatTagIndex : nullptr,
-      ws ? reinterpret_cast<const float*>(ws + kHeaderBytes) : nullptr, (dm.R + prefill::kTile - 1) / prefill::kTile * prefill::kTile));
+      dm, (const T*)q, (const T*)K, (const T*)V, len, evict_idx, max_evict, n_evict, o, o_post, tag, stats, stat_stride,
+      rows_kernel));
   return CAOTE_OK;
 }
 
