@@ -16,6 +16,7 @@
 #include "post_evict.cuh"
 #include "prefill_tc.cuh"
 #include "select_compact.cuh"
+#include "sum_errors_decode.cuh"
 
 namespace caote {
 
@@ -420,7 +421,7 @@ static int launch_decode_cluster(const Dims& dm, const void* q, const void* K, c
 static int launch_decode_score(const Dims& dm, const void* q, const void* K, const void* V, const int* len,
                                float* base, float* o, float* scores, int* status, char* scratch, float* rowstat,
                                int stat_tag, int grid_cap, cudaStream_t st, bool* used, const float* vsum) {
-  // status: the workspace header; scratch: where the plan and the records go; rowstat: [units][8] for the heads'
+  // status: the workspace header; scratch: where the plan and the records go; rowstat: [units][kHeadStatFloats], first 8 of a unit for the heads'
   // log-sum-exp (or null); stat_tag: what the header's statistics tag becomes (< 0: left alone);
   // grid_cap > 0: at most that many CTAs (when the kernel shares the GPU with the cluster kernel)
   *used = false;
@@ -481,9 +482,9 @@ static int launch_decode_score(const Dims& dm, const void* q, const void* K, con
 }
 
 
-// The heads' log-sum-exp of every unit ([units][8] floats) sits right behind the workspace header on the single-
+// The heads' statistics of every unit ([units][kHeadStatFloats] floats) sit right behind the workspace header on the single-
 // query paths; the streaming kernel's plan and records follow it.
-static size_t rowstat_bytes(const Dims& dm) { return align_up(sizeof(float) * 8 * (size_t)dm.units, 256); }
+static size_t rowstat_bytes(const Dims& dm) { return align_up(sizeof(float) * kHeadStatFloats * (size_t)dm.units, 256); }
 
 // The same problem restricted to `count` sequences (the caller offsets the pointers).
 static Dims sub_dims(const Dims& dm, int count) {
@@ -570,6 +571,39 @@ static int side_stream(SideStream* out) {
   }
   *out = ss;
   return CAOTE_OK;
+}
+
+// The sum-of-errors pass that follows the cluster kernel on single-query shapes.
+template <int G>
+static int launch_sum_errors_decode_g(const Dims& dm, const CUtensorMap& tmK, const CUtensorMap& tmV, const void* q,
+                                      const int* len, const float* o, float* scores, char* ws, cudaStream_t st) {
+  int rc = allow_smem(sed::sum_errors_decode_kernel<G>, sed::smem_bytes());
+  if (rc) return rc;
+  dim3 grid((dm.cap + sed::kT - 1) / sed::kT, dm.units);
+  CAOTE_LAUNCH("sum_errors_decode_kernel", st,
+               launch_pdl(sed::sum_errors_decode_kernel<G>, grid, dim3(sed::kT), sed::smem_bytes(), st, tmK, tmV, dm,
+                          (const __nv_bfloat16*)q, len, o, reinterpret_cast<const float*>(ws + kHeaderBytes), scores,
+                          reinterpret_cast<int*>(ws)));
+  return CAOTE_OK;
+}
+static int launch_sum_errors_decode(const Dims& dm, const void* q, const void* K, const void* V, const int* len,
+                                    const float* o, float* scores, char* ws, cudaStream_t st) {
+  TensorMapEncodeFn encode = tensor_map_encoder();
+  if (!encode) return CAOTE_ERR_CUDA;  // (the cluster kernel before it was launched with the same encoder)
+  CUtensorMap tmK, tmV, tmQ;
+  int rc = encode_decode_maps(dm, q, K, V, 8, &tmK, &tmV, &tmQ, encode);
+  if (rc) return rc;
+  switch (dm.G) {
+    case 1: return launch_sum_errors_decode_g<1>(dm, tmK, tmV, q, len, o, scores, ws, st);
+    case 2: return launch_sum_errors_decode_g<2>(dm, tmK, tmV, q, len, o, scores, ws, st);
+    case 3: return launch_sum_errors_decode_g<3>(dm, tmK, tmV, q, len, o, scores, ws, st);
+    case 4: return launch_sum_errors_decode_g<4>(dm, tmK, tmV, q, len, o, scores, ws, st);
+    case 5: return launch_sum_errors_decode_g<5>(dm, tmK, tmV, q, len, o, scores, ws, st);
+    case 6: return launch_sum_errors_decode_g<6>(dm, tmK, tmV, q, len, o, scores, ws, st);
+    case 7: return launch_sum_errors_decode_g<7>(dm, tmK, tmV, q, len, o, scores, ws, st);
+    case 8: return launch_sum_errors_decode_g<8>(dm, tmK, tmV, q, len, o, scores, ws, st);
+    default: return CAOTE_ERR_UNSUPPORTED;
+  }
 }
 
 // Shapes the tensor-core prefill kernels cover.
@@ -827,7 +861,7 @@ static int score_impl(const caote_params_t* p, const void* q, const void* K, con
           bool used_t = false;
           rc = launch_decode_score(dt, (const __nv_bfloat16*)q + qo, (const __nv_bfloat16*)K + uo * dm.cap * dm.D,
                                    (const __nv_bfloat16*)V + uo * dm.cap * dm.D, len + head, base ? base + uo * dm.cap : nullptr,
-                                   o + qo, scores + uo * dm.cap, status, scratch, rowstat + uo * 8, -1,
+                                   o + qo, scores + uo * dm.cap, status, scratch, rowstat + uo * kHeadStatFloats, -1,
                                    g_sm_count - side_clusters_sms(dh, dm.base_mode), ss.stream, &used_t, nullptr);
           if (!rc && !used_t) rc = CAOTE_ERR_CUDA;  // (its preconditions were checked above)
           const cudaError_t e1 = cudaEventRecord(ss.join, ss.stream);
@@ -875,6 +909,13 @@ int caote_score_sum_errors(const caote_params_t* p, const void* q, const void* K
   const Dims dm = make_dims(p);
   cudaStream_t st = (cudaStream_t)stream;
   char* ws = (char*)workspace;
+  if (decode_shape_ok(p)) {
+    // one query per head: the cluster kernel for o and the heads' statistics, then one more pass over K and V
+    bool used = false;
+    rc = launch_decode_cluster(dm, q, K, V, len, nullptr, o, scores, ws, st, &used);
+    if (rc) return rc;
+    if (used) return launch_sum_errors_decode(dm, q, K, V, len, o, scores, ws, st);
+  }
   if (p->dtype == CAOTE_BF16) {
     if (dm.D == 128) return launch_generic_score<__nv_bfloat16, 128>(dm, q, K, V, len, nullptr, o, scores, ws, st, nullptr, true);
     return launch_generic_score<__nv_bfloat16, 64>(dm, q, K, V, len, nullptr, o, scores, ws, st, nullptr, true);

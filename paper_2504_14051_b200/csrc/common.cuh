@@ -15,10 +15,14 @@ namespace caote {
 constexpr size_t kHeaderBytes = 256;
 // Word kStatTagIndex of the workspace header says which softmax statistics the last scoring call left at
 // workspace + kHeaderBytes for the post-eviction output to reuse (reference + log2(sum) of the log2-domain
-// logits): per query head of a unit ([units][8], single-query cluster kernel), per query row of a unit
+// logits): per query head of a unit ([units][kHeadStatFloats], single-query kernels), per query row of a unit
 // ([units][padded rows], tensor-core prefill kernels), or none.
 constexpr int kStatTagIndex = 8;
 constexpr int kStatNone = 0, kStatPerHead = 1, kStatPerRow = 2;
+// Per query head the record is three rows of 8 floats per unit: the log-sum-exp, the largest logit, and the share of
+// all the other tokens next to the token that holds it (sum of the others / sum); the last two only from the
+// cluster kernel, for the sum-of-errors pass that follows it.
+constexpr int kHeadStatFloats = 24;
 
 struct Dims {
   int B, Hq, Hkv, G, D, cap, m, R;  // R = G * m query rows per unit

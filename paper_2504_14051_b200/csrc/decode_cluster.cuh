@@ -965,8 +965,12 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
         }
       }
       // the heads' log-sum-exp, left for the post-eviction output (alpha_j = 2^(s_j - m)); off the merge's path
-      if (bg == 0 && rank == 0 && tok < G)
-        reinterpret_cast<float*>(reinterpret_cast<char*>(status) + kHeaderBytes)[(size_t)w.unit * 8 + tok] = fin->m[tok];
+      if (bg == 0 && rank == 0 && tok < G) {
+        float* hs = reinterpret_cast<float*>(reinterpret_cast<char*>(status) + kHeaderBytes) + (size_t)w.unit * kHeadStatFloats;
+        hs[tok] = fin->m[tok];
+        hs[8 + tok] = fin->smax[tok];
+        hs[16 + tok] = fin->crest[tok];
+      }
       ti += w.T;
       ++mu;
     }

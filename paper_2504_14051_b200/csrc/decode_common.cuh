@@ -70,7 +70,7 @@ struct Plan {
   float* dist;        // [units][capS] ||mean(v) - v_j|| (FastCAOTE only)
   int tpi;            // tiles per item
   int capS;           // cap rounded up to a multiple of kT
-  float* rowstat;     // [units][8] the heads' log-sum-exp (log2 domain), left for the post-eviction output; may be null
+  float* rowstat;     // [units][kHeadStatFloats], first 8 of a unit: the heads' log-sum-exp (log2 domain), left for the post-eviction output; may be null
   int stat_tag;       // what the plan kernel writes into the workspace header's statistics tag; < 0: leaves it alone
 };
 

@@ -681,7 +681,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
                 if (tid == 0) {
                   fr->m[g] = mfin[g];
                   fr->inv_l[g] = inv_l;
-                  if (pl.rowstat) pl.rowstat[(size_t)d.unit * 8 + g] = mfin[g] + log2f(lfin[g]);
+                  if (pl.rowstat) pl.rowstat[(size_t)d.unit * kHeadStatFloats + g] = mfin[g] + log2f(lfin[g]);
                 }
               }
             }

@@ -54,7 +54,7 @@ post_evict_kernel(Dims dm, const T* __restrict__ q, const T* __restrict__ K, con
   const bool have_stat = (tag == kStatPerHead && m == 1) || tag == kStatPerRow;
   float stat2 = 0.f;  // alpha = 2^(log2(e) * scale * <q, k> - stat2)
   if (have_stat && row_ok)
-    stat2 = (tag == kStatPerHead) ? stats[(size_t)unit * 8 + g] : stats[(size_t)unit * prefill_stride + r];
+    stat2 = (tag == kStatPerHead) ? stats[(size_t)unit * kHeadStatFloats + g] : stats[(size_t)unit * prefill_stride + r];
   // pass over the keys: running maximum and sum of exp of this row's logits, two keys per lane and tile
   float mx = -INFINITY, l = 0.f;
   for (int kt = 0; kt < (have_stat ? 0 : n); kt += kKeys) {
