@@ -581,7 +581,7 @@ static int launch_sum_errors_decode_g(const Dims& dm, const CUtensorMap& tmK, co
   if (rc) return rc;
   dim3 grid((dm.cap + sed::kT - 1) / sed::kT, dm.units);
   CAOTE_LAUNCH("sum_errors_decode_kernel", st,
-               launch_pdl(sed::sum_errors_decode_kernel<G>, grid, dim3(sed::kT), sed::smem_bytes(), st, tmK, tmV, dm,
+               launch_pdl(sed::sum_errors_decode_kernel<G>, grid, dim3(sed::kThreads), sed::smem_bytes(), st, tmK, tmV, dm,
                           (const __nv_bfloat16*)q, len, o, reinterpret_cast<const float*>(ws + kHeaderBytes), scores,
                           reinterpret_cast<int*>(ws)));
   return CAOTE_OK;
