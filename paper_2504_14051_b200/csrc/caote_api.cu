@@ -263,7 +263,7 @@ static bool decode_shape_ok(const caote_params_t* p) {
 
 // ---- single-query path on thread-block clusters ---------------------------------------------------------
 typedef void (*ClusterKernel)(const CUtensorMap, const CUtensorMap, const CUtensorMap, Dims, const int*, float*, float*,
-                              float*, int*, long long);
+                              float*, int*, long long, const float*);
 template <int kMode>
 static ClusterKernel cluster_kernel_for_g(int g) {
   switch (g) {
@@ -365,7 +365,8 @@ static int encode_decode_maps(const Dims& dm, const void* q, const void* K, cons
 }
 
 static int launch_decode_cluster(const Dims& dm, const void* q, const void* K, const void* V, const int* len,
-                                 float* base, float* o, float* scores, char* ws, cudaStream_t st, bool* used) {
+                                 float* base, float* o, float* scores, char* ws, cudaStream_t st, bool* used,
+                                 const float* vsum = nullptr) {
   *used = false;
   TensorMapEncodeFn encode = tensor_map_encoder();
   const bool carried = dm.base_mode == CAOTE_BASE_ACCUM || dm.base_mode == CAOTE_BASE_EXTERNAL;
@@ -411,7 +412,7 @@ static int launch_decode_cluster(const Dims& dm, const void* q, const void* K, c
   const long long wait_cycles = g_wait_cycles.load(std::memory_order_relaxed);
   CAOTE_LAUNCH("decode_cluster_kernel", st, {
     cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, tmK, tmV, tmQ, dm, len, base, o, scores, status,
-                                       wait_cycles);
+                                       wait_cycles, vsum);
     if (e != cudaSuccess) return cuda_fail(e, "decode_cluster_kernel");
   });
   *used = true;
@@ -873,6 +874,10 @@ static int score_impl(const caote_params_t* p, const void* q, const void* K, con
         }
       }
       rc = launch_decode_cluster(dm, q, K, V, len, base, o, scores, ws, st, &used);
+      if (rc || used) return rc;
+    } else {
+      // FastCAOTE: the same kernel with the mean of the value rows in the place of X
+      rc = launch_decode_cluster(dm, q, K, V, len, base, o, scores, ws, st, &used, vsum);
       if (rc || used) return rc;
     }
     rc = launch_decode_score(dm, q, K, V, len, base, o, scores, status, scratch, rowstat, kStatPerHead, 0, st, &used, vsum);

@@ -267,7 +267,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 decode_cluster_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                       const __grid_constant__ CUtensorMap tmQ, Dims dm, const int* __restrict__ len,
                       float* __restrict__ base, float* __restrict__ o, float* __restrict__ scores, int* status,
-                      long long wait_cycles) {
+                      long long wait_cycles, const float* __restrict__ vsum) {
   ptx::pdl_wait();
   ptx::pdl_trigger();
   extern __shared__ char smem_raw[];
@@ -850,7 +850,8 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
           float xs = (is_head && counted) ? val : ((act && use_base && r == 7) ? val : 0.f);
 #pragma unroll
           for (int off = 4; off > 0; off >>= 1) xs += __shfl_xor_sync(0xffffffffu, xs, off);
-          const float nxv = -(xs * inv_H);
+          // FastCAOTE (Sec. 3.3): the distances are taken to the mean of the unit's value rows instead of X
+          const float nxv = vsum ? -(act ? __ldg(vsum + (size_t)w.unit * kD + my_ch0 + cl) / (float)w.n : 0.f) : -(xs * inv_H);
           if (act && !ctl[0]) {
             for (int peer = r; peer < C; peer += 8)
               push_f32(map_to_rank(smem_u32(xdst + my_ch0 + cl), peer), nxv, map_to_rank(smem_u32(r2), peer));
