@@ -13,6 +13,7 @@
 #include "decode_tc.cuh"
 #include "generic_score.cuh"
 #include "greedy.cuh"
+#include "greedy_cluster.cuh"
 #include "post_evict.cuh"
 #include "prefill_tc.cuh"
 #include "select_compact.cuh"
@@ -774,6 +775,85 @@ static int launch_greedy(const Dims& dm, const void* V, const float* h, const in
   return CAOTE_OK;
 }
 
+// Greedy eviction with the unit's value rows in the shared memory of a cluster (bf16, d 128). *used = false: the
+// shape does not fit (a unit needs more than 16 CTAs' worth of shared memory, or no cluster can run) and the caller
+// takes the one-CTA kernel. Among the cluster sizes that hold a unit, the largest one of which the GPU can run as
+// many at once as there are units: more CTAs per unit make a pick faster, a second wave of clusters makes the call
+// twice as long.
+static int launch_greedy_cluster(const Dims& dm, const void* V, const float* h, const int* len, const int* budget,
+                                 const int* pos, int* evict_idx, int* order, int max_evict, int* n_evict, int* status,
+                                 cudaStream_t st, bool* used) {
+  *used = false;
+  if (!aligned(V, 16)) return CAOTE_OK;
+  int need = 1;
+  while (need <= greedy_cl::kMaxC && (dm.cap + need - 1) / need > greedy_cl::kMaxRows) need *= 2;
+  if (need > greedy_cl::kMaxC) return CAOTE_OK;
+  CAOTE_CUDA(cudaFuncSetAttribute(greedy_cl::greedy_cluster_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+  int best_c = 0, best_rows = 0, best_got = 0;
+  for (int c = need; c <= greedy_cl::kMaxC; c *= 2) {
+    const int rows = ((dm.cap + c - 1) / c + 7) / 8 * 8;
+    const size_t smem = greedy_cl::smem_bytes(rows);
+    if (cudaFuncSetAttribute(greedy_cl::greedy_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+      (void)cudaGetLastError();
+      continue;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(c * dm.units));
+    cfg.blockDim = dim3(greedy_cl::kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = (unsigned)c;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    int got = 0;
+    if (cudaOccupancyMaxActiveClusters(&got, greedy_cl::greedy_cluster_kernel, &cfg) != cudaSuccess || got <= 0) {
+      (void)cudaGetLastError();
+      continue;
+    }
+    if (best_c == 0 || got >= dm.units) {
+      best_c = c;
+      best_rows = rows;
+      best_got = got;
+    }
+    if (got < dm.units && best_c != c) break;  // larger clusters only fit fewer at once
+  }
+  if (best_c == 0) return CAOTE_OK;
+  {
+    // Worth it? Per pick the one-CTA kernel sweeps the unit's rows from L2 (measured: 12.5 ns per row), this one its
+    // share of them from shared memory plus a cluster barrier (measured: about 6 us + 7 ns per row); but the GPU runs
+    // fewer clusters at once than single CTAs, and with a handful of picks loading the rows is all there is.
+    const double t_one = 0.0125 * dm.cap, t_cluster = 6.0 + 0.007 * best_rows;
+    const double waves_one = (double)((dm.units + g_sm_count - 1) / g_sm_count);
+    const double waves_cluster = (double)((dm.units + best_got - 1) / best_got);
+    if (max_evict < 4 || t_one * waves_one < 1.2 * t_cluster * waves_cluster) return CAOTE_OK;
+  }
+  const size_t smem = greedy_cl::smem_bytes(best_rows);
+  CAOTE_CUDA(cudaFuncSetAttribute(greedy_cl::greedy_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(best_c * dm.units));
+  cfg.blockDim = dim3(greedy_cl::kThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = (unsigned)best_c;
+  at[0].val.clusterDim.y = 1;
+  at[0].val.clusterDim.z = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  CAOTE_LAUNCH("greedy_cluster_kernel", st, {
+    cudaError_t e = cudaLaunchKernelEx(&cfg, greedy_cl::greedy_cluster_kernel, dm.Hkv, dm.cap, best_rows,
+                                       (const __nv_bfloat16*)V, h, len, budget, pos, evict_idx, order, max_evict, n_evict,
+                                       status);
+    if (e != cudaSuccess) return cuda_fail(e, "greedy_cluster_kernel");
+  });
+  *used = true;
+  return CAOTE_OK;
+}
+
 }  // namespace caote
 
 using namespace caote;
@@ -1002,7 +1082,12 @@ int caote_select_evict_greedy(const caote_params_t* p, const void* V, const floa
   cudaStream_t st = (cudaStream_t)stream;
   int* status = (int*)workspace;
   if (p->dtype == CAOTE_BF16) {
-    if (dm.D == 128) return launch_greedy<__nv_bfloat16, 128>(dm, V, h, len, budget, pos, evict_idx, order, max_evict, n_evict, status, st);
+    if (dm.D == 128) {
+      bool used = false;
+      rc = launch_greedy_cluster(dm, V, h, len, budget, pos, evict_idx, order, max_evict, n_evict, status, st, &used);
+      if (rc || used) return rc;
+      return launch_greedy<__nv_bfloat16, 128>(dm, V, h, len, budget, pos, evict_idx, order, max_evict, n_evict, status, st);
+    }
     return launch_greedy<__nv_bfloat16, 64>(dm, V, h, len, budget, pos, evict_idx, order, max_evict, n_evict, status, st);
   }
   if (dm.D == 128) return launch_greedy<float, 128>(dm, V, h, len, budget, pos, evict_idx, order, max_evict, n_evict, status, st);

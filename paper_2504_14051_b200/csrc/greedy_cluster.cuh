@@ -1,0 +1,286 @@
+// Greedy multi-token eviction (Appendix B of the paper, the two-token derivation chained) with a unit's value rows
+// resident on chip: a thread-block cluster per (sequence, KV head) unit, every CTA holding a contiguous share of the
+// unit's value rows in its shared memory (bf16, head_dim 128). Each pick sweeps those rows from shared memory instead
+// of from L2 (the one-CTA kernel in greedy.cuh re-reads all of them from L2 for every pick):
+//   every CTA: distances of its rows to the current output X = Y / H, its best (score bits, position) candidate;
+//   one cluster barrier; every CTA reads all candidates through distributed shared memory and takes the same
+//   minimum; every CTA reads the evicted row from its owner's shared memory and updates its own copy of Y and H
+//   (the same arithmetic everywhere, so the copies never differ).
+// The candidates are double-buffered by the parity of the pick, which is what makes one barrier per pick enough.
+#pragma once
+
+#include "common.cuh"
+
+namespace caote {
+namespace greedy_cl {
+
+constexpr int kThreads = 512;
+constexpr int kWarps = kThreads / 32;
+constexpr int kD = 128;
+constexpr int kMaxRows = 768;   // value rows per CTA (192 KB)
+constexpr int kMaxC = 16;
+
+struct Cand {  // a CTA's best candidate of a pick
+  unsigned long long key;  // (score bits << 32) | position
+  int slot;                // slot in the unit, -1: none
+  float h;                 // its weight
+};
+
+inline size_t smem_bytes(int rows) {
+  return (size_t)rows * kD * 2 + sizeof(float) * (2 * (size_t)rows + kD + (kD + 4) + 2 * kWarps) +
+         sizeof(unsigned long long) * kWarps + sizeof(int) * (2 * kWarps + 8) + 2 * sizeof(Cand) + 64;
+}
+
+__device__ __forceinline__ uint32_t gc_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t gc_size() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t gc_cluster_id() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%clusterid.x;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void gc_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// The same shared-memory location in the CTA of rank `rank`, and loads from it.
+__device__ __forceinline__ uint32_t gc_map(const void* p, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"((uint32_t)__cvta_generic_to_shared(p)), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ float gc_ld_f32(uint32_t a) {
+  float v;
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(a) : "memory");
+  return v;
+}
+__device__ __forceinline__ int gc_ld_s32(uint32_t a) {
+  int v;
+  asm volatile("ld.shared::cluster.s32 %0, [%1];" : "=r"(v) : "r"(a) : "memory");
+  return v;
+}
+__device__ __forceinline__ unsigned long long gc_ld_u64(uint32_t a) {
+  unsigned long long v;
+  asm volatile("ld.shared::cluster.u64 %0, [%1];" : "=l"(v) : "r"(a) : "memory");
+  return v;
+}
+__device__ __forceinline__ unsigned short gc_ld_u16(uint32_t a) {
+  unsigned short v;
+  asm volatile("ld.shared::cluster.u16 %0, [%1];" : "=h"(v) : "r"(a) : "memory");
+  return v;
+}
+
+// grid = units x C CTAs in clusters of C; rows_per = rows of the unit per CTA (the same for every CTA of the grid).
+__global__ void __launch_bounds__(kThreads, 1)
+greedy_cluster_kernel(int Hkv, int cap, int rows_per, const __nv_bfloat16* __restrict__ V, const float* __restrict__ h_in,
+                      const int* __restrict__ len, const int* __restrict__ budget, const int* __restrict__ pos,
+                      int* __restrict__ evict_idx, int* __restrict__ order_out, int max_evict, int* __restrict__ n_evict,
+                      int* status) {
+  extern __shared__ __align__(16) unsigned char gsm[];
+  __nv_bfloat16* Vs = reinterpret_cast<__nv_bfloat16*>(gsm);            // [rows_per][kD]
+  float* hs = reinterpret_cast<float*>(Vs + (size_t)rows_per * kD);     // [rows_per] weight, < 0 once evicted
+  float* ds = hs + rows_per;                                            // [rows_per] || X - v_j || of the current state
+  float* Ys = ds + rows_per;                                            // [kD] sum of h_j v_j over the tokens present
+  float* part = Ys + kD;                                                // [kD + 4] this CTA's share of Y and (at kD) of H
+  float* wsum = part + kD + 4;                                          // [2 * kWarps]
+  unsigned long long* wkey = reinterpret_cast<unsigned long long*>(wsum + 2 * kWarps);  // [kWarps]
+  int* wslot = reinterpret_cast<int*>(wkey + kWarps);                   // [2 * kWarps]
+  int* misc = wslot + 2 * kWarps;                                       // [8]: 0 count of evicted rows here, 1 running count
+  Cand* cand = reinterpret_cast<Cand*>(misc + 8);                       // [2]
+  __shared__ float s_H, s_he;
+  __shared__ int s_e;
+
+  const int C = (int)gc_size(), rank = (int)gc_rank();
+  const int unit = (int)gc_cluster_id(), b = unit / Hkv, hd = unit % Hkv;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int n = len[b];
+  int bud = budget[b];
+  if (bud < 1) bud = 1;
+  int k = n - bud;
+  if (k < 0 || n > cap) k = 0;
+  if (k > max_evict) {
+    if (tid == 0 && rank == 0) set_status(status, CAOTE_ERR_OVERFLOW);
+    k = 0;
+  }
+  if (hd == 0 && rank == 0 && tid == 0) n_evict[b] = k;
+  if (k == 0) return;  // (the whole cluster leaves: no barrier is outstanding)
+  const int r0 = rank * rows_per;
+  const int nr = max(0, min(rows_per, n - r0));  // rows of the unit this CTA holds
+  const __nv_bfloat16* Vu = V + ((size_t)unit * cap + r0) * kD;
+  const float* hu = h_in + (size_t)unit * cap + r0;
+  const int* pu = pos ? pos + (size_t)unit * cap + r0 : nullptr;
+  int* out = evict_idx + (size_t)unit * max_evict;
+  int* ord = order_out ? order_out + (size_t)unit * max_evict : nullptr;
+
+  // ---- the rows into shared memory; H and Y of this CTA's rows (fixed order of the partial sums) ----
+  for (int i = tid; i < nr * (kD / 8); i += kThreads)
+    reinterpret_cast<uint4*>(Vs)[i] = reinterpret_cast<const uint4*>(Vu)[i];
+  float hsum = 0.f;
+  for (int j = tid; j < nr; j += kThreads) {
+    const float hj = fmaxf(hu[j], 0.f);
+    hs[j] = hj;
+    hsum += hj;
+  }
+  hsum = warp_sum(hsum);
+  if (lane == 0) wsum[warp] = hsum;
+  __syncthreads();
+  float yacc[4] = {0.f, 0.f, 0.f, 0.f};
+  for (int j = warp; j < nr; j += kWarps) {
+    const float hj = hs[j];
+    const uint2 raw = *reinterpret_cast<const uint2*>(Vs + (size_t)j * kD + 4 * lane);
+    yacc[0] = fmaf(hj, __uint_as_float(raw.x << 16), yacc[0]);
+    yacc[1] = fmaf(hj, __uint_as_float(raw.x & 0xffff0000u), yacc[1]);
+    yacc[2] = fmaf(hj, __uint_as_float(raw.y << 16), yacc[2]);
+    yacc[3] = fmaf(hj, __uint_as_float(raw.y & 0xffff0000u), yacc[3]);
+  }
+  if (tid < kD + 4) part[tid] = 0.f;
+  __syncthreads();
+  for (int w = 0; w < kWarps; ++w) {  // warps add their parts one after the other: reproducible
+    if (warp == w) {
+#pragma unroll
+      for (int c = 0; c < 4; ++c) part[4 * lane + c] += yacc[c];
+    }
+    __syncthreads();
+  }
+  if (tid == 0) {
+    float H = 0.f;
+    for (int w = 0; w < kWarps; ++w) H += wsum[w];
+    part[kD] = H;
+    misc[0] = 0;
+  }
+  gc_sync();  // every CTA's share is written
+  if (tid <= kD) {  // the unit's Y and H: the shares in rank order, the same sum in every CTA
+    float tot = 0.f;
+    for (int i = 0; i < C; ++i) tot += gc_ld_f32(gc_map(part + tid, (uint32_t)i));
+    if (tid < kD) Ys[tid] = tot; else s_H = tot;
+  }
+  __syncthreads();
+
+  for (int t = 0; t < k; ++t) {
+    const float H = s_H;
+    const float inv_H = (H > 0.f) ? 1.f / H : 0.f;
+    float x[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) x[c] = Ys[4 * lane + c] * inv_H;
+    // ---- distances of this CTA's tokens still present to the current output (a warp per token) ----
+    for (int j = warp; j < nr; j += kWarps) {
+      if (hs[j] < 0.f) continue;  // (warp-uniform)
+      const uint2 raw = *reinterpret_cast<const uint2*>(Vs + (size_t)j * kD + 4 * lane);
+      const float d0 = x[0] - __uint_as_float(raw.x << 16), d1 = x[1] - __uint_as_float(raw.x & 0xffff0000u);
+      const float d2 = x[2] - __uint_as_float(raw.y << 16), d3 = x[3] - __uint_as_float(raw.y & 0xffff0000u);
+      const float acc = warp_sum(fmaf(d0, d0, fmaf(d1, d1, fmaf(d2, d2, d3 * d3))));
+      if (lane == 0) ds[j] = sqrtf(acc);
+    }
+    __syncthreads();
+    // ---- this CTA's arg-min of w_j / (1 - w_j) * dist_j over (score bits, position) (a thread per token; doing
+    //      this inside the sweep, with the division and the position load on every warp's path, was slower) ----
+    unsigned long long best = ~0ull;
+    int best_slot = -1;
+    for (int j = tid; j < nr; j += kThreads) {
+      const float hj = hs[j];
+      if (hj < 0.f) continue;
+      float sc = 0.f;
+      if (H > 0.f && hj > 0.f) {
+        const float rest = H - hj;  // the others' weight (times H)
+        sc = (rest > 0.f) ? hj / rest * ds[j] : INFINITY;
+      }
+      const unsigned long long key = ((unsigned long long)__float_as_uint(sc) << 32) | (unsigned int)(pu ? pu[j] : r0 + j);
+      if (key < best) { best = key; best_slot = j; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const unsigned long long ok = __shfl_xor_sync(0xffffffffu, best, o);
+      const int os = __shfl_xor_sync(0xffffffffu, best_slot, o);
+      if (ok < best || (ok == best && os >= 0 && (best_slot < 0 || os < best_slot))) { best = ok; best_slot = os; }
+    }
+    if (lane == 0) { wkey[warp] = best; wslot[warp] = best_slot; }
+    __syncthreads();
+    if (tid == 0) {
+      unsigned long long bk = wkey[0];
+      int bs = wslot[0];
+      for (int w = 1; w < kWarps; ++w)
+        if (wslot[w] >= 0 && (bs < 0 || wkey[w] < bk || (wkey[w] == bk && wslot[w] < bs))) { bk = wkey[w]; bs = wslot[w]; }
+      Cand cd;
+      cd.key = bk;
+      cd.slot = bs >= 0 ? r0 + bs : -1;
+      cd.h = bs >= 0 ? hs[bs] : 0.f;
+      cand[t & 1] = cd;
+    }
+    gc_sync();  // every CTA's candidate of this pick is written (and everybody is done with the pick before)
+    // ---- the unit's pick: the smallest candidate, lower slot on equal keys; the same in every CTA ----
+    if (warp == 0) {
+      unsigned long long ck = ~0ull;
+      int cs = -1;
+      float ch = 0.f;
+      if (lane < C) {
+        const Cand* rc = cand + (t & 1);
+        cs = gc_ld_s32(gc_map(&rc->slot, (uint32_t)lane));
+        ck = gc_ld_u64(gc_map(&rc->key, (uint32_t)lane));
+        ch = gc_ld_f32(gc_map(&rc->h, (uint32_t)lane));
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const unsigned long long ok = __shfl_xor_sync(0xffffffffu, ck, o);
+        const int os = __shfl_xor_sync(0xffffffffu, cs, o);
+        const float oh = __shfl_xor_sync(0xffffffffu, ch, o);
+        if (os >= 0 && (cs < 0 || ok < ck || (ok == ck && os < cs))) { ck = ok; cs = os; ch = oh; }
+      }
+      if (lane == 0) { s_e = cs; s_he = ch; }
+    }
+    __syncthreads();
+    const int e = s_e;
+    if (e < 0) break;  // (cannot happen with k < n; the same in every CTA, so no barrier is left unmatched)
+    // ---- evict e: Y -= h_e v_e, H -= h_e (the row comes from its owner's shared memory) ----
+    const float he = s_he;
+    const int owner = e / rows_per, el = e - owner * rows_per;
+    if (tid < kD) {
+      const unsigned short raw = gc_ld_u16(gc_map(Vs + (size_t)el * kD + tid, (uint32_t)owner));
+      Ys[tid] -= he * __uint_as_float((uint32_t)raw << 16);
+    }
+    if (tid == 0) {
+      s_H = H - he;
+      if (ord && rank == 0) ord[t] = e;
+      if (owner == rank) {
+        hs[el] = -1.f;
+        misc[0] += 1;
+      }
+    }
+    __syncthreads();
+  }
+  // ---- the evicted slots in ascending order (the layout caote_compact expects): CTAs in rank order ----
+  gc_sync();  // every CTA's count of evicted rows is final
+  if (tid == 0) {
+    int before = 0;
+    for (int i = 0; i < rank; ++i) before += gc_ld_s32(gc_map(misc, (uint32_t)i));
+    misc[1] = before;
+  }
+  __syncthreads();
+  for (int j0 = 0; j0 < nr; j0 += kThreads) {
+    const int j = j0 + tid;
+    const bool gone = j < nr && hs[j] < 0.f;
+    const unsigned m = __ballot_sync(0xffffffffu, gone);
+    if (lane == 0) wslot[kWarps + warp] = __popc(m);
+    __syncthreads();
+    int at = misc[1];
+    for (int w = 0; w < warp; ++w) at += wslot[kWarps + w];
+    if (gone) out[at + __popc(m & ((1u << lane) - 1u))] = r0 + j;
+    __syncthreads();
+    if (tid == 0) {
+      int tot = misc[1];
+      for (int w = 0; w < kWarps; ++w) tot += wslot[kWarps + w];
+      misc[1] = tot;
+    }
+    __syncthreads();
+  }
+  gc_sync();  // no CTA leaves while a peer may still read its shared memory
+}
+
+}  // namespace greedy_cl
+}  // namespace caote

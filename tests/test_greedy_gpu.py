@@ -55,6 +55,8 @@ def follow(order_gpu, h, V, pos, k):
     (1, 3, 64, 100, [97], 40, torch.float32),
     (1, 2, 128, 1300, [1280], 128, torch.bfloat16),     # a reduced prompt block: 1152 kept + 128 new, evict 128
     (1, 1, 128, 40, [33], 32, torch.bfloat16),          # down to a single token
+    (2, 3, 128, 2104, [2000, 777], 64, torch.bfloat16), # the cluster kernel; the short sequence leaves most CTAs of its clusters without rows
+    (1, 2, 128, 6160, [6150], 24, torch.bfloat16),      # the cluster kernel with several hundred rows per CTA
 ])
 def test_greedy_sequence_follows_the_oracle(case):
     B, Hkv, d, cap, lens, k, dtype = case
@@ -69,10 +71,16 @@ def test_greedy_sequence_follows_the_oracle(case):
     ev = torch.full((B, Hkv, k), -1, dtype=torch.int32, device=DEV)
     order = torch.full((B, Hkv, k), -1, dtype=torch.int32, device=DEV)
     ne = torch.zeros((B,), dtype=torch.int32, device=DEV)
+    P.caote_trace_enable(True)
     P.caote_select_evict_greedy(p, V.to(DEV), h.to(DEV), lens_t.to(DEV), budget.to(DEV), pos.to(DEV), ev, order, ne, ws)
     torch.cuda.synchronize()
+    trace = P.caote_trace_collect()
+    P.caote_trace_enable(False)
     assert P.caote_read_status(ws) == 0
     assert ne.cpu().tolist() == [k] * B
+    if dtype == torch.bfloat16 and d == 128 and cap >= 1300:
+        # long units with many picks: the kernel that keeps the value rows in the shared memory of a cluster
+        assert "greedy_cluster_kernel" in trace, trace
     Vn, hn, pn = f32(V), h.numpy(), pos.numpy()
     flips = 0
     for b in range(B):
