@@ -822,10 +822,10 @@ static int launch_greedy_cluster(const Dims& dm, const void* V, const float* h, 
   }
   if (best_c == 0) return CAOTE_OK;
   {
-    // Worth it? Per pick the one-CTA kernel sweeps the unit's rows from L2 (measured: 12.5 ns per row), this one its
+    // Worth it? Per pick the one-CTA kernel sweeps the unit's rows from L2 (measured: 9.5 ns per row), this one its
     // share of them from shared memory plus a cluster barrier (measured: about 6 us + 7 ns per row); but the GPU runs
     // fewer clusters at once than single CTAs, and with a handful of picks loading the rows is all there is.
-    const double t_one = 0.0125 * dm.cap, t_cluster = 6.0 + 0.007 * best_rows;
+    const double t_one = 0.0095 * dm.cap, t_cluster = 6.0 + 0.007 * best_rows;
     const double waves_one = (double)((dm.units + g_sm_count - 1) / g_sm_count);
     const double waves_cluster = (double)((dm.units + best_got - 1) / best_got);
     if (max_evict < 4 || t_one * waves_one < 1.2 * t_cluster * waves_cluster) return CAOTE_OK;

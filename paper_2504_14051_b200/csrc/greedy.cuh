@@ -24,12 +24,35 @@ inline size_t smem_bytes(int cap, int D) {
   return sizeof(float) * ((size_t)2 * cap + 2 * D + 2 * kWarps) + sizeof(unsigned long long) * kWarps + sizeof(int) * kWarps + 64;
 }
 
+// CPL consecutive channels of a row as floats, with one vector load (the row pointer is 16-byte aligned, CPL = 2 or 4).
+template <int CPL>
+__device__ __forceinline__ void load_channels(const __nv_bfloat16* p, float (&f)[CPL]) {
+  if constexpr (CPL == 4) {
+    const uint2 r = *reinterpret_cast<const uint2*>(p);
+    f[0] = __uint_as_float(r.x << 16); f[1] = __uint_as_float(r.x & 0xffff0000u);
+    f[2] = __uint_as_float(r.y << 16); f[3] = __uint_as_float(r.y & 0xffff0000u);
+  } else {
+    const uint32_t r = *reinterpret_cast<const uint32_t*>(p);
+    f[0] = __uint_as_float(r << 16); f[1] = __uint_as_float(r & 0xffff0000u);
+  }
+}
+template <int CPL>
+__device__ __forceinline__ void load_channels(const float* p, float (&f)[CPL]) {
+  if constexpr (CPL == 4) {
+    const float4 r = *reinterpret_cast<const float4*>(p);
+    f[0] = r.x; f[1] = r.y; f[2] = r.z; f[3] = r.w;
+  } else {
+    const float2 r = *reinterpret_cast<const float2*>(p);
+    f[0] = r.x; f[1] = r.y;
+  }
+}
+
 template <typename T, int D>
 __global__ void __launch_bounds__(kThreads, 1)
 greedy_kernel(int Hkv, int cap, const T* __restrict__ V, const float* __restrict__ h_in, const int* __restrict__ len,
               const int* __restrict__ budget, const int* __restrict__ pos, int* __restrict__ evict_idx,
               int* __restrict__ order_out, int max_evict, int* __restrict__ n_evict, int* status) {
-  constexpr int CPL = D / 32;  // channels per lane
+  constexpr int CPL = D / 32;  // channels per lane: lane l owns channels [l * CPL, (l + 1) * CPL)
   extern __shared__ __align__(16) float gsm[];
   float* hs = gsm;                   // [cap] weight of the token, < 0 once evicted
   float* ds = hs + cap;              // [cap] || X - v_j || of the current state
@@ -75,15 +98,17 @@ greedy_kernel(int Hkv, int cap, const T* __restrict__ V, const float* __restrict
   __syncthreads();
   for (int j = warp; j < n; j += kWarps) {
     const float hj = hs[j];
+    float vf[CPL];
+    load_channels<CPL>(Vu + (size_t)j * D + lane * CPL, vf);
 #pragma unroll
-    for (int c = 0; c < CPL; ++c) yacc[c] = fmaf(hj, to_float(Vu[(size_t)j * D + c * 32 + lane]), yacc[c]);
+    for (int c = 0; c < CPL; ++c) yacc[c] = fmaf(hj, vf[c], yacc[c]);
   }
   if (tid < D) Ys[tid] = 0.f;
   __syncthreads();
   for (int w = 0; w < kWarps; ++w) {  // warps add their parts one after the other: reproducible
     if (warp == w) {
 #pragma unroll
-      for (int c = 0; c < CPL; ++c) Ys[c * 32 + lane] += yacc[c];
+      for (int c = 0; c < CPL; ++c) Ys[lane * CPL + c] += yacc[c];
     }
     __syncthreads();
   }
@@ -99,18 +124,31 @@ greedy_kernel(int Hkv, int cap, const T* __restrict__ V, const float* __restrict
     const float inv_H = (H > 0.f) ? 1.f / H : 0.f;
     float x[CPL];
 #pragma unroll
-    for (int c = 0; c < CPL; ++c) x[c] = Ys[c * 32 + lane] * inv_H;
-    // ---- distances of the tokens present to the current output ----
-    for (int j = warp; j < n; j += kWarps) {
-      if (hs[j] < 0.f) continue;  // (warp-uniform)
-      float acc = 0.f;
+    for (int c = 0; c < CPL; ++c) x[c] = Ys[lane * CPL + c] * inv_H;
+    // ---- distances of the tokens present to the current output: a warp takes eight rows at a time, so that eight
+    //      loads are in flight (one row after the other, the sweep ran at the latency of a load from L2 per row) ----
+    constexpr int kInFlight = 8;
+    for (int j0 = warp; j0 < n; j0 += kInFlight * kWarps) {
+      float vf[kInFlight][CPL];
+      bool live[kInFlight];
 #pragma unroll
-      for (int c = 0; c < CPL; ++c) {
-        const float dlt = x[c] - to_float(Vu[(size_t)j * D + c * 32 + lane]);
-        acc = fmaf(dlt, dlt, acc);
+      for (int u = 0; u < kInFlight; ++u) {
+        const int j = j0 + u * kWarps;
+        live[u] = j < n && hs[j] >= 0.f;  // (warp-uniform)
+        if (live[u]) load_channels<CPL>(Vu + (size_t)j * D + lane * CPL, vf[u]);
       }
-      acc = warp_sum(acc);
-      if (lane == 0) ds[j] = sqrtf(acc);
+#pragma unroll
+      for (int u = 0; u < kInFlight; ++u) {
+        if (!live[u]) continue;
+        float acc = 0.f;
+#pragma unroll
+        for (int c = 0; c < CPL; ++c) {
+          const float dlt = x[c] - vf[u][c];
+          acc = fmaf(dlt, dlt, acc);
+        }
+        acc = warp_sum(acc);
+        if (lane == 0) ds[j0 + u * kWarps] = sqrtf(acc);
+      }
     }
     __syncthreads();
     // ---- arg-min of w_j / (1 - w_j) * dist_j over (score bits, position) ----
