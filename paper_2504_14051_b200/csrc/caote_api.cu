@@ -788,15 +788,15 @@ static int launch_greedy_cluster(const Dims& dm, const void* V, const float* h, 
   int need = 1;
   while (need <= greedy_cl::kMaxC && (dm.cap + need - 1) / need > greedy_cl::kMaxRows) need *= 2;
   if (need > greedy_cl::kMaxC) return CAOTE_OK;
+  // (the function's limits are set to the largest any launch may ask for, the same value every time: calls from
+  // several host threads then never see a limit below what they need)
   CAOTE_CUDA(cudaFuncSetAttribute(greedy_cl::greedy_cluster_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
+  CAOTE_CUDA(cudaFuncSetAttribute(greedy_cl::greedy_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  (int)greedy_cl::smem_bytes(greedy_cl::kMaxRows)));
   int best_c = 0, best_rows = 0, best_got = 0;
   for (int c = need; c <= greedy_cl::kMaxC; c *= 2) {
     const int rows = ((dm.cap + c - 1) / c + 7) / 8 * 8;
     const size_t smem = greedy_cl::smem_bytes(rows);
-    if (cudaFuncSetAttribute(greedy_cl::greedy_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
-      (void)cudaGetLastError();
-      continue;
-    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(c * dm.units));
     cfg.blockDim = dim3(greedy_cl::kThreads);
@@ -831,7 +831,6 @@ static int launch_greedy_cluster(const Dims& dm, const void* V, const float* h, 
     if (max_evict < 4 || t_one * waves_one < 1.2 * t_cluster * waves_cluster) return CAOTE_OK;
   }
   const size_t smem = greedy_cl::smem_bytes(best_rows);
-  CAOTE_CUDA(cudaFuncSetAttribute(greedy_cl::greedy_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(best_c * dm.units));
   cfg.blockDim = dim3(greedy_cl::kThreads);
