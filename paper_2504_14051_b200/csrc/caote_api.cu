@@ -655,11 +655,17 @@ static int launch_prefill_score(const Dims& dm, const void* q, const void* K, co
                  launch_pdl(prefill::attn_kernel, dim3(grid), dim3(prefill::kAttnThreads), prefill::attn_smem_bytes(), st, tmQ, tmK64, tmV64, dm, len,
                                                                                                     sc, o, status));
   }
-  if (sc.nsplit > 1) {
+  const bool merged_with_mean = sc.nsplit > 1 && !vsum;  // (small grids: the splits' merge and the column mean in one launch)
+  if (merged_with_mean) {
+    dim3 grid(dm.units, prefill::kD / 16);
+    CAOTE_LAUNCH("prefill_combine_xsum_kernel", st,
+                 launch_pdl(prefill::attn_combine_xsum_kernel, dim3(grid), dim3(prefill::kCxThreads), 0, st, dm, len, sc, o));
+  } else if (sc.nsplit > 1) {
     dim3 grid((dm.R + 3) / 4, dm.units);
     CAOTE_LAUNCH("prefill_attn_combine_kernel", st, launch_pdl(prefill::attn_combine_kernel, dim3(grid), dim3(4 * prefill::kD), 0, st, dm, len, sc, o));
   }
-  if (vsum) {
+  if (merged_with_mean) {
+  } else if (vsum) {
     CAOTE_LAUNCH("fast_mean_kernel", st, fast::mean_kernel<<<dm.units, prefill::kD, 0, st>>>(dm.Hkv, dm.cap, prefill::kD, len, vsum, sc.X));
   } else {
     CAOTE_LAUNCH("prefill_xsum_kernel", st, launch_pdl(prefill::xsum_kernel, dim3(dm.units), dim3(prefill::kXsumLanes * prefill::kD), 0, st, dm, len, o, sc));

@@ -595,6 +595,70 @@ attn_combine_kernel(Dims dm, const int* __restrict__ len, Scratch sc, float* __r
   if (c == 0) sc.stats[(size_t)unit * sc.Mpad + R] = mx + log2f(tot);
 }
 
+// The merge of the key splits and the column mean in one launch (small grids, where every launch counts): a CTA takes
+// 16 channels of a unit and all of its rows, merges the splits row by row exactly as attn_combine_kernel does, writes
+// o and (the CTA of channels 0..15) the rows' statistics, and adds up its 16 columns in a fixed order for X. Units that
+// ran unsplit are only summed. grid = (units, kD / 16), 512 threads: a warp takes 8 rows at a time, 4 lanes per row.
+constexpr int kCxThreads = 512;
+__global__ void __launch_bounds__(kCxThreads)
+attn_combine_xsum_kernel(Dims dm, const int* __restrict__ len, Scratch sc, float* __restrict__ o) {
+  ptx::pdl_wait();
+  ptx::pdl_trigger();
+  __shared__ float4 wpart[kCxThreads / 32][4];
+  const int unit = blockIdx.x, c0 = blockIdx.y * 16;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int n = len[unit / dm.Hkv];
+  if (n == 0 || n < dm.m || n > dm.cap) return;
+  int ts, nsp;
+  split_plan(n, dm.m, sc.nsplit, ts, nsp);
+  const int ch = c0 + 4 * (lane & 3);
+  float4 cs = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int R = warp * 8 + (lane >> 2); R < dm.R; R += (kCxThreads / 32) * 8) {
+    float* orow = o + ((size_t)unit * dm.R + R) * kD + ch;
+    float4 res;
+    if (nsp > 1) {
+      float st[8], mx = -INFINITY;
+      for (int s = 0; s < nsp; ++s) {
+        st[s] = sc.pstat[((size_t)unit * sc.nsplit + s) * sc.Mpad + R];
+        mx = fmaxf(mx, st[s]);
+      }
+      float tot = 0.f;
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int s = 0; s < nsp; ++s) {
+        const float w = exp2f(st[s] - mx);
+        tot += w;
+        const float4 p = *reinterpret_cast<const float4*>(sc.po + (((size_t)unit * sc.nsplit + s) * sc.Mpad + R) * kD + ch);
+        acc.x = fmaf(p.x, w, acc.x); acc.y = fmaf(p.y, w, acc.y); acc.z = fmaf(p.z, w, acc.z); acc.w = fmaf(p.w, w, acc.w);
+      }
+      res = make_float4(acc.x / tot, acc.y / tot, acc.z / tot, acc.w / tot);
+      *reinterpret_cast<float4*>(orow) = res;
+      if (ch == 0) sc.stats[(size_t)unit * sc.Mpad + R] = mx + log2f(tot);
+    } else {
+      res = *reinterpret_cast<const float4*>(orow);
+    }
+    cs.x += res.x; cs.y += res.y; cs.z += res.z; cs.w += res.w;
+  }
+  // the warp's eight row lanes of every channel quad, then the warps in order
+#pragma unroll
+  for (int off = 4; off < 32; off <<= 1) {
+    cs.x += __shfl_xor_sync(0xffffffffu, cs.x, off);
+    cs.y += __shfl_xor_sync(0xffffffffu, cs.y, off);
+    cs.z += __shfl_xor_sync(0xffffffffu, cs.z, off);
+    cs.w += __shfl_xor_sync(0xffffffffu, cs.w, off);
+  }
+  if (lane < 4) wpart[warp][lane] = cs;
+  __syncthreads();
+  if (tid < 4) {
+    float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int w = 0; w < kCxThreads / 32; ++w) {
+      const float4 p = wpart[w][tid];
+      t.x += p.x; t.y += p.y; t.z += p.z; t.w += p.w;
+    }
+    const float inv = 1.f / (float)dm.R;
+    *reinterpret_cast<float4*>(sc.X + (size_t)unit * kD + c0 + 4 * tid) = make_float4(t.x * inv, t.y * inv, t.z * inv, t.w * inv);
+  }
+}
+
 // X[unit] = mean of the unit's M rows of o. grid = units, kXsumLanes x 128 threads (row lanes x channels).
 constexpr int kXsumLanes = 8;  // row lanes per channel: 8 x 128 threads per unit
 __global__ void __launch_bounds__(kXsumLanes * kD)
