@@ -781,9 +781,9 @@ static int launch_greedy(const Dims& dm, const void* V, const float* h, const in
   return CAOTE_OK;
 }
 
-// Greedy eviction with the unit's value rows in the shared memory of a cluster (bf16, d 128). *used = false: the
-// shape does not fit (a unit needs more than 16 CTAs' worth of shared memory, or no cluster can run) and the caller
-// takes the one-CTA kernel. Among the cluster sizes that hold a unit, the largest one of which the GPU can run as
+// Greedy eviction with the unit's value rows in the shared memory of a cluster (bf16, d 128; what 16 CTAs cannot
+// hold of a long unit stays in global memory and is swept from L2). *used = false: the shape does not fit (more
+// than 16 x 2048 tokens, or no cluster can run) or the one-CTA kernel is the better choice, and the caller takes that. Among the cluster sizes that hold a unit, the largest one of which the GPU can run as
 // many at once as there are units: more CTAs per unit make a pick faster, a second wave of clusters makes the call
 // twice as long.
 static int launch_greedy_cluster(const Dims& dm, const void* V, const float* h, const int* len, const int* budget,
@@ -791,18 +791,18 @@ static int launch_greedy_cluster(const Dims& dm, const void* V, const float* h, 
                                  cudaStream_t st, bool* used) {
   *used = false;
   if (!aligned(V, 16)) return CAOTE_OK;
-  int need = 1;
-  while (need <= greedy_cl::kMaxC && (dm.cap + need - 1) / need > greedy_cl::kMaxRows) need *= 2;
-  if (need > greedy_cl::kMaxC) return CAOTE_OK;
+  int need = 1;  // the smallest cluster that holds the unit in shared memory, else the largest cluster
+  while (need < greedy_cl::kMaxC && (dm.cap + need - 1) / need > greedy_cl::kMaxRows) need *= 2;
+  if ((dm.cap + need - 1) / need > greedy_cl::kMaxShare) return CAOTE_OK;
   // (the function's limits are set to the largest any launch may ask for, the same value every time: calls from
   // several host threads then never see a limit below what they need)
   CAOTE_CUDA(cudaFuncSetAttribute(greedy_cl::greedy_cluster_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
   CAOTE_CUDA(cudaFuncSetAttribute(greedy_cl::greedy_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  (int)greedy_cl::smem_bytes(greedy_cl::kMaxRows)));
+                                  (int)greedy_cl::smem_bytes(greedy_cl::kMaxRows, greedy_cl::kMaxShare)));
   int best_c = 0, best_rows = 0, best_got = 0;
   for (int c = need; c <= greedy_cl::kMaxC; c *= 2) {
     const int rows = ((dm.cap + c - 1) / c + 7) / 8 * 8;
-    const size_t smem = greedy_cl::smem_bytes(rows);
+    const size_t smem = greedy_cl::smem_bytes(rows < greedy_cl::kMaxRows ? rows : greedy_cl::kMaxRows, rows);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(c * dm.units));
     cfg.blockDim = dim3(greedy_cl::kThreads);
@@ -831,12 +831,14 @@ static int launch_greedy_cluster(const Dims& dm, const void* V, const float* h, 
     // Worth it? Per pick the one-CTA kernel sweeps the unit's rows from L2 (measured: 9.5 ns per row), this one its
     // share of them from shared memory plus a cluster barrier (measured: about 6 us + 7 ns per row); but the GPU runs
     // fewer clusters at once than single CTAs, and with a handful of picks loading the rows is all there is.
-    const double t_one = 0.0095 * dm.cap, t_cluster = 6.0 + 0.007 * best_rows;
+    const int in_smem = best_rows < greedy_cl::kMaxRows ? best_rows : greedy_cl::kMaxRows;
+    const double t_one = 0.0095 * dm.cap, t_cluster = 6.0 + 0.007 * in_smem + 0.012 * (best_rows - in_smem);
     const double waves_one = (double)((dm.units + g_sm_count - 1) / g_sm_count);
     const double waves_cluster = (double)((dm.units + best_got - 1) / best_got);
     if (max_evict < 4 || t_one * waves_one < 1.2 * t_cluster * waves_cluster) return CAOTE_OK;
   }
-  const size_t smem = greedy_cl::smem_bytes(best_rows);
+  const int rows_smem = best_rows < greedy_cl::kMaxRows ? best_rows : greedy_cl::kMaxRows;
+  const size_t smem = greedy_cl::smem_bytes(rows_smem, best_rows);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(best_c * dm.units));
   cfg.blockDim = dim3(greedy_cl::kThreads);
@@ -850,7 +852,7 @@ static int launch_greedy_cluster(const Dims& dm, const void* V, const float* h, 
   cfg.attrs = at;
   cfg.numAttrs = 1;
   CAOTE_LAUNCH("greedy_cluster_kernel", st, {
-    cudaError_t e = cudaLaunchKernelEx(&cfg, greedy_cl::greedy_cluster_kernel, dm.Hkv, dm.cap, best_rows,
+    cudaError_t e = cudaLaunchKernelEx(&cfg, greedy_cl::greedy_cluster_kernel, dm.Hkv, dm.cap, best_rows, rows_smem,
                                        (const __nv_bfloat16*)V, h, len, budget, pos, evict_idx, order, max_evict, n_evict,
                                        status);
     if (e != cudaSuccess) return cuda_fail(e, "greedy_cluster_kernel");

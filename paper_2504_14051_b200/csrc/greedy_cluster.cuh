@@ -7,6 +7,9 @@
 //   minimum; every CTA reads the evicted row from its owner's shared memory and updates its own copy of Y and H
 //   (the same arithmetic everywhere, so the copies never differ).
 // The candidates are double-buffered by the parity of the pick, which is what makes one barrier per pick enough.
+// A CTA holds up to kMaxRows rows in shared memory; a unit too long for 16 CTAs' worth leaves the rest of every CTA's
+// share in global memory, and the CTA sweeps that part from L2 (several rows in flight per warp): still 16 SMs
+// pulling on a sixteenth each instead of one SM on all of it.
 #pragma once
 
 #include "common.cuh"
@@ -17,7 +20,8 @@ namespace greedy_cl {
 constexpr int kThreads = 512;
 constexpr int kWarps = kThreads / 32;
 constexpr int kD = 128;
-constexpr int kMaxRows = 768;   // value rows per CTA (192 KB)
+constexpr int kMaxRows = 768;   // value rows per CTA in shared memory (192 KB)
+constexpr int kMaxShare = 2048; // rows per CTA in all (the weights and distances of all of them are in shared memory)
 constexpr int kMaxC = 16;
 
 struct Cand {  // a CTA's best candidate of a pick
@@ -26,8 +30,8 @@ struct Cand {  // a CTA's best candidate of a pick
   float h;                 // its weight
 };
 
-inline size_t smem_bytes(int rows) {
-  return (size_t)rows * kD * 2 + sizeof(float) * (2 * (size_t)rows + kD + (kD + 4) + 2 * kWarps) +
+inline size_t smem_bytes(int rows_smem, int rows) {
+  return (size_t)rows_smem * kD * 2 + sizeof(float) * (2 * (size_t)rows + kD + (kD + 4) + 2 * kWarps) +
          sizeof(unsigned long long) * kWarps + sizeof(int) * (2 * kWarps + 8) + 2 * sizeof(Cand) + 64;
 }
 
@@ -77,15 +81,16 @@ __device__ __forceinline__ unsigned short gc_ld_u16(uint32_t a) {
   return v;
 }
 
-// grid = units x C CTAs in clusters of C; rows_per = rows of the unit per CTA (the same for every CTA of the grid).
+// grid = units x C CTAs in clusters of C; rows_per = rows of the unit per CTA (the same for every CTA of the grid),
+// the first rows_smem of them in shared memory.
 __global__ void __launch_bounds__(kThreads, 1)
-greedy_cluster_kernel(int Hkv, int cap, int rows_per, const __nv_bfloat16* __restrict__ V, const float* __restrict__ h_in,
+greedy_cluster_kernel(int Hkv, int cap, int rows_per, int rows_smem, const __nv_bfloat16* __restrict__ V, const float* __restrict__ h_in,
                       const int* __restrict__ len, const int* __restrict__ budget, const int* __restrict__ pos,
                       int* __restrict__ evict_idx, int* __restrict__ order_out, int max_evict, int* __restrict__ n_evict,
                       int* status) {
   extern __shared__ __align__(16) unsigned char gsm[];
-  __nv_bfloat16* Vs = reinterpret_cast<__nv_bfloat16*>(gsm);            // [rows_per][kD]
-  float* hs = reinterpret_cast<float*>(Vs + (size_t)rows_per * kD);     // [rows_per] weight, < 0 once evicted
+  __nv_bfloat16* Vs = reinterpret_cast<__nv_bfloat16*>(gsm);            // [rows_smem][kD]
+  float* hs = reinterpret_cast<float*>(Vs + (size_t)rows_smem * kD);    // [rows_per] weight, < 0 once evicted
   float* ds = hs + rows_per;                                            // [rows_per] || X - v_j || of the current state
   float* Ys = ds + rows_per;                                            // [kD] sum of h_j v_j over the tokens present
   float* part = Ys + kD;                                                // [kD + 4] this CTA's share of Y and (at kD) of H
@@ -120,7 +125,8 @@ greedy_cluster_kernel(int Hkv, int cap, int rows_per, const __nv_bfloat16* __res
   int* ord = order_out ? order_out + (size_t)unit * max_evict : nullptr;
 
   // ---- the rows into shared memory; H and Y of this CTA's rows (fixed order of the partial sums) ----
-  for (int i = tid; i < nr * (kD / 8); i += kThreads)
+  const int ns = min(nr, rows_smem);  // rows held in shared memory; rows [ns, nr) stay in global memory
+  for (int i = tid; i < ns * (kD / 8); i += kThreads)
     reinterpret_cast<uint4*>(Vs)[i] = reinterpret_cast<const uint4*>(Vu)[i];
   float hsum = 0.f;
   for (int j = tid; j < nr; j += kThreads) {
@@ -134,7 +140,7 @@ greedy_cluster_kernel(int Hkv, int cap, int rows_per, const __nv_bfloat16* __res
   float yacc[4] = {0.f, 0.f, 0.f, 0.f};
   for (int j = warp; j < nr; j += kWarps) {
     const float hj = hs[j];
-    const uint2 raw = *reinterpret_cast<const uint2*>(Vs + (size_t)j * kD + 4 * lane);
+    const uint2 raw = *reinterpret_cast<const uint2*>((j < ns ? Vs : Vu) + (size_t)j * kD + 4 * lane);
     yacc[0] = fmaf(hj, __uint_as_float(raw.x << 16), yacc[0]);
     yacc[1] = fmaf(hj, __uint_as_float(raw.x & 0xffff0000u), yacc[1]);
     yacc[2] = fmaf(hj, __uint_as_float(raw.y << 16), yacc[2]);
@@ -170,13 +176,32 @@ greedy_cluster_kernel(int Hkv, int cap, int rows_per, const __nv_bfloat16* __res
 #pragma unroll
     for (int c = 0; c < 4; ++c) x[c] = Ys[4 * lane + c] * inv_H;
     // ---- distances of this CTA's tokens still present to the current output (a warp per token) ----
-    for (int j = warp; j < nr; j += kWarps) {
+    for (int j = warp; j < ns; j += kWarps) {
       if (hs[j] < 0.f) continue;  // (warp-uniform)
       const uint2 raw = *reinterpret_cast<const uint2*>(Vs + (size_t)j * kD + 4 * lane);
       const float d0 = x[0] - __uint_as_float(raw.x << 16), d1 = x[1] - __uint_as_float(raw.x & 0xffff0000u);
       const float d2 = x[2] - __uint_as_float(raw.y << 16), d3 = x[3] - __uint_as_float(raw.y & 0xffff0000u);
       const float acc = warp_sum(fmaf(d0, d0, fmaf(d1, d1, fmaf(d2, d2, d3 * d3))));
       if (lane == 0) ds[j] = sqrtf(acc);
+    }
+    // ... and of the rows it left in global memory: eight loads in flight per warp
+    for (int j0 = ns + warp; j0 < nr; j0 += 8 * kWarps) {
+      uint2 raw[8];
+      bool live[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int j = j0 + u * kWarps;
+        live[u] = j < nr && hs[j] >= 0.f;  // (warp-uniform)
+        if (live[u]) raw[u] = *reinterpret_cast<const uint2*>(Vu + (size_t)j * kD + 4 * lane);
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        if (!live[u]) continue;
+        const float d0 = x[0] - __uint_as_float(raw[u].x << 16), d1 = x[1] - __uint_as_float(raw[u].x & 0xffff0000u);
+        const float d2 = x[2] - __uint_as_float(raw[u].y << 16), d3 = x[3] - __uint_as_float(raw[u].y & 0xffff0000u);
+        const float acc = warp_sum(fmaf(d0, d0, fmaf(d1, d1, fmaf(d2, d2, d3 * d3))));
+        if (lane == 0) ds[j0 + u * kWarps] = sqrtf(acc);
+      }
     }
     __syncthreads();
     // ---- this CTA's arg-min of w_j / (1 - w_j) * dist_j over (score bits, position) (a thread per token; doing
@@ -240,8 +265,9 @@ greedy_cluster_kernel(int Hkv, int cap, int rows_per, const __nv_bfloat16* __res
     // ---- evict e: Y -= h_e v_e, H -= h_e (the row comes from its owner's shared memory) ----
     const float he = s_he;
     const int owner = e / rows_per, el = e - owner * rows_per;
-    if (tid < kD) {
-      const unsigned short raw = gc_ld_u16(gc_map(Vs + (size_t)el * kD + tid, (uint32_t)owner));
+    if (tid < kD) {  // (from its owner's shared memory, or from global memory if the owner left it there)
+      const unsigned short raw = el < rows_smem ? gc_ld_u16(gc_map(Vs + (size_t)el * kD + tid, (uint32_t)owner))
+                                                : __bfloat16_as_ushort(V[((size_t)unit * cap + e) * kD + tid]);
       Ys[tid] -= he * __uint_as_float((uint32_t)raw << 16);
     }
     if (tid == 0) {

@@ -57,6 +57,7 @@ def follow(order_gpu, h, V, pos, k):
     (1, 1, 128, 40, [33], 32, torch.bfloat16),          # down to a single token
     (2, 3, 128, 2104, [2000, 777], 64, torch.bfloat16), # the cluster kernel; the short sequence leaves most CTAs of its clusters without rows
     (1, 2, 128, 6160, [6150], 24, torch.bfloat16),      # the cluster kernel with several hundred rows per CTA
+    (1, 2, 128, 13000, [12900], 24, torch.bfloat16),    # more rows than 16 CTAs hold in shared memory: the rest from L2
 ])
 def test_greedy_sequence_follows_the_oracle(case):
     B, Hkv, d, cap, lens, k, dtype = case
