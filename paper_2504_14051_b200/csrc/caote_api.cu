@@ -655,7 +655,7 @@ static int launch_prefill_score(const Dims& dm, const void* q, const void* K, co
                  launch_pdl(prefill::attn_kernel, dim3(grid), dim3(prefill::kAttnThreads), prefill::attn_smem_bytes(), st, tmQ, tmK64, tmV64, dm, len,
                                                                                                     sc, o, status));
   }
-  const bool merged_with_mean = sc.nsplit > 1 && !vsum;  // (small grids: the splits' merge and the column mean in one launch)
+  const bool merged_with_mean = !vsum;  // the splits' merge (if there are splits) and the column mean in one launch
   if (merged_with_mean) {
     dim3 grid(dm.units, prefill::kD / 16);
     CAOTE_LAUNCH("prefill_combine_xsum_kernel", st,
@@ -664,11 +664,8 @@ static int launch_prefill_score(const Dims& dm, const void* q, const void* K, co
     dim3 grid((dm.R + 3) / 4, dm.units);
     CAOTE_LAUNCH("prefill_attn_combine_kernel", st, launch_pdl(prefill::attn_combine_kernel, dim3(grid), dim3(4 * prefill::kD), 0, st, dm, len, sc, o));
   }
-  if (merged_with_mean) {
-  } else if (vsum) {
+  if (vsum) {
     CAOTE_LAUNCH("fast_mean_kernel", st, fast::mean_kernel<<<dm.units, prefill::kD, 0, st>>>(dm.Hkv, dm.cap, prefill::kD, len, vsum, sc.X));
-  } else {
-    CAOTE_LAUNCH("prefill_xsum_kernel", st, launch_pdl(prefill::xsum_kernel, dim3(dm.units), dim3(prefill::kXsumLanes * prefill::kD), 0, st, dm, len, o, sc));
   }
   {
     dim3 grid((dm.cap + prefill::kScoreKeys - 1) / prefill::kScoreKeys, dm.units);

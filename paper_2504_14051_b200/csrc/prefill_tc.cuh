@@ -10,8 +10,9 @@
 //                 softmax statistics (reference, 1 / sum). One lane each of three extra warps issues
 //                 the products, the K copies and the V copies, so the tensor pipe always has the
 //                 next S queued while the rows are busy with the current one.
-//   xsum_kernel   X = mean of the unit's M output rows (the weights of CHUNK_SUM are the column sums
-//                 of the attention matrix divided by M, so sum_j w_j v_j is the mean output row).
+//   attn_combine_xsum_kernel   merges the key splits of small grids (attn_combine_kernel does only that, for
+//                 FastCAOTE) and forms X = mean of the unit's M output rows (the weights of CHUNK_SUM are the
+//                 column sums of the attention matrix divided by M, so sum_j w_j v_j is the mean output row).
 //   score_kernel  keys x rows. One CTA owns 256 keys of a unit (two key tiles) and walks the unit's
 //                 rows in blocks of 128: S^T = K Q^T lands in TMEM with one key per lane, so each
 //                 thread sums exp2(s - ref_r) / sum_r over the rows of its own key without any
@@ -595,10 +596,11 @@ attn_combine_kernel(Dims dm, const int* __restrict__ len, Scratch sc, float* __r
   if (c == 0) sc.stats[(size_t)unit * sc.Mpad + R] = mx + log2f(tot);
 }
 
-// The merge of the key splits and the column mean in one launch (small grids, where every launch counts): a CTA takes
-// 16 channels of a unit and all of its rows, merges the splits row by row exactly as attn_combine_kernel does, writes
-// o and (the CTA of channels 0..15) the rows' statistics, and adds up its 16 columns in a fixed order for X. Units that
-// ran unsplit are only summed. grid = (units, kD / 16), 512 threads: a warp takes 8 rows at a time, 4 lanes per row.
+// The merge of the key splits and the column mean X (the weights of CHUNK_SUM are the column sums of the attention
+// matrix divided by M, so sum_j w_j v_j is the mean output row) in one launch: a CTA takes 16 channels of a unit and
+// all of its rows, merges the splits row by row exactly as attn_combine_kernel does, writes o and (the CTA of channels
+// 0..15) the rows' statistics, and adds up its 16 columns in a fixed order for X. Units that ran unsplit are only
+// summed. grid = (units, kD / 16), 512 threads: a warp takes 8 rows at a time, 4 lanes per row.
 constexpr int kCxThreads = 512;
 __global__ void __launch_bounds__(kCxThreads)
 attn_combine_xsum_kernel(Dims dm, const int* __restrict__ len, Scratch sc, float* __restrict__ o) {
@@ -656,34 +658,6 @@ attn_combine_xsum_kernel(Dims dm, const int* __restrict__ len, Scratch sc, float
     }
     const float inv = 1.f / (float)dm.R;
     *reinterpret_cast<float4*>(sc.X + (size_t)unit * kD + c0 + 4 * tid) = make_float4(t.x * inv, t.y * inv, t.z * inv, t.w * inv);
-  }
-}
-
-// X[unit] = mean of the unit's M rows of o. grid = units, kXsumLanes x 128 threads (row lanes x channels).
-constexpr int kXsumLanes = 8;  // row lanes per channel: 8 x 128 threads per unit
-__global__ void __launch_bounds__(kXsumLanes * kD)
-xsum_kernel(Dims dm, const int* __restrict__ len, const float* __restrict__ o, Scratch sc) {
-  ptx::pdl_wait();
-  ptx::pdl_trigger();
-  __shared__ float part[kXsumLanes][kD];
-  const int unit = blockIdx.x, c = threadIdx.x % kD, lane = threadIdx.x / kD;
-  const int n = len[unit / dm.Hkv];
-  if (n == 0 || n < dm.m || n > dm.cap) return;
-  const float* base = o + (size_t)unit * dm.R * kD + c;
-  float acc[4] = {0.f, 0.f, 0.f, 0.f};
-  int r = lane;
-  for (; r + 3 * kXsumLanes < dm.R; r += 4 * kXsumLanes) {
-#pragma unroll
-    for (int i = 0; i < 4; ++i) acc[i] += base[(size_t)(r + i * kXsumLanes) * kD];
-  }
-  for (; r < dm.R; r += kXsumLanes) acc[0] += base[(size_t)r * kD];
-  part[lane][c] = (acc[0] + acc[1]) + (acc[2] + acc[3]);
-  __syncthreads();
-  if (lane == 0) {
-    float s = 0.f;
-#pragma unroll
-    for (int l = 0; l < kXsumLanes; ++l) s += part[l][c];  // fixed order: reproducible
-    sc.X[(size_t)unit * kD + c] = s / (float)dm.R;
   }
 }
 
