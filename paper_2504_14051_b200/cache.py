@@ -39,9 +39,13 @@ class EvictionCache:
             budget = torch.full((B,), budget, dtype=torch.int32)
         self.budget = budget.to(device=dev, dtype=torch.int32).contiguous()
         self.max_evict = max_evict if max_evict is not None else max(n_new, 1)
-        self.evict_idx = torch.zeros((B, Hkv, self.max_evict), dtype=torch.int32, device=dev)
-        self.n_evict = torch.zeros((B,), dtype=torch.int32, device=dev)
-        self.o = torch.zeros((B, Hq, m, d), dtype=torch.float32, device=dev)
+        # what a step hands back (o, evict_idx, n_evict) lives in one buffer, so that a caller who wants it on the
+        # host can fetch it with a single copy of `self.results`
+        n_o, n_e = B * Hq * m * d, B * Hkv * self.max_evict
+        self.results = torch.zeros((n_o + n_e + B,), dtype=torch.float32, device=dev)
+        self.o = self.results[:n_o].view(B, Hq, m, d)
+        self.evict_idx = self.results[n_o:n_o + n_e].view(torch.int32).view(B, Hkv, self.max_evict)
+        self.n_evict = self.results[n_o + n_e:].view(torch.int32)
         self.workspace = C.alloc_workspace(self.params, dev)
         # FastCAOTE (Sec. 3.3) scores against the mean of the cached values: the per-unit sum of V rows is state
         assert method in ("caote", "fast", "sum_errors", "post_evict")
