@@ -107,33 +107,13 @@ inline size_t smem_bytes() {
          2 * 32 * 4 /* red */ + 4 * 28 * 4 /* gred */ + kStatFloats * 4 /* mystat */ + kLenTab * 4 + 64 * 8 /* barriers, control words */ + 64;
 }
 
-// ---- cluster PTX ------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t cluster_ctarank() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-  return r;
-}
-__device__ __forceinline__ uint32_t cluster_nctarank() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
-  return r;
-}
-__device__ __forceinline__ uint32_t cluster_id_x() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%clusterid.x;" : "=r"(r));
-  return r;
-}
-__device__ __forceinline__ uint32_t cluster_count_x() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%nclusterid.x;" : "=r"(r));
-  return r;
-}
-// Address of the same shared-memory location in the CTA of rank `rank` of this cluster.
-__device__ __forceinline__ uint32_t map_to_rank(uint32_t local_addr, uint32_t rank) {
-  uint32_t r;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
-  return r;
-}
+// ---- cluster PTX (the register reads, mapa and the cluster barrier are in ptx.cuh) ----------------------
+using ptx::cluster_count_x;
+using ptx::cluster_ctarank;
+using ptx::cluster_id_x;
+using ptx::cluster_nctarank;
+using ptx::cluster_sync_all;
+using ptx::map_to_rank;
 // Floats into a peer's shared memory; the peer's mbarrier counts the bytes when they have landed.
 __device__ __forceinline__ void push_f32(uint32_t remote_addr, float v, uint32_t remote_bar) {
   asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];"
@@ -143,10 +123,6 @@ __device__ __forceinline__ void push_f32x4(uint32_t remote_addr, float a, float 
   asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];"
                ::"r"(remote_addr), "r"(__float_as_uint(a)), "r"(__float_as_uint(b)), "r"(__float_as_uint(c)),
                  "r"(__float_as_uint(d)), "r"(remote_bar) : "memory");
-}
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
 // try_wait that lets the hardware park the thread until the phase completes or `ns` nanoseconds pass: a

@@ -13,6 +13,7 @@
 #pragma once
 
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace caote {
 namespace greedy_cl {
@@ -35,51 +36,16 @@ inline size_t smem_bytes(int rows_smem, int rows) {
          sizeof(unsigned long long) * kWarps + sizeof(int) * (2 * kWarps + 8) + 2 * sizeof(Cand) + 64;
 }
 
-__device__ __forceinline__ uint32_t gc_rank() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-  return r;
-}
-__device__ __forceinline__ uint32_t gc_size() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
-  return r;
-}
-__device__ __forceinline__ uint32_t gc_cluster_id() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%clusterid.x;" : "=r"(r));
-  return r;
-}
-__device__ __forceinline__ void gc_sync() {
-  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// The same shared-memory location in the CTA of rank `rank`, and loads from it.
-__device__ __forceinline__ uint32_t gc_map(const void* p, uint32_t rank) {
-  uint32_t r;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"((uint32_t)__cvta_generic_to_shared(p)), "r"(rank));
-  return r;
-}
-__device__ __forceinline__ float gc_ld_f32(uint32_t a) {
-  float v;
-  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(a) : "memory");
-  return v;
-}
-__device__ __forceinline__ int gc_ld_s32(uint32_t a) {
-  int v;
-  asm volatile("ld.shared::cluster.s32 %0, [%1];" : "=r"(v) : "r"(a) : "memory");
-  return v;
-}
-__device__ __forceinline__ unsigned long long gc_ld_u64(uint32_t a) {
-  unsigned long long v;
-  asm volatile("ld.shared::cluster.u64 %0, [%1];" : "=l"(v) : "r"(a) : "memory");
-  return v;
-}
-__device__ __forceinline__ unsigned short gc_ld_u16(uint32_t a) {
-  unsigned short v;
-  asm volatile("ld.shared::cluster.u16 %0, [%1];" : "=h"(v) : "r"(a) : "memory");
-  return v;
-}
+__device__ __forceinline__ uint32_t gc_rank() { return ptx::cluster_ctarank(); }
+__device__ __forceinline__ uint32_t gc_size() { return ptx::cluster_nctarank(); }
+__device__ __forceinline__ uint32_t gc_cluster_id() { return ptx::cluster_id_x(); }
+__device__ __forceinline__ void gc_sync() { ptx::cluster_sync_all(); }
+// The same shared-memory location in the CTA of rank `rank`.
+__device__ __forceinline__ uint32_t gc_map(const void* p, uint32_t rank) { return ptx::map_to_rank(ptx::smem_u32(p), rank); }
+__device__ __forceinline__ float gc_ld_f32(uint32_t a) { return ptx::ld_dsmem_f32(a); }
+__device__ __forceinline__ int gc_ld_s32(uint32_t a) { return ptx::ld_dsmem_s32(a); }
+__device__ __forceinline__ unsigned long long gc_ld_u64(uint32_t a) { return ptx::ld_dsmem_u64(a); }
+__device__ __forceinline__ unsigned short gc_ld_u16(uint32_t a) { return ptx::ld_dsmem_u16(a); }
 
 // grid = units x C CTAs in clusters of C; rows_per = rows of the unit per CTA (the same for every CTA of the grid),
 // the first rows_smem of them in shared memory.
