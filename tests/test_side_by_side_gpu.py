@@ -79,3 +79,25 @@ def test_side_by_side_matches_the_oracle_and_the_single_kernel(mode):
                                    scale=D ** -0.5, n_new=1)
     for b in range(B):
         assert_close(f32(o_post)[b], ref[b], f"post-eviction output from the statistics [b={b}]")
+
+
+def test_side_by_side_with_empty_sequences():
+    """An empty sequence among those of the cluster kernel and an empty one as the streaming kernel's whole share:
+    their outputs are left alone, the others match the oracle."""
+    lens = [1100, 0, 1152, 0]
+    q, K, V, lens_t = make_case(777, B, HQ, HKV, D, CAP, 1, torch.bfloat16, lens)
+    p = P.make_params(B, HQ, HKV, D, CAP, 1, torch.bfloat16, D ** -0.5, "last_query")
+    ws = P.alloc_workspace(p, DEV)
+    o = torch.full(q.shape, -3.0, dtype=torch.float32, device=DEV)
+    scores = torch.full((B, HKV, CAP), -7.0, dtype=torch.float32, device=DEV)
+    P.caote_set_option(P.OPT_SIDE_BY_SIDE, 2)
+    try:
+        P.caote_score(p, q, K, V, lens_t, None, o, scores, ws)
+        torch.cuda.synchronize()
+    finally:
+        P.caote_set_option(P.OPT_SIDE_BY_SIDE, 1)
+    assert P.caote_read_status(ws) == 0
+    r = oracle_for(q, K, V, lens_t, scale=D ** -0.5, n_new=1, base_mode="last_query")
+    check_scores_and_o(r, scores, o, lens_t, "side by side, empty sequences")
+    for b in (1, 3):
+        assert (f32(scores)[b] == -7.0).all() and (f32(o)[b] == -3.0).all()
