@@ -118,11 +118,11 @@ post_evict_kernel(Dims dm, const T* __restrict__ q, const T* __restrict__ K, con
 }
 
 // The same correction for blocks of queries whose rows' statistics the scoring call left behind (bf16, head_dim 128):
-// does nothing unless the workspace header says so. A CTA takes 32 query rows of a unit (four per warp) and walks
-// the unit's evicted slots 32 at a time: their K and V rows are gathered into shared memory once for all 32 query
+// does nothing unless the workspace header says so. A CTA takes 16 query rows of a unit (two per warp) and walks
+// the unit's evicted slots 32 at a time: their K and V rows are gathered into shared memory once for all its query
 // rows; for the logits a lane is an evicted token (its K row against the warp's four query rows, both from shared
-// memory), for the weighted value sum a lane is four channels. grid = (ceil(R / 32), units), 256 threads.
-constexpr int kBlockRows = 32, kChunk = 32, kRowsD = 128, kKLd = kRowsD + 1;
+// memory), for the weighted value sum a lane is four channels. grid = (ceil(R / 16), units), 256 threads.
+constexpr int kRowsPerWarp = 2, kBlockRows = 8 * kRowsPerWarp, kChunk = 32, kRowsD = 128, kKLd = kRowsD + 1;
 inline size_t rows_smem_bytes() {
   return sizeof(float) * ((size_t)kBlockRows * kRowsD + (size_t)kChunk * kKLd + (size_t)kChunk * kRowsD + (size_t)kBlockRows * kChunk) +
          sizeof(int) * kChunk;
@@ -153,11 +153,12 @@ post_evict_rows_kernel(Dims dm, const __nv_bfloat16* __restrict__ q, const __nv_
     const int rr = idx / D, c = idx % D, r = r0 + rr;
     Qs[idx] = (r < dm.R) ? __bfloat162float(q[row_off(r) + c]) : 0.f;
   }
-  int n_vis[4];
-  float stat[4], A[4], Y[4][4];
+  constexpr int RW = kRowsPerWarp;
+  int n_vis[RW];
+  float stat[RW], A[RW], Y[RW][4];
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int r = r0 + 4 * warp + i;
+  for (int i = 0; i < RW; ++i) {
+    const int r = r0 + RW * warp + i;
     n_vis[i] = (r < dm.R) ? n - m + (r % m) + 1 : 0;
     stat[i] = (r < dm.R) ? stats[(size_t)unit * stat_stride + r] : 0.f;
     A[i] = 0.f;
@@ -194,22 +195,24 @@ post_evict_rows_kernel(Dims dm, const __nv_bfloat16* __restrict__ q, const __nv_
     // weights: lane = evicted token of the chunk
     {
       const int j = js[lane];
-      float s[4] = {0.f, 0.f, 0.f, 0.f};
+      float s[RW];
+#pragma unroll
+      for (int i = 0; i < RW; ++i) s[i] = 0.f;
       const float* kp = Ks + lane * kKLd;
 #pragma unroll 8
       for (int c = 0; c < D; c += 4) {
         const float k0 = kp[c], k1 = kp[c + 1], k2 = kp[c + 2], k3 = kp[c + 3];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const float4 q4 = *reinterpret_cast<const float4*>(Qs + (4 * warp + i) * D + c);
+        for (int i = 0; i < RW; ++i) {
+          const float4 q4 = *reinterpret_cast<const float4*>(Qs + (RW * warp + i) * D + c);
           s[i] = fmaf(q4.x, k0, fmaf(q4.y, k1, fmaf(q4.z, k2, fmaf(q4.w, k3, s[i]))));
         }
       }
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
+      for (int i = 0; i < RW; ++i) {
         const float a = (j >= 0 && j < n_vis[i]) ? exp2f(fmaf(s[i], scale2, -stat[i])) : 0.f;
         A[i] += a;
-        As[(4 * warp + i) * kChunk + lane] = a;
+        As[(RW * warp + i) * kChunk + lane] = a;
       }
     }
     __syncwarp();  // (a warp reads only the weights it wrote)
@@ -218,8 +221,8 @@ post_evict_rows_kernel(Dims dm, const __nv_bfloat16* __restrict__ q, const __nv_
     for (int t = 0; t < kChunk; ++t) {
       const float4 v4 = *reinterpret_cast<const float4*>(Vs + t * D + 4 * lane);
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const float a = As[(4 * warp + i) * kChunk + t];
+      for (int i = 0; i < RW; ++i) {
+        const float a = As[(RW * warp + i) * kChunk + t];
         Y[i][0] = fmaf(a, v4.x, Y[i][0]);
         Y[i][1] = fmaf(a, v4.y, Y[i][1]);
         Y[i][2] = fmaf(a, v4.z, Y[i][2]);
@@ -228,8 +231,8 @@ post_evict_rows_kernel(Dims dm, const __nv_bfloat16* __restrict__ q, const __nv_
     }
   }
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int r = r0 + 4 * warp + i;
+  for (int i = 0; i < RW; ++i) {
+    const int r = r0 + RW * warp + i;
     const float rest = 1.f - warp_sum(A[i]);
     if (r < dm.R) {
       const size_t at = row_off(r) + 4 * lane;
