@@ -902,6 +902,13 @@ int caote_append(const caote_params_t* p, void* K, void* V, float* base, int32_t
   const Dims dm = make_dims(p);
   const int row_bytes = dm.D * (p->dtype == CAOTE_BF16 ? 2 : 4);
   cudaStream_t st = (cudaStream_t)stream;
+  if (dm.Hkv * dm.m <= 16) {  // (single-query decode: a CTA per sequence, which moves its lengths on itself)
+    CAOTE_LAUNCH("append_seq_kernel", st,
+                 launch_pdl(sel::append_seq_kernel, dim3(dm.B), dim3(64 * dm.Hkv * dm.m), 0, st, dm.Hkv, dm.cap, dm.m,
+                            row_bytes, (char*)K, (char*)V, base, pos, len, n_seen, (const char*)k_new,
+                            (const char*)v_new, (int*)workspace));
+    return CAOTE_OK;
+  }
   CAOTE_LAUNCH("append_kernel", st, launch_pdl(sel::append_kernel, dim3(dim3(dm.units, (dm.m + 7) / 8)), dim3(256), 0, st, dm.Hkv, dm.cap, dm.m, row_bytes, (char*)K, (char*)V, base, pos,
                                                len, n_seen, (const char*)k_new, (const char*)v_new,
                                                (int*)workspace, dm.B, (int*)workspace + 4));

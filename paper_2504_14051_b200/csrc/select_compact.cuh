@@ -243,27 +243,94 @@ compact_fill_kernel(int Hkv, int cap, int row_bytes, char* __restrict__ K, char*
   compact_fill_unit(blockIdx.x, n_evict[blockIdx.x / Hkv], Hkv, cap, row_bytes, K, V, base, pos, len, evict_idx, max_evict);
 }
 
-// Selection and FILL compaction of one unit per CTA in one launch, and the length update by whichever
-// CTA finishes last (a ticket counter in the workspace header, which that CTA also resets). Same results
-// as select_kernel + compact_fill_kernel + update_len_kernel.
-__global__ void __launch_bounds__(kSelThreads)
-select_compact_kernel(int B, int Hkv, int cap, int row_bytes, const float* __restrict__ scores, char* __restrict__ K,
-                      char* __restrict__ V, float* __restrict__ base, int* __restrict__ pos, int* __restrict__ len,
-                      const int* __restrict__ budget, int* __restrict__ evict_idx, int max_evict,
-                      int* __restrict__ n_evict, int* status, int* ticket, float* __restrict__ vsum, int elt_bytes) {
-  ptx::pdl_wait();
-  ptx::pdl_trigger();
-  __shared__ int s_last;
-  const int unit = blockIdx.x;
-  const int k = select_unit(unit, Hkv, cap, scores, len, budget, pos, evict_idx, max_evict, n_evict, status);
-  __syncthreads();  // evict_idx of this unit is written
-  if (vsum && k > 0) {  // FastCAOTE: the evicted rows leave the running sum of values before they are overwritten
-    const int* E = evict_idx + (size_t)unit * max_evict;
-    if (elt_bytes == 2) fast::vsum_sub_unit<__nv_bfloat16>(unit, k, cap, row_bytes / 2, (const __nv_bfloat16*)V, E, vsum);
-    else fast::vsum_sub_unit<float>(unit, k, cap, row_bytes / 4, (const float*)V, E, vsum);
-    __syncthreads();
+// A unit that evicts exactly one token, with FILL compaction: the argmin over (score bits, position) and the move of
+// the unit's last row into the hole in one go. The first scores of every thread are fetched before the length is known
+// (slots below cap always exist), the last row of K and V is fetched while the scores are searched, and the pick never
+// travels through global memory. Same results as select_unit + compact_fill_unit. Returns false, with nothing
+// written, unless the unit evicts exactly one token (row_bytes <= 512).
+__device__ __forceinline__ bool select_one_fill_unit(int unit, int Hkv, int cap, int row_bytes,
+                                                     const float* __restrict__ scores, char* __restrict__ K,
+                                                     char* __restrict__ V, float* __restrict__ base,
+                                                     int* __restrict__ pos, const int* __restrict__ len,
+                                                     const int* __restrict__ budget, int* __restrict__ evict_idx,
+                                                     int max_evict, int* __restrict__ n_evict) {
+  __shared__ unsigned long long s_key[kSelThreads / 32];
+  __shared__ int s_slot[kSelThreads / 32];
+  constexpr int kPer = 8;
+  const int b = unit / Hkv, h = unit % Hkv;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const float* sc = scores + (size_t)unit * cap;
+  const int* ps = pos ? pos + (size_t)unit * cap : nullptr;
+  float sv[kPer];
+  int pv[kPer];
+#pragma unroll
+  for (int i = 0; i < kPer; ++i) {
+    const int j = tid + i * kSelThreads;
+    sv[i] = (j < cap) ? sc[j] : 0.f;
+    pv[i] = (ps && j < cap) ? ps[j] : j;
   }
-  compact_fill_unit(unit, k, Hkv, cap, row_bytes, K, V, base, pos, len, evict_idx, max_evict);
+  const int n = len[b];
+  int bud = budget[b];
+  if (bud < 1) bud = 1;
+  if (n > cap || n - bud != 1) return false;
+  if (h == 0 && tid == 0) n_evict[b] = 1;
+  const int last = n - 1;
+  const size_t tail = (size_t)unit * cap + last;
+  const bool row_lane = lane * 16 < row_bytes;
+  uint4 row = make_uint4(0u, 0u, 0u, 0u);
+  float tail_base = 0.f;
+  int tail_pos = 0;
+  if (warp == 1 && row_lane) row = *reinterpret_cast<const uint4*>(K + tail * row_bytes + lane * 16);
+  if (warp == 2 && row_lane) row = *reinterpret_cast<const uint4*>(V + tail * row_bytes + lane * 16);
+  if (warp == 3 && lane == 0) {
+    if (base) tail_base = base[tail];
+    if (pos) tail_pos = pos[tail];
+  }
+  unsigned long long best = ~0ull;
+  int best_slot = 0;
+#pragma unroll
+  for (int i = 0; i < kPer; ++i) {
+    const int j = tid + i * kSelThreads;
+    const unsigned long long key = make_key(sv[i], pv[i]);
+    if (j < n && key < best) { best = key; best_slot = j; }
+  }
+  for (int j = tid + kPer * kSelThreads; j < n; j += kSelThreads) {
+    const unsigned long long key = make_key(sc[j], ps ? ps[j] : j);
+    if (key < best) { best = key; best_slot = j; }
+  }
+  // (key, slot): keys are unique when pos is, else the lower slot wins
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const unsigned long long ok = __shfl_xor_sync(0xffffffffu, best, o);
+    const int os = __shfl_xor_sync(0xffffffffu, best_slot, o);
+    if (ok < best || (ok == best && os < best_slot)) { best = ok; best_slot = os; }
+  }
+  if (lane == 0) { s_key[warp] = best; s_slot[warp] = best_slot; }
+  __syncthreads();
+  best = s_key[lane];  // every warp reduces the 32 partial results for itself
+  best_slot = s_slot[lane];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const unsigned long long ok = __shfl_xor_sync(0xffffffffu, best, o);
+    const int os = __shfl_xor_sync(0xffffffffu, best_slot, o);
+    if (ok < best || (ok == best && os < best_slot)) { best = ok; best_slot = os; }
+  }
+  if (tid == 0) evict_idx[(size_t)unit * max_evict] = best_slot;
+  if (best_slot != last) {  // the last row fills the hole
+    const size_t hole = (size_t)unit * cap + best_slot;
+    if (warp == 1 && row_lane) *reinterpret_cast<uint4*>(K + hole * row_bytes + lane * 16) = row;
+    if (warp == 2 && row_lane) *reinterpret_cast<uint4*>(V + hole * row_bytes + lane * 16) = row;
+    if (warp == 3 && lane == 0) {
+      if (base) base[hole] = tail_base;
+      if (pos) pos[hole] = tail_pos;
+    }
+  }
+  return true;
+}
+
+// The CTA that finishes last (a ticket counter, which it also resets) takes the evicted counts off the lengths.
+__device__ __forceinline__ void finish_lengths(int B, int* __restrict__ len, const int* __restrict__ n_evict, int* ticket) {
+  __shared__ int s_last;
   __syncthreads();
   if (threadIdx.x == 0) {
     __threadfence();
@@ -275,6 +342,34 @@ select_compact_kernel(int B, int Hkv, int cap, int row_bytes, const float* __res
     for (int b = threadIdx.x; b < B; b += blockDim.x) len[b] -= __ldcg(&n_evict[b]);
     if (threadIdx.x == 0) *ticket = 0;
   }
+}
+
+// Selection and FILL compaction of one unit per CTA in one launch, and the length update by whichever
+// CTA finishes last (a ticket counter in the workspace header, which that CTA also resets). Same results
+// as select_kernel + compact_fill_kernel + update_len_kernel.
+__global__ void __launch_bounds__(kSelThreads)
+select_compact_kernel(int B, int Hkv, int cap, int row_bytes, const float* __restrict__ scores, char* __restrict__ K,
+                      char* __restrict__ V, float* __restrict__ base, int* __restrict__ pos, int* __restrict__ len,
+                      const int* __restrict__ budget, int* __restrict__ evict_idx, int max_evict,
+                      int* __restrict__ n_evict, int* status, int* ticket, float* __restrict__ vsum, int elt_bytes) {
+  ptx::pdl_wait();
+  ptx::pdl_trigger();
+  const int unit = blockIdx.x;
+  if (!vsum && row_bytes <= 512 &&
+      select_one_fill_unit(unit, Hkv, cap, row_bytes, scores, K, V, base, pos, len, budget, evict_idx, max_evict, n_evict)) {
+    finish_lengths(B, len, n_evict, ticket);
+    return;
+  }
+  const int k = select_unit(unit, Hkv, cap, scores, len, budget, pos, evict_idx, max_evict, n_evict, status);
+  __syncthreads();  // evict_idx of this unit is written
+  if (vsum && k > 0) {  // FastCAOTE: the evicted rows leave the running sum of values before they are overwritten
+    const int* E = evict_idx + (size_t)unit * max_evict;
+    if (elt_bytes == 2) fast::vsum_sub_unit<__nv_bfloat16>(unit, k, cap, row_bytes / 2, (const __nv_bfloat16*)V, E, vsum);
+    else fast::vsum_sub_unit<float>(unit, k, cap, row_bytes / 4, (const float*)V, E, vsum);
+    __syncthreads();
+  }
+  compact_fill_unit(unit, k, Hkv, cap, row_bytes, K, V, base, pos, len, evict_idx, max_evict);
+  finish_lengths(B, len, n_evict, ticket);
 }
 
 // STABLE compaction: survivors keep their order. grid = (units, 3): y = 0 moves K, 1 moves V,
@@ -382,6 +477,42 @@ append_kernel(int Hkv, int cap, int m, int row_bytes, char* __restrict__ K, char
       }
     }
     if (threadIdx.x == 0) *ticket = 0;
+  }
+}
+
+// Append of a few rows (Hkv * m <= 16): one CTA per sequence, a warp for each K row and each V row. The CTA reads the
+// sequence's length once, so it can move it on itself after a barrier and no counter over the CTAs is needed.
+// block = 64 * Hkv * m threads.
+__global__ void __launch_bounds__(1024)
+append_seq_kernel(int Hkv, int cap, int m, int row_bytes, char* __restrict__ K, char* __restrict__ V,
+                  float* __restrict__ base, int* __restrict__ pos, int* __restrict__ len, int* __restrict__ n_seen,
+                  const char* __restrict__ k_new, const char* __restrict__ v_new, int* status) {
+  ptx::pdl_wait();
+  ptx::pdl_trigger();
+  const int b = blockIdx.x;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int n = len[b];
+  const int seen = n_seen ? n_seen[b] : n;
+  if (n < 0 || n + m > cap) {  // the sequence is skipped, its lengths stay
+    if (threadIdx.x == 0) set_status(status, CAOTE_ERR_OVERFLOW);
+    return;
+  }
+  const int r = warp >> 1, h = r / m, i = r % m;  // row r of the sequence: KV head h, new token i
+  const int unit = b * Hkv + h;
+  const size_t dst = (size_t)unit * cap + n + i, src = (size_t)unit * m + i;
+  if (warp & 1) {
+    warp_copy_row(V + dst * row_bytes, v_new + src * row_bytes, row_bytes, lane);
+  } else {
+    warp_copy_row(K + dst * row_bytes, k_new + src * row_bytes, row_bytes, lane);
+    if (lane == 0) {
+      if (base) base[dst] = 0.f;
+      if (pos) pos[dst] = seen + i;
+    }
+  }
+  __syncthreads();  // every warp has read the lengths
+  if (threadIdx.x == 0) {
+    len[b] = n + m;
+    if (n_seen) n_seen[b] = seen + m;
   }
 }
 
