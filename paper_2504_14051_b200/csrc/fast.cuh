@@ -45,8 +45,8 @@ __global__ void vsum_add_kernel(int Hkv, int cap, int m, int D, const T* __restr
 // The rows listed in evict_idx[unit, 0..k) leave the sum; called by all threads of the unit's CTA before
 // the rows are overwritten.
 template <typename T>
-__device__ inline void vsum_sub_unit(int unit, int k, int cap, int D, const T* __restrict__ V, const int* __restrict__ E,
-                                     float* __restrict__ vsum) {
+__device__ inline void vsum_sub_unit(int unit, int k, int cap, int D, const T* __restrict__ V, const int* E,
+                                     float* __restrict__ vsum) {  // (E: global or shared memory, possibly written by this CTA)
   for (int c = threadIdx.x; c < D; c += blockDim.x) {
     float acc = 0.f;
     for (int r = 0; r < k; ++r) acc += to_float(V[((size_t)unit * cap + E[r]) * D + c]);

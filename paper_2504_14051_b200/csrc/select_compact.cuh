@@ -12,6 +12,7 @@ namespace caote {
 namespace sel {
 
 constexpr int kSelThreads = 1024;
+constexpr int kMaxSharedPicks = 2048;
 
 // 64-bit sort key: score bits in the high word (scores are >= +0, so the unsigned order of the bit
 // patterns is the numeric order; +inf sorts last), original position in the low word.
@@ -21,12 +22,14 @@ __device__ __forceinline__ unsigned long long make_key(float score, int pos) {
 
 // One CTA per unit. k = max(0, n - budget). Finds the k-th smallest key by 8 passes of an 8-bit
 // radix histogram (most significant digit first), then writes the slots whose key is <= that key in
-// ascending slot order with a block-wide ordered compaction.
-// Returns k, the number of slots the unit evicts (the same value in every thread of the CTA).
+// ascending slot order with a block-wide ordered compaction. (Scores of one unit share their leading bytes, but grouping a
+// warp's lanes by digit before the shared-memory atomics, by match_any or by ballots, costs more than the atomics do.)
+// Returns k, the number of slots the unit evicts (the same value in every thread of the CTA). With e_smem (room for
+// kMaxSharedPicks slots) the chosen slots are also left there when k fits, for a compaction in the same kernel.
 __device__ __forceinline__ int select_unit(int unit, int Hkv, int cap, const float* __restrict__ scores,
                                            const int* __restrict__ len, const int* __restrict__ budget,
                                            const int* __restrict__ pos, int* __restrict__ evict_idx, int max_evict,
-                                           int* __restrict__ n_evict, int* status) {
+                                           int* __restrict__ n_evict, int* status, int* e_smem = nullptr) {
   __shared__ unsigned int hist[256];
   __shared__ unsigned long long s_prefix;
   __shared__ int s_remaining;
@@ -148,18 +151,51 @@ __device__ __forceinline__ int select_unit(int unit, int Hkv, int cap, const flo
       break;
     }
   }
+  int* picks = (e_smem && k <= kMaxSharedPicks) ? e_smem : nullptr;
+  if (cached) {
+    // one scan over the (round, warp) counts, which is the ascending order of the slots tid + round * kSelThreads
+    __shared__ int s_cnt[kCached * (kSelThreads / 32)];
+    unsigned int ballots[kCached];
+#pragma unroll
+    for (int i = 0; i < kCached; ++i) {
+      const int j = tid + i * kSelThreads;
+      ballots[i] = __ballot_sync(0xffffffffu, j < n && kreg[i] <= kth);
+      if (lane == 0) s_cnt[i * (kSelThreads / 32) + warp] = __popc(ballots[i]);
+    }
+    __syncthreads();
+    if (warp == 0) {
+      constexpr int kPerLane = kCached * (kSelThreads / 32) / 32;
+      int c[kPerLane], sum = 0;
+#pragma unroll
+      for (int q = 0; q < kPerLane; ++q) { c[q] = s_cnt[kPerLane * lane + q]; sum += c[q]; }
+      int incl = sum;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+      }
+      int run = incl - sum;
+#pragma unroll
+      for (int q = 0; q < kPerLane; ++q) { s_cnt[kPerLane * lane + q] = run; run += c[q]; }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < kCached; ++i) {
+      if (ballots[i] >> lane & 1u) {
+        const int idx = s_cnt[i * (kSelThreads / 32) + warp] + __popc(ballots[i] & ((1u << lane) - 1u));
+        if (idx < k) {
+          out[idx] = tid + i * kSelThreads;
+          if (picks) picks[idx] = tid + i * kSelThreads;
+        }
+      }
+    }
+    return k;
+  }
   if (tid == 0) s_running = 0;
   __syncthreads();
-  for (int j0 = 0, i = 0; j0 < n; j0 += kSelThreads, ++i) {
+  for (int j0 = 0; j0 < n; j0 += kSelThreads) {
     const int j = j0 + tid;
-    unsigned long long key = ~0ull;
-    if (cached) {
-#pragma unroll
-      for (int q = 0; q < kCached; ++q)
-        if (q == i) key = kreg[q];
-    } else if (j < n) {
-      key = make_key(sc[j], ps ? ps[j] : j);
-    }
+    const unsigned long long key = (j < n) ? make_key(sc[j], ps ? ps[j] : j) : ~0ull;
     const int flag = (j < n) && (key <= kth);
     const unsigned int ballot = __ballot_sync(0xffffffffu, flag);
     const int in_warp = __popc(ballot & ((1u << lane) - 1u));
@@ -168,7 +204,10 @@ __device__ __forceinline__ int select_unit(int unit, int Hkv, int cap, const flo
     int before = s_running;
     for (int w = 0; w < warp; ++w) before += s_warp_tot[w];
     const int idx = before + in_warp;
-    if (flag && idx < k) out[idx] = j;
+    if (flag && idx < k) {
+      out[idx] = j;
+      if (picks) picks[idx] = j;
+    }
     __syncthreads();
     if (tid == 0) {
       int tot = s_running;
@@ -208,26 +247,38 @@ __device__ __forceinline__ int lower_bound(const int* a, int n, int x) {
 // FILL compaction, one CTA per unit. With n' = n - k, the evicted slots below n' are holes, and the
 // k slots [n', n) hold exactly as many survivors; the i-th surviving tail slot moves into the i-th
 // hole. Sources lie in [n', n) and destinations in [0, n'), so no move can clobber another's source.
+// E = the unit's k evicted slots in ascending order (global or shared memory). Rows of up to 256 bytes are moved by
+// half a warp each, K and V together.
 __device__ __forceinline__ void compact_fill_unit(int unit, int k, int Hkv, int cap, int row_bytes, char* __restrict__ K,
                                                   char* __restrict__ V, float* __restrict__ base, int* __restrict__ pos,
-                                                  const int* __restrict__ len, const int* __restrict__ evict_idx,
-                                                  int max_evict) {
+                                                  const int* __restrict__ len, const int* E) {
   const int b = unit / Hkv;
   if (k <= 0) return;
   const int n = len[b], n_new = n - k;
-  const int* E = evict_idx + (size_t)unit * max_evict;
   const int nh = lower_bound(E, k, n_new);  // holes = E[0..nh)
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-  for (int t = warp; t < k; t += nwarps) {
+  const int glanes = (row_bytes <= 256) ? 16 : 32;  // lanes that share a row
+  const int gl = lane & (glanes - 1);
+  const int group = warp * (32 / glanes) + lane / glanes, ngroups = nwarps * (32 / glanes);
+  for (int t = group; t < k; t += ngroups) {
     const int s = n_new + t;
     const int lb = nh + lower_bound(E + nh, k - nh, s);
     if (lb < k && E[lb] == s) continue;  // this tail slot is itself evicted
     const int rank = t - (lb - nh);      // its rank among the surviving tail slots
     const int dst = E[rank];
     const size_t so = ((size_t)unit * cap + s), dof = ((size_t)unit * cap + dst);
-    warp_copy_row(K + dof * row_bytes, K + so * row_bytes, row_bytes, lane);
-    warp_copy_row(V + dof * row_bytes, V + so * row_bytes, row_bytes, lane);
-    if (lane == 0) {
+    if (row_bytes <= 512) {
+      if (gl * 16 < row_bytes) {
+        const uint4 kr = *reinterpret_cast<const uint4*>(K + so * row_bytes + gl * 16);
+        const uint4 vr = *reinterpret_cast<const uint4*>(V + so * row_bytes + gl * 16);
+        *reinterpret_cast<uint4*>(K + dof * row_bytes + gl * 16) = kr;
+        *reinterpret_cast<uint4*>(V + dof * row_bytes + gl * 16) = vr;
+      }
+    } else {
+      warp_copy_row(K + dof * row_bytes, K + so * row_bytes, row_bytes, lane);
+      warp_copy_row(V + dof * row_bytes, V + so * row_bytes, row_bytes, lane);
+    }
+    if (gl == 0) {
       if (base) base[dof] = base[so];
       if (pos) pos[dof] = pos[so];
     }
@@ -240,7 +291,8 @@ compact_fill_kernel(int Hkv, int cap, int row_bytes, char* __restrict__ K, char*
                     const int* __restrict__ evict_idx, int max_evict, const int* __restrict__ n_evict) {
   ptx::pdl_wait();
   ptx::pdl_trigger();
-  compact_fill_unit(blockIdx.x, n_evict[blockIdx.x / Hkv], Hkv, cap, row_bytes, K, V, base, pos, len, evict_idx, max_evict);
+  compact_fill_unit(blockIdx.x, n_evict[blockIdx.x / Hkv], Hkv, cap, row_bytes, K, V, base, pos, len,
+                    evict_idx + (size_t)blockIdx.x * max_evict);
 }
 
 // A unit that evicts exactly one token, with FILL compaction: the argmin over (score bits, position) and the move of
@@ -360,15 +412,17 @@ select_compact_kernel(int B, int Hkv, int cap, int row_bytes, const float* __res
     finish_lengths(B, len, n_evict, ticket);
     return;
   }
-  const int k = select_unit(unit, Hkv, cap, scores, len, budget, pos, evict_idx, max_evict, n_evict, status);
-  __syncthreads();  // evict_idx of this unit is written
+  __shared__ int s_picks[kMaxSharedPicks];
+  const int k = select_unit(unit, Hkv, cap, scores, len, budget, pos, evict_idx, max_evict, n_evict, status, s_picks);
+  __syncthreads();  // the unit's picks are written
+  // (read back from shared memory where they fit: the searches below are chains of dependent reads)
+  const int* E = (k <= kMaxSharedPicks && k > 1) ? s_picks : evict_idx + (size_t)unit * max_evict;
   if (vsum && k > 0) {  // FastCAOTE: the evicted rows leave the running sum of values before they are overwritten
-    const int* E = evict_idx + (size_t)unit * max_evict;
     if (elt_bytes == 2) fast::vsum_sub_unit<__nv_bfloat16>(unit, k, cap, row_bytes / 2, (const __nv_bfloat16*)V, E, vsum);
     else fast::vsum_sub_unit<float>(unit, k, cap, row_bytes / 4, (const float*)V, E, vsum);
     __syncthreads();
   }
-  compact_fill_unit(unit, k, Hkv, cap, row_bytes, K, V, base, pos, len, evict_idx, max_evict);
+  compact_fill_unit(unit, k, Hkv, cap, row_bytes, K, V, base, pos, len, E);
   finish_lengths(B, len, n_evict, ticket);
 }
 
