@@ -5,8 +5,10 @@
 // It runs after the cluster kernel, which has written the heads' outputs o_g and left per head the log-sum-exp m_g
 // (alpha_{g,j} = 2^(s_{g,j} - m_g)), the largest logit and the share of all other tokens next to the token that
 // holds it. This pass reads K and V once more: a CTA takes 128 tokens of a unit, their K and V rows land in shared
-// memory by TMA (two boxes of 64 channels each, 128-byte swizzle), two threads share a token, each with half of the
-// heads, and form their logits and distances by plain subtraction (no ||o||^2 - 2 o.v + ||v||^2: for a token that holds nearly all of a head's
+// memory by TMA (two boxes of 64 channels each, 128-byte swizzle), a thread takes four tokens and a quarter of the
+// heads (what bounds the pass on chip is the bytes that shared memory delivers to registers: the heads' q and o rows
+// are fetched once per four tokens, 4 KB per token in all where two threads per token with half of the heads each
+// took 9 KB), and forms logits and distances by plain subtraction (no ||o||^2 - 2 o.v + ||v||^2: for a token that holds nearly all of a head's
 // weight o_g is nearly v_j, and a bf16 cross term from the tensor cores would leave nothing of the difference).
 // 1 - alpha of a head's top token is the stored share of the others, never a difference of nearly equal numbers.
 #pragma once
@@ -18,12 +20,13 @@ namespace caote {
 namespace sed {
 
 constexpr int kT = 128;                      // tokens per CTA
-constexpr int kThreads = 2 * kT;             // two threads per token: the heads are split between them
+constexpr int kTok = 4;                      // tokens per thread: tq, tq + 32, tq + 64, tq + 96
+constexpr int kThreads = 4 * (kT / kTok);    // warp w takes the w-th quarter of the heads
 constexpr int kD = 128;
 constexpr int kTileBytes = kT * kD * 2;      // a K or V tile
 constexpr long long kWaitCycles = 2000000000LL;
 
-inline size_t smem_bytes() { return 1024 + 2 * (size_t)kTileBytes + sizeof(float) * (2 * 8 * kD + 24 + kT) + 64; }
+inline size_t smem_bytes() { return 1024 + 2 * (size_t)kTileBytes + sizeof(float) * (2 * 8 * kD + 24 + 3 * kT) + 64; }
 
 template <int G>
 __global__ void __launch_bounds__(kThreads)
@@ -39,8 +42,8 @@ sum_errors_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
   float* Qs = reinterpret_cast<float*>(Vs + kTileBytes);  // [8][kD]
   float* Os = Qs + 8 * kD;                                  // [8][kD]
   float* St = Os + 8 * kD;                                  // [3][8]
-  float* Cx = St + 24;                                      // [kT] the second thread's part of a token's score
-  uint64_t* bar = reinterpret_cast<uint64_t*>(Cx + kT);
+  float* Cx = St + 24;                                      // [3][kT] the other head quarters' parts of a token's score
+  uint64_t* bar = reinterpret_cast<uint64_t*>(Cx + 3 * kT);
 
   const int unit = blockIdx.y, b = unit / dm.Hkv, h = unit % dm.Hkv;
   const int n = len[b], j0 = blockIdx.x * kT;
@@ -73,57 +76,77 @@ sum_errors_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
       }
     }
   }
-  // thread tok takes heads [0, GH), thread tok + 128 heads [GH, G)
-  constexpr int GH = (G + 1) / 2;
-  const int tok = tid & (kT - 1), g0 = (tid >> 7) * GH;
-  const int j = j0 + tok;
-  float s[GH], d2[GH];
+  // lane tq of warp w: tokens tq + 32 t, heads [w GQ, (w + 1) GQ)
+  constexpr int GQ = (G + 3) / 4;
+  const int tq = tid & 31, g0 = (tid >> 5) * GQ;
+  float s[kTok][GQ], d2[kTok][GQ];
 #pragma unroll
-  for (int g = 0; g < GH; ++g) { s[g] = 0.f; d2[g] = 0.f; }
+  for (int t = 0; t < kTok; ++t)
+#pragma unroll
+    for (int g = 0; g < GQ; ++g) { s[t][g] = 0.f; d2[t][g] = 0.f; }
+  // (a head index beyond G reads rows of the tables that exist, 4 GQ <= 8, and is dropped below)
   const float* Qh = Qs + g0 * kD;
   const float* Oh = Os + g0 * kD;
-#pragma unroll 2
+#pragma unroll 1
   for (int c = 0; c < 16; ++c) {  // 16 chunks of 8 channels
-    const uint4 kr = *reinterpret_cast<const uint4*>(Ks + ptx::tile_off(tok, c));
-    const uint4 vr = *reinterpret_cast<const uint4*>(Vs + ptx::tile_off(tok, c));
-    const uint32_t kw[4] = {kr.x, kr.y, kr.z, kr.w}, vw[4] = {vr.x, vr.y, vr.z, vr.w};
-    float kf[8], vf[8];
+    float qq[GQ][8], oo[GQ][8];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      kf[2 * e] = __uint_as_float(kw[e] << 16);
-      kf[2 * e + 1] = __uint_as_float(kw[e] & 0xffff0000u);
-      vf[2 * e] = __uint_as_float(vw[e] << 16);
-      vf[2 * e + 1] = __uint_as_float(vw[e] & 0xffff0000u);
-    }
-#pragma unroll
-    for (int g = 0; g < GH; ++g) {  // (a head index beyond G reads rows of the tables that exist and is dropped below)
+    for (int g = 0; g < GQ; ++g) {
       const float4 q0 = *reinterpret_cast<const float4*>(Qh + g * kD + 8 * c), q1 = *reinterpret_cast<const float4*>(Qh + g * kD + 8 * c + 4);
       const float4 o0 = *reinterpret_cast<const float4*>(Oh + g * kD + 8 * c), o1 = *reinterpret_cast<const float4*>(Oh + g * kD + 8 * c + 4);
-      const float qq[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
-      const float oo[8] = {o0.x, o0.y, o0.z, o0.w, o1.x, o1.y, o1.z, o1.w};
+      qq[g][0] = q0.x; qq[g][1] = q0.y; qq[g][2] = q0.z; qq[g][3] = q0.w; qq[g][4] = q1.x; qq[g][5] = q1.y; qq[g][6] = q1.z; qq[g][7] = q1.w;
+      oo[g][0] = o0.x; oo[g][1] = o0.y; oo[g][2] = o0.z; oo[g][3] = o0.w; oo[g][4] = o1.x; oo[g][5] = o1.y; oo[g][6] = o1.z; oo[g][7] = o1.w;
+    }
 #pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        s[g] = fmaf(qq[e], kf[e], s[g]);
-        const float df = oo[e] - vf[e];
-        d2[g] = fmaf(df, df, d2[g]);
+    for (int t = 0; t < kTok; ++t) {
+      const int tok = tq + 32 * t;
+      const uint4 kr = *reinterpret_cast<const uint4*>(Ks + ptx::tile_off(tok, c));
+      const uint4 vr = *reinterpret_cast<const uint4*>(Vs + ptx::tile_off(tok, c));
+      const uint32_t kw[4] = {kr.x, kr.y, kr.z, kr.w}, vw[4] = {vr.x, vr.y, vr.z, vr.w};
+      float kf[8], vf[8];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        kf[2 * e] = __uint_as_float(kw[e] << 16);
+        kf[2 * e + 1] = __uint_as_float(kw[e] & 0xffff0000u);
+        vf[2 * e] = __uint_as_float(vw[e] << 16);
+        vf[2 * e + 1] = __uint_as_float(vw[e] & 0xffff0000u);
+      }
+#pragma unroll
+      for (int g = 0; g < GQ; ++g) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          s[t][g] = fmaf(qq[g][e], kf[e], s[t][g]);
+          const float df = oo[g][e] - vf[e];
+          d2[t][g] = fmaf(df, df, d2[t][g]);
+        }
       }
     }
   }
   const float scale2 = dm.scale * 1.4426950408889634f;
-  float cj = 0.f;
+  float cj[kTok];
 #pragma unroll
-  for (int g = 0; g < GH; ++g) {
-    if (g0 + g >= G) continue;
-    const float s2 = s[g] * scale2;
-    const float a = exp2f(s2 - St[g0 + g]);
-    // the head's top token (its logit, formed here in another order than in the attention pass, within 3e-4 of the
-    // largest): the others' share as stored; two tokens that close to the top have weights that close to each other
-    const float rest = (s2 >= St[8 + g0 + g] - 3e-4f) ? St[16 + g0 + g] : 1.f - a;
-    cj += (a == 0.f) ? 0.f : ((rest > 0.f) ? a / rest * sqrtf(d2[g]) : INFINITY);
+  for (int t = 0; t < kTok; ++t) {
+    cj[t] = 0.f;
+#pragma unroll
+    for (int g = 0; g < GQ; ++g) {
+      if (g0 + g >= G) continue;
+      const float s2 = s[t][g] * scale2;
+      const float a = exp2f(s2 - St[g0 + g]);
+      // the head's top token (its logit, formed here in another order than in the attention pass, within 3e-4 of the
+      // largest): the others' share as stored; two tokens that close to the top have weights that close to each other
+      const float rest = (s2 >= St[8 + g0 + g] - 3e-4f) ? St[16 + g0 + g] : 1.f - a;
+      cj[t] += (a == 0.f) ? 0.f : ((rest > 0.f) ? a / rest * sqrtf(d2[t][g]) : INFINITY);
+    }
+    if (tid >= 32) Cx[((tid >> 5) - 1) * kT + tq + 32 * t] = cj[t];
   }
-  if (tid >= kT) Cx[tok] = cj;
   __syncthreads();
-  if (tid < kT && j < n) scores[(size_t)unit * dm.cap + j] = cj + Cx[tok];
+  if (tid < 32) {
+#pragma unroll
+    for (int t = 0; t < kTok; ++t) {
+      const int tok = tq + 32 * t, j = j0 + tok;
+      if (j < n) scores[(size_t)unit * dm.cap + j] = cj[t] + Cx[tok] + Cx[kT + tok] + Cx[2 * kT + tok];
+    }
+  }
 }
 
 }  // namespace sed

@@ -77,6 +77,15 @@ def lockstep(w, steps, units=None, compact="fill", random_base=False):
             keep = np.setdiff1d(np.arange(n), ev[b, h, :k])
             got = np.sort(c.pos[b, h, :n - k].cpu().numpy())
             np.testing.assert_array_equal(got, np.sort(posn[b, h, keep]))
+            # ... and their K and V rows moved with them: slot i of the compacted cache holds the row of the slot that
+            # had its position before the step
+            by_pos = np.argsort(posn[b, h, :n])
+            src = by_pos[np.searchsorted(posn[b, h, :n][by_pos], c.pos[b, h, :n - k].cpu().numpy())]
+            src_t = torch.as_tensor(src, device=DEV)
+            assert torch.equal(c.K[b, h, :n - k], K[b, h][src_t]), what + " K rows after compaction"
+            assert torch.equal(c.V[b, h, :n - k], V[b, h][src_t]), what + " V rows after compaction"
+            if compact == "stable":
+                assert (np.diff(src) > 0).all(), what + " order of the survivors"
             if w.base_mode == "accum":
                 order = np.argsort(c.pos[b, h, :n - k].cpu().numpy())
                 ref_b = r["base"][i, 0, keep][np.argsort(posn[b, h, keep])]
