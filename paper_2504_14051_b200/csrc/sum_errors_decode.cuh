@@ -40,7 +40,7 @@ sum_errors_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
   char* Ks = sm;
   char* Vs = Ks + kTileBytes;
   float* Qs = reinterpret_cast<float*>(Vs + kTileBytes);  // [8][kD]
-  float* Os = Qs + 8 * kD;                                  // [8][kD]
+  float* Os = Qs + 8 * kD;                                  // [8][kD], the heads' outputs negated
   float* St = Os + 8 * kD;                                  // [3][8]
   float* Cx = St + 24;                                      // [3][kT] the other head quarters' parts of a token's score
   uint64_t* bar = reinterpret_cast<uint64_t*>(Cx + 3 * kT);
@@ -63,7 +63,7 @@ sum_errors_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
   const size_t qo = ((size_t)b * dm.Hq + (size_t)h * G) * kD;
   for (int i = tid; i < G * kD; i += kThreads) {
     Qs[i] = __bfloat162float(q[qo + i]);
-    Os[i] = o[qo + i];
+    Os[i] = -o[qo + i];  // (negated: the distance pass forms v - o with a packed add)
   }
   if (tid < 24) St[tid] = head_stats[(size_t)unit * kHeadStatFloats + tid];
   __syncthreads();
@@ -79,23 +79,24 @@ sum_errors_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
   // lane tq of warp w: tokens tq + 32 t, heads [w GQ, (w + 1) GQ)
   constexpr int GQ = (G + 3) / 4;
   const int tq = tid & 31, g0 = (tid >> 5) * GQ;
-  float s[kTok][GQ], d2[kTok][GQ];
+  // logits and squared distances as pairs of partial sums over the even and the odd channels (packed fp32 math)
+  float2 s[kTok][GQ], d2[kTok][GQ];
 #pragma unroll
   for (int t = 0; t < kTok; ++t)
 #pragma unroll
-    for (int g = 0; g < GQ; ++g) { s[t][g] = 0.f; d2[t][g] = 0.f; }
+    for (int g = 0; g < GQ; ++g) { s[t][g] = make_float2(0.f, 0.f); d2[t][g] = make_float2(0.f, 0.f); }
   // (a head index beyond G reads rows of the tables that exist, 4 GQ <= 8, and is dropped below)
   const float* Qh = Qs + g0 * kD;
   const float* Oh = Os + g0 * kD;
 #pragma unroll 1
   for (int c = 0; c < 16; ++c) {  // 16 chunks of 8 channels
-    float qq[GQ][8], oo[GQ][8];
+    float2 qq[GQ][4], no[GQ][4];
 #pragma unroll
     for (int g = 0; g < GQ; ++g) {
       const float4 q0 = *reinterpret_cast<const float4*>(Qh + g * kD + 8 * c), q1 = *reinterpret_cast<const float4*>(Qh + g * kD + 8 * c + 4);
       const float4 o0 = *reinterpret_cast<const float4*>(Oh + g * kD + 8 * c), o1 = *reinterpret_cast<const float4*>(Oh + g * kD + 8 * c + 4);
-      qq[g][0] = q0.x; qq[g][1] = q0.y; qq[g][2] = q0.z; qq[g][3] = q0.w; qq[g][4] = q1.x; qq[g][5] = q1.y; qq[g][6] = q1.z; qq[g][7] = q1.w;
-      oo[g][0] = o0.x; oo[g][1] = o0.y; oo[g][2] = o0.z; oo[g][3] = o0.w; oo[g][4] = o1.x; oo[g][5] = o1.y; oo[g][6] = o1.z; oo[g][7] = o1.w;
+      qq[g][0] = make_float2(q0.x, q0.y); qq[g][1] = make_float2(q0.z, q0.w); qq[g][2] = make_float2(q1.x, q1.y); qq[g][3] = make_float2(q1.z, q1.w);
+      no[g][0] = make_float2(o0.x, o0.y); no[g][1] = make_float2(o0.z, o0.w); no[g][2] = make_float2(o1.x, o1.y); no[g][3] = make_float2(o1.z, o1.w);
     }
 #pragma unroll
     for (int t = 0; t < kTok; ++t) {
@@ -103,21 +104,19 @@ sum_errors_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
       const uint4 kr = *reinterpret_cast<const uint4*>(Ks + ptx::tile_off(tok, c));
       const uint4 vr = *reinterpret_cast<const uint4*>(Vs + ptx::tile_off(tok, c));
       const uint32_t kw[4] = {kr.x, kr.y, kr.z, kr.w}, vw[4] = {vr.x, vr.y, vr.z, vr.w};
-      float kf[8], vf[8];
+      float2 kf[4], vf[4];
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        kf[2 * e] = __uint_as_float(kw[e] << 16);
-        kf[2 * e + 1] = __uint_as_float(kw[e] & 0xffff0000u);
-        vf[2 * e] = __uint_as_float(vw[e] << 16);
-        vf[2 * e + 1] = __uint_as_float(vw[e] & 0xffff0000u);
+        kf[e] = make_float2(__uint_as_float(kw[e] << 16), __uint_as_float(kw[e] & 0xffff0000u));
+        vf[e] = make_float2(__uint_as_float(vw[e] << 16), __uint_as_float(vw[e] & 0xffff0000u));
       }
 #pragma unroll
       for (int g = 0; g < GQ; ++g) {
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          s[t][g] = fmaf(qq[g][e], kf[e], s[t][g]);
-          const float df = oo[g][e] - vf[e];
-          d2[t][g] = fmaf(df, df, d2[t][g]);
+        for (int e = 0; e < 4; ++e) {
+          s[t][g] = __ffma2_rn(qq[g][e], kf[e], s[t][g]);
+          const float2 df = __fadd2_rn(vf[e], no[g][e]);
+          d2[t][g] = __ffma2_rn(df, df, d2[t][g]);
         }
       }
     }
@@ -130,12 +129,12 @@ sum_errors_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
 #pragma unroll
     for (int g = 0; g < GQ; ++g) {
       if (g0 + g >= G) continue;
-      const float s2 = s[t][g] * scale2;
+      const float s2 = (s[t][g].x + s[t][g].y) * scale2;
       const float a = exp2f(s2 - St[g0 + g]);
       // the head's top token (its logit, formed here in another order than in the attention pass, within 3e-4 of the
       // largest): the others' share as stored; two tokens that close to the top have weights that close to each other
       const float rest = (s2 >= St[8 + g0 + g] - 3e-4f) ? St[16 + g0 + g] : 1.f - a;
-      cj[t] += (a == 0.f) ? 0.f : ((rest > 0.f) ? a / rest * sqrtf(d2[t][g]) : INFINITY);
+      cj[t] += (a == 0.f) ? 0.f : ((rest > 0.f) ? a / rest * sqrtf(d2[t][g].x + d2[t][g].y) : INFINITY);
     }
     if (tid >= 32) Cx[((tid >> 5) - 1) * kT + tq + 32 * t] = cj[t];
   }
