@@ -602,7 +602,7 @@ attn_combine_kernel(Dims dm, const int* __restrict__ len, Scratch sc, float* __r
 // 0..15) the rows' statistics, and adds up its 16 columns in a fixed order for X. Units that ran unsplit are only
 // summed. grid = (units, kD / 16), 512 threads: a warp takes 8 rows at a time, 4 lanes per row.
 constexpr int kCxThreads = 512;
-__global__ void __launch_bounds__(kCxThreads)
+__global__ void __launch_bounds__(kCxThreads, 2)
 attn_combine_xsum_kernel(Dims dm, const int* __restrict__ len, Scratch sc, float* __restrict__ o) {
   ptx::pdl_wait();
   ptx::pdl_trigger();
@@ -615,30 +615,52 @@ attn_combine_xsum_kernel(Dims dm, const int* __restrict__ len, Scratch sc, float
   split_plan(n, dm.m, sc.nsplit, ts, nsp);
   const int ch = c0 + 4 * (lane & 3);
   float4 cs = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int R = warp * 8 + (lane >> 2); R < dm.R; R += (kCxThreads / 32) * 8) {
-    float* orow = o + ((size_t)unit * dm.R + R) * kD + ch;
-    float4 res;
-    if (nsp > 1) {
-      float st[8], mx = -INFINITY;
-      for (int s = 0; s < nsp; ++s) {
-        st[s] = sc.pstat[((size_t)unit * sc.nsplit + s) * sc.Mpad + R];
-        mx = fmaxf(mx, st[s]);
+  // A warp's time here is round trips to L2, not arithmetic: every load of a pass is issued before the first use.
+  constexpr int kStep = (kCxThreads / 32) * 8;
+  if (nsp > 1) {
+    // (splits beyond nsp count as weight zero, which leaves every sum as it is)
+    for (int R = warp * 8 + (lane >> 2); R < dm.R; R += kStep) {
+      float st[8];
+      float4 p[8];
+#pragma unroll
+      for (int s = 0; s < 8; ++s) {
+        st[s] = -INFINITY;
+        p[s] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (s < nsp) {
+          st[s] = sc.pstat[((size_t)unit * sc.nsplit + s) * sc.Mpad + R];
+          p[s] = *reinterpret_cast<const float4*>(sc.po + (((size_t)unit * sc.nsplit + s) * sc.Mpad + R) * kD + ch);
+        }
       }
+      float mx = -INFINITY;
+#pragma unroll
+      for (int s = 0; s < 8; ++s) mx = fmaxf(mx, st[s]);
       float tot = 0.f;
       float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-      for (int s = 0; s < nsp; ++s) {
-        const float w = exp2f(st[s] - mx);
+#pragma unroll
+      for (int s = 0; s < 8; ++s) {
+        const float w = (s < nsp) ? exp2f(st[s] - mx) : 0.f;
         tot += w;
-        const float4 p = *reinterpret_cast<const float4*>(sc.po + (((size_t)unit * sc.nsplit + s) * sc.Mpad + R) * kD + ch);
-        acc.x = fmaf(p.x, w, acc.x); acc.y = fmaf(p.y, w, acc.y); acc.z = fmaf(p.z, w, acc.z); acc.w = fmaf(p.w, w, acc.w);
+        acc.x = fmaf(p[s].x, w, acc.x); acc.y = fmaf(p[s].y, w, acc.y);
+        acc.z = fmaf(p[s].z, w, acc.z); acc.w = fmaf(p[s].w, w, acc.w);
       }
-      res = make_float4(acc.x / tot, acc.y / tot, acc.z / tot, acc.w / tot);
-      *reinterpret_cast<float4*>(orow) = res;
+      const float4 res = make_float4(acc.x / tot, acc.y / tot, acc.z / tot, acc.w / tot);
+      *reinterpret_cast<float4*>(o + ((size_t)unit * dm.R + R) * kD + ch) = res;
       if (ch == 0) sc.stats[(size_t)unit * sc.Mpad + R] = mx + log2f(tot);
-    } else {
-      res = *reinterpret_cast<const float4*>(orow);
+      cs.x += res.x; cs.y += res.y; cs.z += res.z; cs.w += res.w;
     }
-    cs.x += res.x; cs.y += res.y; cs.z += res.z; cs.w += res.w;
+  } else {
+    for (int R0 = warp * 8 + (lane >> 2); R0 < dm.R; R0 += 4 * kStep) {  // four rows in flight, summed in row order
+      float4 r[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int R = R0 + u * kStep;
+        r[u] = (R < dm.R) ? *reinterpret_cast<const float4*>(o + ((size_t)unit * dm.R + R) * kD + ch)
+                          : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (R0 + u * kStep < dm.R) { cs.x += r[u].x; cs.y += r[u].y; cs.z += r[u].z; cs.w += r[u].w; }
+    }
   }
   // the warp's eight row lanes of every channel quad, then the warps in order
 #pragma unroll
