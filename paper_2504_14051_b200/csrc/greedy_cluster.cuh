@@ -3,9 +3,11 @@
 // unit's value rows in its shared memory (bf16, head_dim 128). Each pick sweeps those rows from shared memory instead
 // of from L2 (the one-CTA kernel in greedy.cuh re-reads all of them from L2 for every pick):
 //   every CTA: distances of its rows to the current output X = Y / H, its best (score bits, position) candidate;
-//   one cluster barrier; every CTA reads all candidates through distributed shared memory and takes the same
-//   minimum; every CTA reads the evicted row from its owner's shared memory and updates its own copy of Y and H
-//   (the same arithmetic everywhere, so the copies never differ).
+//   every CTA stores its candidate and the candidate's value row into every CTA's shared memory (distributed shared
+//   memory stores: nobody waits for them); one cluster barrier; every CTA takes the same minimum of the candidates it
+//   now holds and updates its own copy of Y and H with the winner's row (the same arithmetic everywhere, so the
+//   copies never differ). Reading the candidates and then the row from their owners after the barrier cost two more
+//   round trips through distributed shared memory per pick.
 // The candidates are double-buffered by the parity of the pick, which is what makes one barrier per pick enough.
 // A CTA holds up to kMaxRows rows in shared memory; a unit too long for 16 CTAs' worth leaves the rest of every CTA's
 // share in global memory, and the CTA sweeps that part from L2 (several rows in flight per warp): still 16 SMs
@@ -33,7 +35,7 @@ struct Cand {  // a CTA's best candidate of a pick
 
 inline size_t smem_bytes(int rows_smem, int rows) {
   return (size_t)rows_smem * kD * 2 + sizeof(float) * (2 * (size_t)rows + kD + (kD + 4) + 2 * kWarps) +
-         sizeof(unsigned long long) * kWarps + sizeof(int) * (2 * kWarps + 8) + 2 * sizeof(Cand) + 64;
+         sizeof(unsigned long long) * kWarps + sizeof(int) * (2 * kWarps + 8) + 64;
 }
 
 __device__ __forceinline__ uint32_t gc_rank() { return ptx::cluster_ctarank(); }
@@ -44,8 +46,6 @@ __device__ __forceinline__ void gc_sync() { ptx::cluster_sync_all(); }
 __device__ __forceinline__ uint32_t gc_map(const void* p, uint32_t rank) { return ptx::map_to_rank(ptx::smem_u32(p), rank); }
 __device__ __forceinline__ float gc_ld_f32(uint32_t a) { return ptx::ld_dsmem_f32(a); }
 __device__ __forceinline__ int gc_ld_s32(uint32_t a) { return ptx::ld_dsmem_s32(a); }
-__device__ __forceinline__ unsigned long long gc_ld_u64(uint32_t a) { return ptx::ld_dsmem_u64(a); }
-__device__ __forceinline__ unsigned short gc_ld_u16(uint32_t a) { return ptx::ld_dsmem_u16(a); }
 
 // grid = units x C CTAs in clusters of C; rows_per = rows of the unit per CTA (the same for every CTA of the grid),
 // the first rows_smem of them in shared memory.
@@ -64,9 +64,10 @@ greedy_cluster_kernel(int Hkv, int cap, int rows_per, int rows_smem, const __nv_
   unsigned long long* wkey = reinterpret_cast<unsigned long long*>(wsum + 2 * kWarps);  // [kWarps]
   int* wslot = reinterpret_cast<int*>(wkey + kWarps);                   // [2 * kWarps]
   int* misc = wslot + 2 * kWarps;                                       // [8]: 0 count of evicted rows here, 1 running count
-  Cand* cand = reinterpret_cast<Cand*>(misc + 8);                       // [2]
   __shared__ float s_H, s_he;
   __shared__ int s_e;
+  __shared__ __align__(16) Cand pcand[2][kMaxC];                 // [parity of the pick][rank]: every CTA's candidate
+  __shared__ __align__(16) __nv_bfloat16 prow[2][kMaxC][kD];     // ... and its value row
 
   const int C = (int)gc_size(), rank = (int)gc_rank();
   const int unit = (int)gc_cluster_id(), b = unit / Hkv, hd = unit % Hkv;
@@ -193,28 +194,42 @@ greedy_cluster_kernel(int Hkv, int cap, int rows_per, int rows_smem, const __nv_
     }
     if (lane == 0) { wkey[warp] = best; wslot[warp] = best_slot; }
     __syncthreads();
-    if (tid == 0) {
-      unsigned long long bk = wkey[0];
-      int bs = wslot[0];
-      for (int w = 1; w < kWarps; ++w)
-        if (wslot[w] >= 0 && (bs < 0 || wkey[w] < bk || (wkey[w] == bk && wslot[w] < bs))) { bk = wkey[w]; bs = wslot[w]; }
-      Cand cd;
-      cd.key = bk;
-      cd.slot = bs >= 0 ? r0 + bs : -1;
-      cd.h = bs >= 0 ? hs[bs] : 0.f;
-      cand[t & 1] = cd;
+    // every warp reduces the warps' results for itself: this CTA's candidate (local slot bs, -1: none)
+    unsigned long long bk = lane < kWarps ? wkey[lane] : ~0ull;
+    int bs = lane < kWarps ? wslot[lane] : -1;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const unsigned long long ok = __shfl_xor_sync(0xffffffffu, bk, o);
+      const int os = __shfl_xor_sync(0xffffffffu, bs, o);
+      if (os >= 0 && (bs < 0 || ok < bk || (ok == bk && os < bs))) { bk = ok; bs = os; }
     }
-    gc_sync();  // every CTA's candidate of this pick is written (and everybody is done with the pick before)
+    // ---- the candidate and its value row go to every CTA of the cluster (this one included) ----
+    const int par = t & 1;
+    if (tid < 16 * C) {  // 16 bytes of the row per thread, 16 threads per peer
+      const int peer = tid >> 4, chunk = tid & 15;
+      if (bs >= 0) {
+        const uint4 v = *reinterpret_cast<const uint4*>((bs < ns ? Vs : Vu) + (size_t)bs * kD + 8 * chunk);
+        ptx::st_dsmem_v4(gc_map(&prow[par][rank][8 * chunk], (uint32_t)peer), v);
+      }
+    } else if (tid >= 256 && tid < 256 + C) {
+      uint4 cd;
+      cd.x = (uint32_t)bk;
+      cd.y = (uint32_t)(bk >> 32);
+      cd.z = (uint32_t)(bs >= 0 ? r0 + bs : -1);
+      cd.w = __float_as_uint(bs >= 0 ? hs[bs] : 0.f);
+      ptx::st_dsmem_v4(gc_map(&pcand[par][rank], (uint32_t)(tid - 256)), cd);
+    }
+    gc_sync();  // every CTA's candidate of this pick has arrived (and everybody is done with the pick before)
     // ---- the unit's pick: the smallest candidate, lower slot on equal keys; the same in every CTA ----
     if (warp == 0) {
       unsigned long long ck = ~0ull;
       int cs = -1;
       float ch = 0.f;
       if (lane < C) {
-        const Cand* rc = cand + (t & 1);
-        cs = gc_ld_s32(gc_map(&rc->slot, (uint32_t)lane));
-        ck = gc_ld_u64(gc_map(&rc->key, (uint32_t)lane));
-        ch = gc_ld_f32(gc_map(&rc->h, (uint32_t)lane));
+        const Cand rc = pcand[par][lane];
+        cs = rc.slot;
+        ck = rc.key;
+        ch = rc.h;
       }
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) {
@@ -228,14 +243,10 @@ greedy_cluster_kernel(int Hkv, int cap, int rows_per, int rows_smem, const __nv_
     __syncthreads();
     const int e = s_e;
     if (e < 0) break;  // (cannot happen with k < n; the same in every CTA, so no barrier is left unmatched)
-    // ---- evict e: Y -= h_e v_e, H -= h_e (the row comes from its owner's shared memory) ----
+    // ---- evict e: Y -= h_e v_e, H -= h_e (the row came with its owner's candidate) ----
     const float he = s_he;
     const int owner = e / rows_per, el = e - owner * rows_per;
-    if (tid < kD) {  // (from its owner's shared memory, or from global memory if the owner left it there)
-      const unsigned short raw = el < rows_smem ? gc_ld_u16(gc_map(Vs + (size_t)el * kD + tid, (uint32_t)owner))
-                                                : __bfloat16_as_ushort(V[((size_t)unit * cap + e) * kD + tid]);
-      Ys[tid] -= he * __uint_as_float((uint32_t)raw << 16);
-    }
+    if (tid < kD) Ys[tid] -= he * __bfloat162float(prow[par][owner][tid]);
     if (tid == 0) {
       s_H = H - he;
       if (ord && rank == 0) ord[t] = e;

@@ -145,6 +145,11 @@ __device__ __forceinline__ unsigned short ld_dsmem_u16(uint32_t a) {
   asm volatile("ld.shared::cluster.u16 %0, [%1];" : "=h"(v) : "r"(a) : "memory");
   return v;
 }
+// Store of 16 bytes into the shared memory of another CTA of the cluster (address from map_to_rank, 16-byte
+// aligned); visible to that CTA after the next cluster barrier (arrive.release / wait.acquire).
+__device__ __forceinline__ void st_dsmem_v4(uint32_t a, uint4 v) {
+  asm volatile("st.shared::cluster.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
 
 }  // namespace ptx
 }  // namespace caote
