@@ -825,11 +825,13 @@ static int launch_greedy_cluster(const Dims& dm, const void* V, const float* h, 
   }
   if (best_c == 0) return CAOTE_OK;
   {
-    // Worth it? Per pick the one-CTA kernel sweeps the unit's rows from L2 (measured: 9.5 ns per row), this one its
-    // share of them from shared memory plus a cluster barrier (measured: about 6 us + 7 ns per row); but the GPU runs
-    // fewer clusters at once than single CTAs, and with a handful of picks loading the rows is all there is.
+    // Worth it? Per pick the one-CTA kernel sweeps the unit's rows from L2 (measured: 19 us at 4224 rows, taken as
+    // 3 us + 3.8 ns per row), this one its share of them from shared memory plus a cluster barrier (measured: 5.25 us at
+    // 528 rows per CTA, 8.35 us at 768 + 288 left in global memory: about 4.2 us + 2 ns per row + 9 ns per row from
+    // L2); but the GPU runs fewer clusters at once than single CTAs, and with a handful of picks loading the rows is
+    // all there is.
     const int in_smem = best_rows < greedy_cl::kMaxRows ? best_rows : greedy_cl::kMaxRows;
-    const double t_one = 0.0095 * dm.cap, t_cluster = 6.0 + 0.007 * in_smem + 0.012 * (best_rows - in_smem);
+    const double t_one = 3.0 + 0.0038 * dm.cap, t_cluster = 4.2 + 0.002 * in_smem + 0.009 * (best_rows - in_smem);
     const double waves_one = (double)((dm.units + g_sm_count - 1) / g_sm_count);
     const double waves_cluster = (double)((dm.units + best_got - 1) / best_got);
     if (max_evict < 4 || t_one * waves_one < 1.2 * t_cluster * waves_cluster) return CAOTE_OK;

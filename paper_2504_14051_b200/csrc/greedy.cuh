@@ -122,32 +122,58 @@ greedy_kernel(int Hkv, int cap, const T* __restrict__ V, const float* __restrict
   for (int t = 0; t < k; ++t) {
     const float H = s_H;
     const float inv_H = (H > 0.f) ? 1.f / H : 0.f;
-    float x[CPL];
+    // ---- distances of the tokens present to the current output: four rows per warp at a time, eight lanes per
+    //      row, each with the 16-byte pieces l, l + 8, ... of the row (a row's loads are contiguous over its lanes) and
+    //      three shuffle steps per sum; four such passes' loads in flight (a warp per row with a five-step sum kept
+    //      the SM's one shuffle per clock busy for most of the sweep) ----
+    {
+      constexpr int E = 16 / (int)sizeof(T);  // elements per 16-byte piece
+      constexpr int NCH = D / 8 / E;          // pieces per lane
+      constexpr int kPasses = 4;
+      const int sub = lane >> 3, l8 = lane & 7;
+      float x[NCH][E];
 #pragma unroll
-    for (int c = 0; c < CPL; ++c) x[c] = Ys[lane * CPL + c] * inv_H;
-    // ---- distances of the tokens present to the current output: a warp takes eight rows at a time, so that eight
-    //      loads are in flight (one row after the other, the sweep ran at the latency of a load from L2 per row) ----
-    constexpr int kInFlight = 8;
-    for (int j0 = warp; j0 < n; j0 += kInFlight * kWarps) {
-      float vf[kInFlight][CPL];
-      bool live[kInFlight];
+      for (int i = 0; i < NCH; ++i)
 #pragma unroll
-      for (int u = 0; u < kInFlight; ++u) {
-        const int j = j0 + u * kWarps;
-        live[u] = j < n && hs[j] >= 0.f;  // (warp-uniform)
-        if (live[u]) load_channels<CPL>(Vu + (size_t)j * D + lane * CPL, vf[u]);
-      }
+        for (int e = 0; e < E; ++e) x[i][e] = Ys[(l8 + 8 * i) * E + e] * inv_H;
+      for (int j0 = 4 * warp; j0 < n; j0 += 4 * kWarps * kPasses) {
+        uint4 raw[kPasses][NCH];
+        bool live[kPasses];
 #pragma unroll
-      for (int u = 0; u < kInFlight; ++u) {
-        if (!live[u]) continue;
-        float acc = 0.f;
+        for (int u = 0; u < kPasses; ++u) {
+          const int j = j0 + u * 4 * kWarps + sub;
+          live[u] = j < n && hs[j] >= 0.f;
+          if (live[u]) {
+            const uint4* row = reinterpret_cast<const uint4*>(Vu + (size_t)j * D);
 #pragma unroll
-        for (int c = 0; c < CPL; ++c) {
-          const float dlt = x[c] - vf[u][c];
-          acc = fmaf(dlt, dlt, acc);
+            for (int i = 0; i < NCH; ++i) raw[u][i] = row[l8 + 8 * i];
+          }
         }
-        acc = warp_sum(acc);
-        if (lane == 0) ds[j0 + u * kWarps] = sqrtf(acc);
+#pragma unroll
+        for (int u = 0; u < kPasses; ++u) {
+          float acc = 0.f;
+          if (live[u]) {
+#pragma unroll
+            for (int i = 0; i < NCH; ++i) {
+              const uint32_t w[4] = {raw[u][i].x, raw[u][i].y, raw[u][i].z, raw[u][i].w};
+#pragma unroll
+              for (int c = 0; c < 4; ++c) {
+                if constexpr (sizeof(T) == 2) {
+                  const float d0 = x[i][2 * c] - __uint_as_float(w[c] << 16);
+                  const float d1 = x[i][2 * c + 1] - __uint_as_float(w[c] & 0xffff0000u);
+                  acc = fmaf(d0, d0, fmaf(d1, d1, acc));
+                } else {
+                  const float d0 = x[i][c] - __uint_as_float(w[c]);
+                  acc = fmaf(d0, d0, acc);
+                }
+              }
+            }
+          }
+          acc += __shfl_xor_sync(0xffffffffu, acc, 4);
+          acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+          acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+          if (live[u] && l8 == 0) ds[j0 + u * 4 * kWarps + sub] = sqrtf(acc);
+        }
       }
     }
     __syncthreads();

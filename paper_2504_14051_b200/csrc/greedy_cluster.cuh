@@ -139,35 +139,84 @@ greedy_cluster_kernel(int Hkv, int cap, int rows_per, int rows_smem, const __nv_
   for (int t = 0; t < k; ++t) {
     const float H = s_H;
     const float inv_H = (H > 0.f) ? 1.f / H : 0.f;
-    float x[4];
+    // ---- distances of this CTA's tokens still present to the current output: four tokens per warp at a time, eight
+    //      lanes per token (channels [8 l, 8 l + 8) and [64 + 8 l, 64 + 8 l + 8): both 16-byte loads of a token are
+    //      contiguous over its lanes), three shuffle steps per sum; a warp per token with five steps spent most of the
+    //      sweep waiting for its own shuffles ----
+    {
+      const int sub = lane >> 3, l8 = lane & 7;
+      float xa[8], xb[8];
 #pragma unroll
-    for (int c = 0; c < 4; ++c) x[c] = Ys[4 * lane + c] * inv_H;
-    // ---- distances of this CTA's tokens still present to the current output (a warp per token) ----
-    for (int j = warp; j < ns; j += kWarps) {
-      if (hs[j] < 0.f) continue;  // (warp-uniform)
-      const uint2 raw = *reinterpret_cast<const uint2*>(Vs + (size_t)j * kD + 4 * lane);
-      const float d0 = x[0] - __uint_as_float(raw.x << 16), d1 = x[1] - __uint_as_float(raw.x & 0xffff0000u);
-      const float d2 = x[2] - __uint_as_float(raw.y << 16), d3 = x[3] - __uint_as_float(raw.y & 0xffff0000u);
-      const float acc = warp_sum(fmaf(d0, d0, fmaf(d1, d1, fmaf(d2, d2, d3 * d3))));
-      if (lane == 0) ds[j] = sqrtf(acc);
-    }
-    // ... and of the rows it left in global memory: eight loads in flight per warp
-    for (int j0 = ns + warp; j0 < nr; j0 += 8 * kWarps) {
-      uint2 raw[8];
-      bool live[8];
-#pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const int j = j0 + u * kWarps;
-        live[u] = j < nr && hs[j] >= 0.f;  // (warp-uniform)
-        if (live[u]) raw[u] = *reinterpret_cast<const uint2*>(Vu + (size_t)j * kD + 4 * lane);
+      for (int c = 0; c < 8; ++c) {
+        xa[c] = Ys[8 * l8 + c] * inv_H;
+        xb[c] = Ys[64 + 8 * l8 + c] * inv_H;
       }
+      for (int j0 = 4 * warp; j0 < ns; j0 += 4 * kWarps) {
+        const int j = j0 + sub;
+        const bool live = j < ns && hs[j] >= 0.f;
+        float acc = 0.f;
+        if (live) {
+          const uint4 ra = *reinterpret_cast<const uint4*>(Vs + (size_t)j * kD + 8 * l8);
+          const uint4 rb = *reinterpret_cast<const uint4*>(Vs + (size_t)j * kD + 64 + 8 * l8);
+          const uint32_t wa[4] = {ra.x, ra.y, ra.z, ra.w}, wb[4] = {rb.x, rb.y, rb.z, rb.w};
+          float acc2 = 0.f;
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        if (!live[u]) continue;
-        const float d0 = x[0] - __uint_as_float(raw[u].x << 16), d1 = x[1] - __uint_as_float(raw[u].x & 0xffff0000u);
-        const float d2 = x[2] - __uint_as_float(raw[u].y << 16), d3 = x[3] - __uint_as_float(raw[u].y & 0xffff0000u);
-        const float acc = warp_sum(fmaf(d0, d0, fmaf(d1, d1, fmaf(d2, d2, d3 * d3))));
-        if (lane == 0) ds[j0 + u * kWarps] = sqrtf(acc);
+          for (int c = 0; c < 4; ++c) {
+            const float a0 = xa[2 * c] - __uint_as_float(wa[c] << 16), a1 = xa[2 * c + 1] - __uint_as_float(wa[c] & 0xffff0000u);
+            const float b0 = xb[2 * c] - __uint_as_float(wb[c] << 16), b1 = xb[2 * c + 1] - __uint_as_float(wb[c] & 0xffff0000u);
+            acc = fmaf(a0, a0, fmaf(a1, a1, acc));
+            acc2 = fmaf(b0, b0, fmaf(b1, b1, acc2));
+          }
+          acc += acc2;
+        }
+        acc += __shfl_xor_sync(0xffffffffu, acc, 4);
+        acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+        acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+        if (live && l8 == 0) ds[j] = sqrtf(acc);
+      }
+    }
+    // ... and of the rows it left in global memory, the same way with four passes' loads in flight per warp
+    {
+      constexpr int kPasses = 4;
+      const int sub = lane >> 3, l8 = lane & 7;
+      float xa[8], xb[8];
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        xa[c] = Ys[8 * l8 + c] * inv_H;
+        xb[c] = Ys[64 + 8 * l8 + c] * inv_H;
+      }
+      for (int j0 = ns + 4 * warp; j0 < nr; j0 += 4 * kWarps * kPasses) {
+        uint4 ra[kPasses], rb[kPasses];
+        bool live[kPasses];
+#pragma unroll
+        for (int u = 0; u < kPasses; ++u) {
+          const int j = j0 + u * 4 * kWarps + sub;
+          live[u] = j < nr && hs[j] >= 0.f;
+          if (live[u]) {
+            ra[u] = *reinterpret_cast<const uint4*>(Vu + (size_t)j * kD + 8 * l8);
+            rb[u] = *reinterpret_cast<const uint4*>(Vu + (size_t)j * kD + 64 + 8 * l8);
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < kPasses; ++u) {
+          float acc = 0.f;
+          if (live[u]) {
+            const uint32_t wa[4] = {ra[u].x, ra[u].y, ra[u].z, ra[u].w}, wb[4] = {rb[u].x, rb[u].y, rb[u].z, rb[u].w};
+            float acc2 = 0.f;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              const float a0 = xa[2 * c] - __uint_as_float(wa[c] << 16), a1 = xa[2 * c + 1] - __uint_as_float(wa[c] & 0xffff0000u);
+              const float b0 = xb[2 * c] - __uint_as_float(wb[c] << 16), b1 = xb[2 * c + 1] - __uint_as_float(wb[c] & 0xffff0000u);
+              acc = fmaf(a0, a0, fmaf(a1, a1, acc));
+              acc2 = fmaf(b0, b0, fmaf(b1, b1, acc2));
+            }
+            acc += acc2;
+          }
+          acc += __shfl_xor_sync(0xffffffffu, acc, 4);
+          acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+          acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+          if (live[u] && l8 == 0) ds[j0 + u * 4 * kWarps + sub] = sqrtf(acc);
+        }
       }
     }
     __syncthreads();
