@@ -36,7 +36,9 @@ sum_errors_decode_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_c
   ptx::pdl_wait();
   ptx::pdl_trigger();
   extern __shared__ char smem_raw[];
-  char* sm = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  // (1024-byte alignment by an offset into the array, not by a round trip through an integer: the pointer keeps its
+  // address space, so what is read through it compiles to shared-memory loads, not generic ones)
+  char* sm = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
   char* Ks = sm;
   char* Vs = Ks + kTileBytes;
   float* Qs = reinterpret_cast<float*>(Vs + kTileBytes);  // [8][kD]
