@@ -247,7 +247,9 @@ decode_cluster_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
   ptx::pdl_wait();
   ptx::pdl_trigger();
   extern __shared__ char smem_raw[];
-  char* sm = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  // (aligned by an offset into the array, not through an integer: the pointer keeps its address space, and what is
+  // read and written through it compiles to shared-memory accesses, not generic ones)
+  char* sm = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
   char* tilesK = sm;                                                   // [kKS][kTileBytes]
   char* tilesV = tilesK + kKS * kTileBytes;                            // [kVS][kTileBytes]
   char* qbuf = tilesV + kVS * kTileBytes;                              // [2][kQBufBytes]

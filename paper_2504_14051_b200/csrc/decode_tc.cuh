@@ -176,7 +176,9 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   constexpr int kQ = kFast ? kQBufsFast : kQBufs;  // a buffer is reused only after every reader of its item has moved on:
                                                    // that takes one more buffer with the deeper ring
   extern __shared__ char smem_raw[];
-  char* sm = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  // (aligned by an offset into the array, not through an integer: the pointer keeps its address space, and what is
+  // read and written through it compiles to shared-memory accesses, not generic ones)
+  char* sm = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
   char* tilesA = sm;                                                     // [kA][kTileBytes]
   char* tilesB = tilesA + kA * kTileBytes;                               // [kBSlots][kTileBytes] (none with kFast)
   char* qbuf = tilesB + (kFast ? 0 : kBSlots * kTileBytes);                            // [kQ][kQBytes]

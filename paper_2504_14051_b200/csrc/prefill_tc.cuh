@@ -320,7 +320,9 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
   ptx::pdl_wait();
   ptx::pdl_trigger();
   extern __shared__ char smem_raw[];
-  char* sm = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  // (aligned by an offset into the array, not through an integer: the pointer keeps its address space, and what is
+  // read and written through it compiles to shared-memory accesses, not generic ones)
+  char* sm = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
   char* Qs = sm;
   char* Ksm = Qs + kTileBytes;                 // [kKStages]
   char* Vsm = Ksm + kKStages * kKvTile;        // [kVStages]
@@ -764,7 +766,9 @@ score_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
   ptx::pdl_wait();
   ptx::pdl_trigger();
   extern __shared__ char smem_raw[];
-  char* sm = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  // (aligned by an offset into the array, not through an integer: the pointer keeps its address space, and what is
+  // read and written through it compiles to shared-memory accesses, not generic ones)
+  char* sm = smem_raw + ((1024u - (ptx::smem_u32(smem_raw) & 1023u)) & 1023u);
   char* Ks = sm;                                                     // [2] key tiles
   char* Qst = Ks + 2 * kTileBytes;                                   // [kQStages] Q blocks
   float* Sst = reinterpret_cast<float*>(Qst + kQStages * kTileBytes);  // [kSStages][kTile] row statistics
