@@ -894,9 +894,15 @@ size_t caote_workspace_bytes(const caote_params_t* params) {
   return workspace_bytes(params);
 }
 
-int caote_append(const caote_params_t* p, void* K, void* V, float* base, int32_t* pos, int32_t* len,
-                 int32_t* n_seen, const void* k_new, const void* v_new, void* workspace,
-                 size_t workspace_bytes_, caote_stream_t stream) {
+// Whether the append of this shape runs a CTA per sequence, and can then also add the one new value row of every unit
+// to FastCAOTE's running sum (m = 1).
+static bool append_per_sequence(const Dims& dm) { return dm.Hkv * dm.m <= 16; }
+
+// caote_append, and the append inside caote_step_fast (vsum: the units' running sums, folded in where
+// append_per_sequence(dm) and m = 1).
+static int append_impl(const caote_params_t* p, void* K, void* V, float* base, int32_t* pos, int32_t* len,
+                       int32_t* n_seen, const void* k_new, const void* v_new, void* workspace,
+                       size_t workspace_bytes_, caote_stream_t stream, float* vsum) {
   int rc = append_args_check(p, K, V, len, k_new, v_new, workspace, workspace_bytes_);
   if (rc) return rc;
   rc = check_device();
@@ -904,17 +910,24 @@ int caote_append(const caote_params_t* p, void* K, void* V, float* base, int32_t
   const Dims dm = make_dims(p);
   const int row_bytes = dm.D * (p->dtype == CAOTE_BF16 ? 2 : 4);
   cudaStream_t st = (cudaStream_t)stream;
-  if (dm.Hkv * dm.m <= 16) {  // (single-query decode: a CTA per sequence, which moves its lengths on itself)
+  if (append_per_sequence(dm)) {  // (single-query decode: a CTA per sequence, which moves its lengths on itself)
     CAOTE_LAUNCH("append_seq_kernel", st,
                  launch_pdl(sel::append_seq_kernel, dim3(dm.B), dim3(64 * dm.Hkv * dm.m), 0, st, dm.Hkv, dm.cap, dm.m,
                             row_bytes, (char*)K, (char*)V, base, pos, len, n_seen, (const char*)k_new,
-                            (const char*)v_new, (int*)workspace));
+                            (const char*)v_new, (int*)workspace, dm.m == 1 ? vsum : nullptr,
+                            p->dtype == CAOTE_BF16 ? 2 : 4));
     return CAOTE_OK;
   }
   CAOTE_LAUNCH("append_kernel", st, launch_pdl(sel::append_kernel, dim3(dim3(dm.units, (dm.m + 7) / 8)), dim3(256), 0, st, dm.Hkv, dm.cap, dm.m, row_bytes, (char*)K, (char*)V, base, pos,
                                                len, n_seen, (const char*)k_new, (const char*)v_new,
                                                (int*)workspace, dm.B, (int*)workspace + 4));
   return CAOTE_OK;
+}
+
+int caote_append(const caote_params_t* p, void* K, void* V, float* base, int32_t* pos, int32_t* len,
+                 int32_t* n_seen, const void* k_new, const void* v_new, void* workspace,
+                 size_t workspace_bytes_, caote_stream_t stream) {
+  return append_impl(p, K, V, base, pos, len, n_seen, k_new, v_new, workspace, workspace_bytes_, stream, nullptr);
 }
 
 // caote_score (vsum == NULL) and caote_score_fast (vsum: the per-unit sums of the cached value rows).
@@ -1148,7 +1161,9 @@ static int step_impl(const caote_params_t* p, const void* q, const void* k_new, 
   if (rc) return rc;
   const bool bf16 = p->dtype == CAOTE_BF16;
   if (k_new || v_new) {
-    if (vsum) {
+    const Dims dma = make_dims(p);
+    const bool fold = vsum && dma.m == 1 && append_per_sequence(dma);  // the append adds the new value rows itself
+    if (vsum && !fold) {
       const Dims dm = make_dims(p);
       cudaStream_t st = (cudaStream_t)stream;
       if (bf16) {
@@ -1159,7 +1174,8 @@ static int step_impl(const caote_params_t* p, const void* q, const void* k_new, 
             dm.Hkv, dm.cap, dm.m, dm.D, (const float*)v_new, len, vsum));
       }
     }
-    rc = caote_append(p, K, V, base, pos, len, n_seen, k_new, v_new, workspace, workspace_bytes_, stream);
+    rc = append_impl(p, K, V, base, pos, len, n_seen, k_new, v_new, workspace, workspace_bytes_, stream,
+                     fold ? vsum : nullptr);
     if (rc) return rc;
   }
   rc = score_impl(p, q, K, V, len, base, vsum, o, scores, workspace, workspace_bytes_, stream);

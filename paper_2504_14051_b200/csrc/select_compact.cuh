@@ -305,7 +305,8 @@ __device__ __forceinline__ bool select_one_fill_unit(int unit, int Hkv, int cap,
                                                      char* __restrict__ V, float* __restrict__ base,
                                                      int* __restrict__ pos, const int* __restrict__ len,
                                                      const int* __restrict__ budget, int* __restrict__ evict_idx,
-                                                     int max_evict, int* __restrict__ n_evict) {
+                                                     int max_evict, int* __restrict__ n_evict, float* __restrict__ vsum,
+                                                     int elt_bytes) {
   __shared__ unsigned long long s_key[kSelThreads / 32];
   __shared__ int s_slot[kSelThreads / 32];
   constexpr int kPer = 8;
@@ -368,6 +369,16 @@ __device__ __forceinline__ bool select_one_fill_unit(int unit, int Hkv, int cap,
     if (ok < best || (ok == best && os < best_slot)) { best = ok; best_slot = os; }
   }
   if (tid == 0) evict_idx[(size_t)unit * max_evict] = best_slot;
+  if (vsum) {  // FastCAOTE: the evicted row leaves the running sum of values before the last row lands on it
+    const int D = row_bytes / elt_bytes, c = tid - 128;
+    if (c >= 0 && c < D) {
+      const char* vrow = V + ((size_t)unit * cap + best_slot) * row_bytes;
+      const float v = (elt_bytes == 2) ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(vrow)[c])
+                                       : reinterpret_cast<const float*>(vrow)[c];
+      vsum[(size_t)unit * D + c] -= v;
+    }
+    __syncthreads();
+  }
   if (best_slot != last) {  // the last row fills the hole
     const size_t hole = (size_t)unit * cap + best_slot;
     if (warp == 1 && row_lane) *reinterpret_cast<uint4*>(K + hole * row_bytes + lane * 16) = row;
@@ -407,8 +418,9 @@ select_compact_kernel(int B, int Hkv, int cap, int row_bytes, const float* __res
   ptx::pdl_wait();
   ptx::pdl_trigger();
   const int unit = blockIdx.x;
-  if (!vsum && row_bytes <= 512 &&
-      select_one_fill_unit(unit, Hkv, cap, row_bytes, scores, K, V, base, pos, len, budget, evict_idx, max_evict, n_evict)) {
+  if (row_bytes <= 512 &&
+      select_one_fill_unit(unit, Hkv, cap, row_bytes, scores, K, V, base, pos, len, budget, evict_idx, max_evict, n_evict,
+                           vsum, elt_bytes)) {
     finish_lengths(B, len, n_evict, ticket);
     return;
   }
@@ -536,11 +548,13 @@ append_kernel(int Hkv, int cap, int m, int row_bytes, char* __restrict__ K, char
 
 // Append of a few rows (Hkv * m <= 16): one CTA per sequence, a warp for each K row and each V row. The CTA reads the
 // sequence's length once, so it can move it on itself after a barrier and no counter over the CTAs is needed.
-// block = 64 * Hkv * m threads.
+// block = 64 * Hkv * m threads. With vsum (FastCAOTE, m = 1 only: one row per unit, so nobody else touches the unit's
+// sums) the new value row is also added to the unit's running sum of value rows.
 __global__ void __launch_bounds__(1024)
 append_seq_kernel(int Hkv, int cap, int m, int row_bytes, char* __restrict__ K, char* __restrict__ V,
                   float* __restrict__ base, int* __restrict__ pos, int* __restrict__ len, int* __restrict__ n_seen,
-                  const char* __restrict__ k_new, const char* __restrict__ v_new, int* status) {
+                  const char* __restrict__ k_new, const char* __restrict__ v_new, int* status, float* __restrict__ vsum,
+                  int elt_bytes) {
   ptx::pdl_wait();
   ptx::pdl_trigger();
   const int b = blockIdx.x;
@@ -555,7 +569,25 @@ append_seq_kernel(int Hkv, int cap, int m, int row_bytes, char* __restrict__ K, 
   const int unit = b * Hkv + h;
   const size_t dst = (size_t)unit * cap + n + i, src = (size_t)unit * m + i;
   if (warp & 1) {
-    warp_copy_row(V + dst * row_bytes, v_new + src * row_bytes, row_bytes, lane);
+    if (vsum) {
+      for (int o = lane * 16; o < row_bytes; o += 32 * 16) {
+        const uint4 v = *reinterpret_cast<const uint4*>(v_new + src * row_bytes + o);
+        *reinterpret_cast<uint4*>(V + dst * row_bytes + o) = v;
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        float* vs = vsum + (size_t)unit * (row_bytes / elt_bytes) + o / elt_bytes;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          if (elt_bytes == 2) {
+            vs[2 * e] += __uint_as_float(w[e] << 16);
+            vs[2 * e + 1] += __uint_as_float(w[e] & 0xffff0000u);
+          } else {
+            vs[e] += __uint_as_float(w[e]);
+          }
+        }
+      }
+    } else {
+      warp_copy_row(V + dst * row_bytes, v_new + src * row_bytes, row_bytes, lane);
+    }
   } else {
     warp_copy_row(K + dst * row_bytes, k_new + src * row_bytes, row_bytes, lane);
     if (lane == 0) {
