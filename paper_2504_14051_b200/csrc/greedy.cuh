@@ -129,7 +129,7 @@ greedy_kernel(int Hkv, int cap, const T* __restrict__ V, const float* __restrict
     {
       constexpr int E = 16 / (int)sizeof(T);  // elements per 16-byte piece
       constexpr int NCH = D / 8 / E;          // pieces per lane
-      constexpr int kPasses = 4;
+      constexpr int kPasses = 8 / NCH;  // the passes in flight hold 32 registers of row pieces
       const int sub = lane >> 3, l8 = lane & 7;
       float x[NCH][E];
 #pragma unroll
