@@ -204,3 +204,27 @@ def test_fast_full_size_step_on_sampled_units(name, units):
         assert_close(f32(c.o)[b, h * G:(h + 1) * G], r["o"][0], f"{name} unit ({b},{h}) o")
         k = max(0, n - int(c.budget[b]))
         check_evicted(ref, pu.cpu().numpy(), n, k, ev[b, h, :k], f"{name} unit ({b},{h})")
+
+
+def test_a_sequence_without_room_keeps_its_running_sum():
+    """caote_step_fast on single-query shapes adds the new value row to the running sum inside the append: a sequence
+    whose cache has no room for the new token is skipped by the append (status: overflow), and its sum, its rows and
+    its length stay as they were; the other sequence's sum takes its new row and gives up the evicted one."""
+    B, Hq, Hkv, d, cap = 2, 8, 2, 128, 300
+    g = torch.Generator(device="cpu").manual_seed(99)
+    c = P.EvictionCache(B, Hq, Hkv, d, cap, 1, torch.bfloat16, torch.tensor([256, 300], dtype=torch.int32, device=DEV),
+                        "last_query", "fill", d ** -0.5, max_evict=1, device=DEV, method="fast")
+    K0 = torch.randn((B, Hkv, cap, d), generator=g).to(torch.bfloat16).to(DEV)
+    V0 = torch.randn((B, Hkv, cap, d), generator=g).to(torch.bfloat16).to(DEV)
+    c.load(K0, V0, torch.tensor([256, 300], dtype=torch.int32, device=DEV))  # the second one is full
+    q = torch.randn((B, Hq, 1, d), generator=g).to(torch.bfloat16).to(DEV)
+    kn = torch.randn((B, Hkv, 1, d), generator=g).to(torch.bfloat16).to(DEV)
+    vn = torch.randn((B, Hkv, 1, d), generator=g).to(torch.bfloat16).to(DEV)
+    vsum0, V1 = c.vsum.clone(), c.V.clone()
+    c.step(q, kn, vn)
+    torch.cuda.synchronize()
+    assert c.status() == P.binding.ERR_OVERFLOW
+    assert c.lens.tolist() == [256, 300] and c.n_evict.tolist() == [1, 0]
+    assert torch.equal(c.vsum[1], vsum0[1]) and torch.equal(c.V[1], V1[1])
+    ref = c.V[0, :, :256].double().sum(dim=1).cpu().numpy()
+    assert_close(c.vsum[0].double().cpu().numpy(), ref, "running sum of the sequence that took its new row", rtol=1e-5, atol=2e-3)
