@@ -21,7 +21,7 @@ def make_cache(B, H, d, n, cap, dtype, seed):
     return c, q, vn, g
 
 
-@pytest.mark.parametrize("dtype,d", [(torch.bfloat16, 128), (torch.float32, 64)])
+@pytest.mark.parametrize("dtype,d", [(torch.bfloat16, 128), (torch.float32, 64), (torch.float32, 128)])
 @pytest.mark.parametrize("n", [37, 2049, 9000])
 def test_new_token_with_the_lowest_score_is_evicted_in_place(dtype, d, n):
     """One head per unit; the new key points away from the query (logit -20 below zero), so the new token has by far
@@ -40,7 +40,7 @@ def test_new_token_with_the_lowest_score_is_evicted_in_place(dtype, d, n):
     assert torch.equal(c.pos[:, :, :n], pos0[:, :, :n])
 
 
-@pytest.mark.parametrize("dtype,d", [(torch.bfloat16, 128), (torch.float32, 64)])
+@pytest.mark.parametrize("dtype,d", [(torch.bfloat16, 128), (torch.float32, 64), (torch.float32, 128)])
 @pytest.mark.parametrize("n", [37, 2049, 9000])
 def test_last_row_fills_the_hole(dtype, d, n):
     """The new key is the query's direction (the largest weight by far), so some older token goes: the new token's row
