@@ -69,3 +69,39 @@ def test_last_row_fills_the_hole(dtype, d, n):
             assert torch.equal(c.V[b, h, :n][keep], V0[b, h, :n][keep])
             assert torch.equal(c.K[b, h, e], kn[b, h, 0]) and torch.equal(c.V[b, h, e], vn[b, h, 0])
             assert int(c.pos[b, h, e]) == n and torch.equal(c.pos[b, h, :n][keep], pos0[b, h, :n][keep])
+
+
+@pytest.mark.parametrize("dtype,d", [(torch.bfloat16, 128), (torch.float32, 64)])
+@pytest.mark.parametrize("n", [300, 9000])
+def test_equal_lowest_scores_go_by_position(dtype, d, n):
+    """Three cached tokens of every unit are copies of one another (same key, same value) with by far the smallest
+    weight, so their scores are the unit's lowest and, computed the same way, equal; positions are a permutation, so the
+    copy in the highest slot can have the lowest position. The evicted slot is the arg-min over (score bits, position)
+    of the scores this call wrote."""
+    B, H, cap = 2, 2, n + 8
+    c, q, vn, g = make_cache(B, H, d, n, cap, dtype, 300 + n)
+    qf = q.float()
+    low = (-(20.0 / (d ** -0.5 * (qf * qf).sum(-1, keepdim=True))) * qf).to(dtype)  # [B, H, 1, d]
+    K0, V0 = c.K.clone(), c.V.clone()
+    copies = [5, n // 2, n - 2]
+    for j in copies:
+        K0[:, :, j] = low[:, :, 0]
+        V0[:, :, j] = V0[:, :, 5]
+    pos0 = torch.stack([torch.stack([torch.randperm(cap, generator=g) for _ in range(H)]) for _ in range(B)]).to(torch.int32).to(DEV)
+    c.load(K0, V0, torch.full((B,), n, dtype=torch.int32, device=DEV), pos=pos0)
+    c.n_seen.fill_(cap)  # the new token's position: above every cached one
+    kn = ((12.0 / (d ** -0.5 * (qf * qf).sum(-1, keepdim=True))) * qf).to(dtype)
+    c.step(q, kn, vn)
+    torch.cuda.synchronize()
+    assert c.status() == 0 and c.n_evict.tolist() == [1] * B
+    ties = 0
+    for b in range(B):
+        for h in range(H):
+            sc = c.scores[b, h, :n + 1]
+            cand = torch.nonzero(sc == sc.min()).flatten()
+            ties += int(len(cand) > 1)
+            pos_pre = torch.cat([pos0[b, h, :n], torch.tensor([cap], dtype=torch.int32, device=DEV)])
+            want = int(cand[torch.argmin(pos_pre[cand])])
+            assert int(c.evict_idx[b, h, 0]) == want
+            assert want in copies
+    assert ties > 0, "the copies' scores were expected to be equal in at least one unit"
